@@ -1,0 +1,56 @@
+"""CPU oracle: GEMM-ready weight repack (naive) -- TEST INFRASTRUCTURE ONLY.
+
+The paper's sgemm/pack kernels use a "simpler weights transformation" than
+Winograd (its Section 3.1.1 and the sgemm-pack4 / pack4 rows of Table 2): a
+pure re-ordering of the raw weights into the layout the GEMM consumes.  The
+paper does not print that layout (it is the substrate library's), so the
+layout is defined here:
+
+    raw   W[k][c][r][s]                      (OIHW, fp32)
+    pack  P[k][q],  q = (r*S + s)*C + c,     row length Qp = ceil(R*S*C / 8) * 8,
+          entries with q >= R*S*C are +0.0
+
+In bf16 mode every element is additionally rounded fp32 -> bf16 with
+round-to-nearest-even, done with integer bit operations.
+"""
+import numpy as np
+
+
+def padded_q(C, R, S):
+    return -(-(R * S * C) // 8) * 8
+
+
+def pack_offset(k, c, r, s, C, R, S):
+    """Element offset of raw weight (k,c,r,s) inside the packed array."""
+    return k * padded_q(C, R, S) + (r * S + s) * C + c
+
+
+def bf16_bits_rne(a):
+    """fp32 array -> uint16 bf16 bit patterns, round to nearest even (finite inputs)."""
+    bits = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bias = np.uint64(0x7FFF) + ((bits >> np.uint64(16)) & np.uint64(1))
+    return ((bits + bias) >> np.uint64(16)).astype(np.uint16)
+
+
+def bf16_to_f32(bits16):
+    return (np.asarray(bits16, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def pack_weights(w, bf16=False):
+    """Naive repack (loops over c, r, s; numpy over k) of w (K,C,R,S) fp32.
+
+    Returns a (K, Qp) array: fp32 (bit-identical copies) or uint16 bf16 bits.
+    """
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    K, C, R, S = w.shape
+    Qp = padded_q(C, R, S)
+    flat = np.zeros(K * Qp, dtype=np.float32)
+    rows = np.arange(K) * Qp                     # pack_offset is linear in k with stride Qp
+    for c in range(C):
+        for r in range(R):
+            for s in range(S):
+                flat[rows + pack_offset(0, c, r, s, C, R, S)] = w[:, c, r, s]
+    P = flat.reshape(K, Qp)
+    if bf16:
+        return bf16_bits_rne(P)
+    return P
