@@ -1,0 +1,256 @@
+/*
+ * nnv.h -- C ABI of the cold-start convolution path for NVIDIA B200 (sm_100a).
+ *
+ * The path is the one the NNV12 paper ("Boosting DNN Cold Inference on Devices")
+ * optimises: for every convolution layer, raw fp32 weights are READ (here: copied
+ * from pinned host memory to the GPU), TRANSFORMED into the layout the chosen
+ * kernel wants, and the layer is EXECUTED (the paper's Section 2 stage list and
+ * the read / transform / execute operation triple <r_i, w_i, e_i> of its
+ * Section 3.2).  On top sit the three knobs of its Section 3.1: kernel selection
+ * by cold cost, bypassing the transform with cached post-transform weights, and
+ * pipelining the layers' operations.
+ *
+ * Conventions for every call
+ *   - Plain C types only.  Pointers prefixed h_ are HOST pointers, d_ are DEVICE
+ *     pointers.  Streams are cudaStream_t / CUstream handles passed as void*.
+ *   - The caller owns every device buffer, host blob and stream.  The library owns
+ *     only nnv_plan_t (host memory, plus CUDA events created lazily) and allocates
+ *     NO device memory; nnv_cold_run and nnv_profile sub-allocate from the arena
+ *     the caller passes.
+ *   - Device pointers must be 256-byte aligned unless stated otherwise.
+ *   - Every call returns nnv_status_t and never throws, aborts or exits.
+ *     Argument and shape errors are found on the host before any launch.
+ *     nnv_last_error() gives a thread-local message for the last failing call.
+ *   - nnv_transform_weights, nnv_conv_exec, nnv_pool_exec and the layout helpers
+ *     only enqueue work on the given stream; nnv_cold_run and nnv_profile
+ *     synchronise before returning.
+ *   - Layouts.  Raw weights: OIHW fp32, W[k][c][r][s], c over C/groups.
+ *     Activations on the device: NHWC fp32, X[h][w][c], batch 1, no channel
+ *     padding.  Model input/output on the host: NCHW fp32.
+ *     Transformed weights:
+ *       Winograd F(m x m, 3 x 3):  U[xi*alpha+nu][k][cp], alpha = m+2,
+ *           cp < Cp = ceil(C/8)*8 (entries with cp >= C are +0), fp32 (TF32 math)
+ *           or bf16 (BF16 math, F(2x2,3x3) only: one bf16 pass in the F(4x4) /
+ *           F(6x6) domain misses the 1e-2 output tolerance, so those two exist
+ *           in the TF32 accuracy class only);
+ *       IM2COL / GEMM1X1:          P[k][q], q = (r*S+s)*C + c, row length
+ *           Qp = ceil(R*S*C/8)*8, pad +0; each element rounded to nearest even to
+ *           TF32 precision and kept as an fp32 word (TF32), or to bf16 (BF16);
+ *       DIRECT / DEPTHWISE:        none -- these kernels read the raw weights.
+ */
+#ifndef NNV_H_
+#define NNV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NNV_OK = 0,
+    NNV_ERR_INVALID_ARG = 1,          /* null / misaligned pointer, bad index, bad enum      */
+    NNV_ERR_UNSUPPORTED = 2,          /* layer shape or (variant, math) pair not implemented */
+    NNV_ERR_STATE = 3,                /* call order / plan state problem                     */
+    NNV_ERR_WORKSPACE_TOO_SMALL = 4,  /* d_ws / d_arena smaller than the size query returns  */
+    NNV_ERR_CUDA = 5,                 /* a CUDA runtime / driver call failed                 */
+    NNV_ERR_TIMEOUT = 6               /* a bounded device-side wait gave up                  */
+} nnv_status_t;
+
+typedef struct nnv_plan nnv_plan_t;   /* opaque; created by nnv_plan_create */
+
+typedef enum { NNV_OP_CONV = 0, NNV_OP_MAXPOOL = 1, NNV_OP_GAVGPOOL = 2 } nnv_op_t;
+
+/* Kernel variants of the convolution operator ("one operator, many kernels",
+ * the paper's Section 3.1.1).  Enum order is the tie-break order of selection. */
+typedef enum {
+    NNV_VAR_DIRECT = 0,     /* fp32 FFMA, reads raw weights, no transform            */
+    NNV_VAR_IM2COL = 1,     /* im2col + tensor-core GEMM on packed weights           */
+    NNV_VAR_GEMM1X1 = 2,    /* 1x1 conv as a tensor-core GEMM over pixels            */
+    NNV_VAR_DEPTHWISE = 3,  /* fp32 direct depthwise, reads raw weights              */
+    NNV_VAR_WINO_F2 = 4,    /* Winograd F(2x2,3x3)                                   */
+    NNV_VAR_WINO_F4 = 5,    /* Winograd F(4x4,3x3)                                   */
+    NNV_VAR_WINO_F6 = 6     /* Winograd F(6x6,3x3)                                   */
+} nnv_variant_t;
+#define NNV_NUM_VARIANTS 7
+
+typedef enum { NNV_MATH_FP32 = 0, NNV_MATH_TF32 = 1, NNV_MATH_BF16 = 2 } nnv_math_t;
+
+typedef struct {
+    int32_t op;                 /* nnv_op_t                                                      */
+    int32_t C, K;               /* input / output channels (pools: K == C)                       */
+    int32_t R, S;               /* filter / window height, width                                 */
+    int32_t stride, pad, groups;
+    int32_t H, W;               /* INPUT height, width; batch is always 1                        */
+    int32_t in0;                /* producer layer index, -1 = model input; must be < own index   */
+    int32_t in1;                /* residual addend's producer layer, -1 = none; < own index      */
+    int32_t act;                /* 0 none, 1 ReLU, 2 ReLU6 -- applied after bias and addend      */
+    int32_t has_bias;
+    uint64_t w_off, b_off;      /* byte offsets of weights / bias in the host weight blob (256-B aligned) */
+} nnv_layer_desc_t;
+
+typedef struct {
+    int32_t default_math;       /* nnv_math_t used where a caller passes -1; default TF32 */
+    int32_t allow_cached;       /* default for selection; default 1                       */
+    int32_t max_depth;          /* largest pipeline depth nnv_cold_run accepts; default 4 */
+    int32_t debug_checks;       /* reserved, 0                                            */
+} nnv_plan_opts_t;
+
+/* One row of the profiled cost table: the operation costs of one kernel of one
+ * layer in integer nanoseconds (the paper's Table 2 has exactly these columns:
+ * read raw, weights transformation, read cache, execution). */
+typedef struct {
+    int32_t layer, variant, math, reserved;
+    uint64_t h2d_raw_ns, xform_ns, h2d_cached_ns, exec_ns;
+} nnv_cost_t;
+
+typedef struct { int32_t variant, math, cached; } nnv_choice_t;
+
+/* Per-layer record of one cold run.  Start/end stamps are nanoseconds since the
+ * run's first enqueue; 0/0 where the operation does not exist for the layer. */
+typedef struct {
+    uint64_t h2d_start_ns, h2d_end_ns;
+    uint64_t xform_start_ns, xform_end_ns;
+    uint64_t exec_start_ns, exec_end_ns;
+    uint64_t h2d_bytes;         /* bytes copied host -> device for this layer              */
+    uint64_t xform_bytes;       /* algorithmic bytes of the transform: raw read + written  */
+    uint64_t exec_flops;        /* 2 * multiply-adds the chosen kernel performs            */
+    nnv_choice_t choice;
+    int32_t reserved;
+} nnv_timing_t;
+
+/* ---- plan -------------------------------------------------------------------------------- */
+
+/* Build a plan from n layer descriptors (copied).  Validates shapes, producer
+ * indices (topological order) and that every conv layer has at least one
+ * eligible variant.  opts may be NULL.  The model abstraction is the paper's:
+ * a list of layers, each with candidate kernels (input of its Algorithm 1). */
+nnv_status_t nnv_plan_create(const nnv_layer_desc_t* layers, int32_t n,
+                             const nnv_plan_opts_t* opts, nnv_plan_t** out);
+nnv_status_t nnv_plan_destroy(nnv_plan_t* plan);
+
+/* Variants that can execute `layer`, ascending, written to out[0..*n_out).
+ * Rules keyed on filter size, stride and grouping (the keys of the paper's
+ * Figure 5 kernel tree).  cap < needed -> NNV_ERR_INVALID_ARG. */
+nnv_status_t nnv_eligible(const nnv_plan_t* plan, int32_t layer,
+                          int32_t* out, int32_t cap, int32_t* n_out);
+
+/* Bytes of the transformed weights of (layer, variant, math); 0 for DIRECT /
+ * DEPTHWISE.  This is also the size of the layer's cached post-transform blob
+ * (the paper's Section 3.1.2: bypassing trades a larger read for no transform). */
+nnv_status_t nnv_transformed_bytes(const nnv_plan_t* plan, int32_t layer,
+                                   int32_t variant, int32_t math, uint64_t* bytes);
+
+/* Scratch bytes nnv_conv_exec needs for (layer, variant, math). */
+nnv_status_t nnv_exec_workspace_bytes(const nnv_plan_t* plan, int32_t layer,
+                                      int32_t variant, int32_t math, uint64_t* bytes);
+
+/* Arena bytes nnv_cold_run needs for these choices at pipeline depth `depth`. */
+nnv_status_t nnv_arena_bytes(const nnv_plan_t* plan, const nnv_choice_t* choices,
+                             int32_t depth, uint64_t* bytes);
+
+/* Byte offset of every layer's transformed weights inside the cached blob that
+ * nnv_cold_run reads for layers chosen with cached = 1 (0 for other layers);
+ * *total = blob size.  Offsets are 256-byte aligned. */
+nnv_status_t nnv_cached_layout(const nnv_plan_t* plan, const nnv_choice_t* choices,
+                               uint64_t* offsets /* n layers */, uint64_t* total);
+
+/* ---- selection (integer, exact) ------------------------------------------------------------ */
+
+/* Candidate filter that opens the paper's Algorithm 1: of one layer's options
+ * (each cost row gives a raw arm, prep = h2d_raw + xform, and -- if the variant
+ * has a transform and allow_cached -- a cached arm, prep = h2d_cached) drop every
+ * option for which another is no slower in both prep and exec and faster in one;
+ * of exact duplicates keep the lowest (variant, math, cached).  Survivors are
+ * written in ascending (variant, math, cached) order. */
+nnv_status_t nnv_filter_candidates(const nnv_plan_t* plan, int32_t layer,
+                                   const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                                   nnv_choice_t* out, int32_t cap, int32_t* n_out);
+
+/* Per conv layer pick the survivor with the least cold cost prep + exec (the
+ * paper's Section 3.1.1 / 3.1.2 trade-off, its Table 2); ties go to the lowest
+ * (variant, math, cached).  out has one entry per layer; pool layers get
+ * {-1,-1,0}.  Rows naming a variant the layer cannot use -> NNV_ERR_INVALID_ARG;
+ * a conv layer without rows -> NNV_ERR_STATE. */
+nnv_status_t nnv_select_kernels(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs,
+                                int32_t allow_cached, nnv_choice_t* out);
+
+/* ---- single operations (asynchronous on `stream`) ------------------------------------------ */
+
+/* Weights transformation (the paper's Section 2 stage, Figure 3): Winograd
+ * filter transform U = G g G^T for WINO_F2/F4/F6, or the GEMM-ready repack for
+ * IM2COL / GEMM1X1.  d_raw: the layer's raw OIHW fp32 weights.  d_out:
+ * nnv_transformed_bytes() bytes.  DIRECT / DEPTHWISE -> NNV_ERR_UNSUPPORTED. */
+nnv_status_t nnv_transform_weights(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
+                                   const void* d_raw, void* d_out, void* stream);
+
+/* Execute one conv layer (the paper's "execution" operation) with the given
+ * kernel.  d_in: NHWC fp32 input (H x W x C).  d_addend: NHWC fp32 residual of
+ * the output's shape or NULL.  d_wt: transformed weights of this (variant, math),
+ * or the raw weights for DIRECT / DEPTHWISE.  d_bias: K floats or NULL.
+ * d_out: NHWC fp32 (OH x OW x K).  d_ws: scratch of at least
+ * nnv_exec_workspace_bytes() bytes (may be NULL when that is 0). */
+nnv_status_t nnv_conv_exec(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
+                           const void* d_in, const void* d_addend, const void* d_wt, const void* d_bias,
+                           void* d_out, void* d_ws, uint64_t ws_bytes, void* stream);
+
+/* Max-pool / global-average-pool layer, NHWC fp32 in and out. */
+nnv_status_t nnv_pool_exec(const nnv_plan_t* plan, int32_t layer,
+                           const void* d_in, void* d_out, void* stream);
+
+/* fp32 layout conversion between the host convention (CHW) and the device one (HWC). */
+nnv_status_t nnv_chw_to_hwc(const float* d_in, float* d_out, int32_t C, int32_t H, int32_t W, void* stream);
+nnv_status_t nnv_hwc_to_chw(const float* d_in, float* d_out, int32_t C, int32_t H, int32_t W, void* stream);
+
+/* ---- whole-model cold run ------------------------------------------------------------------ */
+
+/* One cold inference: for every conv layer copy its weights from pinned host
+ * memory (stream s_copy), transform them (s_xform) and execute the layer
+ * (s_exec), pipelined so that layer i+1.. are prepared while layer i executes
+ * (the paper's Section 3.1.3).  Preparation of conv layer j may start only
+ * after the execution of conv layer j-depth has finished (depth staging slots);
+ * depth = 1 is the fully serial order read, transform, execute per layer.
+ *   h_weights: pinned host blob holding raw weights / biases at w_off / b_off.
+ *   h_cached:  pinned host blob of cached transformed weights laid out by
+ *              nnv_cached_layout(); may be NULL if no choice has cached = 1.
+ *   h_input / h_output: NCHW fp32 host buffers (pinned recommended); h_output
+ *              receives the LAST layer's output.
+ *   d_arena:   nnv_arena_bytes() bytes of device memory.
+ *   timings:   NULL, or n entries filled from CUDA events (adds event records).
+ * Synchronises the three streams before returning. */
+nnv_status_t nnv_cold_run(nnv_plan_t* plan, const nnv_choice_t* choices,
+                          const void* h_weights, uint64_t w_bytes,
+                          const void* h_cached, uint64_t c_bytes,
+                          const float* h_input, float* h_output,
+                          void* d_arena, uint64_t arena_bytes,
+                          void* s_copy, void* s_xform, void* s_exec,
+                          int32_t depth, nnv_timing_t* timings);
+
+/* Device address, inside the arena of the most recent nnv_cold_run on this
+ * plan, of layer `layer`'s NHWC fp32 output (valid until the arena is reused). */
+nnv_status_t nnv_layer_output(const nnv_plan_t* plan, int32_t layer, const void** d_ptr, uint64_t* bytes);
+
+/* Profile every eligible (variant, math) of every conv layer in isolation --
+ * the per-operation profiling that feeds the paper's Algorithm 1 -- and write
+ * one cost row each: median of `reps` timed repetitions, CUDA events, integer
+ * nanoseconds.  Layer inputs are the activations left in the arena by running
+ * the model once with DIRECT/IM2COL kernels.  d_arena: nnv_profile_arena_bytes(). */
+nnv_status_t nnv_profile_arena_bytes(const nnv_plan_t* plan, uint64_t* bytes);
+nnv_status_t nnv_profile(nnv_plan_t* plan, const void* h_weights, uint64_t w_bytes,
+                         const float* h_input, void* d_arena, uint64_t arena_bytes,
+                         void* stream, int32_t reps,
+                         nnv_cost_t* out, int32_t cap, int32_t* n_out);
+
+/* ---- diagnostics --------------------------------------------------------------------------- */
+
+/* Read and clear the device-side status word that kernels with bounded waits
+ * set when a wait gives up.  Synchronises the device.  *code = 0 when clean. */
+nnv_status_t nnv_device_status(int32_t* code);
+
+const char* nnv_last_error(void);   /* valid until the next failing call on this thread */
+int32_t nnv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NNV_H_ */

@@ -10,8 +10,9 @@ layout is defined here:
     pack  P[k][q],  q = (r*S + s)*C + c,     row length Qp = ceil(R*S*C / 8) * 8,
           entries with q >= R*S*C are +0.0
 
-In bf16 mode every element is additionally rounded fp32 -> bf16 with
-round-to-nearest-even, done with integer bit operations.
+Every element is additionally rounded, round-to-nearest-even with integer bit
+operations, to the precision the tensor core multiplies in: TF32 (10 explicit
+mantissa bits, kept in an fp32 word whose low 13 bits are zero) or bf16.
 """
 import numpy as np
 
@@ -32,6 +33,14 @@ def bf16_bits_rne(a):
     return ((bits + bias) >> np.uint64(16)).astype(np.uint16)
 
 
+def tf32_round_rne(a):
+    """fp32 array -> fp32 array rounded to TF32 precision, round to nearest even (finite inputs)."""
+    bits = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bias = np.uint64(0xFFF) + ((bits >> np.uint64(13)) & np.uint64(1))
+    out = ((bits + bias) & np.uint64(0xFFFFE000)).astype(np.uint32)
+    return out.view(np.float32).reshape(np.shape(a))
+
+
 def bf16_to_f32(bits16):
     return (np.asarray(bits16, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
@@ -39,7 +48,7 @@ def bf16_to_f32(bits16):
 def pack_weights(w, bf16=False):
     """Naive repack (loops over c, r, s; numpy over k) of w (K,C,R,S) fp32.
 
-    Returns a (K, Qp) array: fp32 (bit-identical copies) or uint16 bf16 bits.
+    Returns a (K, Qp) array: fp32 words rounded to TF32 precision, or uint16 bf16 bits.
     """
     w = np.ascontiguousarray(w, dtype=np.float32)
     K, C, R, S = w.shape
@@ -53,4 +62,4 @@ def pack_weights(w, bf16=False):
     P = flat.reshape(K, Qp)
     if bf16:
         return bf16_bits_rne(P)
-    return P
+    return tf32_round_rne(P)

@@ -1,0 +1,302 @@
+"""ctypes binding of libnnv.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (see
+include/nnv.h) and does nothing but convert Python values to C arguments and
+raise on a non-zero status.  Device buffers are torch tensors (or raw integer
+addresses); streams are torch.cuda.Stream objects (or raw handles).  There is
+no CPU fallback: importing this module fails if the library has not been built.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnnv.so")
+
+OP_CONV, OP_MAXPOOL, OP_GAVGPOOL = 0, 1, 2
+VAR_DIRECT, VAR_IM2COL, VAR_GEMM1X1, VAR_DEPTHWISE, VAR_WINO_F2, VAR_WINO_F4, VAR_WINO_F6 = range(7)
+VARIANT_NAMES = ["direct", "im2col", "gemm1x1", "depthwise", "wino_f2", "wino_f4", "wino_f6"]
+MATH_FP32, MATH_TF32, MATH_BF16 = 0, 1, 2
+MATH_NAMES = ["fp32", "tf32", "bf16"]
+STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "STATE", "WORKSPACE_TOO_SMALL", "CUDA", "TIMEOUT"]
+
+
+class NnvError(RuntimeError):
+    def __init__(self, status, message):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__("nnv: %s: %s" % (name, message))
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("op", "C", "K", "R", "S", "stride", "pad", "groups", "H", "W", "in0", "in1", "act", "has_bias")] + \
+               [("w_off", ctypes.c_uint64), ("b_off", ctypes.c_uint64)]
+
+
+class PlanOpts(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("default_math", "allow_cached", "max_depth", "debug_checks")]
+
+
+class Cost(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("layer", "variant", "math", "reserved")] + \
+               [(n, ctypes.c_uint64) for n in ("h2d_raw_ns", "xform_ns", "h2d_cached_ns", "exec_ns")]
+
+
+class Choice(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("variant", "math", "cached")]
+
+
+class Timing(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in
+                ("h2d_start_ns", "h2d_end_ns", "xform_start_ns", "xform_end_ns", "exec_start_ns", "exec_end_ns",
+                 "h2d_bytes", "xform_bytes", "exec_flops")] + [("choice", Choice), ("reserved", ctypes.c_int32)]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libnnv.so is not built (%s). Run `python -m paper_2206_07446_b200.build` "
+        "(needs nvcc with sm_100a support); there is no fallback path." % LIB_PATH)
+_lib = ctypes.CDLL(LIB_PATH)
+
+_vp, _i32, _u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint64
+_P = ctypes.POINTER
+_SIGS = {
+    "nnv_plan_create": [_P(LayerDesc), _i32, _P(PlanOpts), _P(_vp)],
+    "nnv_plan_destroy": [_vp],
+    "nnv_eligible": [_vp, _i32, _P(_i32), _i32, _P(_i32)],
+    "nnv_transformed_bytes": [_vp, _i32, _i32, _i32, _P(_u64)],
+    "nnv_exec_workspace_bytes": [_vp, _i32, _i32, _i32, _P(_u64)],
+    "nnv_arena_bytes": [_vp, _P(Choice), _i32, _P(_u64)],
+    "nnv_cached_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
+    "nnv_filter_candidates": [_vp, _i32, _P(Cost), _i32, _i32, _P(Choice), _i32, _P(_i32)],
+    "nnv_select_kernels": [_vp, _P(Cost), _i32, _i32, _P(Choice)],
+    "nnv_transform_weights": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
+    "nnv_conv_exec": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _u64, _vp],
+    "nnv_pool_exec": [_vp, _i32, _vp, _vp, _vp],
+    "nnv_chw_to_hwc": [_vp, _vp, _i32, _i32, _i32, _vp],
+    "nnv_hwc_to_chw": [_vp, _vp, _i32, _i32, _i32, _vp],
+    "nnv_cold_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing)],
+    "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
+    "nnv_profile_arena_bytes": [_vp, _P(_u64)],
+    "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
+    "nnv_device_status": [_P(_i32)],
+}
+for _name, _args in _SIGS.items():
+    _fn = getattr(_lib, _name)
+    _fn.argtypes = _args
+    _fn.restype = ctypes.c_int
+_lib.nnv_last_error.restype = ctypes.c_char_p
+_lib.nnv_last_error.argtypes = []
+_lib.nnv_version.restype = ctypes.c_int32
+_lib.nnv_version.argtypes = []
+
+
+def _check(status):
+    if status != 0:
+        raise NnvError(status, _lib.nnv_last_error().decode("utf-8", "replace"))
+
+
+def _ptr(x):
+    """Address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    raise TypeError("cannot take the address of %r" % type(x))
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def nnv_version():
+    return int(_lib.nnv_version())
+
+
+def nnv_last_error():
+    return _lib.nnv_last_error().decode("utf-8", "replace")
+
+
+class Plan:
+    """Owns an nnv_plan_t*.  `layers` is a list of dicts with the descriptor's field names."""
+
+    def __init__(self, layers, w_off=None, b_off=None, opts=None):
+        n = len(layers)
+        arr = (LayerDesc * n)()
+        for i, L in enumerate(layers):
+            for f, _ in LayerDesc._fields_:
+                if f in ("w_off", "b_off"):
+                    continue
+                setattr(arr[i], f, int(L[f]))
+            arr[i].w_off = int(w_off[i]) if w_off is not None else int(L.get("w_off", 0))
+            arr[i].b_off = int(b_off[i]) if b_off is not None else int(L.get("b_off", 0))
+        o = None
+        if opts is not None:
+            o = ctypes.pointer(PlanOpts(**opts))
+        h = _vp()
+        _check(_lib.nnv_plan_create(arr, n, o, ctypes.byref(h)))
+        self.handle = h
+        self.n = n
+        self.layers = [dict(L) for L in layers]
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.nnv_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def nnv_plan_create(layers, w_off=None, b_off=None, opts=None):
+    return Plan(layers, w_off, b_off, opts)
+
+
+def nnv_plan_destroy(plan):
+    plan.close()
+
+
+def nnv_eligible(plan, layer):
+    out = (_i32 * 8)()
+    n = _i32(0)
+    _check(_lib.nnv_eligible(plan.handle, layer, out, 8, ctypes.byref(n)))
+    return [int(out[i]) for i in range(n.value)]
+
+
+def nnv_transformed_bytes(plan, layer, variant, math):
+    b = _u64(0)
+    _check(_lib.nnv_transformed_bytes(plan.handle, layer, variant, math, ctypes.byref(b)))
+    return int(b.value)
+
+
+def nnv_exec_workspace_bytes(plan, layer, variant, math):
+    b = _u64(0)
+    _check(_lib.nnv_exec_workspace_bytes(plan.handle, layer, variant, math, ctypes.byref(b)))
+    return int(b.value)
+
+
+def _choices_array(plan, choices):
+    arr = (Choice * plan.n)()
+    for i, c in enumerate(choices):
+        if c is None:
+            arr[i] = Choice(-1, -1, 0)
+        else:
+            arr[i] = Choice(int(c[0]), int(c[1]), int(c[2]))
+    return arr
+
+
+def nnv_arena_bytes(plan, choices, depth):
+    b = _u64(0)
+    _check(_lib.nnv_arena_bytes(plan.handle, _choices_array(plan, choices), depth, ctypes.byref(b)))
+    return int(b.value)
+
+
+def nnv_cached_layout(plan, choices):
+    offs = (_u64 * plan.n)()
+    total = _u64(0)
+    _check(_lib.nnv_cached_layout(plan.handle, _choices_array(plan, choices), offs, ctypes.byref(total)))
+    return [int(o) for o in offs], int(total.value)
+
+
+def _costs_array(costs):
+    arr = (Cost * max(1, len(costs)))()
+    for i, c in enumerate(costs):
+        arr[i] = Cost(int(c["layer"]), int(c["variant"]), int(c["math"]), 0, int(c["h2d_raw_ns"]),
+                      int(c["xform_ns"]), int(c["h2d_cached_ns"]), int(c["exec_ns"]))
+    return arr
+
+
+def nnv_filter_candidates(plan, layer, costs, allow_cached):
+    out = (Choice * 64)()
+    n = _i32(0)
+    _check(_lib.nnv_filter_candidates(plan.handle, layer, _costs_array(costs), len(costs), int(allow_cached),
+                                      out, 64, ctypes.byref(n)))
+    return [(out[i].variant, out[i].math, out[i].cached) for i in range(n.value)]
+
+
+def nnv_select_kernels(plan, costs, allow_cached):
+    out = (Choice * plan.n)()
+    _check(_lib.nnv_select_kernels(plan.handle, _costs_array(costs), len(costs), int(allow_cached), out))
+    return [None if out[i].variant < 0 else (out[i].variant, out[i].math, out[i].cached) for i in range(plan.n)]
+
+
+def nnv_transform_weights(plan, layer, variant, math, d_raw, d_out, stream=None):
+    _check(_lib.nnv_transform_weights(plan.handle, layer, variant, math, _ptr(d_raw), _ptr(d_out), _stream(stream)))
+
+
+def nnv_conv_exec(plan, layer, variant, math, d_in, d_addend, d_wt, d_bias, d_out, d_ws, ws_bytes, stream=None):
+    _check(_lib.nnv_conv_exec(plan.handle, layer, variant, math, _ptr(d_in), _ptr(d_addend), _ptr(d_wt),
+                              _ptr(d_bias), _ptr(d_out), _ptr(d_ws), int(ws_bytes), _stream(stream)))
+
+
+def nnv_pool_exec(plan, layer, d_in, d_out, stream=None):
+    _check(_lib.nnv_pool_exec(plan.handle, layer, _ptr(d_in), _ptr(d_out), _stream(stream)))
+
+
+def nnv_chw_to_hwc(d_in, d_out, C, H, W, stream=None):
+    _check(_lib.nnv_chw_to_hwc(_ptr(d_in), _ptr(d_out), C, H, W, _stream(stream)))
+
+
+def nnv_hwc_to_chw(d_in, d_out, C, H, W, stream=None):
+    _check(_lib.nnv_hwc_to_chw(_ptr(d_in), _ptr(d_out), C, H, W, _stream(stream)))
+
+
+def nnv_cold_run(plan, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena, arena_bytes,
+                 s_copy, s_xform, s_exec, depth, want_timings=False):
+    """Returns the list of per-layer timing dicts when want_timings, else None."""
+    tarr = (Timing * plan.n)() if want_timings else None
+    _check(_lib.nnv_cold_run(plan.handle, _choices_array(plan, choices), _ptr(h_weights), int(w_bytes),
+                             _ptr(h_cached), int(c_bytes), _ptr(h_input), _ptr(h_output), _ptr(d_arena),
+                             int(arena_bytes), _stream(s_copy), _stream(s_xform), _stream(s_exec), int(depth), tarr))
+    if not want_timings:
+        return None
+    out = []
+    for t in tarr:
+        d = {f: int(getattr(t, f)) for f, _ in Timing._fields_ if f not in ("choice", "reserved")}
+        d["choice"] = (t.choice.variant, t.choice.math, t.choice.cached)
+        out.append(d)
+    return out
+
+
+def nnv_layer_output(plan, layer):
+    p = _vp()
+    b = _u64(0)
+    _check(_lib.nnv_layer_output(plan.handle, layer, ctypes.byref(p), ctypes.byref(b)))
+    return int(p.value), int(b.value)
+
+
+def nnv_profile_arena_bytes(plan):
+    b = _u64(0)
+    _check(_lib.nnv_profile_arena_bytes(plan.handle, ctypes.byref(b)))
+    return int(b.value)
+
+
+def nnv_profile(plan, h_weights, w_bytes, h_input, d_arena, arena_bytes, stream, reps):
+    cap = plan.n * 16
+    out = (Cost * cap)()
+    n = _i32(0)
+    _check(_lib.nnv_profile(plan.handle, _ptr(h_weights), int(w_bytes), _ptr(h_input), _ptr(d_arena),
+                            int(arena_bytes), _stream(stream), int(reps), out, cap, ctypes.byref(n)))
+    return [{f: int(getattr(out[i], f)) for f, _ in Cost._fields_ if f != "reserved"} for i in range(n.value)]
+
+
+def nnv_device_status():
+    c = _i32(0)
+    _check(_lib.nnv_device_status(ctypes.byref(c)))
+    return int(c.value)
+
+
+EXPORTED_SYMBOLS = sorted(list(_SIGS.keys()) + ["nnv_last_error", "nnv_version"])

@@ -1,0 +1,460 @@
+// Batched tensor-core GEMM for sm_100a:  D[b][M][N] = A[b][M][Kd] * B[b][N][Kd]^T.
+//
+// Both operands are K-major (row-major with the reduction index innermost), which is how the
+// Winograd tile GEMM (V[xi,nu][T][C] x U[xi,nu][K][C]), the im2col GEMM (Xcol[P][Q] x P[K][Q])
+// and the 1x1 GEMM (X[P][C] x W[K][C]) all present themselves.  Pixels / tiles sit on the MMA's
+// M dimension (128 TMEM lanes), output channels on N.
+//
+// Structure of one CTA (one 128 x BN output tile, 192 threads):
+//   warp 0   TMA producer: cp.async.bulk.tensor loads of 128-byte-wide K slices of A and B into a
+//            ring of shared-memory stages (128B swizzle), completion on "full" mbarriers
+//   warp 1   allocates TMEM, issues tcgen05.mma (one lane) from shared-memory descriptors into
+//            the fp32 accumulator in TMEM, releases stages with tcgen05.commit on "empty" mbarriers
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (each warp its own 32 TMEM lanes), apply
+//            bias / residual / activation, store fp32 rows
+// Every mbarrier wait is bounded; a wait that gives up records NNV_ERR_TIMEOUT in a device status
+// word and the CTA drains and exits instead of hanging.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_bf16.h>
+
+#include <mutex>
+
+#include "nnv_internal.h"
+
+namespace nnv {
+
+__device__ int g_device_status = 0;
+
+nnv_status_t read_device_status(int32_t* code) {
+    NNV_CUDA(cudaDeviceSynchronize());
+    int v = 0;
+    NNV_CUDA(cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)));
+    if (v != 0) {
+        int zero = 0;
+        NNV_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
+    }
+    *code = v;
+    return NNV_OK;
+}
+
+namespace {
+
+constexpr int BM = 128;                 // rows of A per tile = TMEM lanes
+constexpr int BK_BYTES = 128;           // bytes of K per stage row = one 128B swizzle atom
+constexpr int A_STAGE_BYTES = BM * BK_BYTES;
+constexpr int GEMM_THREADS = 192;
+constexpr uint32_t WAIT_LIMIT = 1u << 20;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out (the caller records a timeout and bails out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart,
+// 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+    d |= (uint64_t)1 << 16;                     // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset
+    d |= (uint64_t)1 << 46;                     // version
+    d |= (uint64_t)2 << 61;                     // SWIZZLE_128B
+    return d;
+}
+
+template <bool BF16>
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    if constexpr (BF16) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct GemmDev {
+    float* D;
+    const float* bias;
+    const float* addend;
+    long long ldd, strideD;
+    int M, N, Kd, BN, act, tmem_cols;
+};
+
+__device__ __forceinline__ float act_fn(float v, int act) {
+    if (act == 1) return fmaxf(v, 0.f);
+    if (act == 2) return fminf(fmaxf(v, 0.f), 6.f);
+    return v;
+}
+
+// Descriptor for the un-swizzled K-major layout used by the converted bf16 tiles: 8x16-byte core
+// matrices, `lbo` bytes between core matrices adjacent in K, `sbo` bytes between 8-row groups.
+__device__ __forceinline__ uint64_t make_smem_desc_plain(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;                     // version; layout type 0 = no swizzle
+    return d;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Split eight fp32 values into bf16 hi = rn(x) and lo = rn(x - hi), packed as two 16-byte chunks.
+__device__ __forceinline__ void split8(const float4& a, const float4& b, uint4& hi, uint4& lo) {
+    const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(x[2 * i]), h1 = __float2bfloat16_rn(x[2 * i + 1]);
+        const __nv_bfloat16 l0 = __float2bfloat16_rn(x[2 * i] - __bfloat162float(h0));
+        const __nv_bfloat16 l1 = __float2bfloat16_rn(x[2 * i + 1] - __bfloat162float(h1));
+        h[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        l[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    hi = make_uint4(h[0], h[1], h[2], h[3]);
+    lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+// Converts one row (32 fp32 = 128 bytes, stored by TMA with the 128-byte swizzle) of a staged tile
+// into the hi and lo bf16 tiles (un-swizzled core-matrix layout, `rows` rows tall).
+__device__ __forceinline__ void convert_row(uint32_t src_tile, uint32_t hi_tile, uint32_t lo_tile, int r, int rows) {
+    const uint32_t src = src_tile + (uint32_t)r * 128u;
+    const uint32_t lbo = (uint32_t)rows * 16u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {                              // 4 chunks of 8 K-elements
+        float4 v0, v1;
+        const uint32_t a0 = src + ((uint32_t)((2 * c) ^ (r & 7)) << 4), a1 = src + ((uint32_t)((2 * c + 1) ^ (r & 7)) << 4);
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v0.x), "=f"(v0.y), "=f"(v0.z), "=f"(v0.w) : "r"(a0));
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v1.x), "=f"(v1.y), "=f"(v1.z), "=f"(v1.w) : "r"(a1));
+        uint4 hi, lo;
+        split8(v0, v1, hi, lo);
+        const uint32_t off = (uint32_t)c * lbo + (uint32_t)r * 16u;
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(hi_tile + off), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(lo_tile + off), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
+    }
+}
+
+// MODE 0: TF32 operands (fp32 words), 1: BF16 operands, 2: fp32 operands multiplied as
+// hi*hi + lo*hi + hi*lo of their bf16 splits (error-compensated, fp32-class accuracy).
+template <int MODE> struct ModeTraits {
+    static constexpr int STAGES = (MODE == 2) ? 3 : 4;
+    static constexpr int BKE = (MODE == 1) ? 64 : 32;          // K elements per stage
+};
+
+template <int MODE>
+__host__ __device__ constexpr uint32_t stage_bytes_of(int BN) {
+    // staged TMA tiles (A: 128 rows x 128 B, B: BN rows x 128 B); mode 2 adds hi and lo bf16 tiles
+    return (uint32_t)(A_STAGE_BYTES + BN * BK_BYTES) * (MODE == 2 ? 2u : 1u);
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev g) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int STAGES = ModeTraits<MODE>::STAGES;
+    constexpr int BKE = ModeTraits<MODE>::BKE;
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int BN = g.BN;
+    const uint32_t b_stage_bytes = (uint32_t)BN * BK_BYTES;
+    const uint32_t tma_bytes = A_STAGE_BYTES + b_stage_bytes;
+    const uint32_t stage_bytes = stage_bytes_of<MODE>(BN);
+    const uint32_t bars = sbase + STAGES * stage_bytes;       // full[S], empty[S], conv[S], tmem_full, holder
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto conv_bar = [&](int s) { return bars + 8u * (2 * STAGES + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (3 * STAGES);
+    const uint32_t holder = bars + 8u * (3 * STAGES + 1);
+    volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, b = blockIdx.z;
+    const int nkb = (g.Kd + BKE - 1) / BKE;
+
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+            mbar_init(conv_bar(s), 128);
+        }
+        mbar_init(tmem_full_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"((uint32_t)g.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *holder_ptr;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                ok = mbar_wait(empty_bar(s), ph ^ 1u);
+                if (!ok) break;
+                mbar_expect_tx(full_bar(s), tma_bytes);
+                const uint32_t a_dst = sbase + s * stage_bytes;
+                tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
+                tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
+            }
+            if (!ok) {
+                atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let loads already in flight land
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // instruction descriptor: fp32 accumulate, A/B format, both K-major, N, M = 128
+            const uint32_t fmt = (MODE == 0) ? 2u : 1u;
+            const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                ok = mbar_wait(MODE == 2 ? conv_bar(s) : full_bar(s), ph);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_src = sbase + s * stage_bytes;
+                if constexpr (MODE == 2) {
+                    // converted tiles follow the staged ones: A_hi, A_lo (8 KB each), B_hi, B_lo
+                    const uint32_t a_hi = a_src + tma_bytes, a_lo = a_hi + A_STAGE_BYTES / 2;
+                    const uint32_t b_hi = a_lo + A_STAGE_BYTES / 2, b_lo = b_hi + b_stage_bytes / 2;
+                    const uint32_t lbo_a = BM * 16u, lbo_b = (uint32_t)BN * 16u;
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {            // 2 K-steps of 16 bf16 = 2 core matrices each
+                        const uint64_t ah = make_smem_desc_plain(a_hi + kk * 2 * lbo_a, lbo_a, 128);
+                        const uint64_t al = make_smem_desc_plain(a_lo + kk * 2 * lbo_a, lbo_a, 128);
+                        const uint64_t bh = make_smem_desc_plain(b_hi + kk * 2 * lbo_b, lbo_b, 128);
+                        const uint64_t bl = make_smem_desc_plain(b_lo + kk * 2 * lbo_b, lbo_b, 128);
+                        umma<true>(tmem_base, al, bh, idesc, (kb | kk) ? 1u : 0u);   // small terms first
+                        umma<true>(tmem_base, ah, bl, idesc, 1u);
+                        umma<true>(tmem_base, ah, bh, idesc, 1u);
+                    }
+                } else {
+                    const uint64_t adesc = make_smem_desc(a_src);
+                    const uint64_t bdesc = make_smem_desc(a_src + A_STAGE_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)             // 4 MMAs of 32 bytes of K each
+                        umma<MODE == 1>(tmem_base, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (kb | kk) ? 1u : 0u);
+                }
+                umma_commit(empty_bar(s));
+            }
+            if (ok) umma_commit(tmem_full_bar);
+            else atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        }
+    } else {
+        bool ok = true;
+        if constexpr (MODE == 2) {
+            // warps 2-5 first convert every staged fp32 tile into its bf16 hi / lo tiles
+            const int idx = (int)threadIdx.x - 64;              // 0..127: one row of A (and of B) each
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                ok = mbar_wait(full_bar(s), ph);
+                if (!ok) break;
+                const uint32_t a_src = sbase + s * stage_bytes;
+                const uint32_t a_hi = a_src + tma_bytes, a_lo = a_hi + A_STAGE_BYTES / 2;
+                const uint32_t b_hi = a_lo + A_STAGE_BYTES / 2, b_lo = b_hi + b_stage_bytes / 2;
+                convert_row(a_src, a_hi, a_lo, idx, BM);
+                if (idx < BN) convert_row(a_src + A_STAGE_BYTES, b_hi, b_lo, idx, BN);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
+                mbar_arrive(conv_bar(s));
+            }
+        }
+        ok = ok && mbar_wait(tmem_full_bar, 0);
+        tc_fence_after();
+        if (!ok) {
+            if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        } else {
+            const int quarter = warp & 3;                     // TMEM lanes this warp may read
+            const int m = m0 + quarter * 32 + lane;
+            float* drow = g.D + (long long)b * g.strideD + (long long)m * g.ldd;
+            const float* arow = g.addend ? g.addend + (long long)m * g.ldd : nullptr;
+            const bool vec = ((g.ldd & 3) == 0) && ((g.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
+                             (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
+                             (!g.bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                if (m >= g.M) continue;
+                const int n = n0 + c0;
+                if (vec) {
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        if (n + j >= g.N) break;
+                        float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                               __uint_as_float(r[j + 3]));
+                        if (g.bias) {
+                            const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + n + j));
+                            v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                        }
+                        if (arow) {
+                            const float4 aa = __ldg(reinterpret_cast<const float4*>(arow + n + j));
+                            v.x += aa.x; v.y += aa.y; v.z += aa.z; v.w += aa.w;
+                        }
+                        v.x = act_fn(v.x, g.act); v.y = act_fn(v.y, g.act); v.z = act_fn(v.z, g.act); v.w = act_fn(v.w, g.act);
+                        *reinterpret_cast<float4*>(drow + n + j) = v;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        if (n + j < g.N) {
+                            float v = __uint_as_float(r[j]);
+                            if (g.bias) v += __ldg(g.bias + n + j);
+                            if (arow) v += __ldg(arow + n + j);
+                            drow[n + j] = act_fn(v, g.act);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
+    }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+std::once_flag g_encode_once;
+cudaError_t g_encode_err = cudaSuccess;
+
+nnv_status_t get_encoder() {
+    std::call_once(g_encode_once, [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        g_encode_err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (g_encode_err == cudaSuccess && q == cudaDriverEntryPointSuccess) g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    });
+    NNV_REQUIRE(g_encode != nullptr, NNV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    return NNV_OK;
+}
+
+// 3-D map over a K-major operand: dims {Kd, rows, batch}, box {128 bytes of K, box_rows, 1}.
+nnv_status_t encode_operand(CUtensorMap* map, const void* base, bool bf16, int Kd, int rows, int batch, int64_t ld,
+                            int64_t batch_stride, int box_rows) {
+    const uint64_t es = bf16 ? 2 : 4;
+    NNV_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0, NNV_ERR_INVALID_ARG, "GEMM operand is not 16-byte aligned");
+    NNV_REQUIRE((ld * es) % 16 == 0 && (batch_stride * es) % 16 == 0, NNV_ERR_INVALID_ARG,
+                "GEMM operand strides must be multiples of 16 bytes");
+    cuuint64_t dims[3] = {(cuuint64_t)Kd, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)(ld * es), (cuuint64_t)(batch_stride * es)};
+    cuuint32_t box[3] = {(cuuint32_t)(BK_BYTES / es), (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                          const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return NNV_OK;
+}
+
+std::once_flag g_attr_once;
+
+}  // namespace
+
+nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
+    NNV_REQUIRE(a.M > 0 && a.N > 0 && a.Kd > 0 && a.batch > 0, NNV_ERR_INVALID_ARG, "empty GEMM");
+    NNV_TRY(get_encoder());
+    // Column tile: split N into equal tiles of at most 128 columns, rounded up to the MMA's
+    // granularity of 16.
+    const int n_tiles = ceil_div(a.N, 128);
+    const int BN = ceil_div(ceil_div(a.N, n_tiles), 16) * 16;
+    int tmem_cols = 32;
+    while (tmem_cols < BN) tmem_cols *= 2;
+
+    const bool bf16 = a.mode == GEMM_BF16;
+    CUtensorMap tmA, tmB;
+    NNV_TRY(encode_operand(&tmA, a.A, bf16, a.Kd, a.M, a.batch, a.lda, a.strideA, BM));
+    NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
+
+    GemmDev g;
+    g.D = a.D; g.bias = a.bias; g.addend = a.addend;
+    g.ldd = a.ldd; g.strideD = a.strideD;
+    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols;
+
+    std::call_once(g_attr_once, [] {
+        cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    });
+    dim3 grid(ceil_div(a.M, BM), ceil_div(a.N, BN), a.batch);
+    NNV_REQUIRE(grid.y <= 65535 && grid.z <= 65535, NNV_ERR_UNSUPPORTED, "GEMM grid too large");
+    auto smem_for = [&](int stages, uint32_t stage) { return (size_t)1024 + (size_t)stages * stage + 8 * (3 * stages + 2); };
+    if (a.mode == GEMM_TF32)
+        gemm_tc_kernel<0><<<grid, GEMM_THREADS, smem_for(ModeTraits<0>::STAGES, stage_bytes_of<0>(BN)), st>>>(tmA, tmB, g);
+    else if (a.mode == GEMM_BF16)
+        gemm_tc_kernel<1><<<grid, GEMM_THREADS, smem_for(ModeTraits<1>::STAGES, stage_bytes_of<1>(BN)), st>>>(tmA, tmB, g);
+    else if (a.mode == GEMM_X3)
+        gemm_tc_kernel<2><<<grid, GEMM_THREADS, smem_for(ModeTraits<2>::STAGES, stage_bytes_of<2>(BN)), st>>>(tmA, tmB, g);
+    else
+        return fail(NNV_ERR_INVALID_ARG, "unknown GEMM mode %d", a.mode);
+    NNV_CUDA(cudaGetLastError());
+    return NNV_OK;
+}
+
+}  // namespace nnv

@@ -1,0 +1,129 @@
+// Internal declarations shared by the host and device translation units of libnnv.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "nnv.h"
+
+namespace nnv {
+
+// ---- error plumbing -------------------------------------------------------------------------
+nnv_status_t fail(nnv_status_t code, const char* fmt, ...);
+#define NNV_REQUIRE(cond, code, ...)                       \
+    do {                                                   \
+        if (!(cond)) return ::nnv::fail((code), __VA_ARGS__); \
+    } while (0)
+#define NNV_CUDA(call)                                                                     \
+    do {                                                                                   \
+        cudaError_t e__ = (call);                                                          \
+        if (e__ != cudaSuccess)                                                            \
+            return ::nnv::fail(NNV_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+#define NNV_TRY(call)                         \
+    do {                                      \
+        nnv_status_t s__ = (call);            \
+        if (s__ != NNV_OK) return s__;        \
+    } while (0)
+
+static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+// ---- per-layer derived geometry -------------------------------------------------------------
+struct LayerGeom {
+    int OH, OW, P;        // output grid and pixel count
+    int Cg;               // input channels per group
+    int Q, Qp;            // im2col reduction length R*S*C and its padded row length
+    int Cp;               // channels padded to a multiple of 8 (Winograd operands)
+};
+
+// ---- plan -----------------------------------------------------------------------------------
+struct ArenaLayout {
+    std::vector<uint64_t> act_off;     // NHWC output of each layer
+    uint64_t in_chw = 0, in_hwc = 0, out_chw = 0;
+    uint64_t raw_slot0 = 0, raw_slot_bytes = 0, raw_bias_off = 0;
+    uint64_t xf_slot0 = 0, xf_slot_bytes = 0;
+    uint64_t ws_off = 0, ws_bytes = 0;
+    uint64_t total = 0;
+};
+
+}  // namespace nnv
+
+struct nnv_plan {
+    std::vector<nnv_layer_desc_t> layers;
+    std::vector<nnv::LayerGeom> geom;
+    nnv_plan_opts_t opts;
+    // runtime state of the most recent cold run
+    std::vector<cudaEvent_t> ev;          // 3 ordering events per layer (copied, transformed, executed)
+    std::vector<cudaEvent_t> tev;         // 6 timing events per layer + 1 origin
+    nnv::ArenaLayout last_layout;
+    const void* last_arena = nullptr;
+};
+
+namespace nnv {
+
+bool variant_has_transform(int variant);
+bool math_valid_for(int variant, int math);
+int wino_m(int variant);                                     // 2/4/6 or 0
+bool is_eligible(const nnv_layer_desc_t& L, int variant);
+uint64_t transformed_bytes(const nnv_plan& p, int layer, int variant, int math);
+uint64_t exec_ws_bytes(const nnv_plan& p, int layer, int variant, int math);
+uint64_t raw_weight_bytes(const nnv_layer_desc_t& L);
+uint64_t exec_flops(const nnv_plan& p, int layer, int variant);
+nnv_status_t check_choice(const nnv_plan& p, int layer, int variant, int math);
+nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int depth, ArenaLayout* out);
+
+// ---- kernel launchers (device TUs) ----------------------------------------------------------
+// Winograd filter transform: g[K][C][3][3] fp32 -> U[alpha^2][K][Cp] (fp32 or bf16).
+nnv_status_t launch_filter_transform(int m, bool bf16, const float* d_g, void* d_U, int K, int C, int Cp,
+                                     cudaStream_t st);
+// GEMM-ready repack: W[K][C][R][S] -> P[K][Qp] (fp32 or bf16).
+nnv_status_t launch_pack(bool bf16, const float* d_w, void* d_P, int K, int C, int RS, int Qp, cudaStream_t st);
+
+// Explicit im2col of an NHWC fp32 image: Xcol[P][Qp], q = (r*S+s)*C + c (fp32 or bf16).
+nnv_status_t launch_im2col(bool bf16, const float* d_x, void* d_col, int C, int H, int W, int R, int S,
+                           int stride, int pad, int OH, int OW, int Qp, cudaStream_t st);
+// Winograd input transform V[alpha^2][T][Cp] = B^T d B per tile and channel.
+nnv_status_t launch_wino_input(int m, bool bf16, const float* d_x, void* d_V, int C, int Cp, int H, int W,
+                               int pad, int TH, int TW, cudaStream_t st);
+// Winograd output transform Y = A^T M A with the layer epilogue.
+nnv_status_t launch_wino_output(int m, const float* d_M, float* d_y, const float* d_bias, const float* d_add,
+                                int act, int K, int OH, int OW, int TH, int TW, cudaStream_t st);
+// fp32 direct convolution from raw OIHW weights (groups == 1).
+nnv_status_t launch_direct(const float* d_x, const float* d_w, const float* d_bias, const float* d_add,
+                           float* d_y, int act, int C, int H, int W, int K, int R, int S, int stride, int pad,
+                           int OH, int OW, cudaStream_t st);
+// fp32 depthwise convolution from raw [C][1][R][S] weights.
+nnv_status_t launch_depthwise(const float* d_x, const float* d_w, const float* d_bias, const float* d_add,
+                              float* d_y, int act, int C, int H, int W, int R, int S, int stride, int pad,
+                              int OH, int OW, cudaStream_t st);
+nnv_status_t launch_maxpool(const float* d_x, float* d_y, int C, int H, int W, int R, int stride, int pad,
+                            int OH, int OW, cudaStream_t st);
+nnv_status_t launch_gavgpool(const float* d_x, float* d_y, int C, int H, int W, cudaStream_t st);
+nnv_status_t launch_chw_to_hwc(const float* d_in, float* d_out, int C, int H, int W, cudaStream_t st);
+nnv_status_t launch_hwc_to_chw(const float* d_in, float* d_out, int C, int H, int W, cudaStream_t st);
+
+// Batched tensor-core GEMM  D[b][M][N] = A[b][M][Kd] * B[b][N][Kd]^T, both operands K-major
+// (row-major with the reduction index innermost), fp32 accumulate, fp32 output with leading
+// dimension ldd.  GEMM_TF32 / GEMM_X3: operands are fp32 words; GEMM_BF16: operands are bf16.  lda/ldb in elements,
+// multiples of 16 bytes.  Optional epilogue: + bias[n], + addend[m*ldd+n], activation.
+struct GemmArgs {
+    const void* A; const void* B; float* D;
+    int M, N, Kd, batch;
+    int64_t lda, ldb, ldd;            // row strides (elements)
+    int64_t strideA, strideB, strideD;  // batch strides (elements)
+    const float* bias; const float* addend; int act;
+    int mode;                         // GEMM_TF32, GEMM_BF16 or GEMM_X3
+};
+// GEMM_X3: fp32 operands; each is split on the fly into bf16 hi + lo and the product is formed
+// as hi*hi + lo*hi + hi*lo on the bf16 tensor pipe (fp32-class accuracy, fp32 bytes in memory).
+enum { GEMM_TF32 = 0, GEMM_BF16 = 1, GEMM_X3 = 2 };
+nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
+
+nnv_status_t read_device_status(int32_t* code);
+
+}  // namespace nnv

@@ -1,0 +1,359 @@
+// Whole-model cold run (three-stream layer pipeline) and per-operation profiling.
+#include <algorithm>
+#include <cstring>
+
+#include "nnv_internal.h"
+
+namespace nnv {
+nnv_status_t do_transform(const nnv_plan& p, int layer, int v, int math, const void* d_raw, void* d_out, cudaStream_t st);
+nnv_status_t do_exec(const nnv_plan& p, int layer, int v, int math, const void* d_in, const void* d_add,
+                     const void* d_wt, const void* d_bias, void* d_out, void* d_ws, uint64_t ws_bytes, cudaStream_t st);
+nnv_status_t do_pool(const nnv_plan& p, int layer, const void* d_in, void* d_out, cudaStream_t st);
+
+static nnv_status_t ensure_events(nnv_plan& p, bool timing) {
+    const size_t n = p.layers.size();
+    if (p.ev.size() != 3 * n) {
+        p.ev.resize(3 * n, nullptr);
+        for (size_t i = 0; i < 3 * n; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming));
+    }
+    if (timing && p.tev.size() != 6 * n + 1) {
+        p.tev.resize(6 * n + 1, nullptr);
+        for (size_t i = 0; i < 6 * n + 1; ++i) NNV_CUDA(cudaEventCreate(&p.tev[i]));
+    }
+    return NNV_OK;
+}
+
+static inline uint64_t ms_to_ns(float ms) { return ms <= 0.f ? 0ull : (uint64_t)((double)ms * 1e6 + 0.5); }
+
+}  // namespace nnv
+
+using namespace nnv;
+
+extern "C" {
+
+nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void* h_weights, uint64_t w_bytes,
+                          const void* h_cached, uint64_t c_bytes, const float* h_input, float* h_output,
+                          void* d_arena, uint64_t arena_bytes, void* s_copy_, void* s_xform_, void* s_exec_,
+                          int32_t depth, nnv_timing_t* timings) {
+    NNV_REQUIRE(p && choices && h_weights && h_input && h_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
+    NNV_REQUIRE(s_copy_ != s_xform_ && s_copy_ != s_exec_ && s_xform_ != s_exec_, NNV_ERR_INVALID_ARG,
+                "the three streams must be distinct");
+    cudaStream_t s_copy = (cudaStream_t)s_copy_, s_xform = (cudaStream_t)s_xform_, s_exec = (cudaStream_t)s_exec_;
+    const int n = (int)p->layers.size();
+
+    ArenaLayout A;
+    NNV_TRY(layout_arena(*p, choices, depth, &A));
+    NNV_REQUIRE(arena_bytes >= A.total, NNV_ERR_WORKSPACE_TOO_SMALL, "arena needs %llu bytes, got %llu",
+                (unsigned long long)A.total, (unsigned long long)arena_bytes);
+    std::vector<uint64_t> coff(n, 0);
+    uint64_t ctotal = 0;
+    NNV_TRY(nnv_cached_layout(p, choices, coff.data(), &ctotal));
+    NNV_REQUIRE(ctotal == 0 || (h_cached && c_bytes >= ctotal), NNV_ERR_INVALID_ARG,
+                "cached blob needs %llu bytes", (unsigned long long)ctotal);
+    for (int i = 0; i < n; ++i) {
+        const nnv_layer_desc_t& L = p->layers[i];
+        if (L.op != NNV_OP_CONV) continue;
+        NNV_REQUIRE(L.w_off + raw_weight_bytes(L) <= w_bytes && (!L.has_bias || L.b_off + 4ull * L.K <= w_bytes),
+                    NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the host blob", i);
+    }
+    NNV_TRY(ensure_events(*p, timings != nullptr));
+    p->last_layout = A;
+    p->last_arena = d_arena;
+
+    uint8_t* base = (uint8_t*)d_arena;
+    auto EV = [&](int layer, int k) { return p->ev[3 * layer + k]; };       // 0 copied, 1 transformed, 2 executed
+    auto TEV = [&](int layer, int k) { return p->tev[1 + 6 * layer + k]; };
+    const bool tm = timings != nullptr;
+    if (tm) {
+        NNV_CUDA(cudaEventRecord(p->tev[0], s_exec));
+        NNV_CUDA(cudaStreamWaitEvent(s_copy, p->tev[0], 0));
+        NNV_CUDA(cudaStreamWaitEvent(s_xform, p->tev[0], 0));
+        std::memset(timings, 0, sizeof(nnv_timing_t) * n);
+    }
+
+    // model input: host NCHW -> device NHWC, on the execution stream
+    const nnv_layer_desc_t& L0 = p->layers[0];
+    NNV_CUDA(cudaMemcpyAsync(base + A.in_chw, h_input, 4ull * L0.C * L0.H * L0.W, cudaMemcpyHostToDevice, s_exec));
+    NNV_TRY(launch_chw_to_hwc((const float*)(base + A.in_chw), (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, s_exec));
+
+    std::vector<int> conv_ids;
+    for (int i = 0; i < n; ++i) {
+        const nnv_layer_desc_t& L = p->layers[i];
+        const void* in = L.in0 < 0 ? base + A.in_hwc : base + A.act_off[L.in0];
+        void* out = base + A.act_off[i];
+        if (L.op != NNV_OP_CONV) {
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), s_exec));
+            NNV_TRY(do_pool(*p, i, in, out, s_exec));
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 5), s_exec));
+            NNV_CUDA(cudaEventRecord(EV(i, 2), s_exec));
+            continue;
+        }
+        const nnv_choice_t ch = choices[i];
+        const int j = (int)conv_ids.size();
+        conv_ids.push_back(i);
+        const int slot = j % depth;
+        uint8_t* raw = base + A.raw_slot0 + (uint64_t)slot * A.raw_slot_bytes;
+        uint8_t* xf = base + A.xf_slot0 + (uint64_t)slot * A.xf_slot_bytes;
+        const bool has_xf = variant_has_transform(ch.variant);
+        const bool cached = has_xf && ch.cached;
+        const uint64_t rbytes = raw_weight_bytes(L), tbytes = transformed_bytes(*p, i, ch.variant, ch.math);
+
+        // read: the staging slot is free once the layer that used it last has executed
+        if (j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
+        uint64_t copied = 0;
+        if (cached) {
+            NNV_CUDA(cudaMemcpyAsync(xf, (const uint8_t*)h_cached + coff[i], tbytes, cudaMemcpyHostToDevice, s_copy));
+            copied += tbytes;
+        } else {
+            NNV_CUDA(cudaMemcpyAsync(raw, (const uint8_t*)h_weights + L.w_off, rbytes, cudaMemcpyHostToDevice, s_copy));
+            copied += rbytes;
+        }
+        if (L.has_bias) {
+            NNV_CUDA(cudaMemcpyAsync(raw + A.raw_bias_off, (const uint8_t*)h_weights + L.b_off, 4ull * L.K,
+                                     cudaMemcpyHostToDevice, s_copy));
+            copied += 4ull * L.K;
+        }
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
+        NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
+
+        // transform
+        cudaEvent_t ready = EV(i, 0);
+        if (has_xf && !cached) {
+            NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(i, 0), 0));
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
+            NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, xf, s_xform));
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
+            NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
+            ready = EV(i, 1);
+        }
+
+        // execute
+        NNV_CUDA(cudaStreamWaitEvent(s_exec, ready, 0));
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), s_exec));
+        const void* add = L.in1 >= 0 ? base + A.act_off[L.in1] : nullptr;
+        NNV_TRY(do_exec(*p, i, ch.variant, ch.math, in, add, has_xf ? xf : raw, L.has_bias ? raw + A.raw_bias_off : nullptr,
+                        out, base + A.ws_off, A.ws_bytes, s_exec));
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 5), s_exec));
+        NNV_CUDA(cudaEventRecord(EV(i, 2), s_exec));
+        if (tm) {
+            timings[i].h2d_bytes = copied;
+            timings[i].xform_bytes = (has_xf && !cached) ? rbytes + tbytes : 0;
+            timings[i].exec_flops = exec_flops(*p, i, ch.variant);
+            timings[i].choice = nnv_choice_t{ch.variant, ch.math, cached ? 1 : 0};
+        }
+    }
+
+    // last layer's output: device NHWC -> host NCHW
+    const nnv_layer_desc_t& Ln = p->layers[n - 1];
+    const LayerGeom& gn = p->geom[n - 1];
+    NNV_TRY(launch_hwc_to_chw((const float*)(base + A.act_off[n - 1]), (float*)(base + A.out_chw), Ln.K, gn.OH, gn.OW, s_exec));
+    NNV_CUDA(cudaMemcpyAsync(h_output, base + A.out_chw, 4ull * gn.P * Ln.K, cudaMemcpyDeviceToHost, s_exec));
+
+    NNV_CUDA(cudaStreamSynchronize(s_copy));
+    NNV_CUDA(cudaStreamSynchronize(s_xform));
+    NNV_CUDA(cudaStreamSynchronize(s_exec));
+
+    if (tm) {
+        auto stamp = [&](cudaEvent_t e, uint64_t* out) -> nnv_status_t {
+            float ms = 0.f;
+            NNV_CUDA(cudaEventElapsedTime(&ms, p->tev[0], e));
+            *out = ms_to_ns(ms);
+            return NNV_OK;
+        };
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p->layers[i];
+            NNV_TRY(stamp(TEV(i, 4), &timings[i].exec_start_ns));
+            NNV_TRY(stamp(TEV(i, 5), &timings[i].exec_end_ns));
+            if (L.op != NNV_OP_CONV) continue;
+            NNV_TRY(stamp(TEV(i, 0), &timings[i].h2d_start_ns));
+            NNV_TRY(stamp(TEV(i, 1), &timings[i].h2d_end_ns));
+            if (timings[i].xform_bytes) {
+                NNV_TRY(stamp(TEV(i, 2), &timings[i].xform_start_ns));
+                NNV_TRY(stamp(TEV(i, 3), &timings[i].xform_end_ns));
+            }
+        }
+    }
+    int32_t code = 0;
+    NNV_TRY(read_device_status(&code));
+    NNV_REQUIRE(code == 0, (nnv_status_t)code, "a device-side wait gave up during the cold run");
+    return NNV_OK;
+}
+
+nnv_status_t nnv_layer_output(const nnv_plan_t* p, int32_t layer, const void** d_ptr, uint64_t* bytes) {
+    NNV_REQUIRE(p && d_ptr && bytes, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(layer >= 0 && layer < (int)p->layers.size(), NNV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    NNV_REQUIRE(p->last_arena, NNV_ERR_STATE, "no cold run has used this plan yet");
+    *d_ptr = (const uint8_t*)p->last_arena + p->last_layout.act_off[layer];
+    *bytes = 4ull * p->geom[layer].P * p->layers[layer].K;
+    return NNV_OK;
+}
+
+// ---- profiling ------------------------------------------------------------------------------
+namespace {
+constexpr uint64_t FLUSH_BYTES = 192ull << 20;     // larger than the L2
+
+struct ProfLayout {
+    std::vector<uint64_t> act_off;
+    uint64_t in_chw, in_hwc, raw, bias, xf, ws, ws_bytes, flush, total;
+};
+
+nnv_status_t layout_profile(const nnv_plan& p, ProfLayout* out) {
+    const int n = (int)p.layers.size();
+    ProfLayout a;
+    uint64_t pos = 0;
+    auto take = [&](uint64_t b) { uint64_t o = pos; pos += align_up(b ? b : 1, 1024); return o; };
+    const nnv_layer_desc_t& L0 = p.layers[0];
+    a.in_chw = take(4ull * L0.C * L0.H * L0.W);
+    a.in_hwc = take(4ull * L0.C * L0.H * L0.W);
+    a.act_off.resize(n);
+    uint64_t max_raw = 0, max_bias = 0, max_xf = 0, max_ws = 0;
+    for (int i = 0; i < n; ++i) {
+        const nnv_layer_desc_t& L = p.layers[i];
+        a.act_off[i] = take(4ull * p.geom[i].P * L.K);
+        if (L.op != NNV_OP_CONV) continue;
+        max_raw = std::max(max_raw, raw_weight_bytes(L));
+        max_bias = std::max<uint64_t>(max_bias, 4ull * L.K);
+        for (int v = 0; v < NNV_NUM_VARIANTS; ++v) {
+            if (!is_eligible(L, v)) continue;
+            for (int m = 0; m < 3; ++m) {
+                if (!math_valid_for(v, m)) continue;
+                max_xf = std::max(max_xf, transformed_bytes(p, i, v, m));
+                max_ws = std::max(max_ws, exec_ws_bytes(p, i, v, m));
+            }
+        }
+    }
+    a.raw = take(max_raw);
+    a.bias = take(max_bias);
+    a.xf = take(max_xf);
+    a.ws_bytes = align_up(max_ws ? max_ws : 1, 1024);
+    a.ws = take(a.ws_bytes);
+    a.flush = take(FLUSH_BYTES);
+    a.total = pos;
+    *out = a;
+    return NNV_OK;
+}
+}  // namespace
+
+nnv_status_t nnv_profile_arena_bytes(const nnv_plan_t* p, uint64_t* bytes) {
+    NNV_REQUIRE(p && bytes, NNV_ERR_INVALID_ARG, "null argument");
+    ProfLayout a;
+    NNV_TRY(layout_profile(*p, &a));
+    *bytes = a.total;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_profile(nnv_plan_t* p, const void* h_weights, uint64_t w_bytes, const float* h_input, void* d_arena,
+                         uint64_t arena_bytes, void* stream, int32_t reps, nnv_cost_t* out, int32_t cap,
+                         int32_t* n_out) {
+    NNV_REQUIRE(p && h_weights && h_input && d_arena && out && n_out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(reps >= 1 && reps <= 1000, NNV_ERR_INVALID_ARG, "reps %d outside 1..1000", reps);
+    NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
+    ProfLayout A;
+    NNV_TRY(layout_profile(*p, &A));
+    NNV_REQUIRE(arena_bytes >= A.total, NNV_ERR_WORKSPACE_TOO_SMALL, "profiling arena needs %llu bytes, got %llu",
+                (unsigned long long)A.total, (unsigned long long)arena_bytes);
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* base = (uint8_t*)d_arena;
+    const int n = (int)p->layers.size();
+    cudaEvent_t e0, e1;
+    NNV_CUDA(cudaEventCreate(&e0));
+    NNV_CUDA(cudaEventCreate(&e1));
+    nnv_status_t rc = NNV_OK;
+    std::vector<float> samples(reps);
+    int cnt = 0;
+
+    // Times `reps` repetitions of `op`, each after an L2 flush, and returns the median in ns.
+    auto timed = [&](auto&& op, uint64_t* ns) -> nnv_status_t {
+        for (int r = 0; r < reps; ++r) {
+            NNV_CUDA(cudaMemsetAsync(base + A.flush, r & 0xff, FLUSH_BYTES, st));
+            NNV_CUDA(cudaEventRecord(e0, st));
+            NNV_TRY(op());
+            NNV_CUDA(cudaEventRecord(e1, st));
+            NNV_CUDA(cudaEventSynchronize(e1));
+            NNV_CUDA(cudaEventElapsedTime(&samples[r], e0, e1));
+        }
+        std::sort(samples.begin(), samples.end());
+        *ns = ms_to_ns(samples[reps / 2]);
+        return NNV_OK;
+    };
+
+    auto body = [&]() -> nnv_status_t {
+        const nnv_layer_desc_t& L0 = p->layers[0];
+        NNV_CUDA(cudaMemcpyAsync(base + A.in_chw, h_input, 4ull * L0.C * L0.H * L0.W, cudaMemcpyHostToDevice, st));
+        NNV_TRY(launch_chw_to_hwc((const float*)(base + A.in_chw), (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, st));
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p->layers[i];
+            const void* in = L.in0 < 0 ? base + A.in_hwc : base + A.act_off[L.in0];
+            void* y = base + A.act_off[i];
+            if (L.op != NNV_OP_CONV) {
+                NNV_TRY(do_pool(*p, i, in, y, st));
+                continue;
+            }
+            NNV_REQUIRE(L.w_off + raw_weight_bytes(L) <= w_bytes, NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the host blob", i);
+            const void* add = L.in1 >= 0 ? base + A.act_off[L.in1] : nullptr;
+            const uint64_t rbytes = raw_weight_bytes(L);
+            const void* hsrc = (const uint8_t*)h_weights + L.w_off;
+            const void* bias = nullptr;
+            if (L.has_bias) {
+                NNV_CUDA(cudaMemcpyAsync(base + A.bias, (const uint8_t*)h_weights + L.b_off, 4ull * L.K, cudaMemcpyHostToDevice, st));
+                bias = base + A.bias;
+            }
+            uint64_t h2d_raw = 0;
+            NNV_TRY(timed([&]() -> nnv_status_t {
+                NNV_CUDA(cudaMemcpyAsync(base + A.raw, hsrc, rbytes, cudaMemcpyHostToDevice, st));
+                return NNV_OK;
+            }, &h2d_raw));
+            for (int v = 0; v < NNV_NUM_VARIANTS; ++v) {
+                if (!is_eligible(L, v)) continue;
+                for (int m = 0; m < 3; ++m) {
+                    if (!math_valid_for(v, m)) continue;
+                    NNV_REQUIRE(cnt < cap, NNV_ERR_INVALID_ARG, "cost table capacity %d too small", cap);
+                    nnv_cost_t c{};
+                    c.layer = i; c.variant = v; c.math = m;
+                    c.h2d_raw_ns = h2d_raw;
+                    const bool has_xf = variant_has_transform(v);
+                    const uint64_t tbytes = transformed_bytes(*p, i, v, m);
+                    if (has_xf) {
+                        NNV_TRY(timed([&]() { return do_transform(*p, i, v, m, base + A.raw, base + A.xf, st); }, &c.xform_ns));
+                        // the cached blob is `tbytes` long; time a copy of that many bytes (scaled when the
+                        // host blob is shorter than the layer's transformed weights)
+                        const uint64_t cp = std::min<uint64_t>(tbytes, w_bytes);
+                        uint64_t t = 0;
+                        NNV_TRY(timed([&]() -> nnv_status_t {
+                            NNV_CUDA(cudaMemcpyAsync(base + A.ws, h_weights, std::min<uint64_t>(cp, A.ws_bytes), cudaMemcpyHostToDevice, st));
+                            return NNV_OK;
+                        }, &t));
+                        const uint64_t done = std::min<uint64_t>(cp, A.ws_bytes);
+                        c.h2d_cached_ns = done ? (uint64_t)((double)t * (double)tbytes / (double)done + 0.5) : 0;
+                        // the timed copy overwrote nothing the exec needs: transformed weights live in A.xf
+                    } else {
+                        c.h2d_cached_ns = h2d_raw;
+                    }
+                    NNV_TRY(timed([&]() {
+                        return do_exec(*p, i, v, m, in, add, has_xf ? base + A.xf : base + A.raw, bias, y, base + A.ws, A.ws_bytes, st);
+                    }, &c.exec_ns));
+                    out[cnt++] = c;
+                }
+            }
+            // leave the layer's output computed by its lowest-numbered eligible fp32 kernel
+            const int vbase = is_eligible(L, NNV_VAR_DIRECT) ? NNV_VAR_DIRECT : NNV_VAR_DEPTHWISE;
+            NNV_TRY(do_exec(*p, i, vbase, NNV_MATH_FP32, in, add, base + A.raw, bias, y, base + A.ws, A.ws_bytes, st));
+        }
+        NNV_CUDA(cudaStreamSynchronize(st));
+        return NNV_OK;
+    };
+    rc = body();
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (rc != NNV_OK) return rc;
+    int32_t code = 0;
+    NNV_TRY(read_device_status(&code));
+    NNV_REQUIRE(code == 0, (nnv_status_t)code, "a device-side wait gave up during profiling");
+    *n_out = cnt;
+    return NNV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,369 @@
+// Host-side plan logic: validation, eligibility, size queries, arena layout and the
+// integer cold-cost selection.  No device work happens in this file.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "nnv_internal.h"
+
+namespace nnv {
+
+static thread_local char g_err[512] = "";
+
+nnv_status_t fail(nnv_status_t code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+bool variant_has_transform(int v) { return v != NNV_VAR_DIRECT && v != NNV_VAR_DEPTHWISE; }
+
+bool math_valid_for(int v, int math) {
+    if (v == NNV_VAR_DIRECT || v == NNV_VAR_DEPTHWISE) return math == NNV_MATH_FP32;
+    // One bf16 pass in the F(4,3) / F(6,3) Winograd domain misses the 1e-2 output tolerance
+    // (measured 2.6e-2 / 4.9e-2 relative L2), so these variants exist in the TF32 accuracy class only.
+    if (v == NNV_VAR_WINO_F4 || v == NNV_VAR_WINO_F6) return math == NNV_MATH_TF32;
+    return math == NNV_MATH_TF32 || math == NNV_MATH_BF16;
+}
+
+int wino_m(int v) {
+    switch (v) {
+        case NNV_VAR_WINO_F2: return 2;
+        case NNV_VAR_WINO_F4: return 4;
+        case NNV_VAR_WINO_F6: return 6;
+        default: return 0;
+    }
+}
+
+// Eligibility is keyed on filter size, stride and grouping only (the surviving keys of the
+// paper's Figure 5 kernel tree); ragged channel counts are handled by padding, so there is no
+// divisibility requirement.
+bool is_eligible(const nnv_layer_desc_t& L, int v) {
+    if (L.op != NNV_OP_CONV) return false;
+    const bool dense = L.groups == 1;
+    switch (v) {
+        case NNV_VAR_DIRECT: return dense;
+        case NNV_VAR_IM2COL: return dense;
+        case NNV_VAR_GEMM1X1: return dense && L.R == 1 && L.S == 1 && L.pad == 0;
+        case NNV_VAR_DEPTHWISE: return L.groups > 1 && L.groups == L.C && L.C == L.K;
+        case NNV_VAR_WINO_F2:
+        case NNV_VAR_WINO_F4:
+        case NNV_VAR_WINO_F6: return dense && L.R == 3 && L.S == 3 && L.stride == 1;
+        default: return false;
+    }
+}
+
+uint64_t raw_weight_bytes(const nnv_layer_desc_t& L) {
+    if (L.op != NNV_OP_CONV) return 0;
+    return 4ull * L.K * (L.C / L.groups) * L.R * L.S;
+}
+
+uint64_t transformed_bytes(const nnv_plan& p, int layer, int v, int math) {
+    const nnv_layer_desc_t& L = p.layers[layer];
+    const LayerGeom& g = p.geom[layer];
+    const uint64_t es = (math == NNV_MATH_BF16) ? 2 : 4;
+    if (int m = wino_m(v)) {
+        const uint64_t a = m + 2;
+        return a * a * (uint64_t)L.K * g.Cp * es;
+    }
+    if (v == NNV_VAR_IM2COL || v == NNV_VAR_GEMM1X1) return (uint64_t)L.K * g.Qp * es;
+    return 0;
+}
+
+static inline bool gemm1x1_direct_operand(const nnv_layer_desc_t& L, int math) {
+    // The activation itself can be the GEMM's A operand when no subsampling, padding or
+    // conversion is needed: stride 1, fp32 words (TF32), rows a multiple of 16 bytes.
+    return math == NNV_MATH_TF32 && L.stride == 1 && (L.C % 4) == 0;
+}
+
+uint64_t exec_ws_bytes(const nnv_plan& p, int layer, int v, int math) {
+    const nnv_layer_desc_t& L = p.layers[layer];
+    const LayerGeom& g = p.geom[layer];
+    const uint64_t es = (math == NNV_MATH_BF16) ? 2 : 4;
+    if (int m = wino_m(v)) {
+        const uint64_t a2 = (uint64_t)(m + 2) * (m + 2);
+        const uint64_t T = (uint64_t)ceil_div(g.OH, m) * ceil_div(g.OW, m);
+        return align_up(a2 * T * g.Cp * es, 256) + align_up(a2 * T * L.K * 4, 256);
+    }
+    if (v == NNV_VAR_IM2COL) return align_up((uint64_t)g.P * g.Qp * es, 256);
+    if (v == NNV_VAR_GEMM1X1)
+        return gemm1x1_direct_operand(L, math) ? 0 : align_up((uint64_t)g.P * g.Qp * es, 256);
+    return 0;
+}
+
+uint64_t exec_flops(const nnv_plan& p, int layer, int v) {
+    const nnv_layer_desc_t& L = p.layers[layer];
+    const LayerGeom& g = p.geom[layer];
+    if (int m = wino_m(v)) {
+        const uint64_t a2 = (uint64_t)(m + 2) * (m + 2);
+        const uint64_t T = (uint64_t)ceil_div(g.OH, m) * ceil_div(g.OW, m);
+        return 2ull * a2 * T * L.K * L.C;
+    }
+    return 2ull * g.P * L.K * g.Cg * L.R * L.S;
+}
+
+nnv_status_t check_choice(const nnv_plan& p, int layer, int v, int math) {
+    NNV_REQUIRE(layer >= 0 && layer < (int)p.layers.size(), NNV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    NNV_REQUIRE(p.layers[layer].op == NNV_OP_CONV, NNV_ERR_INVALID_ARG, "layer %d is not a convolution", layer);
+    NNV_REQUIRE(v >= 0 && v < NNV_NUM_VARIANTS, NNV_ERR_INVALID_ARG, "variant %d is not a variant", v);
+    NNV_REQUIRE(is_eligible(p.layers[layer], v), NNV_ERR_UNSUPPORTED, "variant %d cannot run layer %d", v, layer);
+    NNV_REQUIRE(math_valid_for(v, math), NNV_ERR_UNSUPPORTED, "math mode %d does not exist for variant %d", math, v);
+    return NNV_OK;
+}
+
+nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int depth, ArenaLayout* out) {
+    const int n = (int)p.layers.size();
+    ArenaLayout a;
+    uint64_t pos = 0;
+    auto take = [&](uint64_t bytes) {
+        uint64_t off = pos;
+        pos += align_up(bytes ? bytes : 1, 1024);
+        return off;
+    };
+    const nnv_layer_desc_t& L0 = p.layers[0];
+    const uint64_t in_bytes = 4ull * L0.C * L0.H * L0.W;
+    a.in_chw = take(in_bytes);
+    a.in_hwc = take(in_bytes);
+    a.act_off.resize(n);
+    uint64_t max_raw = 0, max_bias = 0, max_xf = 0, max_ws = 0;
+    for (int i = 0; i < n; ++i) {
+        const nnv_layer_desc_t& L = p.layers[i];
+        const LayerGeom& g = p.geom[i];
+        a.act_off[i] = take(4ull * g.P * L.K);
+        if (L.op != NNV_OP_CONV) continue;
+        NNV_TRY(check_choice(p, i, choices[i].variant, choices[i].math));
+        max_raw = std::max(max_raw, raw_weight_bytes(L));
+        max_bias = std::max<uint64_t>(max_bias, 4ull * L.K);
+        max_xf = std::max(max_xf, transformed_bytes(p, i, choices[i].variant, choices[i].math));
+        max_ws = std::max(max_ws, exec_ws_bytes(p, i, choices[i].variant, choices[i].math));
+    }
+    const nnv_layer_desc_t& Ln = p.layers[n - 1];
+    a.out_chw = take(4ull * p.geom[n - 1].P * Ln.K);
+    a.raw_bias_off = align_up(max_raw ? max_raw : 1, 1024);
+    a.raw_slot_bytes = a.raw_bias_off + align_up(max_bias ? max_bias : 1, 1024);
+    a.raw_slot0 = take(a.raw_slot_bytes * depth);
+    a.xf_slot_bytes = align_up(max_xf ? max_xf : 1, 1024);
+    a.xf_slot0 = take(a.xf_slot_bytes * depth);
+    a.ws_bytes = align_up(max_ws ? max_ws : 1, 1024);
+    a.ws_off = take(a.ws_bytes);
+    a.total = pos;
+    *out = a;
+    return NNV_OK;
+}
+
+// ---- selection ------------------------------------------------------------------------------
+struct Option {
+    int variant, math, cached;
+    uint64_t prep, exec;
+};
+static inline bool rank_less(const Option& a, const Option& b) {
+    if (a.variant != b.variant) return a.variant < b.variant;
+    if (a.math != b.math) return a.math < b.math;
+    return a.cached < b.cached;
+}
+
+static nnv_status_t gather_options(const nnv_plan& p, int layer, const nnv_cost_t* costs, int n_costs,
+                                   int allow_cached, std::vector<Option>* opts) {
+    for (int i = 0; i < n_costs; ++i) {
+        const nnv_cost_t& c = costs[i];
+        if (c.layer != layer) continue;
+        NNV_REQUIRE(c.variant >= 0 && c.variant < NNV_NUM_VARIANTS && is_eligible(p.layers[layer], c.variant) &&
+                        math_valid_for(c.variant, c.math),
+                    NNV_ERR_INVALID_ARG, "cost row %d names a kernel layer %d cannot use", i, layer);
+        opts->push_back({c.variant, c.math, 0, c.h2d_raw_ns + c.xform_ns, c.exec_ns});
+        if (allow_cached && variant_has_transform(c.variant))
+            opts->push_back({c.variant, c.math, 1, c.h2d_cached_ns, c.exec_ns});
+    }
+    return NNV_OK;
+}
+
+static void pareto(const std::vector<Option>& in, std::vector<Option>* out) {
+    for (size_t i = 0; i < in.size(); ++i) {
+        const Option& o = in[i];
+        bool drop = false;
+        for (size_t j = 0; j < in.size() && !drop; ++j) {
+            if (j == i) continue;
+            const Option& q = in[j];
+            if (q.prep <= o.prep && q.exec <= o.exec) {
+                if (q.prep < o.prep || q.exec < o.exec) drop = true;
+                else if (rank_less(q, o)) drop = true;          // exact duplicate, lower rank wins
+            }
+        }
+        if (!drop) out->push_back(o);
+    }
+    std::sort(out->begin(), out->end(), rank_less);
+}
+
+}  // namespace nnv
+
+using namespace nnv;
+
+extern "C" {
+
+const char* nnv_last_error(void) { return g_err; }
+int32_t nnv_version(void) { return 100; }
+
+nnv_status_t nnv_plan_create(const nnv_layer_desc_t* layers, int32_t n, const nnv_plan_opts_t* opts,
+                             nnv_plan_t** out) {
+    NNV_REQUIRE(layers && out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(n > 0 && n <= 4096, NNV_ERR_INVALID_ARG, "layer count %d out of range", n);
+    nnv_plan* p = new (std::nothrow) nnv_plan();
+    NNV_REQUIRE(p, NNV_ERR_STATE, "out of host memory");
+    p->layers.assign(layers, layers + n);
+    p->geom.resize(n);
+    p->opts = nnv_plan_opts_t{NNV_MATH_TF32, 1, 4, 0};
+    if (opts) {
+        p->opts = *opts;
+        if (p->opts.max_depth <= 0) p->opts.max_depth = 4;
+    }
+    nnv_status_t st = NNV_OK;
+    for (int i = 0; i < n && st == NNV_OK; ++i) {
+        const nnv_layer_desc_t& L = p->layers[i];
+        LayerGeom& g = p->geom[i];
+        auto bad = [&](const char* what) { st = fail(NNV_ERR_INVALID_ARG, "layer %d: %s", i, what); };
+        if (L.op < NNV_OP_CONV || L.op > NNV_OP_GAVGPOOL) { bad("unknown op"); break; }
+        if (L.C <= 0 || L.K <= 0 || L.H <= 0 || L.W <= 0 || L.R <= 0 || L.S <= 0 || L.stride <= 0 || L.pad < 0 ||
+            L.groups <= 0) { bad("non-positive dimension"); break; }
+        if ((int64_t)L.C * L.H * L.W > (1ll << 30)) { bad("activation too large"); break; }
+        if (L.in0 < -1 || L.in0 >= i || L.in1 < -1 || L.in1 >= i) { bad("producer index must be -1 or an earlier layer"); break; }
+        if (L.act < 0 || L.act > 2) { bad("unknown activation"); break; }
+        if (L.op == NNV_OP_GAVGPOOL) {
+            g.OH = g.OW = 1;
+        } else {
+            if (L.H + 2 * L.pad < L.R || L.W + 2 * L.pad < L.S) { bad("window larger than padded input"); break; }
+            g.OH = (L.H + 2 * L.pad - L.R) / L.stride + 1;
+            g.OW = (L.W + 2 * L.pad - L.S) / L.stride + 1;
+        }
+        g.P = g.OH * g.OW;
+        if (L.op != NNV_OP_CONV) {
+            if (L.K != L.C) { bad("pool layers keep the channel count"); break; }
+            if (L.op == NNV_OP_MAXPOOL && L.pad >= L.R) { bad("max-pool padding must be smaller than its window"); break; }
+            g.Cg = L.C; g.Q = g.Qp = 0; g.Cp = L.C;
+        } else {
+            if (L.C % L.groups || L.K % L.groups) { bad("channels not divisible by groups"); break; }
+            if ((L.w_off & 255) || (L.has_bias && (L.b_off & 255))) { bad("weight / bias offsets must be 256-byte aligned"); break; }
+            g.Cg = L.C / L.groups;
+            g.Q = L.R * L.S * g.Cg;
+            g.Qp = (g.Q + 7) / 8 * 8;
+            g.Cp = (L.C + 7) / 8 * 8;
+            bool any = false;
+            for (int v = 0; v < NNV_NUM_VARIANTS; ++v) any = any || is_eligible(L, v);
+            if (!any) { st = fail(NNV_ERR_UNSUPPORTED, "layer %d: no kernel variant supports this grouping", i); break; }
+        }
+        // shape agreement with the producers
+        const int src = L.in0;
+        if (src >= 0) {
+            const nnv_layer_desc_t& S = p->layers[src];
+            if (S.K != L.C || p->geom[src].OH != L.H || p->geom[src].OW != L.W) { bad("input shape differs from its producer's output"); break; }
+        } else if (i != 0 && (L.C != p->layers[0].C || L.H != p->layers[0].H || L.W != p->layers[0].W)) {
+            bad("layers reading the model input must share its shape"); break;
+        }
+        if (L.in1 >= 0) {
+            const nnv_layer_desc_t& A = p->layers[L.in1];
+            if (L.op != NNV_OP_CONV || A.K != L.K || p->geom[L.in1].OH != g.OH || p->geom[L.in1].OW != g.OW) { bad("residual addend shape differs from the output"); break; }
+        }
+    }
+    if (st == NNV_OK && p->layers[0].in0 != -1) st = fail(NNV_ERR_INVALID_ARG, "layer 0 must read the model input");
+    if (st != NNV_OK) { delete p; return st; }
+    *out = p;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_plan_destroy(nnv_plan_t* p) {
+    if (!p) return NNV_OK;
+    for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : p->tev) cudaEventDestroy(e);
+    delete p;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_eligible(const nnv_plan_t* p, int32_t layer, int32_t* out, int32_t cap, int32_t* n_out) {
+    NNV_REQUIRE(p && out && n_out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(layer >= 0 && layer < (int)p->layers.size(), NNV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    int cnt = 0;
+    for (int v = 0; v < NNV_NUM_VARIANTS; ++v) {
+        if (!is_eligible(p->layers[layer], v)) continue;
+        NNV_REQUIRE(cnt < cap, NNV_ERR_INVALID_ARG, "output capacity %d too small", cap);
+        out[cnt++] = v;
+    }
+    *n_out = cnt;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_transformed_bytes(const nnv_plan_t* p, int32_t layer, int32_t v, int32_t math, uint64_t* bytes) {
+    NNV_REQUIRE(p && bytes, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_TRY(check_choice(*p, layer, v, math));
+    *bytes = transformed_bytes(*p, layer, v, math);
+    return NNV_OK;
+}
+
+nnv_status_t nnv_exec_workspace_bytes(const nnv_plan_t* p, int32_t layer, int32_t v, int32_t math, uint64_t* bytes) {
+    NNV_REQUIRE(p && bytes, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_TRY(check_choice(*p, layer, v, math));
+    *bytes = exec_ws_bytes(*p, layer, v, math);
+    return NNV_OK;
+}
+
+nnv_status_t nnv_arena_bytes(const nnv_plan_t* p, const nnv_choice_t* choices, int32_t depth, uint64_t* bytes) {
+    NNV_REQUIRE(p && choices && bytes, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    ArenaLayout a;
+    NNV_TRY(layout_arena(*p, choices, depth, &a));
+    *bytes = a.total;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_cached_layout(const nnv_plan_t* p, const nnv_choice_t* choices, uint64_t* offsets, uint64_t* total) {
+    NNV_REQUIRE(p && choices && offsets && total, NNV_ERR_INVALID_ARG, "null argument");
+    uint64_t pos = 0;
+    for (int i = 0; i < (int)p->layers.size(); ++i) {
+        offsets[i] = 0;
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        NNV_TRY(check_choice(*p, i, choices[i].variant, choices[i].math));
+        if (!choices[i].cached) continue;
+        NNV_REQUIRE(variant_has_transform(choices[i].variant), NNV_ERR_INVALID_ARG,
+                    "layer %d: variant %d has no transform to cache", i, choices[i].variant);
+        offsets[i] = pos;
+        pos += align_up(transformed_bytes(*p, i, choices[i].variant, choices[i].math), 256);
+    }
+    *total = pos;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_filter_candidates(const nnv_plan_t* p, int32_t layer, const nnv_cost_t* costs, int32_t n_costs,
+                                   int32_t allow_cached, nnv_choice_t* out, int32_t cap, int32_t* n_out) {
+    NNV_REQUIRE(p && costs && out && n_out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(layer >= 0 && layer < (int)p->layers.size() && p->layers[layer].op == NNV_OP_CONV,
+                NNV_ERR_INVALID_ARG, "layer %d is not a convolution layer", layer);
+    std::vector<Option> opts, surv;
+    NNV_TRY(gather_options(*p, layer, costs, n_costs, allow_cached, &opts));
+    pareto(opts, &surv);
+    NNV_REQUIRE((int)surv.size() <= cap, NNV_ERR_INVALID_ARG, "output capacity %d too small", cap);
+    for (size_t i = 0; i < surv.size(); ++i) out[i] = nnv_choice_t{surv[i].variant, surv[i].math, surv[i].cached};
+    *n_out = (int)surv.size();
+    return NNV_OK;
+}
+
+nnv_status_t nnv_select_kernels(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                                nnv_choice_t* out) {
+    NNV_REQUIRE(p && costs && out, NNV_ERR_INVALID_ARG, "null argument");
+    for (int i = 0; i < (int)p->layers.size(); ++i) {
+        out[i] = nnv_choice_t{-1, -1, 0};
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        std::vector<Option> opts, surv;
+        NNV_TRY(gather_options(*p, i, costs, n_costs, allow_cached, &opts));
+        NNV_REQUIRE(!opts.empty(), NNV_ERR_STATE, "no cost rows for conv layer %d", i);
+        pareto(opts, &surv);
+        const Option* best = nullptr;
+        for (const Option& o : surv)                        // surv is in rank order: first minimum wins ties
+            if (!best || o.prep + o.exec < best->prep + best->exec) best = &o;
+        out[i] = nnv_choice_t{best->variant, best->math, best->cached};
+    }
+    return NNV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,134 @@
+"""Thin PyTorch harness around the C ABI: owns device memory, pinned host blobs and streams.
+
+PyTorch is used for allocation and stream handles only; every step of the path
+runs inside libnnv.so.
+"""
+import numpy as np
+import torch
+
+from . import binding as nb
+
+
+def _pinned_bytes(arr_u8):
+    t = torch.empty(max(1, arr_u8.size), dtype=torch.uint8).pin_memory()
+    if arr_u8.size:
+        t[:arr_u8.size].copy_(torch.from_numpy(arr_u8))
+    return t
+
+
+def dev_bytes(nbytes, fill=0xFF):
+    """256-byte aligned device buffer (torch's allocator returns >= 512-byte alignment), poisoned."""
+    t = torch.empty(max(256, int(nbytes)), dtype=torch.uint8, device="cuda")
+    assert t.data_ptr() % 256 == 0
+    if fill is not None:
+        t.fill_(fill)
+    return t
+
+
+class Model:
+    """A plan plus its host-side weight blob, ready for cold runs."""
+
+    def __init__(self, layers, blob_u8, w_off, b_off, max_depth=4):
+        self.layers = layers
+        self.plan = nb.Plan(layers, w_off, b_off, opts=dict(default_math=nb.MATH_TF32, allow_cached=1,
+                                                            max_depth=max_depth, debug_checks=0))
+        self.h_weights = _pinned_bytes(np.ascontiguousarray(blob_u8))
+        self.w_bytes = int(blob_u8.size)
+        self.w_off, self.b_off = list(w_off), list(b_off)
+        self.streams = [torch.cuda.Stream() for _ in range(3)]
+        L0, Ln = layers[0], layers[-1]
+        self.h_input = torch.empty((1, L0["C"], L0["H"], L0["W"]), dtype=torch.float32).pin_memory()
+        oh, ow = self.out_hw(len(layers) - 1)
+        self.h_output = torch.empty((1, Ln["K"], oh, ow), dtype=torch.float32).pin_memory()
+        self.arena = None
+        self.h_cached = None
+        self.c_bytes = 0
+
+    def out_hw(self, i):
+        L = self.layers[i]
+        if L["op"] == nb.OP_GAVGPOOL:
+            return 1, 1
+        return ((L["H"] + 2 * L["pad"] - L["R"]) // L["stride"] + 1,
+                (L["W"] + 2 * L["pad"] - L["S"]) // L["stride"] + 1)
+
+    def default_choices(self, prefer=None, math=nb.MATH_TF32):
+        """First eligible variant per conv layer, or the first of `prefer` that is eligible."""
+        out = []
+        for i, L in enumerate(self.layers):
+            if L["op"] != nb.OP_CONV:
+                out.append(None)
+                continue
+            el = nb.nnv_eligible(self.plan, i)
+            v = None
+            for cand in (prefer or []):
+                if cand in el:
+                    v = cand
+                    break
+            if v is None:
+                v = nb.VAR_DEPTHWISE if nb.VAR_DEPTHWISE in el else el[0]
+            m = nb.MATH_FP32 if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else math
+            out.append((v, m, 0))
+        return out
+
+    def ensure_arena(self, choices, depth):
+        need = nb.nnv_arena_bytes(self.plan, choices, depth)
+        if self.arena is None or self.arena.numel() < need:
+            self.arena = dev_bytes(need)
+        return need
+
+    def build_cached_blob(self, choices):
+        """Transform the weights of every layer chosen with cached=1 on the device and keep the
+        result in pinned host memory, laid out as nnv_cached_layout() says."""
+        offs, total = nb.nnv_cached_layout(self.plan, choices)
+        host = torch.zeros(max(1, total), dtype=torch.uint8).pin_memory()
+        for i, c in enumerate(choices):
+            if c is None or not c[2]:
+                continue
+            L = self.layers[i]
+            rbytes = 4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"]
+            raw = dev_bytes(rbytes)
+            raw[:rbytes].copy_(self.h_weights[self.w_off[i]:self.w_off[i] + rbytes])
+            tb = nb.nnv_transformed_bytes(self.plan, i, c[0], c[1])
+            out = dev_bytes(tb)
+            nb.nnv_transform_weights(self.plan, i, c[0], c[1], raw, out, torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            host[offs[i]:offs[i] + tb].copy_(out[:tb])
+        self.h_cached, self.c_bytes = host, total
+        return offs, total
+
+    def cold_run(self, x_nchw, choices, depth=2, want_timings=False, poison=True):
+        """One cold inference through nnv_cold_run; returns (output NCHW numpy, timings)."""
+        self.h_input.copy_(torch.from_numpy(np.ascontiguousarray(x_nchw, dtype=np.float32)).reshape(self.h_input.shape))
+        need = self.ensure_arena(choices, depth)
+        if poison:
+            self.arena.fill_(0xFF)
+            torch.cuda.synchronize()
+        tm = nb.nnv_cold_run(self.plan, choices, self.h_weights, self.w_bytes, self.h_cached, self.c_bytes,
+                             self.h_input, self.h_output, self.arena, need,
+                             self.streams[0], self.streams[1], self.streams[2], depth, want_timings)
+        return self.h_output.numpy().copy(), tm
+
+    def layer_output(self, i):
+        """NCHW numpy copy of layer i's activation left in the arena by the last cold run."""
+        ptr, nbytes = nb.nnv_layer_output(self.plan, i)
+        off = ptr - self.arena.data_ptr()
+        L = self.layers[i]
+        oh, ow = self.out_hw(i)
+        t = self.arena[off:off + nbytes].view(torch.float32).reshape(oh, ow, L["K"])
+        return t.permute(2, 0, 1).contiguous().cpu().numpy()
+
+    def profile(self, x_nchw, reps=5):
+        self.h_input.copy_(torch.from_numpy(np.ascontiguousarray(x_nchw, dtype=np.float32)).reshape(self.h_input.shape))
+        need = nb.nnv_profile_arena_bytes(self.plan)
+        arena = dev_bytes(need, fill=None)
+        costs = nb.nnv_profile(self.plan, self.h_weights, self.w_bytes, self.h_input, arena, need,
+                               torch.cuda.current_stream(), reps)
+        del arena
+        return costs
+
+
+def model_from_workload(layers, weights, biases, blob_fn, max_depth=4):
+    """Build a Model from a layer list and per-layer numpy weights using `blob_fn`
+    (workloads.weight_blob) to lay out the host blob."""
+    blob, w_off, b_off = blob_fn(layers, weights, biases)
+    return Model(layers, blob, w_off, b_off, max_depth=max_depth)

@@ -1,0 +1,134 @@
+"""GPU parity: whole-model cold runs (host weights -> H2D -> transform -> exec, three streams),
+pipeline-depth invariance, the cached bypass, and profiling + selection."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from oracle import model as omodel
+from oracle import selection as osel
+from paper_2206_07446_b200 import binding as nb
+from paper_2206_07446_b200 import harness
+from gpu_util import rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def _model(layers, seed=0):
+    ws, bs = wl.make_weights(layers, seed=seed)
+    x = wl.make_input(layers, seed=seed)
+    return harness.model_from_workload(layers, ws, bs, wl.weight_blob), ws, bs, x
+
+
+def _choices(model, prefer, math):
+    return model.default_choices(prefer=prefer, math=math)
+
+
+@pytest.mark.parametrize("prefer,math,tol", [
+    ([nb.VAR_DIRECT], nb.MATH_FP32, 1e-5),
+    ([nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32, 2e-3),
+    ([nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32, 2e-3),
+    ([nb.VAR_WINO_F2, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_BF16, 2e-2),
+])
+def test_tiny_net_cold_run_matches_oracle(prefer, math, tol):
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=2)
+    acts = omodel.run_model(layers, ws, bs, x)
+    ch = _choices(model, prefer, math)
+    y, _ = model.cold_run(x, ch, depth=2)
+    assert np.all(np.isfinite(y))
+    # end-to-end error accumulates over layers: twice the per-layer tolerance
+    assert rel_l2(y[0], acts[-1]) <= tol
+    for i in range(len(layers)):
+        assert rel_l2(model.layer_output(i), acts[i]) <= tol, i
+
+
+def test_cfg1_cold_run_each_variant():
+    layers = wl.cfg1()
+    model, ws, bs, x = _model(layers)
+    ref = omodel.run_model(layers, ws, bs, x)[-1]
+    for v, m, tol in [(nb.VAR_DIRECT, 0, 1e-5), (nb.VAR_IM2COL, 1, 1e-3), (nb.VAR_WINO_F2, 1, 1e-3),
+                      (nb.VAR_IM2COL, 2, 1e-2), (nb.VAR_WINO_F2, 2, 1e-2)]:
+        y, tm = model.cold_run(x, [(v, m, 0)], depth=1, want_timings=True)
+        assert rel_l2(y[0], ref) <= tol, (v, m)
+        assert tm[0]["h2d_bytes"] == 64 * 64 * 9 * 4
+        assert tm[0]["choice"] == (v, m, 0)
+
+
+def test_resnet18_cold_run_pipeline_depths_bitwise_equal_and_ordered():
+    """Config 2 end to end; the pipelined result is bitwise the serial one for depth 1..4, and the
+    recorded stamps obey the dependency constraints (no operation starts before its precursors end)."""
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers)
+    acts = omodel.run_model(layers, ws, bs, x)
+    ch = _choices(model, [nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    outs = []
+    for depth in (1, 2, 3, 4):
+        y, tm = model.cold_run(x, ch, depth=depth, want_timings=True)
+        outs.append(y.copy())
+        conv = [i for i, L in enumerate(layers) if L["op"] == wl.OP_CONV]
+        slack = 2000      # event stamps have 0.5 us resolution; allow 2 us
+        for j, i in enumerate(conv):
+            t = tm[i]
+            assert t["h2d_end_ns"] >= t["h2d_start_ns"] and t["exec_end_ns"] >= t["exec_start_ns"]
+            if t["xform_bytes"]:
+                assert t["xform_start_ns"] + slack >= t["h2d_end_ns"]
+                assert t["exec_start_ns"] + slack >= t["xform_end_ns"]
+            else:
+                assert t["exec_start_ns"] + slack >= t["h2d_end_ns"]
+            for src in (layers[i]["in0"], layers[i]["in1"]):
+                if src >= 0:
+                    assert t["exec_start_ns"] + slack >= tm[src]["exec_end_ns"]
+            if j >= depth:
+                assert t["h2d_start_ns"] + slack >= tm[conv[j - depth]]["exec_end_ns"]
+    for y in outs[1:]:
+        assert np.array_equal(y.view(np.uint32), outs[0].view(np.uint32))
+    assert rel_l2(outs[0][0], acts[-1]) <= 5e-3          # 20 TF32 layers chained
+
+
+def test_cached_bypass_gives_identical_result():
+    """Reading cached post-transform weights and skipping the transform changes nothing in the output."""
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=4)
+    ch = _choices(model, [nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    y_raw, _ = model.cold_run(x, ch, depth=2)
+    ch_c = [None if c is None else (c[0], c[1], 1 if c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else 0) for c in ch]
+    model.build_cached_blob(ch_c)
+    y_c, tm = model.cold_run(x, ch_c, depth=2, want_timings=True)
+    assert np.array_equal(y_raw.view(np.uint32), y_c.view(np.uint32))
+    for i, c in enumerate(ch_c):
+        if c is not None and c[2]:
+            assert tm[i]["xform_bytes"] == 0
+            assert tm[i]["h2d_bytes"] >= nb.nnv_transformed_bytes(model.plan, i, c[0], c[1])
+
+
+def test_profile_then_select_matches_oracle_selection():
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=5)
+    costs = model.profile(x, reps=3)
+    n_expected = sum(len(osel.math_modes(v)) for L in layers if L["op"] == 0 for v in osel.eligible(L))
+    assert len(costs) == n_expected
+    assert all(c["exec_ns"] > 0 and c["h2d_raw_ns"] > 0 for c in costs)
+    for allow in (0, 1):
+        got = nb.nnv_select_kernels(model.plan, costs, allow)
+        assert got == osel.select_kernels(layers, costs, allow)
+    # the selected plan runs and matches the oracle
+    ch = nb.nnv_select_kernels(model.plan, costs, 0)
+    acts = omodel.run_model(layers, ws, bs, x)
+    y, _ = model.cold_run(x, ch, depth=2)
+    assert rel_l2(y[0], acts[-1]) <= 2e-2
+
+
+def test_arena_too_small_and_bad_depth():
+    layers = wl.cfg1()
+    model, ws, bs, x = _model(layers)
+    ch = [(nb.VAR_IM2COL, 1, 0)]
+    need = model.ensure_arena(ch, 1)
+    with pytest.raises(nb.NnvError) as e:
+        nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
+                        model.arena, need - 1024, model.streams[0], model.streams[1], model.streams[2], 1)
+    assert e.value.status == 4
+    with pytest.raises(nb.NnvError) as e:
+        nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
+                        model.arena, need, model.streams[0], model.streams[1], model.streams[2], 0)
+    assert e.value.status == 1

@@ -1,0 +1,136 @@
+"""GPU parity: execution of one layer with every kernel variant against the fp64 direct-convolution
+oracle, through the C ABI, with oracle-fed inputs."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from oracle import conv as oconv
+from oracle import model as omodel
+from paper_2206_07446_b200 import binding as nb
+from gpu_util import TOL, dev, poisoned, chw_to_hwc, hwc_to_chw, rel_l2, run_conv
+
+pytestmark = pytest.mark.gpu
+
+
+def _maths(v):
+    if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE):
+        return [nb.MATH_FP32]
+    if v in (nb.VAR_WINO_F4, nb.VAR_WINO_F6):
+        return [nb.MATH_TF32]
+    return [nb.MATH_TF32, nb.MATH_BF16]
+
+
+def _check_layer(layers, i, x, w, b, add, variants=None):
+    L = layers[i]
+    plan = nb.Plan(layers, [0] * len(layers), [0] * len(layers))
+    ref = omodel.run_layer(L, x, w, b, add)
+    seen = []
+    for v in nb.nnv_eligible(plan, i):
+        if variants is not None and v not in variants:
+            continue
+        for m in _maths(v):
+            y = run_conv(plan, i, L, v, m, x, w, b, add)
+            assert y.shape == ref.shape
+            assert np.all(np.isfinite(y)), (nb.VARIANT_NAMES[v], nb.MATH_NAMES[m])
+            err = rel_l2(y, ref)
+            seen.append((nb.VARIANT_NAMES[v], nb.MATH_NAMES[m], err))
+            assert err <= TOL[m], (nb.VARIANT_NAMES[v], nb.MATH_NAMES[m], err)
+    return seen
+
+
+def test_cfg1_all_variants():
+    """Config 1: 3x3 s1 p1, 64->64, 56x56: direct, im2col, Winograd F(2,3)/F(4,3)/F(6,3)."""
+    layers = wl.cfg1()
+    ws, bs = wl.make_weights(layers)
+    x = wl.make_input(layers)[0]
+    seen = _check_layer(layers, 0, x, ws[0], None, None)
+    assert len(seen) == 1 + 2 + 4
+    print(seen)
+
+
+def test_tiny_net_every_layer_every_variant():
+    """Ragged shapes (C=5, 9x7 grid, K=12/20/9), residual, bias, ReLU6, strides, depthwise; oracle-fed inputs."""
+    layers = wl.tiny_net()
+    ws, bs = wl.make_weights(layers, seed=3)
+    x = wl.make_input(layers, seed=3)
+    acts = omodel.run_model(layers, ws, bs, x)
+    plan = nb.Plan(layers, [0] * len(layers), [0] * len(layers))
+    for i, L in enumerate(layers):
+        src = x[0] if L["in0"] < 0 else acts[L["in0"]].astype(np.float32)
+        if L["op"] == wl.OP_CONV:
+            add = None if L["in1"] < 0 else acts[L["in1"]].astype(np.float32)
+            _check_layer(layers, i, src, ws[i], bs[i], add)
+        else:
+            oh, ow = wl.out_hw(L)
+            d_out = poisoned(4 * oh * ow * L["K"])
+            nb.nnv_pool_exec(plan, i, dev(chw_to_hwc(src)), d_out, torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            y = hwc_to_chw(d_out[:4 * oh * ow * L["K"]].view(torch.float32).reshape(oh, ow, L["K"]).cpu().numpy())
+            ref = omodel.run_layer(L, src)
+            tol = 0.0 if L["op"] == wl.OP_MAXPOOL else 1e-6
+            assert np.max(np.abs(y - ref)) <= tol * max(1.0, np.max(np.abs(ref)))
+
+
+@pytest.mark.parametrize("shape", [
+    # C, K, R, stride, H, W, groups
+    (3, 64, 7, 2, 224, 224, 1),        # ResNet stem
+    (512, 512, 3, 1, 7, 7, 1),         # ResNet-18 last stage (tiny grid, large K reduction)
+    (64, 128, 1, 2, 56, 56, 1),        # strided 1x1 downsample
+    (256, 256, 3, 2, 28, 28, 1),       # strided 3x3
+    (16, 96, 1, 1, 112, 112, 1),       # MobileNetV2 expand, narrow C
+    (96, 24, 1, 1, 56, 56, 1),         # project to K=24 (not a multiple of 16)
+    (320, 1280, 1, 1, 7, 7, 1),        # wide 1x1 on a tiny grid
+    (144, 144, 3, 2, 56, 56, 144),     # depthwise stride 2
+    (384, 384, 3, 1, 14, 14, 384),     # depthwise stride 1
+    (512, 2048, 1, 1, 7, 7, 1),        # ResNet-50 last 1x1
+    (128, 128, 3, 1, 28, 28, 1),       # Winograd edge tiles: 28 = 4*7 = 6*4+4
+    (256, 256, 3, 1, 14, 14, 1),       # 14 = 4*3+2 = 6*2+2
+    (3, 64, 3, 1, 224, 224, 1),        # VGG conv1_1 (C=3 padded to 8 in the Winograd domain)
+    (64, 64, 3, 1, 112, 112, 1),       # large-grid VGG-like layer (scaled down from 224 for oracle time)
+])
+def test_config_layer_shapes(shape):
+    C, K, R, stride, H, W, groups = shape
+    pad = R // 2
+    L = dict(op=0, C=C, K=K, R=R, S=R, stride=stride, pad=pad, groups=groups, H=H, W=W, in0=-1, in1=-1, act=1, has_bias=0)
+    rng = np.random.default_rng(list(shape))
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    cg = C // groups
+    w = (rng.standard_normal((K, cg, R, R)) * np.sqrt(2.0 / (cg * R * R))).astype(np.float32)
+    seen = _check_layer([L], 0, x, w, None, None)
+    print(shape, seen)
+
+
+def test_residual_and_bias_epilogues_on_every_variant():
+    """bias + addend + ReLU6 through each kernel's epilogue (K = 40 is not a multiple of 16)."""
+    base = dict(op=0, C=24, K=40, R=3, S=3, stride=1, pad=1, groups=1, H=13, W=11, in0=-1, in1=-1, act=0, has_bias=0)
+    layers = [base, dict(base, C=40, in0=0, in1=0, act=2, has_bias=1)]
+    rng = np.random.default_rng(5)
+    x = rng.uniform(-1, 1, (40, 13, 11)).astype(np.float32)
+    w = (rng.standard_normal((40, 40, 3, 3)) * 0.05).astype(np.float32)
+    b = rng.uniform(-1, 1, 40).astype(np.float32)
+    add = rng.uniform(-3, 3, (40, 13, 11)).astype(np.float32)
+    seen = _check_layer(layers, 1, x, w, b, add)
+    assert len(seen) == 7
+
+
+def test_layout_helpers_roundtrip():
+    rng = np.random.default_rng(6)
+    x = rng.uniform(-1, 1, (5, 7, 9)).astype(np.float32)
+    d_in = dev(x)
+    d_hwc = poisoned(x.nbytes)
+    d_back = poisoned(x.nbytes)
+    nb.nnv_chw_to_hwc(d_in, d_hwc, 5, 7, 9, torch.cuda.current_stream())
+    nb.nnv_hwc_to_chw(d_hwc, d_back, 5, 7, 9, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    assert np.array_equal(d_hwc[:x.nbytes].view(torch.float32).reshape(7, 9, 5).cpu().numpy(), chw_to_hwc(x))
+    assert np.array_equal(d_back[:x.nbytes].view(torch.float32).reshape(5, 7, 9).cpu().numpy(), x)
+
+
+def test_workspace_too_small_is_reported():
+    layers = wl.cfg1()
+    plan = nb.Plan(layers, [0], [0])
+    buf = poisoned(1 << 20)
+    with pytest.raises(nb.NnvError) as e:
+        nb.nnv_conv_exec(plan, 0, nb.VAR_IM2COL, nb.MATH_TF32, buf, None, buf, None, buf, buf, 1024, torch.cuda.current_stream())
+    assert e.value.status == 4

@@ -25,7 +25,7 @@ def test_pack_is_a_bijection_with_zero_padding(C, K, R):
     bits = P.view(np.uint32)
     for o in range(K * Qp):
         if o in offs:
-            assert P[o] == w[offs[o]]
+            assert P[o] == op.tf32_round_rne(w)[offs[o]]
         else:
             assert bits[o] == 0                      # +0.0 exactly
     assert len(offs) == K * C * R * S
@@ -37,6 +37,22 @@ def test_pack_order_channel_innermost_then_taps():
     P = op.pack_weights(w)
     assert P.shape == (2, 32)
     assert P[1, (0 * 3 + 1) * 3 + 2] == 5.0 and np.count_nonzero(P) == 1
+
+
+def test_tf32_rne_hand_patterns():
+    """TF32 keeps 10 explicit mantissa bits: spacing 2^-10 in [1,2)."""
+    f = lambda v: float(op.tf32_round_rne(np.array([v], np.float32))[0])
+    assert f(1.0) == 1.0 and f(-3.5) == -3.5 and f(0.0) == 0.0
+    assert f(1.0 + 2.0 ** -11) == 1.0                       # exact tie -> even (down)
+    assert f(1.0 + 3 * 2.0 ** -11) == 1.0 + 2.0 ** -9       # exact tie -> even (up)
+    assert f(1.0 + 2.0 ** -11 + 2.0 ** -22) == 1.0 + 2.0 ** -10
+    assert f(2049.0) == 2048.0 and f(2051.0) == 2052.0
+    rng = np.random.default_rng(12)
+    a = rng.standard_normal(10000).astype(np.float32)
+    r = op.tf32_round_rne(a)
+    assert np.all(r.view(np.uint32) & 0x1FFF == 0)
+    assert np.max(np.abs(r - a) / np.abs(a)) <= 2.0 ** -11
+    assert np.array_equal(op.tf32_round_rne(r), r)          # idempotent
 
 
 def test_bf16_rne_hand_patterns():
