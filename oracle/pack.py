@@ -45,11 +45,8 @@ def bf16_to_f32(bits16):
     return (np.asarray(bits16, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
-def pack_weights(w, bf16=False):
-    """Naive repack (loops over c, r, s; numpy over k) of w (K,C,R,S) fp32.
-
-    Returns a (K, Qp) array: fp32 words rounded to TF32 precision, or uint16 bf16 bits.
-    """
+def permute_weights(w):
+    """The pure re-ordering (loops over c, r, s; numpy over k): (K,C,R,S) fp32 -> (K,Qp) fp32, pad +0."""
     w = np.ascontiguousarray(w, dtype=np.float32)
     K, C, R, S = w.shape
     Qp = padded_q(C, R, S)
@@ -59,7 +56,12 @@ def pack_weights(w, bf16=False):
         for r in range(R):
             for s in range(S):
                 flat[rows + pack_offset(0, c, r, s, C, R, S)] = w[:, c, r, s]
-    P = flat.reshape(K, Qp)
+    return flat.reshape(K, Qp)
+
+
+def pack_weights(w, bf16=False):
+    """Repack then round: returns (K, Qp) fp32 words of TF32 precision, or uint16 bf16 bits."""
+    P = permute_weights(w)
     if bf16:
         return bf16_bits_rne(P)
     return tf32_round_rne(P)

@@ -81,7 +81,8 @@ def test_bf16_rne_vs_library_conversion():
     assert np.max(np.abs(back - a) / np.abs(a)) <= 2.0 ** -8
 
 
-def test_pack_bf16_is_rounding_of_pack_fp32():
+def test_pack_rounding_is_applied_to_the_permuted_raw_weights():
     rng = np.random.default_rng(10)
     w = rng.standard_normal((5, 3, 3, 3)).astype(np.float32)
-    assert np.array_equal(op.pack_weights(w, bf16=True), op.bf16_bits_rne(op.pack_weights(w)))
+    assert np.array_equal(op.pack_weights(w, bf16=True), op.bf16_bits_rne(op.permute_weights(w)))
+    assert np.array_equal(op.pack_weights(w), op.tf32_round_rne(op.permute_weights(w)))

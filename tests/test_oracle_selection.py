@@ -89,8 +89,8 @@ def test_select_kernels_over_layers():
               dict(op=1, C=8, K=8, R=2, S=2, stride=2, pad=0, groups=1),
               dict(op=0, C=8, K=8, R=3, S=3, stride=1, pad=1, groups=8)]
     costs = [dict(layer=0, variant=sel.DIRECT, math=sel.FP32, h2d_raw_ns=10, xform_ns=0, h2d_cached_ns=10, exec_ns=100),
-             dict(layer=0, variant=sel.WINO_F4, math=sel.TF32, h2d_raw_ns=10, xform_ns=80, h2d_cached_ns=40, exec_ns=30),
-             dict(layer=0, variant=sel.WINO_F4, math=sel.BF16, h2d_raw_ns=10, xform_ns=80, h2d_cached_ns=20, exec_ns=50),
+             dict(layer=0, variant=sel.WINO_F2, math=sel.TF32, h2d_raw_ns=10, xform_ns=80, h2d_cached_ns=40, exec_ns=30),
+             dict(layer=0, variant=sel.WINO_F2, math=sel.BF16, h2d_raw_ns=10, xform_ns=80, h2d_cached_ns=20, exec_ns=50),
              dict(layer=2, variant=sel.DEPTHWISE, math=sel.FP32, h2d_raw_ns=1, xform_ns=0, h2d_cached_ns=1, exec_ns=5)]
-    assert sel.select_kernels(layers, costs, True) == [(sel.WINO_F4, sel.TF32, 1), None, (sel.DEPTHWISE, sel.FP32, 0)]
+    assert sel.select_kernels(layers, costs, True) == [(sel.WINO_F2, sel.TF32, 1), None, (sel.DEPTHWISE, sel.FP32, 0)]
     assert sel.select_kernels(layers, costs, False) == [(sel.DIRECT, sel.FP32, 0), None, (sel.DEPTHWISE, sel.FP32, 0)]
