@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the cold-start convolution path on B200.
+
+One step = one cold inference of the workload at batch 1: per-layer kernel selection on the
+profiled cost table, then for every conv layer the weights are read (host -> HBM), transformed
+(Winograd filter transform or GEMM repack) and the layer is executed, pipelined over streams.
+
+  value   cold ms with weights and input already resident in HBM (transform + exec only)
+  e2e     cold ms through nnv_cold_run with pinned HOST weights / input / output (H2D, D2H inside)
+
+Run `python bench.py` (1 GPU) or under torch.distributed.run with --gpus N (independent replicas,
+the path does not shard).  `--impl reference` times the CPU oracle instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "cold_inference_ms_batch1"
+UNIT = "ms"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2_resnet18", choices=list(wl.CONFIGS))
+    ap.add_argument("--depth", type=int, default=3)
+    ap.add_argument("--math", default="tf32", choices=["tf32", "bf16"])
+    ap.add_argument("--cpu-passes", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+def oracle_pass(layers, ws, bs, x):
+    """One whole cold pass of the oracle: literal filter transform / naive pack per layer, then the
+    fp64 direct-convolution chain.  Returns seconds."""
+    from oracle import model as omodel
+    from oracle import pack as opack
+    from oracle import winograd as owin
+    t0 = time.perf_counter()
+    for i, L in enumerate(layers):
+        if L["op"] != wl.OP_CONV or L["groups"] != 1:
+            continue
+        if L["R"] == 3 and L["S"] == 3 and L["stride"] == 1:
+            owin.filter_transform(ws[i], 4)
+        else:
+            opack.pack_weights(ws[i])
+    omodel.run_model(layers, ws, bs, x)
+    return time.perf_counter() - t0
+
+
+def cpu_threads():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import conv as oconv
+    oconv.build()
+    os.environ.setdefault("OMP_NUM_THREADS", str(cpu_threads()))
+    layers = wl.CONFIGS[args.config]()
+    ws, bs = wl.make_weights(layers)
+    x = wl.make_input(layers)
+    for _ in range(min(args.warmup, 2)):
+        oracle_pass(layers, ws, bs, x)
+    ts = [oracle_pass(layers, ws, bs, x) for _ in range(args.steps)]
+    ms = 1e3 * sum(ts) / len(ts)
+    sample = "whole %s workload per step: F(4,3) literal filter transform / naive pack of every conv layer + fp64 direct-conv chain" % args.config
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": args.config, "batch": 1},
+        "cpu_baseline": {"value": ms, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": ms, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        f = tempfile.NamedTemporaryFile(prefix="nnv_clocks_", suffix=".csv", delete=False)
+        self.path = f.name
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+        f.close()
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        try:
+            rows = [r.strip().split(",") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except OSError:
+            rows = []
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, r[4:8]):
+                if v.strip().lower() == "active":
+                    reasons.add(nme)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def count_launches(layers, choices, plan, nb):
+    """Kernels of this library launched by one pass (layout conversion in, per-layer kernels, out)."""
+    n = 2
+    for i, L in enumerate(layers):
+        if L["op"] != wl.OP_CONV:
+            n += 1
+            continue
+        v, m, cached = choices[i]
+        if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE):
+            n += 1
+            continue
+        if not cached:
+            n += 1                                           # transform
+        if v in (nb.VAR_WINO_F2, nb.VAR_WINO_F4, nb.VAR_WINO_F6):
+            n += 3
+        else:
+            n += 1 + (1 if nb.nnv_exec_workspace_bytes(plan, i, v, m) else 0)
+    return n
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2206_07446_b200 import binding as nb
+    from paper_2206_07446_b200 import harness
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    layers = wl.CONFIGS[args.config]()
+    ws, bs = wl.make_weights(layers)
+    x = wl.make_input(layers)
+    model = harness.model_from_workload(layers, ws, bs, wl.weight_blob)
+    math = nb.MATH_BF16 if args.math == "bf16" else nb.MATH_TF32
+
+    # offline decision stage: profile every candidate kernel, select per layer by cold cost
+    costs = model.profile(x, reps=5)
+    costs = [c for c in costs if c["math"] in (nb.MATH_FP32, math) or c["variant"] in (nb.VAR_WINO_F4, nb.VAR_WINO_F6)]
+    choices_cold = nb.nnv_select_kernels(model.plan, costs, 1)
+    if any(c is not None and c[2] for c in choices_cold):
+        model.build_cached_blob(choices_cold)
+    # with the read stage removed (weights resident) h2d costs vanish: select on transform + exec only
+    costs_res = [dict(c, h2d_raw_ns=0, h2d_cached_ns=0) for c in costs]
+    choices_res = nb.nnv_select_kernels(model.plan, costs_res, 0)
+    model.to_device()
+    model.d_input.copy_(torch.from_numpy(x))
+    model.h_input.copy_(torch.from_numpy(x))
+    need_cold = model.ensure_arena(choices_cold, args.depth)
+    need_res = model.ensure_arena(choices_res, args.depth)
+    need = max(need_cold, need_res)
+    model.arena.fill_(0xFF)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    s_copy, s_xform, s_exec = model.streams
+    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step_resident(k, timed, want_timings=False):
+        flush.fill_(k & 0xFF)                                # evict L2 between steps
+        torch.cuda.synchronize()
+        ch = nb.nnv_select_kernels(model.plan, costs_res, 0)
+        if timed:
+            ev0[k].record(s_exec)
+            s_xform.wait_event(ev0[k])
+        tm = nb.nnv_resident_run(model.plan, ch, model.d_weights, model.w_bytes, model.d_cached, model.c_bytes,
+                                 model.d_input, model.d_output, model.arena, need, s_xform, s_exec, args.depth, want_timings)
+        if timed:
+            ev1[k].record(s_exec)
+        return tm
+
+    def step_cold(k, timed):
+        flush.fill_(k & 0xFF)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ch = nb.nnv_select_kernels(model.plan, costs, 1)
+        if timed:
+            ev0[k].record(s_exec)
+            s_copy.wait_event(ev0[k])
+            s_xform.wait_event(ev0[k])
+        nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes, model.h_input,
+                        model.h_output, model.arena, need, s_copy, s_xform, s_exec, args.depth)
+        if timed:
+            ev1[k].record(s_exec)
+        return time.perf_counter() - t0
+
+    def reduce_max(v):
+        if world > 1:
+            t = torch.tensor([v], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return v
+
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+
+    # ---- timed region 1: weights resident in HBM ------------------------------------------------
+    sampler.start()
+    for k in range(args.warmup):
+        step_resident(k, False)
+    barrier()
+    for k in range(args.steps):
+        step_resident(k, True)
+    barrier()
+    res_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
+    value = reduce_max(sum(res_ms) / len(res_ms))
+
+    # ---- timed region 2: end to end from pinned host memory -------------------------------------
+    for k in range(args.warmup):
+        step_cold(k, False)
+    barrier()
+    wall = [step_cold(k, True) for k in range(args.steps)]
+    barrier()
+    cold_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
+    e2e = reduce_max(sum(cold_ms) / len(cold_ms))
+    e2e_wall = reduce_max(1e3 * sum(wall) / len(wall))
+
+    # ---- per-kernel durations for the roofline (same resident steps, with per-operation events) --
+    xf = {}          # layer -> [ns]
+    ex = {}
+    for k in range(args.steps):
+        tm = step_resident(k, False, want_timings=True)
+        for i, t in enumerate(tm):
+            if t["xform_bytes"]:
+                xf.setdefault(i, []).append(t["xform_end_ns"] - t["xform_start_ns"])
+            if layers[i]["op"] == wl.OP_CONV:
+                ex.setdefault(i, []).append(t["exec_end_ns"] - t["exec_start_ns"])
+    clocks = sampler.stop()
+    last_tm = tm
+    y_gpu = model.d_output.cpu().numpy()
+
+    peaks = load_peaks()
+    # dominant memory-bound kernel: the Winograd filter transform (one launch per Winograd layer)
+    wino = [i for i in xf if choices_res[i][0] in (nb.VAR_WINO_F2, nb.VAR_WINO_F4, nb.VAR_WINO_F6)]
+    tb = sum(last_tm[i]["xform_bytes"] for i in wino)
+    tns = sum(statistics.mean(xf[i]) for i in wino)
+    roof = None
+    if wino and tns > 0:
+        ach = tb / tns                                        # bytes per ns = GB/s
+        big = max(wino, key=lambda i: last_tm[i]["xform_bytes"])
+        roof = {"kernel": "filter_transform_kernel", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "launches_per_step": len(wino), "bytes_per_step": tb, "avg_launch_us": tns / len(wino) / 1e3,
+                "largest_launch": {"layer": big, "bytes": last_tm[big]["xform_bytes"],
+                                   "us": statistics.mean(xf[big]) / 1e3,
+                                   "gbs": last_tm[big]["xform_bytes"] / statistics.mean(xf[big])}}
+    flops = sum(last_tm[i]["exec_flops"] for i in ex)
+    exec_ns = sum(statistics.mean(v) for v in ex.values())
+    xform_ns = sum(statistics.mean(v) for v in xf.values())
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": value, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "tf32" if math == nb.MATH_TF32 else "bf16", "data": "synthetic",
+        "config": {"workload": args.config, "batch": 1, "pipeline_depth": args.depth, "l2": "flushed between steps (256 MiB write)",
+                   "replicas": world, "weights_bytes": int(model.w_bytes)},
+        "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": None,
+                "d2h_bytes_per_step": int(model.h_output.numel() * 4), "host_wall_ms": e2e_wall},
+        "gpu_launches": (count_launches(layers, choices_res, model.plan, nb) + count_launches(layers, choices_cold, model.plan, nb)) * args.steps,
+        "clocks": clocks,
+        "roofline": roof,
+        "breakdown": {"sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3, "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
+                      "choices_resident": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_res],
+                      "choices_cold": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_cold]},
+    }
+    # bytes that cross the host link per cold step: weights (raw or cached) + biases + the input
+    h2d = int(x.nbytes)
+    for i, c in enumerate(choices_cold):
+        if c is None:
+            continue
+        L = layers[i]
+        h2d += nb.nnv_transformed_bytes(model.plan, i, c[0], c[1]) if c[2] else 4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"]
+        h2d += 4 * L["K"] if L["has_bias"] else 0
+    line["e2e"]["h2d_bytes_per_step"] = h2d
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import conv as oconv
+        from oracle import model as omodel
+        oconv.build()
+        os.environ.setdefault("OMP_NUM_THREADS", str(cpu_threads()))
+        oracle_pass(layers, ws, bs, x)
+        ts = [oracle_pass(layers, ws, bs, x) for _ in range(args.cpu_passes)]
+        line["cpu_baseline"] = {"value": 1e3 * sum(ts) / len(ts), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": "whole %s workload, %d passes: literal filter transform / naive pack + fp64 direct-conv chain"
+                                          % (args.config, args.cpu_passes)}
+        ref = omodel.run_model(layers, ws, bs, x)[-1]
+        den = float(np.sqrt(np.sum(ref * ref)))
+        line["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_gpu[0] - ref) ** 2)) / den)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -226,6 +226,20 @@ nnv_status_t nnv_cold_run(nnv_plan_t* plan, const nnv_choice_t* choices,
                           void* s_copy, void* s_xform, void* s_exec,
                           int32_t depth, nnv_timing_t* timings);
 
+/* The same pass with the read stage already done (the paper's Tables 1 and 2
+ * separate reading from transformation and execution; this call measures the
+ * latter two alone).  d_weights / d_cached are DEVICE copies of the two blobs
+ * (256-byte aligned), d_input / d_output are DEVICE NCHW fp32 buffers; nothing
+ * crosses the host link.  Transforms run on s_xform, layers on s_exec; the
+ * transform of conv layer j waits for the execution of conv layer j-depth. */
+nnv_status_t nnv_resident_run(nnv_plan_t* plan, const nnv_choice_t* choices,
+                              const void* d_weights, uint64_t w_bytes,
+                              const void* d_cached, uint64_t c_bytes,
+                              const float* d_input, float* d_output,
+                              void* d_arena, uint64_t arena_bytes,
+                              void* s_xform, void* s_exec,
+                              int32_t depth, nnv_timing_t* timings);
+
 /* Device address, inside the arena of the most recent nnv_cold_run on this
  * plan, of layer `layer`'s NHWC fp32 output (valid until the arena is reused). */
 nnv_status_t nnv_layer_output(const nnv_plan_t* plan, int32_t layer, const void** d_ptr, uint64_t* bytes);

@@ -78,6 +78,7 @@ _SIGS = {
     "nnv_chw_to_hwc": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_hwc_to_chw": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_cold_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing)],
+    "nnv_resident_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _i32, _P(Timing)],
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
     "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
@@ -261,7 +262,11 @@ def nnv_cold_run(plan, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, 
     _check(_lib.nnv_cold_run(plan.handle, _choices_array(plan, choices), _ptr(h_weights), int(w_bytes),
                              _ptr(h_cached), int(c_bytes), _ptr(h_input), _ptr(h_output), _ptr(d_arena),
                              int(arena_bytes), _stream(s_copy), _stream(s_xform), _stream(s_exec), int(depth), tarr))
-    if not want_timings:
+    return _timings_list(tarr)
+
+
+def _timings_list(tarr):
+    if tarr is None:
         return None
     out = []
     for t in tarr:
@@ -269,6 +274,15 @@ def nnv_cold_run(plan, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, 
         d["choice"] = (t.choice.variant, t.choice.math, t.choice.cached)
         out.append(d)
     return out
+
+
+def nnv_resident_run(plan, choices, d_weights, w_bytes, d_cached, c_bytes, d_input, d_output, d_arena, arena_bytes,
+                     s_xform, s_exec, depth, want_timings=False):
+    tarr = (Timing * plan.n)() if want_timings else None
+    _check(_lib.nnv_resident_run(plan.handle, _choices_array(plan, choices), _ptr(d_weights), int(w_bytes),
+                                 _ptr(d_cached), int(c_bytes), _ptr(d_input), _ptr(d_output), _ptr(d_arena),
+                                 int(arena_bytes), _stream(s_xform), _stream(s_exec), int(depth), tarr))
+    return _timings_list(tarr)
 
 
 def nnv_layer_output(plan, layer):

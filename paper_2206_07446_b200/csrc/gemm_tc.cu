@@ -38,6 +38,11 @@ nnv_status_t read_device_status(int32_t* code) {
     return NNV_OK;
 }
 
+nnv_status_t enqueue_status_read(int* h_pinned, cudaStream_t st) {
+    NNV_CUDA(cudaMemcpyFromSymbolAsync(h_pinned, g_device_status, sizeof(int), 0, cudaMemcpyDeviceToHost, st));
+    return NNV_OK;
+}
+
 namespace {
 
 constexpr int BM = 128;                 // rows of A per tile = TMEM lanes

@@ -62,6 +62,7 @@ struct nnv_plan {
     std::vector<cudaEvent_t> tev;         // 6 timing events per layer + 1 origin
     nnv::ArenaLayout last_layout;
     const void* last_arena = nullptr;
+    int* h_status = nullptr;              // pinned host word the device status is copied into
 };
 
 namespace nnv {
@@ -125,5 +126,7 @@ enum { GEMM_TF32 = 0, GEMM_BF16 = 1, GEMM_X3 = 2 };
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
 
 nnv_status_t read_device_status(int32_t* code);
+// Enqueue a copy of the device status word into pinned host memory on `st` (no synchronisation).
+nnv_status_t enqueue_status_read(int* h_pinned, cudaStream_t st);
 
 }  // namespace nnv

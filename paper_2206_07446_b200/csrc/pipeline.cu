@@ -28,21 +28,15 @@ static inline uint64_t ms_to_ns(float ms) { return ms <= 0.f ? 0ull : (uint64_t)
 }  // namespace nnv
 
 using namespace nnv;
+namespace nnv {
 
-extern "C" {
-
-nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void* h_weights, uint64_t w_bytes,
-                          const void* h_cached, uint64_t c_bytes, const float* h_input, float* h_output,
-                          void* d_arena, uint64_t arena_bytes, void* s_copy_, void* s_xform_, void* s_exec_,
-                          int32_t depth, nnv_timing_t* timings) {
-    NNV_REQUIRE(p && choices && h_weights && h_input && h_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
-    NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
-    NNV_REQUIRE(s_copy_ != s_xform_ && s_copy_ != s_exec_ && s_xform_ != s_exec_, NNV_ERR_INVALID_ARG,
-                "the three streams must be distinct");
-    cudaStream_t s_copy = (cudaStream_t)s_copy_, s_xform = (cudaStream_t)s_xform_, s_exec = (cudaStream_t)s_exec_;
+// One pass over the layer list.  `resident` = the read stage is already done: weights, cached
+// blob, input and output are device buffers and nothing crosses the host link.
+static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const void* weights, uint64_t w_bytes,
+                              const void* cached_blob, uint64_t c_bytes, const float* input, float* output,
+                              void* d_arena, uint64_t arena_bytes, cudaStream_t s_copy, cudaStream_t s_xform,
+                              cudaStream_t s_exec, int depth, nnv_timing_t* timings, bool resident) {
     const int n = (int)p->layers.size();
-
     ArenaLayout A;
     NNV_TRY(layout_arena(*p, choices, depth, &A));
     NNV_REQUIRE(arena_bytes >= A.total, NNV_ERR_WORKSPACE_TOO_SMALL, "arena needs %llu bytes, got %llu",
@@ -50,15 +44,18 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
     std::vector<uint64_t> coff(n, 0);
     uint64_t ctotal = 0;
     NNV_TRY(nnv_cached_layout(p, choices, coff.data(), &ctotal));
-    NNV_REQUIRE(ctotal == 0 || (h_cached && c_bytes >= ctotal), NNV_ERR_INVALID_ARG,
+    NNV_REQUIRE(ctotal == 0 || (cached_blob && c_bytes >= ctotal), NNV_ERR_INVALID_ARG,
                 "cached blob needs %llu bytes", (unsigned long long)ctotal);
+    NNV_REQUIRE(!resident || (aligned256(weights) && (!cached_blob || aligned256(cached_blob))), NNV_ERR_INVALID_ARG,
+                "device-resident blobs must be 256-byte aligned");
     for (int i = 0; i < n; ++i) {
         const nnv_layer_desc_t& L = p->layers[i];
         if (L.op != NNV_OP_CONV) continue;
         NNV_REQUIRE(L.w_off + raw_weight_bytes(L) <= w_bytes && (!L.has_bias || L.b_off + 4ull * L.K <= w_bytes),
-                    NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the host blob", i);
+                    NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the weight blob", i);
     }
     NNV_TRY(ensure_events(*p, timings != nullptr));
+    if (!p->h_status) NNV_CUDA(cudaHostAlloc((void**)&p->h_status, sizeof(int), cudaHostAllocDefault));
     p->last_layout = A;
     p->last_arena = d_arena;
 
@@ -68,15 +65,19 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
     const bool tm = timings != nullptr;
     if (tm) {
         NNV_CUDA(cudaEventRecord(p->tev[0], s_exec));
-        NNV_CUDA(cudaStreamWaitEvent(s_copy, p->tev[0], 0));
+        if (!resident) NNV_CUDA(cudaStreamWaitEvent(s_copy, p->tev[0], 0));
         NNV_CUDA(cudaStreamWaitEvent(s_xform, p->tev[0], 0));
         std::memset(timings, 0, sizeof(nnv_timing_t) * n);
     }
 
-    // model input: host NCHW -> device NHWC, on the execution stream
+    // model input: NCHW -> device NHWC, on the execution stream
     const nnv_layer_desc_t& L0 = p->layers[0];
-    NNV_CUDA(cudaMemcpyAsync(base + A.in_chw, h_input, 4ull * L0.C * L0.H * L0.W, cudaMemcpyHostToDevice, s_exec));
-    NNV_TRY(launch_chw_to_hwc((const float*)(base + A.in_chw), (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, s_exec));
+    const float* in_chw = input;
+    if (!resident) {
+        NNV_CUDA(cudaMemcpyAsync(base + A.in_chw, input, 4ull * L0.C * L0.H * L0.W, cudaMemcpyHostToDevice, s_exec));
+        in_chw = (const float*)(base + A.in_chw);
+    }
+    NNV_TRY(launch_chw_to_hwc(in_chw, (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, s_exec));
 
     std::vector<int> conv_ids;
     for (int i = 0; i < n; ++i) {
@@ -94,48 +95,56 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
         const int j = (int)conv_ids.size();
         conv_ids.push_back(i);
         const int slot = j % depth;
-        uint8_t* raw = base + A.raw_slot0 + (uint64_t)slot * A.raw_slot_bytes;
-        uint8_t* xf = base + A.xf_slot0 + (uint64_t)slot * A.xf_slot_bytes;
+        const uint8_t* raw = base + A.raw_slot0 + (uint64_t)slot * A.raw_slot_bytes;
+        const uint8_t* bias = raw + A.raw_bias_off;
+        const uint8_t* xf = base + A.xf_slot0 + (uint64_t)slot * A.xf_slot_bytes;
         const bool has_xf = variant_has_transform(ch.variant);
         const bool cached = has_xf && ch.cached;
         const uint64_t rbytes = raw_weight_bytes(L), tbytes = transformed_bytes(*p, i, ch.variant, ch.math);
-
-        // read: the staging slot is free once the layer that used it last has executed
-        if (j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
-        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
+        cudaEvent_t ready = nullptr;
         uint64_t copied = 0;
-        if (cached) {
-            NNV_CUDA(cudaMemcpyAsync(xf, (const uint8_t*)h_cached + coff[i], tbytes, cudaMemcpyHostToDevice, s_copy));
-            copied += tbytes;
+
+        if (resident) {
+            raw = (const uint8_t*)weights + L.w_off;
+            bias = (const uint8_t*)weights + L.b_off;
+            if (cached) xf = (const uint8_t*)cached_blob + coff[i];
         } else {
-            NNV_CUDA(cudaMemcpyAsync(raw, (const uint8_t*)h_weights + L.w_off, rbytes, cudaMemcpyHostToDevice, s_copy));
-            copied += rbytes;
+            // read: the staging slot is free once the layer that used it last has executed
+            if (j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
+            if (cached) {
+                NNV_CUDA(cudaMemcpyAsync((void*)xf, (const uint8_t*)cached_blob + coff[i], tbytes, cudaMemcpyHostToDevice, s_copy));
+                copied += tbytes;
+            } else {
+                NNV_CUDA(cudaMemcpyAsync((void*)raw, (const uint8_t*)weights + L.w_off, rbytes, cudaMemcpyHostToDevice, s_copy));
+                copied += rbytes;
+            }
+            if (L.has_bias) {
+                NNV_CUDA(cudaMemcpyAsync((void*)bias, (const uint8_t*)weights + L.b_off, 4ull * L.K, cudaMemcpyHostToDevice, s_copy));
+                copied += 4ull * L.K;
+            }
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
+            NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
+            ready = EV(i, 0);
         }
-        if (L.has_bias) {
-            NNV_CUDA(cudaMemcpyAsync(raw + A.raw_bias_off, (const uint8_t*)h_weights + L.b_off, 4ull * L.K,
-                                     cudaMemcpyHostToDevice, s_copy));
-            copied += 4ull * L.K;
-        }
-        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
-        NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
 
         // transform
-        cudaEvent_t ready = EV(i, 0);
         if (has_xf && !cached) {
-            NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(i, 0), 0));
+            if (ready) NNV_CUDA(cudaStreamWaitEvent(s_xform, ready, 0));
+            else if (j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
-            NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, xf, s_xform));
+            NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, (void*)xf, s_xform));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
             NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
             ready = EV(i, 1);
         }
 
         // execute
-        NNV_CUDA(cudaStreamWaitEvent(s_exec, ready, 0));
+        if (ready) NNV_CUDA(cudaStreamWaitEvent(s_exec, ready, 0));
         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), s_exec));
         const void* add = L.in1 >= 0 ? base + A.act_off[L.in1] : nullptr;
-        NNV_TRY(do_exec(*p, i, ch.variant, ch.math, in, add, has_xf ? xf : raw, L.has_bias ? raw + A.raw_bias_off : nullptr,
-                        out, base + A.ws_off, A.ws_bytes, s_exec));
+        NNV_TRY(do_exec(*p, i, ch.variant, ch.math, in, add, has_xf ? xf : raw, L.has_bias ? bias : nullptr, out,
+                        base + A.ws_off, A.ws_bytes, s_exec));
         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 5), s_exec));
         NNV_CUDA(cudaEventRecord(EV(i, 2), s_exec));
         if (tm) {
@@ -146,13 +155,15 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
         }
     }
 
-    // last layer's output: device NHWC -> host NCHW
+    // last layer's output: device NHWC -> NCHW
     const nnv_layer_desc_t& Ln = p->layers[n - 1];
     const LayerGeom& gn = p->geom[n - 1];
-    NNV_TRY(launch_hwc_to_chw((const float*)(base + A.act_off[n - 1]), (float*)(base + A.out_chw), Ln.K, gn.OH, gn.OW, s_exec));
-    NNV_CUDA(cudaMemcpyAsync(h_output, base + A.out_chw, 4ull * gn.P * Ln.K, cudaMemcpyDeviceToHost, s_exec));
+    float* out_chw = resident ? output : (float*)(base + A.out_chw);
+    NNV_TRY(launch_hwc_to_chw((const float*)(base + A.act_off[n - 1]), out_chw, Ln.K, gn.OH, gn.OW, s_exec));
+    if (!resident) NNV_CUDA(cudaMemcpyAsync(output, out_chw, 4ull * gn.P * Ln.K, cudaMemcpyDeviceToHost, s_exec));
+    NNV_TRY(enqueue_status_read(p->h_status, s_exec));
 
-    NNV_CUDA(cudaStreamSynchronize(s_copy));
+    if (!resident) NNV_CUDA(cudaStreamSynchronize(s_copy));
     NNV_CUDA(cudaStreamSynchronize(s_xform));
     NNV_CUDA(cudaStreamSynchronize(s_exec));
 
@@ -168,18 +179,53 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
             NNV_TRY(stamp(TEV(i, 4), &timings[i].exec_start_ns));
             NNV_TRY(stamp(TEV(i, 5), &timings[i].exec_end_ns));
             if (L.op != NNV_OP_CONV) continue;
-            NNV_TRY(stamp(TEV(i, 0), &timings[i].h2d_start_ns));
-            NNV_TRY(stamp(TEV(i, 1), &timings[i].h2d_end_ns));
+            if (!resident) {
+                NNV_TRY(stamp(TEV(i, 0), &timings[i].h2d_start_ns));
+                NNV_TRY(stamp(TEV(i, 1), &timings[i].h2d_end_ns));
+            }
             if (timings[i].xform_bytes) {
                 NNV_TRY(stamp(TEV(i, 2), &timings[i].xform_start_ns));
                 NNV_TRY(stamp(TEV(i, 3), &timings[i].xform_end_ns));
             }
         }
     }
-    int32_t code = 0;
-    NNV_TRY(read_device_status(&code));
-    NNV_REQUIRE(code == 0, (nnv_status_t)code, "a device-side wait gave up during the cold run");
+    if (*p->h_status != 0) {
+        const int code = *p->h_status;
+        int32_t dummy = 0;
+        read_device_status(&dummy);                 // clears the device word
+        return fail((nnv_status_t)code, "a device-side wait gave up during the run");
+    }
     return NNV_OK;
+}
+
+}  // namespace nnv
+
+extern "C" {
+
+nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void* h_weights, uint64_t w_bytes,
+                          const void* h_cached, uint64_t c_bytes, const float* h_input, float* h_output,
+                          void* d_arena, uint64_t arena_bytes, void* s_copy, void* s_xform, void* s_exec,
+                          int32_t depth, nnv_timing_t* timings) {
+    NNV_REQUIRE(p && choices && h_weights && h_input && h_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
+    NNV_REQUIRE(s_copy != s_xform && s_copy != s_exec && s_xform != s_exec, NNV_ERR_INVALID_ARG,
+                "the three streams must be distinct");
+    return run_model(p, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena, arena_bytes,
+                     (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings, false);
+}
+
+nnv_status_t nnv_resident_run(nnv_plan_t* p, const nnv_choice_t* choices, const void* d_weights, uint64_t w_bytes,
+                              const void* d_cached, uint64_t c_bytes, const float* d_input, float* d_output,
+                              void* d_arena, uint64_t arena_bytes, void* s_xform, void* s_exec, int32_t depth,
+                              nnv_timing_t* timings) {
+    NNV_REQUIRE(p && choices && d_weights && d_input && d_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(aligned256(d_arena) && aligned256(d_input) && aligned256(d_output), NNV_ERR_INVALID_ARG,
+                "device pointers must be 256-byte aligned");
+    NNV_REQUIRE(s_xform != s_exec, NNV_ERR_INVALID_ARG, "the two streams must be distinct");
+    return run_model(p, choices, d_weights, w_bytes, d_cached, c_bytes, d_input, d_output, d_arena, arena_bytes,
+                     nullptr, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings, true);
 }
 
 nnv_status_t nnv_layer_output(const nnv_plan_t* p, int32_t layer, const void** d_ptr, uint64_t* bytes) {

@@ -277,6 +277,7 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* p) {
     if (!p) return NNV_OK;
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     for (cudaEvent_t e : p->tev) cudaEventDestroy(e);
+    if (p->h_status) cudaFreeHost(p->h_status);
     delete p;
     return NNV_OK;
 }

@@ -86,6 +86,18 @@ def test_resnet18_cold_run_pipeline_depths_bitwise_equal_and_ordered():
     assert rel_l2(outs[0][0], acts[-1]) <= 5e-3          # 20 TF32 layers chained
 
 
+def test_resident_run_equals_cold_run_bitwise():
+    """With the read stage already done the result is bit-identical to the run that copies from the host."""
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=6)
+    ch = _choices(model, [nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    y_cold, _ = model.cold_run(x, ch, depth=2)
+    for depth in (1, 3):
+        y_res, tm = model.resident_run(x, ch, depth=depth, want_timings=True)
+        assert np.array_equal(y_cold.view(np.uint32), y_res.view(np.uint32))
+        assert all(t["h2d_bytes"] == 0 for t in tm)
+
+
 def test_cached_bypass_gives_identical_result():
     """Reading cached post-transform weights and skipping the transform changes nothing in the output."""
     layers = wl.tiny_net()
