@@ -194,6 +194,32 @@ nnv_status_t nnv_conv_exec(const nnv_plan_t* plan, int32_t layer, int32_t varian
                            const void* d_in, const void* d_addend, const void* d_wt, const void* d_bias,
                            void* d_out, void* d_ws, uint64_t ws_bytes, void* stream);
 
+/* nnv_conv_exec without a scratch argument.  (The paper has no counterpart to
+ * this call; it is a convenience of this library.)  It is for callers that cannot
+ * hand over device scratch because they cannot allocate any: a plug-in inside an
+ * application that owns all device memory, a latency-bound loop that must avoid
+ * cudaMalloc's device-wide synchronisation, set-up code that runs before a memory
+ * pool exists.  The scratch is a fixed array of NNV_STATIC_SCRATCH_BYTES compiled
+ * into the library; every GPU that loads the library holds that much memory until
+ * the process ends.  The call allocates and frees nothing.
+ *   - Same arguments, layouts, alignment rules and result as nnv_conv_exec; inputs
+ *     and outputs are still the caller's.
+ *   - A (layer, variant, math) whose nnv_exec_workspace_bytes() exceeds
+ *     NNV_STATIC_SCRATCH_BYTES is refused with NNV_ERR_WORKSPACE_TOO_SMALL before
+ *     anything is launched; use nnv_conv_exec with your own buffer for those.
+ *   - The first call on each device (with that device current) looks up the
+ *     array's device address; make that first call before any stream capture
+ *     begins on the device.  Later calls only enqueue kernels.
+ *   - All calls on a device share the one array, and it keeps whatever the last
+ *     call left in it.  Nothing in it has to start at zero -- every kernel of the
+ *     chain fully writes what the next one reads -- so it is never cleared.  Two
+ *     calls whose kernels may overlap on the GPU (different streams without an
+ *     ordering between them) race on it: serialise them. */
+#define NNV_STATIC_SCRATCH_BYTES (16u << 20)
+nnv_status_t nnv_conv_exec_static(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
+                                  const void* d_in, const void* d_addend, const void* d_wt, const void* d_bias,
+                                  void* d_out, void* stream);
+
 /* Max-pool / global-average-pool layer, NHWC fp32 in and out. */
 nnv_status_t nnv_pool_exec(const nnv_plan_t* plan, int32_t layer,
                            const void* d_in, void* d_out, void* stream);

@@ -74,6 +74,7 @@ _SIGS = {
     "nnv_select_kernels": [_vp, _P(Cost), _i32, _i32, _P(Choice)],
     "nnv_transform_weights": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
     "nnv_conv_exec": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _u64, _vp],
+    "nnv_conv_exec_static": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp],
     "nnv_pool_exec": [_vp, _i32, _vp, _vp, _vp],
     "nnv_chw_to_hwc": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_hwc_to_chw": [_vp, _vp, _i32, _i32, _i32, _vp],
@@ -241,6 +242,16 @@ def nnv_transform_weights(plan, layer, variant, math, d_raw, d_out, stream=None)
 def nnv_conv_exec(plan, layer, variant, math, d_in, d_addend, d_wt, d_bias, d_out, d_ws, ws_bytes, stream=None):
     _check(_lib.nnv_conv_exec(plan.handle, layer, variant, math, _ptr(d_in), _ptr(d_addend), _ptr(d_wt),
                               _ptr(d_bias), _ptr(d_out), _ptr(d_ws), int(ws_bytes), _stream(stream)))
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def nnv_conv_exec_static(plan, layer, variant, math, d_in, d_addend, d_wt, d_bias, d_out, stream=None):
+    """nnv_conv_exec for callers without device scratch of their own: the scratch is a fixed array
+    inside the library (STATIC_SCRATCH_BYTES); nothing is allocated by this call."""
+    _check(_lib.nnv_conv_exec_static(plan.handle, layer, variant, math, _ptr(d_in), _ptr(d_addend), _ptr(d_wt),
+                                     _ptr(d_bias), _ptr(d_out), _stream(stream)))
 
 
 def nnv_pool_exec(plan, layer, d_in, d_out, stream=None):
