@@ -94,6 +94,10 @@ typedef struct {
     int32_t allow_cached;       /* default for selection; default 1                       */
     int32_t max_depth;          /* largest pipeline depth nnv_cold_run accepts; default 4 */
     int32_t debug_checks;       /* reserved, 0                                            */
+    int32_t use_graphs;         /* 1: nnv_cold_run / nnv_resident_run record their stream work into a
+                                   CUDA graph on the first call with a given argument set (choices,
+                                   buffer addresses, depth) and replay it afterwards; 0: always enqueue
+                                   call by call.  Calls that ask for timings never use a graph.        */
 } nnv_plan_opts_t;
 
 /* One row of the profiled cost table: the operation costs of one kernel of one

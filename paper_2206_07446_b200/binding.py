@@ -36,7 +36,7 @@ class LayerDesc(ctypes.Structure):
 
 
 class PlanOpts(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("default_math", "allow_cached", "max_depth", "debug_checks")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("default_math", "allow_cached", "max_depth", "debug_checks", "use_graphs")]
 
 
 class Cost(ctypes.Structure):

@@ -422,9 +422,19 @@ std::once_flag g_attr_once;
 
 }  // namespace
 
+nnv_status_t gemm_tc_init() {
+    NNV_TRY(get_encoder());
+    std::call_once(g_attr_once, [] {
+        cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    });
+    return NNV_OK;
+}
+
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     NNV_REQUIRE(a.M > 0 && a.N > 0 && a.Kd > 0 && a.batch > 0, NNV_ERR_INVALID_ARG, "empty GEMM");
-    NNV_TRY(get_encoder());
+    NNV_TRY(gemm_tc_init());
     // Column tile: split N into equal tiles of at most 128 columns, rounded up to the MMA's
     // granularity of 16.
     const int n_tiles = ceil_div(a.N, 128);
@@ -442,11 +452,6 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     g.ldd = a.ldd; g.strideD = a.strideD;
     g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols;
 
-    std::call_once(g_attr_once, [] {
-        cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-    });
     dim3 grid(ceil_div(a.M, BM), ceil_div(a.N, BN), a.batch);
     NNV_REQUIRE(grid.y <= 65535 && grid.z <= 65535, NNV_ERR_UNSUPPORTED, "GEMM grid too large");
     auto smem_for = [&](int stages, uint32_t stage) { return (size_t)1024 + (size_t)stages * stage + 8 * (3 * stages + 2); };

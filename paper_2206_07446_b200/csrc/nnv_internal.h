@@ -53,6 +53,30 @@ struct ArenaLayout {
 
 }  // namespace nnv
 
+namespace nnv {
+struct GraphKey {
+    std::vector<nnv_choice_t> choices;
+    std::vector<const void*> ptrs;
+    uint64_t w_bytes = 0;
+    int depth = 0;
+    bool resident = false;
+    bool operator==(const GraphKey& o) const {
+        if (ptrs != o.ptrs || w_bytes != o.w_bytes || depth != o.depth || resident != o.resident ||
+            choices.size() != o.choices.size())
+            return false;
+        for (size_t i = 0; i < choices.size(); ++i)
+            if (choices[i].variant != o.choices[i].variant || choices[i].math != o.choices[i].math ||
+                choices[i].cached != o.choices[i].cached)
+                return false;
+        return true;
+    }
+};
+struct CachedGraph {
+    GraphKey key;
+    cudaGraphExec_t exec = nullptr;       // null: recording failed, this argument set runs eagerly
+};
+}  // namespace nnv
+
 struct nnv_plan {
     std::vector<nnv_layer_desc_t> layers;
     std::vector<nnv::LayerGeom> geom;
@@ -62,6 +86,7 @@ struct nnv_plan {
     std::vector<cudaEvent_t> tev;         // 6 timing events per layer + 1 origin
     nnv::ArenaLayout last_layout;
     const void* last_arena = nullptr;
+    std::vector<nnv::CachedGraph> graphs;   // recorded passes, one per distinct argument set
     int* h_status = nullptr;              // pinned host word the device status is copied into
 };
 
@@ -124,6 +149,9 @@ struct GemmArgs {
 // as hi*hi + lo*hi + hi*lo on the bf16 tensor pipe (fp32-class accuracy, fp32 bytes in memory).
 enum { GEMM_TF32 = 0, GEMM_BF16 = 1, GEMM_X3 = 2 };
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
+// One-time host set-up of the GEMM (driver entry point, shared-memory attributes); call before
+// stream capture.
+nnv_status_t gemm_tc_init();
 
 nnv_status_t read_device_status(int32_t* code);
 // Enqueue a copy of the device status word into pinned host memory on `st` (no synchronisation).

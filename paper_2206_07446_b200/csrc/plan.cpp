@@ -215,7 +215,7 @@ nnv_status_t nnv_plan_create(const nnv_layer_desc_t* layers, int32_t n, const nn
     NNV_REQUIRE(p, NNV_ERR_STATE, "out of host memory");
     p->layers.assign(layers, layers + n);
     p->geom.resize(n);
-    p->opts = nnv_plan_opts_t{NNV_MATH_TF32, 1, 4, 0};
+    p->opts = nnv_plan_opts_t{NNV_MATH_TF32, 1, 4, 0, 1};
     if (opts) {
         p->opts = *opts;
         if (p->opts.max_depth <= 0) p->opts.max_depth = 4;
@@ -278,6 +278,8 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* p) {
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     for (cudaEvent_t e : p->tev) cudaEventDestroy(e);
     if (p->h_status) cudaFreeHost(p->h_status);
+    for (nnv::CachedGraph& g : p->graphs)
+        if (g.exec) cudaGraphExecDestroy(g.exec);
     delete p;
     return NNV_OK;
 }

@@ -28,10 +28,11 @@ def dev_bytes(nbytes, fill=0xFF):
 class Model:
     """A plan plus its host-side weight blob, ready for cold runs."""
 
-    def __init__(self, layers, blob_u8, w_off, b_off, max_depth=4):
+    def __init__(self, layers, blob_u8, w_off, b_off, max_depth=4, use_graphs=1):
         self.layers = layers
         self.plan = nb.Plan(layers, w_off, b_off, opts=dict(default_math=nb.MATH_TF32, allow_cached=1,
-                                                            max_depth=max_depth, debug_checks=0))
+                                                            max_depth=max_depth, debug_checks=0,
+                                                            use_graphs=use_graphs))
         self.h_weights = _pinned_bytes(np.ascontiguousarray(blob_u8))
         self.w_bytes = int(blob_u8.size)
         self.w_off, self.b_off = list(w_off), list(b_off)
@@ -154,8 +155,8 @@ class Model:
         return costs
 
 
-def model_from_workload(layers, weights, biases, blob_fn, max_depth=4):
+def model_from_workload(layers, weights, biases, blob_fn, max_depth=4, use_graphs=1):
     """Build a Model from a layer list and per-layer numpy weights using `blob_fn`
     (workloads.weight_blob) to lay out the host blob."""
     blob, w_off, b_off = blob_fn(layers, weights, biases)
-    return Model(layers, blob, w_off, b_off, max_depth=max_depth)
+    return Model(layers, blob, w_off, b_off, max_depth=max_depth, use_graphs=use_graphs)
