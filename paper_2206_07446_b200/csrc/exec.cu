@@ -66,9 +66,14 @@ nnv_status_t do_exec(const nnv_plan& p, int layer, int v, int math, const void* 
     // IM2COL and GEMM1X1: Y[P][K] = Xcol[P][Qp] * P[K][Qp]^T
     a.M = g.P; a.Kd = g.Qp; a.batch = 1;
     a.B = d_wt; a.ldb = g.Qp; a.strideB = (int64_t)L.K * g.Qp;
-    const bool direct_operand = (v == NNV_VAR_GEMM1X1) && need == 0;
+    const bool direct_operand = (v == NNV_VAR_GEMM1X1) && need == 0 && L.stride == 1;
     if (direct_operand) {
         a.A = x; a.lda = L.C; a.Kd = L.C;                      // rows of X are the GEMM's rows
+    } else if (need == 0) {
+        // implicit GEMM: the TMA gathers the filter-window pixels from the activation itself
+        a.A = x; a.lda = L.C;
+        a.ic.on = 1; a.ic.C = L.C; a.ic.H = L.H; a.ic.W = L.W; a.ic.R = L.R; a.ic.S = L.S;
+        a.ic.stride = L.stride; a.ic.pad = L.pad; a.ic.OW = g.OW;
     } else {
         NNV_TRY(launch_im2col(bf16, x, d_ws, L.C, L.H, L.W, L.R, L.S, L.stride, L.pad, g.OH, g.OW, g.Qp, st));
         a.A = d_ws; a.lda = g.Qp;

@@ -29,6 +29,7 @@ template <typename OutT>
 __global__ void __launch_bounds__(256)
 im2col_kernel(const float* __restrict__ x, OutT* __restrict__ col, int C, int H, int W, int R, int S, int stride,
               int pad, int OH, int OW, int Qp) {
+    pdl_enter();
     const long long n = (long long)OH * OW * Qp;
     const int Q = R * S * C;
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
@@ -50,6 +51,7 @@ template <typename OutT>
 __global__ void __launch_bounds__(256)
 im2col_vec4_kernel(const float* __restrict__ x, OutT* __restrict__ col, int C, int H, int W, int R, int S, int stride,
                    int pad, int OH, int OW, int Qp) {
+    pdl_enter();
     const int Qv = Qp / 4;
     const long long n = (long long)OH * OW * Qv;
     const int Q = R * S * C;
@@ -83,11 +85,11 @@ nnv_status_t launch_im2col(bool bf16, const float* x, void* col, int C, int H, i
     const long long n = (long long)OH * OW * (vec ? Qp / 4 : Qp);
     const unsigned grid = (unsigned)std::min<long long>((n + 255) / 256, 148ll * 32);
     if (vec) {
-        if (bf16) im2col_vec4_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
-        else im2col_vec4_kernel<float><<<grid, 256, 0, st>>>(x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
+        if (bf16) NNV_LAUNCH((im2col_vec4_kernel<__nv_bfloat16>), grid, 256, 0, st, x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
+        else NNV_LAUNCH((im2col_vec4_kernel<float>), grid, 256, 0, st, x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
     } else {
-        if (bf16) im2col_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
-        else im2col_kernel<float><<<grid, 256, 0, st>>>(x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
+        if (bf16) NNV_LAUNCH((im2col_kernel<__nv_bfloat16>), grid, 256, 0, st, x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
+        else NNV_LAUNCH((im2col_kernel<float>), grid, 256, 0, st, x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
     }
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
@@ -150,6 +152,7 @@ template <int M_, typename OutT>
 __global__ void __launch_bounds__(128)
 wino_input_kernel(const float* __restrict__ x, OutT* __restrict__ V, int C, int Cp, int H, int W, int pad, int TH,
                   int TW) {
+    pdl_enter();
     constexpr int A = WinoBA<M_>::A;
     const long long T = (long long)TH * TW;
     const long long idx = (long long)blockIdx.x * 128 + threadIdx.x;
@@ -196,8 +199,8 @@ nnv_status_t launch_wino_input(int m, bool bf16, const float* x, void* V, int C,
     const long long n = (long long)TH * TW * Cp;
     const unsigned grid = (unsigned)((n + 127) / 128);
 #define NNV_WI(MM)                                                                                              \
-    if (bf16) wino_input_kernel<MM, __nv_bfloat16><<<grid, 128, 0, st>>>(x, (__nv_bfloat16*)V, C, Cp, H, W, pad, TH, TW); \
-    else wino_input_kernel<MM, float><<<grid, 128, 0, st>>>(x, (float*)V, C, Cp, H, W, pad, TH, TW);
+    if (bf16) NNV_LAUNCH((wino_input_kernel<MM, __nv_bfloat16>), grid, 128, 0, st, x, (__nv_bfloat16*)V, C, Cp, H, W, pad, TH, TW); \
+    else NNV_LAUNCH((wino_input_kernel<MM, float>), grid, 128, 0, st, x, (float*)V, C, Cp, H, W, pad, TH, TW);
     if (m == 2) { NNV_WI(2) } else if (m == 4) { NNV_WI(4) } else if (m == 6) { NNV_WI(6) }
     else return fail(NNV_ERR_INVALID_ARG, "no Winograd tile size %d", m);
 #undef NNV_WI
@@ -211,6 +214,7 @@ template <int M_>
 __global__ void __launch_bounds__(128)
 wino_output_kernel(const float* __restrict__ Mt, float* __restrict__ y, const float* __restrict__ bias,
                    const float* __restrict__ add, int act, int K, int OH, int OW, int TH, int TW) {
+    pdl_enter();
     constexpr int A = WinoBA<M_>::A;
     const long long T = (long long)TH * TW;
     const long long idx = (long long)blockIdx.x * 128 + threadIdx.x;
@@ -260,9 +264,9 @@ nnv_status_t launch_wino_output(int m, const float* Mt, float* y, const float* b
                                 int K, int OH, int OW, int TH, int TW, cudaStream_t st) {
     const long long n = (long long)TH * TW * K;
     const unsigned grid = (unsigned)((n + 127) / 128);
-    if (m == 2) wino_output_kernel<2><<<grid, 128, 0, st>>>(Mt, y, bias, add, act, K, OH, OW, TH, TW);
-    else if (m == 4) wino_output_kernel<4><<<grid, 128, 0, st>>>(Mt, y, bias, add, act, K, OH, OW, TH, TW);
-    else if (m == 6) wino_output_kernel<6><<<grid, 128, 0, st>>>(Mt, y, bias, add, act, K, OH, OW, TH, TW);
+    if (m == 2) NNV_LAUNCH((wino_output_kernel<2>), grid, 128, 0, st, Mt, y, bias, add, act, K, OH, OW, TH, TW);
+    else if (m == 4) NNV_LAUNCH((wino_output_kernel<4>), grid, 128, 0, st, Mt, y, bias, add, act, K, OH, OW, TH, TW);
+    else if (m == 6) NNV_LAUNCH((wino_output_kernel<6>), grid, 128, 0, st, Mt, y, bias, add, act, K, OH, OW, TH, TW);
     else return fail(NNV_ERR_INVALID_ARG, "no Winograd tile size %d", m);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
@@ -277,6 +281,7 @@ __global__ void __launch_bounds__(256)
 direct_conv_kernel(const float* __restrict__ x, const float* __restrict__ w, const float* __restrict__ bias,
                    const float* __restrict__ add, float* __restrict__ y, int act, int C, int H, int W, int K, int R,
                    int S, int stride, int pad, int OH, int OW) {
+    pdl_enter();
     __shared__ float As[DC_BK][DC_BM + 4];
     __shared__ float Bs[DC_BK][DC_BN + 4];
     const int P = OH * OW, RS = R * S, Q = C * RS;
@@ -347,7 +352,7 @@ nnv_status_t launch_direct(const float* x, const float* w, const float* bias, co
                            int C, int H, int W, int K, int R, int S, int stride, int pad, int OH, int OW,
                            cudaStream_t st) {
     dim3 grid(ceil_div(OH * OW, DC_BM), ceil_div(K, DC_BN));
-    direct_conv_kernel<<<grid, 256, 0, st>>>(x, w, bias, add, y, act, C, H, W, K, R, S, stride, pad, OH, OW);
+    NNV_LAUNCH((direct_conv_kernel), grid, 256, 0, st, x, w, bias, add, y, act, C, H, W, K, R, S, stride, pad, OH, OW);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
@@ -358,6 +363,7 @@ __global__ void __launch_bounds__(256)
 depthwise_kernel(const float* __restrict__ x, const float* __restrict__ w, const float* __restrict__ bias,
                  const float* __restrict__ add, float* __restrict__ y, int act, int C, int H, int W, int R, int S,
                  int stride, int pad, int OH, int OW) {
+    pdl_enter();
     const long long n = (long long)OH * OW * C;
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
         const int p = (int)(i / C), c = (int)(i - (long long)p * C);
@@ -382,7 +388,7 @@ nnv_status_t launch_depthwise(const float* x, const float* w, const float* bias,
                               cudaStream_t st) {
     const long long n = (long long)OH * OW * C;
     const unsigned grid = (unsigned)std::min<long long>((n + 255) / 256, 148ll * 32);
-    depthwise_kernel<<<grid, 256, 0, st>>>(x, w, bias, add, y, act, C, H, W, R, S, stride, pad, OH, OW);
+    NNV_LAUNCH((depthwise_kernel), grid, 256, 0, st, x, w, bias, add, y, act, C, H, W, R, S, stride, pad, OH, OW);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
@@ -391,6 +397,7 @@ nnv_status_t launch_depthwise(const float* x, const float* w, const float* bias,
 __global__ void __launch_bounds__(256)
 maxpool_kernel(const float* __restrict__ x, float* __restrict__ y, int C, int H, int W, int R, int stride, int pad,
                int OH, int OW) {
+    pdl_enter();
     const long long n = (long long)OH * OW * C;
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
         const int p = (int)(i / C), c = (int)(i - (long long)p * C);
@@ -411,6 +418,7 @@ maxpool_kernel(const float* __restrict__ x, float* __restrict__ y, int C, int H,
 
 __global__ void __launch_bounds__(256)
 gavgpool_kernel(const float* __restrict__ x, float* __restrict__ y, int C, int HW) {
+    pdl_enter();
     const int c = blockIdx.x * 256 + threadIdx.x;
     if (c >= C) return;
     float s = 0.f;
@@ -420,6 +428,7 @@ gavgpool_kernel(const float* __restrict__ x, float* __restrict__ y, int C, int H
 
 __global__ void __launch_bounds__(256)
 chw_to_hwc_kernel(const float* __restrict__ in, float* __restrict__ out, int C, int HW) {
+    pdl_enter();
     const long long n = (long long)C * HW;
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
         const int p = (int)(i / C), c = (int)(i - (long long)p * C);
@@ -429,6 +438,7 @@ chw_to_hwc_kernel(const float* __restrict__ in, float* __restrict__ out, int C, 
 
 __global__ void __launch_bounds__(256)
 hwc_to_chw_kernel(const float* __restrict__ in, float* __restrict__ out, int C, int HW) {
+    pdl_enter();
     const long long n = (long long)C * HW;
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
         const int c = (int)(i / HW), p = (int)(i - (long long)c * HW);
@@ -440,22 +450,22 @@ static inline unsigned grid_for(long long n) { return (unsigned)std::min<long lo
 
 nnv_status_t launch_maxpool(const float* x, float* y, int C, int H, int W, int R, int stride, int pad, int OH,
                             int OW, cudaStream_t st) {
-    maxpool_kernel<<<grid_for((long long)OH * OW * C), 256, 0, st>>>(x, y, C, H, W, R, stride, pad, OH, OW);
+    NNV_LAUNCH((maxpool_kernel), grid_for((long long)OH * OW * C), 256, 0, st, x, y, C, H, W, R, stride, pad, OH, OW);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
 nnv_status_t launch_gavgpool(const float* x, float* y, int C, int H, int W, cudaStream_t st) {
-    gavgpool_kernel<<<ceil_div(C, 256), 256, 0, st>>>(x, y, C, H * W);
+    NNV_LAUNCH((gavgpool_kernel), ceil_div(C, 256), 256, 0, st, x, y, C, H * W);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
 nnv_status_t launch_chw_to_hwc(const float* in, float* out, int C, int H, int W, cudaStream_t st) {
-    chw_to_hwc_kernel<<<grid_for((long long)C * H * W), 256, 0, st>>>(in, out, C, H * W);
+    NNV_LAUNCH((chw_to_hwc_kernel), grid_for((long long)C * H * W), 256, 0, st, in, out, C, H * W);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
 nnv_status_t launch_hwc_to_chw(const float* in, float* out, int C, int H, int W, cudaStream_t st) {
-    hwc_to_chw_kernel<<<grid_for((long long)C * H * W), 256, 0, st>>>(in, out, C, H * W);
+    NNV_LAUNCH((hwc_to_chw_kernel), grid_for((long long)C * H * W), 256, 0, st, in, out, C, H * W);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }

@@ -84,6 +84,23 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// im2col-mode load: `pixelsPerColumn` consecutive output pixels starting at the filter window whose
+// top-left input coordinate is (w, h), each shifted by the tap offset (off_w, off_h); channels
+// [c, c + channelsPerPixel).  Positions outside the image read as zero.
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                   uint16_t off_w, uint16_t off_h, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+
+// Barrier over every thread of every CTA in the cluster (release / acquire).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -135,7 +152,9 @@ struct GemmDev {
     const float* bias;
     const float* addend;
     long long ldd, strideD;
-    int M, N, Kd, BN, act, tmem_cols;
+    int M, N, Kd, BN, act, tmem_cols, splits;
+    // implicit im2col (A is the NHWC activation itself): 0 = off
+    int ic_on, ic_C, ic_cblk, ic_S, ic_OW, ic_stride, ic_pad;
 };
 
 __device__ __forceinline__ float act_fn(float v, int act) {
@@ -211,6 +230,7 @@ template <int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev g) {
     extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();
     constexpr int STAGES = ModeTraits<MODE>::STAGES;
     constexpr int BKE = ModeTraits<MODE>::BKE;
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -227,8 +247,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, b = blockIdx.z;
-    const int nkb = (g.Kd + BKE - 1) / BKE;
+    // blockIdx.z = batch * splits + split; the `splits` CTAs of one output tile form a thread-block
+    // cluster, each reducing its own contiguous range of K blocks.
+    const int splits = g.splits;
+    const int sp = (int)blockIdx.z % splits, b = (int)blockIdx.z / splits;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const int nkb_all = g.ic_on ? g.Kd : (g.Kd + BKE - 1) / BKE;  // implicit mode: Kd already counts K blocks
+    const int kb0 = (int)(((long long)nkb_all * sp) / splits);
+    const int nkb = (int)(((long long)nkb_all * (sp + 1)) / splits) - kb0;
 
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
@@ -249,19 +275,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *holder_ptr;
+    pdl_wait();                                               // set-up above overlaps the previous kernel's tail
 
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
+            for (int it = 0; it < nkb && ok; ++it) {
+                const int kb = kb0 + it;
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
                 ok = mbar_wait(empty_bar(s), ph ^ 1u);
                 if (!ok) break;
                 mbar_expect_tx(full_bar(s), tma_bytes);
                 const uint32_t a_dst = sbase + s * stage_bytes;
-                tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
-                tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
+                if (g.ic_on) {
+                    // K runs over (filter tap, channel block): A comes straight from the activation
+                    const int tap = kb / g.ic_cblk, cb = kb - tap * g.ic_cblk;
+                    const int fr = tap / g.ic_S, fs = tap - fr * g.ic_S;
+                    const int p0 = m0 / g.ic_OW, q0 = m0 - p0 * g.ic_OW;
+                    tma_load_im2col_4d(a_dst, &tmA, cb * BKE, q0 * g.ic_stride - g.ic_pad, p0 * g.ic_stride - g.ic_pad, 0,
+                                       (uint16_t)fs, (uint16_t)fr, full_bar(s));
+                    tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, tap * g.ic_C + cb * BKE, n0, b, full_bar(s));
+                } else {
+                    tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
+                    tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
+                }
             }
             if (!ok) {
                 atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
@@ -274,9 +312,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t fmt = (MODE == 0) ? 2u : 1u;
             const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             bool ok = true;
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
+            for (int it = 0; it < nkb; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
                 ok = mbar_wait(MODE == 2 ? conv_bar(s) : full_bar(s), ph);
                 if (!ok) break;
                 tc_fence_after();
@@ -292,7 +330,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const uint64_t al = make_smem_desc_plain(a_lo + kk * 2 * lbo_a, lbo_a, 128);
                         const uint64_t bh = make_smem_desc_plain(b_hi + kk * 2 * lbo_b, lbo_b, 128);
                         const uint64_t bl = make_smem_desc_plain(b_lo + kk * 2 * lbo_b, lbo_b, 128);
-                        umma<true>(tmem_base, al, bh, idesc, (kb | kk) ? 1u : 0u);   // small terms first
+                        umma<true>(tmem_base, al, bh, idesc, (it | kk) ? 1u : 0u);   // small terms first
                         umma<true>(tmem_base, ah, bl, idesc, 1u);
                         umma<true>(tmem_base, ah, bh, idesc, 1u);
                     }
@@ -301,7 +339,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint64_t bdesc = make_smem_desc(a_src + A_STAGE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)             // 4 MMAs of 32 bytes of K each
-                        umma<MODE == 1>(tmem_base, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (kb | kk) ? 1u : 0u);
+                        umma<MODE == 1>(tmem_base, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (it | kk) ? 1u : 0u);
                 }
                 umma_commit(empty_bar(s));
             }
@@ -313,9 +351,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if constexpr (MODE == 2) {
             // warps 2-5 first convert every staged fp32 tile into its bf16 hi / lo tiles
             const int idx = (int)threadIdx.x - 64;              // 0..127: one row of A (and of B) each
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
+            for (int it = 0; it < nkb; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
                 ok = mbar_wait(full_bar(s), ph);
                 if (!ok) break;
                 const uint32_t a_src = sbase + s * stage_bytes;
@@ -331,6 +369,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         if (!ok) {
             if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        } else if (splits > 1) {
+            // park this CTA's partial tile in its own shared memory (the stage ring is idle by now):
+            // P[row][col], row pitch BN + 4 words
+            const int quarter = warp & 3;
+            const int row = quarter * 32 + lane;
+            const uint32_t prow = sbase + (uint32_t)row * (uint32_t)(BN + 4) * 4u;
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+#pragma unroll
+                for (int j = 0; j < 16; j += 4)
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (uint32_t)(c0 + j) * 4u), "r"(r[j]),
+                                 "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]) : "memory");
+            }
         } else {
             const int quarter = warp & 3;                     // TMEM lanes this warp may read
             const int m = m0 + quarter * 32 + lane;
@@ -375,6 +427,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         }
     }
+    __syncwarp();
+    if (splits > 1) {
+        // Split-K reduction through distributed shared memory: once every CTA of the cluster has
+        // parked its partial tile, CTA `sp` sums rows [sp*128/splits, (sp+1)*128/splits) over the
+        // cluster in rank order (a fixed order: the result does not depend on timing) and applies
+        // the epilogue.  Both cluster barriers are reached by every thread on every path.
+        cluster_sync_all();
+        if (warp >= 2 && g_device_status == 0) {
+            const int t = (int)threadIdx.x - 64;
+            const int rows_per = BM / splits, r0 = sp * rows_per;
+            const int c4n = BN / 4;
+            const bool vec = ((g.ldd & 3) == 0) && ((g.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
+                             (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
+                             (!g.bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+            for (int idx = t; idx < rows_per * c4n; idx += 128) {
+                const int row = r0 + idx / c4n, col = (idx % c4n) * 4;
+                const uint32_t local = sbase + ((uint32_t)row * (uint32_t)(BN + 4) + (uint32_t)col) * 4u;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int rk = 0; rk < splits; ++rk) {
+                    uint32_t remote;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rk));
+                    float4 v;
+                    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+                const int m = m0 + row, n = n0 + col;
+                if (m >= g.M || n >= g.N) continue;
+                float* drow = g.D + (long long)b * g.strideD + (long long)m * g.ldd;
+                const float* arow = g.addend ? g.addend + (long long)m * g.ldd : nullptr;
+                float vv[4] = {acc.x, acc.y, acc.z, acc.w};
+                if (vec) {
+                    if (g.bias) { const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + n)); vv[0] += bb.x; vv[1] += bb.y; vv[2] += bb.z; vv[3] += bb.w; }
+                    if (arow) { const float4 aa = __ldg(reinterpret_cast<const float4*>(arow + n)); vv[0] += aa.x; vv[1] += aa.y; vv[2] += aa.z; vv[3] += aa.w; }
+                    *reinterpret_cast<float4*>(drow + n) = make_float4(act_fn(vv[0], g.act), act_fn(vv[1], g.act), act_fn(vv[2], g.act), act_fn(vv[3], g.act));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (n + j < g.N) {
+                            float v = vv[j];
+                            if (g.bias) v += __ldg(g.bias + n + j);
+                            if (arow) v += __ldg(arow + n + j);
+                            drow[n + j] = act_fn(v, g.act);
+                        }
+                    }
+                }
+            }
+        }
+        cluster_sync_all();                                   // nobody leaves while its tile may still be read
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -385,6 +486,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // ---- host side --------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+PFN_cuTensorMapEncodeIm2col_v12000 g_encode_im2col = nullptr;
 std::once_flag g_encode_once;
 cudaError_t g_encode_err = cudaSuccess;
 
@@ -394,6 +496,10 @@ nnv_status_t get_encoder() {
         cudaDriverEntryPointQueryResult q;
         g_encode_err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
         if (g_encode_err == cudaSuccess && q == cudaDriverEntryPointSuccess) g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+        void* fn2 = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn2, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            g_encode_im2col = (PFN_cuTensorMapEncodeIm2col_v12000)fn2;
     });
     NNV_REQUIRE(g_encode != nullptr, NNV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     return NNV_OK;
@@ -418,6 +524,24 @@ nnv_status_t encode_operand(CUtensorMap* map, const void* base, bool bf16, int K
     return NNV_OK;
 }
 
+// 4-D im2col map over an NHWC fp32 activation {C, W, H, 1}: 32 channels x 128 output pixels per load.
+nnv_status_t encode_im2col_operand(CUtensorMap* map, const void* base, int C, int H, int W, int R, int S, int stride,
+                                   int pad) {
+    NNV_REQUIRE(g_encode_im2col != nullptr, NNV_ERR_CUDA, "cuTensorMapEncodeIm2col is not available from this driver");
+    NNV_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0 && (C % 4) == 0, NNV_ERR_INVALID_ARG,
+                "implicit-GEMM activation must be 16-byte aligned with C a multiple of 4");
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, 1};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 4, (cuuint64_t)W * C * 4, (cuuint64_t)H * W * C * 4};
+    int lower[2] = {-pad, -pad};
+    int upper[2] = {pad - (S - 1), pad - (R - 1)};
+    cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
+    CUresult r = g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, lower,
+                                 upper, 32, BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeIm2col failed with code %d", (int)r);
+    return NNV_OK;
+}
+
 std::once_flag g_attr_once;
 
 }  // namespace
@@ -435,32 +559,51 @@ nnv_status_t gemm_tc_init() {
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     NNV_REQUIRE(a.M > 0 && a.N > 0 && a.Kd > 0 && a.batch > 0, NNV_ERR_INVALID_ARG, "empty GEMM");
     NNV_TRY(gemm_tc_init());
-    // Column tile: split N into equal tiles of at most 128 columns, rounded up to the MMA's
-    // granularity of 16.
-    const int n_tiles = ceil_div(a.N, 128);
-    const int BN = ceil_div(ceil_div(a.N, n_tiles), 16) * 16;
+    // Tiling.  Start from equal column tiles of at most 128 (rounded up to the MMA's granularity of
+    // 16).  These layers are small for 148 SMs and a CTA can pull operands out of L2 only so fast, so
+    // while the grid is short of one wave first halve the column tile (down to 32), then split the
+    // K loop over a thread-block cluster of up to 8 CTAs that reduce through shared memory.
+    const int bke = (a.mode == GEMM_BF16) ? 64 : 32;
+    const int nkb_all = a.ic.on ? a.ic.R * a.ic.S * ceil_div(a.ic.C, 32) : ceil_div(a.Kd, bke);
+    const int m_tiles = ceil_div(a.M, BM);
+    int n_tiles = ceil_div(a.N, 128);
+    int BN = ceil_div(ceil_div(a.N, n_tiles), 16) * 16;
+    while ((long long)m_tiles * n_tiles * a.batch < 100 && BN > 32) {
+        n_tiles = ceil_div(a.N, BN / 2);
+        BN = ceil_div(ceil_div(a.N, n_tiles), 16) * 16;
+    }
+    int splits = 1;
+    while ((long long)m_tiles * n_tiles * a.batch * splits * 2 <= 160 && splits < 8 && nkb_all / (splits * 2) >= 2) splits *= 2;
     int tmem_cols = 32;
     while (tmem_cols < BN) tmem_cols *= 2;
 
     const bool bf16 = a.mode == GEMM_BF16;
     CUtensorMap tmA, tmB;
-    NNV_TRY(encode_operand(&tmA, a.A, bf16, a.Kd, a.M, a.batch, a.lda, a.strideA, BM));
-    NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
-
     GemmDev g;
     g.D = a.D; g.bias = a.bias; g.addend = a.addend;
     g.ldd = a.ldd; g.strideD = a.strideD;
-    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols;
+    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits;
+    g.ic_on = 0; g.ic_C = g.ic_cblk = g.ic_S = g.ic_OW = g.ic_stride = g.ic_pad = 0;
+    if (a.ic.on) {
+        NNV_REQUIRE(a.mode == GEMM_TF32 && a.batch == 1, NNV_ERR_INVALID_ARG, "implicit im2col needs the TF32 mode and one batch");
+        NNV_TRY(encode_im2col_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, a.ic.R, a.ic.S, a.ic.stride, a.ic.pad));
+        g.ic_on = 1; g.ic_C = a.ic.C; g.ic_cblk = ceil_div(a.ic.C, 32); g.ic_S = a.ic.S; g.ic_OW = a.ic.OW;
+        g.ic_stride = a.ic.stride; g.ic_pad = a.ic.pad;
+        g.Kd = a.ic.R * a.ic.S * g.ic_cblk;                       // number of K blocks
+    } else {
+        NNV_TRY(encode_operand(&tmA, a.A, bf16, a.Kd, a.M, a.batch, a.lda, a.strideA, BM));
+    }
+    NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
 
-    dim3 grid(ceil_div(a.M, BM), ceil_div(a.N, BN), a.batch);
+    dim3 grid(m_tiles, ceil_div(a.N, BN), a.batch * splits);
     NNV_REQUIRE(grid.y <= 65535 && grid.z <= 65535, NNV_ERR_UNSUPPORTED, "GEMM grid too large");
     auto smem_for = [&](int stages, uint32_t stage) { return (size_t)1024 + (size_t)stages * stage + 8 * (3 * stages + 2); };
     if (a.mode == GEMM_TF32)
-        gemm_tc_kernel<0><<<grid, GEMM_THREADS, smem_for(ModeTraits<0>::STAGES, stage_bytes_of<0>(BN)), st>>>(tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<0>, grid, dim3(GEMM_THREADS), smem_for(ModeTraits<0>::STAGES, stage_bytes_of<0>(BN)), st, splits, tmA, tmB, g);
     else if (a.mode == GEMM_BF16)
-        gemm_tc_kernel<1><<<grid, GEMM_THREADS, smem_for(ModeTraits<1>::STAGES, stage_bytes_of<1>(BN)), st>>>(tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<1>, grid, dim3(GEMM_THREADS), smem_for(ModeTraits<1>::STAGES, stage_bytes_of<1>(BN)), st, splits, tmA, tmB, g);
     else if (a.mode == GEMM_X3)
-        gemm_tc_kernel<2><<<grid, GEMM_THREADS, smem_for(ModeTraits<2>::STAGES, stage_bytes_of<2>(BN)), st>>>(tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<2>, grid, dim3(GEMM_THREADS), smem_for(ModeTraits<2>::STAGES, stage_bytes_of<2>(BN)), st, splits, tmA, tmB, g);
     else
         return fail(NNV_ERR_INVALID_ARG, "unknown GEMM mode %d", a.mode);
     NNV_CUDA(cudaGetLastError());

@@ -29,6 +29,55 @@ nnv_status_t fail(nnv_status_t code, const char* fmt, ...);
         if (s__ != NNV_OK) return s__;        \
     } while (0)
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// Every kernel is launched with the programmatic-stream-serialization attribute and starts with
+// pdl_enter(): it lets the next kernel in the stream be launched at once (its blocks get scheduled
+// and run their own preamble while this grid is still working) and then waits until the previous
+// grid has completed and its writes are visible.  Because every kernel waits before it touches
+// global memory, completion is transitive along the stream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_trigger(); pdl_wait(); }
+
+template <typename... Params, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+// Same, as thread-block clusters of `cluster_z` consecutive CTAs along grid z (1 = no cluster).
+template <typename... Params, typename... Args>
+inline cudaError_t launch_pdl_cluster(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                      int cluster_z, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = (unsigned)cluster_z;
+    cfg.attrs = attr;
+    cfg.numAttrs = cluster_z > 1 ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+#define NNV_LAUNCH(kernel, grid, block, smem, st, ...) \
+    (void)::nnv::launch_pdl(kernel, dim3(grid), dim3(block), (size_t)(smem), st, __VA_ARGS__)
+#endif
+
 static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -144,6 +193,9 @@ struct GemmArgs {
     int64_t strideA, strideB, strideD;  // batch strides (elements)
     const float* bias; const float* addend; int act;
     int mode;                         // GEMM_TF32, GEMM_BF16 or GEMM_X3
+    // Implicit im2col: A is the NHWC fp32 activation (C % 4 == 0) read by the TMA in im2col mode;
+    // B is the packed weight P[K][Qp] with Kd = Qp; M = OH*OW output pixels.  TF32 mode, batch 1.
+    struct { int on, C, H, W, R, S, stride, pad, OW; } ic;
 };
 // GEMM_X3: fp32 operands; each is split on the fly into bf16 hi + lo and the product is formed
 // as hi*hi + lo*hi + hi*lo on the bf16 tensor pipe (fp32-class accuracy, fp32 bytes in memory).

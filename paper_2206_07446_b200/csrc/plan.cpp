@@ -80,6 +80,14 @@ static inline bool gemm1x1_direct_operand(const nnv_layer_desc_t& L, int math) {
     return math == NNV_MATH_TF32 && L.stride == 1 && (L.C % 4) == 0;
 }
 
+static inline bool implicit_gemm_operand(const nnv_layer_desc_t& L, int math) {
+    // The TMA's im2col mode gathers filter-window pixels straight from the NHWC activation, so no
+    // Xcol matrix is materialised: fp32 words (TF32), pixel rows a multiple of 16 bytes, and an
+    // activation of at least 128 KiB (smaller tensors take the explicit path).
+    return math == NNV_MATH_TF32 && (L.C % 4) == 0 && 4ull * L.C * L.H * L.W >= 131072ull && L.R <= 16 && L.S <= 16 &&
+           L.pad <= 8;
+}
+
 uint64_t exec_ws_bytes(const nnv_plan& p, int layer, int v, int math) {
     const nnv_layer_desc_t& L = p.layers[layer];
     const LayerGeom& g = p.geom[layer];
@@ -89,9 +97,10 @@ uint64_t exec_ws_bytes(const nnv_plan& p, int layer, int v, int math) {
         const uint64_t T = (uint64_t)ceil_div(g.OH, m) * ceil_div(g.OW, m);
         return align_up(a2 * T * g.Cp * es, 256) + align_up(a2 * T * L.K * 4, 256);
     }
-    if (v == NNV_VAR_IM2COL) return align_up((uint64_t)g.P * g.Qp * es, 256);
+    if (v == NNV_VAR_IM2COL) return implicit_gemm_operand(L, math) ? 0 : align_up((uint64_t)g.P * g.Qp * es, 256);
     if (v == NNV_VAR_GEMM1X1)
-        return gemm1x1_direct_operand(L, math) ? 0 : align_up((uint64_t)g.P * g.Qp * es, 256);
+        return (gemm1x1_direct_operand(L, math) || implicit_gemm_operand(L, math)) ? 0
+                                                                                  : align_up((uint64_t)g.P * g.Qp * es, 256);
     return 0;
 }
 

@@ -81,6 +81,7 @@ constexpr int FT_THREADS = 256;
 template <int M_, typename OutT, int NF>
 __global__ void __launch_bounds__(FT_THREADS)
 filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp) {
+    pdl_enter();
     constexpr int A = WinoG<M_>::A;
     __shared__ __align__(16) float sg[FT_THREADS * NF * 9];
     const long long F = (long long)K * Cp;                      // padded filter count = plane size
@@ -154,7 +155,7 @@ static nnv_status_t launch_ft(const float* g, void* U, int K, int C, int Cp, cud
     const long long F = (long long)K * Cp;
     const long long per_block = (long long)FT_THREADS * NF;
     const unsigned grid = (unsigned)((F + per_block - 1) / per_block);
-    filter_transform_kernel<M_, OutT, NF><<<grid, FT_THREADS, 0, st>>>(g, reinterpret_cast<OutT*>(U), K, C, Cp);
+    NNV_LAUNCH((filter_transform_kernel<M_, OutT, NF>), grid, FT_THREADS, 0, st, g, reinterpret_cast<OutT*>(U), K, C, Cp);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
@@ -192,6 +193,7 @@ constexpr int PACK_SMEM_FLOATS = 8192;
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
 pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int C, int RS, int Qp) {
+    pdl_enter();
     __shared__ float sw[PACK_SMEM_FLOATS];
     const int k = blockIdx.x;
     const long long Q = (long long)C * RS;
@@ -216,6 +218,7 @@ pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int C, int RS, in
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
 pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp) {
+    pdl_enter();
     const long long n = (long long)K * Qp;
     for (long long i = (long long)blockIdx.x * PACK_THREADS + threadIdx.x; i < n; i += (long long)gridDim.x * PACK_THREADS) {
         const int k = (int)(i / Qp), q = (int)(i - (long long)k * Qp);
@@ -227,12 +230,12 @@ nnv_status_t launch_pack(bool bf16, const float* w, void* P, int K, int C, int R
     if (RS == 1) {
         const long long n = (long long)K * Qp;
         const unsigned grid = (unsigned)std::min<long long>((n + PACK_THREADS - 1) / PACK_THREADS, 148 * 16);
-        if (bf16) pack1x1_kernel<__nv_bfloat16><<<grid, PACK_THREADS, 0, st>>>(w, (__nv_bfloat16*)P, K, C, Qp);
-        else pack1x1_kernel<float><<<grid, PACK_THREADS, 0, st>>>(w, (float*)P, K, C, Qp);
+        if (bf16) NNV_LAUNCH((pack1x1_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, Qp);
+        else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp);
     } else {
         NNV_REQUIRE(RS <= PACK_SMEM_FLOATS, NNV_ERR_UNSUPPORTED, "filter window of %d taps is too large to repack", RS);
-        if (bf16) pack_kernel<__nv_bfloat16><<<K, PACK_THREADS, 0, st>>>(w, (__nv_bfloat16*)P, C, RS, Qp);
-        else pack_kernel<float><<<K, PACK_THREADS, 0, st>>>(w, (float*)P, C, RS, Qp);
+        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), K, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, C, RS, Qp);
+        else NNV_LAUNCH((pack_kernel<float>), K, PACK_THREADS, 0, st, w, (float*)P, C, RS, Qp);
     }
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;

@@ -132,5 +132,5 @@ def test_workspace_too_small_is_reported():
     plan = nb.Plan(layers, [0], [0])
     buf = poisoned(1 << 20)
     with pytest.raises(nb.NnvError) as e:
-        nb.nnv_conv_exec(plan, 0, nb.VAR_IM2COL, nb.MATH_TF32, buf, None, buf, None, buf, buf, 1024, torch.cuda.current_stream())
+        nb.nnv_conv_exec(plan, 0, nb.VAR_IM2COL, nb.MATH_BF16, buf, None, buf, None, buf, buf, 1024, torch.cuda.current_stream())
     assert e.value.status == 4
