@@ -18,6 +18,10 @@
 #include <cudaTypedefs.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "nnv_internal.h"
@@ -152,7 +156,7 @@ struct GemmDev {
     const float* bias;
     const float* addend;
     long long ldd, strideD;
-    int M, N, Kd, BN, act, tmem_cols, splits;
+    int M, N, Kd, BN, act, tmem_cols, splits, stages, prefill;
     // implicit im2col (A is the NHWC activation itself): 0 = off
     int ic_on, ic_C, ic_cblk, ic_S, ic_OW, ic_stride, ic_pad;
 };
@@ -216,7 +220,6 @@ __device__ __forceinline__ void convert_row(uint32_t src_tile, uint32_t hi_tile,
 // MODE 0: TF32 operands (fp32 words), 1: BF16 operands, 2: fp32 operands multiplied as
 // hi*hi + lo*hi + hi*lo of their bf16 splits (error-compensated, fp32-class accuracy).
 template <int MODE> struct ModeTraits {
-    static constexpr int STAGES = (MODE == 2) ? 3 : 4;
     static constexpr int BKE = (MODE == 1) ? 64 : 32;          // K elements per stage
 };
 
@@ -231,7 +234,8 @@ __global__ void __launch_bounds__(GEMM_THREADS)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev g) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();
-    constexpr int STAGES = ModeTraits<MODE>::STAGES;
+    const int STAGES = g.stages;                              // depth of the shared-memory ring (2..8)
+    constexpr int MAXS = 8;
     constexpr int BKE = ModeTraits<MODE>::BKE;
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int BN = g.BN;
@@ -240,10 +244,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t stage_bytes = stage_bytes_of<MODE>(BN);
     const uint32_t bars = sbase + STAGES * stage_bytes;       // full[S], empty[S], conv[S], tmem_full, holder
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto conv_bar = [&](int s) { return bars + 8u * (2 * STAGES + s); };
-    const uint32_t tmem_full_bar = bars + 8u * (3 * STAGES);
-    const uint32_t holder = bars + 8u * (3 * STAGES + 1);
+    auto empty_bar = [&](int s) { return bars + 8u * (MAXS + s); };
+    auto conv_bar = [&](int s) { return bars + 8u * (2 * MAXS + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (3 * MAXS);
+    const uint32_t holder = bars + 8u * (3 * MAXS + 1);
     volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -271,35 +275,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"((uint32_t)g.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // One K block: operand tiles of iteration `it` into ring slot it % STAGES.
+    auto issue_stage = [&](int it) {
+        const int kb = kb0 + it;
+        const int s = it % STAGES;
+        mbar_expect_tx(full_bar(s), tma_bytes);
+        const uint32_t a_dst = sbase + s * stage_bytes;
+        if (g.ic_on) {
+            // K runs over (filter tap, channel block): A comes straight from the activation
+            const int tap = kb / g.ic_cblk, cb = kb - tap * g.ic_cblk;
+            const int fr = tap / g.ic_S, fs = tap - fr * g.ic_S;
+            const int p0 = m0 / g.ic_OW, q0 = m0 - p0 * g.ic_OW;
+            tma_load_im2col_4d(a_dst, &tmA, cb * BKE, q0 * g.ic_stride - g.ic_pad, p0 * g.ic_stride - g.ic_pad, 0,
+                               (uint16_t)fs, (uint16_t)fr, full_bar(s));
+            tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, tap * g.ic_C + cb * BKE, n0, b, full_bar(s));
+        } else {
+            tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
+            tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
+        }
+    };
+    // The producer fills the whole ring before the CTA-wide barrier: the first loads fly while
+    // TMEM is being allocated.  It only needs its own barrier initialisation and the previous
+    // kernel's results (pdl_wait).
+    const int prefill = g.prefill ? (nkb < STAGES ? nkb : STAGES) : 0;
+    if (warp == 0 && lane == 0) {
+        pdl_wait();
+        for (int it = 0; it < prefill; ++it) issue_stage(it);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *holder_ptr;
     pdl_wait();                                               // set-up above overlaps the previous kernel's tail
 
+    bool epi_ok = false;
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
-            for (int it = 0; it < nkb && ok; ++it) {
-                const int kb = kb0 + it;
+            for (int it = prefill; it < nkb && ok; ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (it / STAGES) & 1;
                 ok = mbar_wait(empty_bar(s), ph ^ 1u);
                 if (!ok) break;
-                mbar_expect_tx(full_bar(s), tma_bytes);
-                const uint32_t a_dst = sbase + s * stage_bytes;
-                if (g.ic_on) {
-                    // K runs over (filter tap, channel block): A comes straight from the activation
-                    const int tap = kb / g.ic_cblk, cb = kb - tap * g.ic_cblk;
-                    const int fr = tap / g.ic_S, fs = tap - fr * g.ic_S;
-                    const int p0 = m0 / g.ic_OW, q0 = m0 - p0 * g.ic_OW;
-                    tma_load_im2col_4d(a_dst, &tmA, cb * BKE, q0 * g.ic_stride - g.ic_pad, p0 * g.ic_stride - g.ic_pad, 0,
-                                       (uint16_t)fs, (uint16_t)fr, full_bar(s));
-                    tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, tap * g.ic_C + cb * BKE, n0, b, full_bar(s));
-                } else {
-                    tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
-                    tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
-                }
+                issue_stage(it);
             }
             if (!ok) {
                 atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
@@ -369,21 +387,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         if (!ok) {
             if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
-        } else if (splits > 1) {
-            // park this CTA's partial tile in its own shared memory (the stage ring is idle by now):
-            // P[row][col], row pitch BN + 4 words
-            const int quarter = warp & 3;
-            const int row = quarter * 32 + lane;
-            const uint32_t prow = sbase + (uint32_t)row * (uint32_t)(BN + 4) * 4u;
-            for (int c0 = 0; c0 < BN; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
-#pragma unroll
-                for (int j = 0; j < 16; j += 4)
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (uint32_t)(c0 + j) * 4u), "r"(r[j]),
-                                 "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]) : "memory");
-            }
-        } else {
+        } else if (splits == 1) {
             const int quarter = warp & 3;                     // TMEM lanes this warp may read
             const int m = m0 + quarter * 32 + lane;
             float* drow = g.D + (long long)b * g.strideD + (long long)m * g.ldd;
@@ -425,56 +429,88 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
+        } else {
+            epi_ok = true;
+            // park this CTA's (partial) tile in its own shared memory (the stage ring is idle by now):
+            // P[row][col], row pitch BN + 4 words
+            const int quarter = warp & 3;
+            const int row = quarter * 32 + lane;
+            const uint32_t prow = sbase + (uint32_t)row * (uint32_t)(BN + 4) * 4u;
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+#pragma unroll
+                for (int j = 0; j < 16; j += 4)
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (uint32_t)(c0 + j) * 4u), "r"(r[j]),
+                                 "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]) : "memory");
+            }
         }
     }
     __syncwarp();
-    if (splits > 1) {
-        // Split-K reduction through distributed shared memory: once every CTA of the cluster has
-        // parked its partial tile, CTA `sp` sums rows [sp*128/splits, (sp+1)*128/splits) over the
-        // cluster in rank order (a fixed order: the result does not depend on timing) and applies
-        // the epilogue.  Both cluster barriers are reached by every thread on every path.
-        cluster_sync_all();
-        if (warp >= 2 && g_device_status == 0) {
+    {
+        // Split-K write-out.  Every CTA of the cluster has parked its partial tile in shared memory;
+        // CTA `sp` sums rows [sp*128/splits, (sp+1)*128/splits) over the cluster through distributed
+        // shared memory in rank order (a fixed order: the result does not depend on timing), then
+        // applies bias / residual / activation and stores row-contiguous 128-bit words.  The
+        // cluster barriers are reached by every thread on every path.
+        if (splits > 1) cluster_sync_all();
+        if (splits > 1 && warp >= 2 && g_device_status == 0) {
             const int t = (int)threadIdx.x - 64;
             const int rows_per = BM / splits, r0 = sp * rows_per;
             const int c4n = BN / 4;
             const bool vec = ((g.ldd & 3) == 0) && ((g.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
                              (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
                              (!g.bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
-            for (int idx = t; idx < rows_per * c4n; idx += 128) {
-                const int row = r0 + idx / c4n, col = (idx % c4n) * 4;
-                const uint32_t local = sbase + ((uint32_t)row * (uint32_t)(BN + 4) + (uint32_t)col) * 4u;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int rk = 0; rk < splits; ++rk) {
-                    uint32_t remote;
-                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rk));
-                    float4 v;
-                    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
-                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            // Thread t walks the (row, 4-column group) grid in steps of 128 without divisions.  The loop
+            // is kept small on purpose (no unrolling): each CTA runs it once, and instruction fetch of
+            // cold code costs more here than the arithmetic.
+            const int total = rows_per * c4n;
+            const int qstep = 128 / c4n, rstep = 128 - qstep * c4n;
+            int row = r0 + t / c4n, col4 = t % c4n;
+            float* const dbase = g.D + (long long)b * g.strideD;
+#pragma unroll 1
+            for (int idx = t; idx < total; idx += 128) {
+                const int rr = row, cc = col4 * 4;
+                row += qstep; col4 += rstep;
+                if (col4 >= c4n) { col4 -= c4n; ++row; }
+                const uint32_t local = sbase + ((uint32_t)rr * (uint32_t)(BN + 4) + (uint32_t)cc) * 4u;
+                // all remote loads are issued before the first is consumed, so their latencies overlap
+                float4 v[8];
+#pragma unroll
+                for (int rk = 0; rk < 8; ++rk) {
+                    if (rk < splits) {
+                        uint32_t remote;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rk));
+                        asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v[rk].x), "=f"(v[rk].y), "=f"(v[rk].z), "=f"(v[rk].w) : "r"(remote));
+                    }
                 }
-                const int m = m0 + row, n = n0 + col;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int rk = 0; rk < 8; ++rk)
+                    if (rk < splits) { acc.x += v[rk].x; acc.y += v[rk].y; acc.z += v[rk].z; acc.w += v[rk].w; }
+                const int m = m0 + rr, n = n0 + cc;
                 if (m >= g.M || n >= g.N) continue;
-                float* drow = g.D + (long long)b * g.strideD + (long long)m * g.ldd;
+                float* drow = dbase + (long long)m * g.ldd;
                 const float* arow = g.addend ? g.addend + (long long)m * g.ldd : nullptr;
                 float vv[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (vec || n + j < g.N) {
+                        if (g.bias) vv[j] += __ldg(g.bias + n + j);
+                        if (arow) vv[j] += __ldg(arow + n + j);
+                        vv[j] = act_fn(vv[j], g.act);
+                    }
+                }
                 if (vec) {
-                    if (g.bias) { const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + n)); vv[0] += bb.x; vv[1] += bb.y; vv[2] += bb.z; vv[3] += bb.w; }
-                    if (arow) { const float4 aa = __ldg(reinterpret_cast<const float4*>(arow + n)); vv[0] += aa.x; vv[1] += aa.y; vv[2] += aa.z; vv[3] += aa.w; }
-                    *reinterpret_cast<float4*>(drow + n) = make_float4(act_fn(vv[0], g.act), act_fn(vv[1], g.act), act_fn(vv[2], g.act), act_fn(vv[3], g.act));
+                    *reinterpret_cast<float4*>(drow + n) = make_float4(vv[0], vv[1], vv[2], vv[3]);
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (n + j < g.N) {
-                            float v = vv[j];
-                            if (g.bias) v += __ldg(g.bias + n + j);
-                            if (arow) v += __ldg(arow + n + j);
-                            drow[n + j] = act_fn(v, g.act);
-                        }
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        if (n + j < g.N) drow[n + j] = vv[j];
                 }
             }
         }
-        cluster_sync_all();                                   // nobody leaves while its tile may still be read
+        if (splits > 1) cluster_sync_all();                   // nobody leaves while its tile may still be read
     }
     tc_fence_before();
     __syncthreads();
@@ -559,30 +595,54 @@ nnv_status_t gemm_tc_init() {
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     NNV_REQUIRE(a.M > 0 && a.N > 0 && a.Kd > 0 && a.batch > 0, NNV_ERR_INVALID_ARG, "empty GEMM");
     NNV_TRY(gemm_tc_init());
-    // Tiling.  Start from equal column tiles of at most 128 (rounded up to the MMA's granularity of
-    // 16).  These layers are small for 148 SMs and a CTA can pull operands out of L2 only so fast, so
-    // while the grid is short of one wave first halve the column tile (down to 32), then split the
-    // K loop over a thread-block cluster of up to 8 CTAs that reduce through shared memory.
+    // Tiling.  These layers are small for 148 SMs, and one CTA can pull operand tiles out of L2 only
+    // so fast (~90 GB/s measured), so the column tile BN and the number of K splits (a thread-block
+    // cluster of up to 8 CTAs reducing through shared memory) are picked by a small cost model:
+    // waves x (fixed cost + K blocks per CTA x bytes per K block / per-SM bandwidth).
     const int bke = (a.mode == GEMM_BF16) ? 64 : 32;
     const int nkb_all = a.ic.on ? a.ic.R * a.ic.S * ceil_div(a.ic.C, 32) : ceil_div(a.Kd, bke);
     const int m_tiles = ceil_div(a.M, BM);
-    int n_tiles = ceil_div(a.N, 128);
-    int BN = ceil_div(ceil_div(a.N, n_tiles), 16) * 16;
-    while ((long long)m_tiles * n_tiles * a.batch < 100 && BN > 32) {
-        n_tiles = ceil_div(a.N, BN / 2);
-        BN = ceil_div(ceil_div(a.N, n_tiles), 16) * 16;
+    const int stages = (a.mode == GEMM_X3) ? 3 : 4;               // ring depth assumed by the cost model
+    int BN = 0, splits = 1;
+    double best = 1e30;
+    for (int nt = ceil_div(a.N, 128); nt <= ceil_div(a.N, 16); nt *= 2) {
+        const int bn = ceil_div(ceil_div(a.N, nt), 16) * 16;
+        const int n_tiles = ceil_div(a.N, bn);
+        const double kb_bytes = (double)(A_STAGE_BYTES + bn * BK_BYTES);
+        const double smem = 1024.0 + stages * kb_bytes * (a.mode == GEMM_X3 ? 2 : 1);
+        const int occ = std::max(1, std::min(4, (int)(220.0 * 1024.0 / smem)));
+        for (int sp = 1; sp <= 8 && sp <= nkb_all; sp *= 2) {
+            const long long ctas = (long long)m_tiles * n_tiles * a.batch * sp;
+            const double waves = std::ceil((double)ctas / (148.0 * occ));
+            const double per_kb_us = std::max(kb_bytes * occ / 90e3, 0.12);   // bytes / (90 GB/s) in us, shared by co-resident CTAs
+            const double t = waves * (2.0 + (sp > 1 ? 4.5 : 0.0) + std::ceil((double)nkb_all / sp) * per_kb_us + bn * 0.004);
+            if (t < best - 1e-9) { best = t; BN = bn; splits = sp; }
+        }
+        if (bn <= 16) break;
     }
-    int splits = 1;
-    while ((long long)m_tiles * n_tiles * a.batch * splits * 2 <= 160 && splits < 8 && nkb_all / (splits * 2) >= 2) splits *= 2;
+    if (const char* e = std::getenv("NNV_DEBUG_GEMM_TILE")) {      // debug only: "BN,splits"
+        int fb = 0, fs = 0;
+        if (std::sscanf(e, "%d,%d", &fb, &fs) == 2 && fb >= 16 && fb <= 128 && fb % 16 == 0 && fs >= 1 && fs <= 8 &&
+            (fs & (fs - 1)) == 0 && fs <= nkb_all) { BN = fb; splits = fs; }
+    }
     int tmem_cols = 32;
     while (tmem_cols < BN) tmem_cols *= 2;
+    // Ring depth.  Measured: the K loop moves ~90 GB/s per SM whatever the depth beyond 4 (it is bound
+    // by the SM's L2 read rate, not by latency), so 4 stages (3 with the extra converted tiles).
+    const uint32_t sb = (a.mode == GEMM_X3) ? stage_bytes_of<2>(BN) : stage_bytes_of<0>(BN);
+    int ring = (a.mode == GEMM_X3) ? 3 : 4;
+    if (const char* e = std::getenv("NNV_DEBUG_GEMM_RING")) {      // debug only: ring depth
+        const int r = std::atoi(e);
+        if (r >= 2 && r <= 8 && (size_t)r * sb <= 210u * 1024u) ring = r;
+    }
+    while (splits > 1 && (uint32_t)ring * sb < (uint32_t)BM * (BN + 4) * 4u) ++ring;   // room to park the partial tile
 
     const bool bf16 = a.mode == GEMM_BF16;
     CUtensorMap tmA, tmB;
     GemmDev g;
     g.D = a.D; g.bias = a.bias; g.addend = a.addend;
     g.ldd = a.ldd; g.strideD = a.strideD;
-    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits;
+    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits; g.stages = ring; g.prefill = std::getenv("NNV_DEBUG_GEMM_NOPREFILL") ? 0 : 1;
     g.ic_on = 0; g.ic_C = g.ic_cblk = g.ic_S = g.ic_OW = g.ic_stride = g.ic_pad = 0;
     if (a.ic.on) {
         NNV_REQUIRE(a.mode == GEMM_TF32 && a.batch == 1, NNV_ERR_INVALID_ARG, "implicit im2col needs the TF32 mode and one batch");
@@ -597,13 +657,13 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
 
     dim3 grid(m_tiles, ceil_div(a.N, BN), a.batch * splits);
     NNV_REQUIRE(grid.y <= 65535 && grid.z <= 65535, NNV_ERR_UNSUPPORTED, "GEMM grid too large");
-    auto smem_for = [&](int stages, uint32_t stage) { return (size_t)1024 + (size_t)stages * stage + 8 * (3 * stages + 2); };
+    const size_t smem_bytes = (size_t)1024 + (size_t)ring * sb + 8 * (3 * 8 + 2);
     if (a.mode == GEMM_TF32)
-        (void)launch_pdl_cluster(gemm_tc_kernel<0>, grid, dim3(GEMM_THREADS), smem_for(ModeTraits<0>::STAGES, stage_bytes_of<0>(BN)), st, splits, tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<0>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, g);
     else if (a.mode == GEMM_BF16)
-        (void)launch_pdl_cluster(gemm_tc_kernel<1>, grid, dim3(GEMM_THREADS), smem_for(ModeTraits<1>::STAGES, stage_bytes_of<1>(BN)), st, splits, tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<1>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, g);
     else if (a.mode == GEMM_X3)
-        (void)launch_pdl_cluster(gemm_tc_kernel<2>, grid, dim3(GEMM_THREADS), smem_for(ModeTraits<2>::STAGES, stage_bytes_of<2>(BN)), st, splits, tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<2>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, g);
     else
         return fail(NNV_ERR_INVALID_ARG, "unknown GEMM mode %d", a.mode);
     NNV_CUDA(cudaGetLastError());
