@@ -188,6 +188,18 @@ nnv_status_t nnv_select_kernels(const nnv_plan_t* plan, const nnv_cost_t* costs,
 nnv_status_t nnv_transform_weights(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
                                    const void* d_raw, void* d_out, void* stream);
 
+/* The weights transformation of EVERY layer in one launch (the paper's decision
+ * stage writes all post-transformed weights out once, its Section 3.1.2; the
+ * same job builds the cached blob here).  d_weights: device copy of the weight
+ * blob (raw weights at w_off).  d_out: nnv_transformed_layout() bytes; layer i's
+ * transformed weights land at offsets[i] (256-byte aligned; 0 for layers without
+ * a transform).  Bit-identical to calling nnv_transform_weights per layer. */
+nnv_status_t nnv_transformed_layout(const nnv_plan_t* plan, const nnv_choice_t* choices,
+                                    uint64_t* offsets /* n layers */, uint64_t* total);
+nnv_status_t nnv_transform_all(const nnv_plan_t* plan, const nnv_choice_t* choices,
+                               const void* d_weights, uint64_t w_bytes,
+                               void* d_out, uint64_t out_bytes, void* stream);
+
 /* Execute one conv layer (the paper's "execution" operation) with the given
  * kernel.  d_in: NHWC fp32 input (H x W x C).  d_addend: NHWC fp32 residual of
  * the output's shape or NULL.  d_wt: transformed weights of this (variant, math),
@@ -239,7 +251,10 @@ nnv_status_t nnv_hwc_to_chw(const float* d_in, float* d_out, int32_t C, int32_t 
  * (s_exec), pipelined so that layer i+1.. are prepared while layer i executes
  * (the paper's Section 3.1.3).  Preparation of conv layer j may start only
  * after the execution of conv layer j-depth has finished (depth staging slots);
- * depth = 1 is the fully serial order read, transform, execute per layer.
+ * depth = 1 is the fully serial order read, transform, execute per layer;
+ * depth = 0 lifts the limit: every layer gets its own raw and transformed buffer
+ * in the arena and preparation never waits for execution (the paper's pipeline,
+ * whose little cores run ahead freely).
  *   h_weights: pinned host blob holding raw weights / biases at w_off / b_off.
  *   h_cached:  pinned host blob of cached transformed weights laid out by
  *              nnv_cached_layout(); may be NULL if no choice has cached = 1.
@@ -261,7 +276,9 @@ nnv_status_t nnv_cold_run(nnv_plan_t* plan, const nnv_choice_t* choices,
  * latter two alone).  d_weights / d_cached are DEVICE copies of the two blobs
  * (256-byte aligned), d_input / d_output are DEVICE NCHW fp32 buffers; nothing
  * crosses the host link.  Transforms run on s_xform, layers on s_exec; the
- * transform of conv layer j waits for the execution of conv layer j-depth. */
+ * transform of conv layer j waits for the execution of conv layer j-depth.  With
+ * depth = 0 nothing orders the transforms, and they are issued as two multi-layer
+ * launches (the first layers, then all the rest) instead of one per layer. */
 nnv_status_t nnv_resident_run(nnv_plan_t* plan, const nnv_choice_t* choices,
                               const void* d_weights, uint64_t w_bytes,
                               const void* d_cached, uint64_t c_bytes,

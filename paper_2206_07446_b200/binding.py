@@ -73,6 +73,8 @@ _SIGS = {
     "nnv_filter_candidates": [_vp, _i32, _P(Cost), _i32, _i32, _P(Choice), _i32, _P(_i32)],
     "nnv_select_kernels": [_vp, _P(Cost), _i32, _i32, _P(Choice)],
     "nnv_transform_weights": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
+    "nnv_transformed_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
+    "nnv_transform_all": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp],
     "nnv_conv_exec": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _u64, _vp],
     "nnv_conv_exec_static": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp],
     "nnv_pool_exec": [_vp, _i32, _vp, _vp, _vp],
@@ -237,6 +239,18 @@ def nnv_select_kernels(plan, costs, allow_cached):
 
 def nnv_transform_weights(plan, layer, variant, math, d_raw, d_out, stream=None):
     _check(_lib.nnv_transform_weights(plan.handle, layer, variant, math, _ptr(d_raw), _ptr(d_out), _stream(stream)))
+
+
+def nnv_transformed_layout(plan, choices):
+    offs = (_u64 * plan.n)()
+    total = _u64(0)
+    _check(_lib.nnv_transformed_layout(plan.handle, _choices_array(plan, choices), offs, ctypes.byref(total)))
+    return [int(o) for o in offs], int(total.value)
+
+
+def nnv_transform_all(plan, choices, d_weights, w_bytes, d_out, out_bytes, stream=None):
+    _check(_lib.nnv_transform_all(plan.handle, _choices_array(plan, choices), _ptr(d_weights), int(w_bytes),
+                                  _ptr(d_out), int(out_bytes), _stream(stream)))
 
 
 def nnv_conv_exec(plan, layer, variant, math, d_in, d_addend, d_wt, d_bias, d_out, d_ws, ws_bytes, stream=None):

@@ -103,6 +103,49 @@ nnv_status_t nnv_transform_weights(const nnv_plan_t* p, int32_t layer, int32_t v
     return do_transform(*p, layer, v, math, d_raw, d_out, (cudaStream_t)stream);
 }
 
+nnv_status_t nnv_transformed_layout(const nnv_plan_t* p, const nnv_choice_t* choices, uint64_t* offsets, uint64_t* total) {
+    NNV_REQUIRE(p && choices && offsets && total, NNV_ERR_INVALID_ARG, "null argument");
+    uint64_t pos = 0;
+    for (int i = 0; i < (int)p->layers.size(); ++i) {
+        offsets[i] = 0;
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        NNV_TRY(check_choice(*p, i, choices[i].variant, choices[i].math));
+        if (!variant_has_transform(choices[i].variant)) continue;
+        offsets[i] = pos;
+        pos += align_up(transformed_bytes(*p, i, choices[i].variant, choices[i].math), 256);
+    }
+    *total = pos;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_transform_all(const nnv_plan_t* p, const nnv_choice_t* choices, const void* d_weights, uint64_t w_bytes,
+                               void* d_out, uint64_t out_bytes, void* stream) {
+    NNV_REQUIRE(p && choices && d_weights && d_out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(aligned256(d_weights) && aligned256(d_out), NNV_ERR_INVALID_ARG, "device pointers must be 256-byte aligned");
+    const int n = (int)p->layers.size();
+    std::vector<uint64_t> offs(n);
+    uint64_t total = 0;
+    NNV_TRY(nnv_transformed_layout(p, choices, offs.data(), &total));
+    NNV_REQUIRE(out_bytes >= total, NNV_ERR_WORKSPACE_TOO_SMALL, "output needs %llu bytes, got %llu",
+                (unsigned long long)total, (unsigned long long)out_bytes);
+    std::vector<XformDesc> descs;
+    for (int i = 0; i < n; ++i) {
+        const nnv_layer_desc_t& L = p->layers[i];
+        if (L.op != NNV_OP_CONV || !variant_has_transform(choices[i].variant)) continue;
+        NNV_REQUIRE(L.w_off + raw_weight_bytes(L) <= w_bytes, NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the weight blob", i);
+        XformDesc d{};
+        d.src = (const uint8_t*)d_weights + L.w_off;
+        d.dst = (uint8_t*)d_out + offs[i];
+        d.K = L.K; d.C = L.C; d.Cp = p->geom[i].Cp; d.RS = L.R * L.S; d.Qp = p->geom[i].Qp;
+        d.bf16 = choices[i].math == NNV_MATH_BF16;
+        const int m = wino_m(choices[i].variant);
+        d.kind = m == 2 ? XF_WINO2 : m == 4 ? XF_WINO4 : m == 6 ? XF_WINO6 : (d.RS == 1 ? XF_PACK1X1 : XF_PACK);
+        descs.push_back(d);
+    }
+    if (descs.empty()) return NNV_OK;
+    return launch_transform_batch(descs.data(), (int)descs.size(), (cudaStream_t)stream);
+}
+
 nnv_status_t nnv_conv_exec(const nnv_plan_t* p, int32_t layer, int32_t v, int32_t math, const void* d_in,
                            const void* d_addend, const void* d_wt, const void* d_bias, void* d_out, void* d_ws,
                            uint64_t ws_bytes, void* stream) {

@@ -96,6 +96,7 @@ struct ArenaLayout {
     uint64_t in_chw = 0, in_hwc = 0, out_chw = 0;
     uint64_t raw_slot0 = 0, raw_slot_bytes = 0, raw_bias_off = 0;
     uint64_t xf_slot0 = 0, xf_slot_bytes = 0;
+    std::vector<uint64_t> raw_off, bias_off, xf_off;   // depth 0: one buffer set per conv layer
     uint64_t ws_off = 0, ws_bytes = 0;
     uint64_t total = 0;
 };
@@ -158,6 +159,17 @@ nnv_status_t launch_filter_transform(int m, bool bf16, const float* d_g, void* d
                                      cudaStream_t st);
 // GEMM-ready repack: W[K][C][R][S] -> P[K][Qp] (fp32 or bf16).
 nnv_status_t launch_pack(bool bf16, const float* d_w, void* d_P, int K, int C, int RS, int Qp, cudaStream_t st);
+
+// Several layers' weight transforms in one launch.
+enum { XF_PACK = 0, XF_PACK1X1 = 1, XF_WINO2 = 2, XF_WINO4 = 3, XF_WINO6 = 4 };
+struct XformDesc {
+    const void* src; void* dst;
+    int K, C, Cp, RS, Qp;
+    int kind, bf16, block0;
+};
+constexpr int XF_BATCH_MAX = 56;
+struct XformBatch { int n; int total_blocks; XformDesc d[XF_BATCH_MAX]; };
+nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st);
 
 // Explicit im2col of an NHWC fp32 image: Xcol[P][Qp], q = (r*S+s)*C + c (fp32 or bf16).
 nnv_status_t launch_im2col(bool bf16, const float* d_x, void* d_col, int C, int H, int W, int R, int S,

@@ -1,5 +1,6 @@
 // Whole-model cold run (three-stream layer pipeline) and per-operation profiling.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 
 #include "nnv_internal.h"
@@ -12,13 +13,13 @@ nnv_status_t do_pool(const nnv_plan& p, int layer, const void* d_in, void* d_out
 
 static nnv_status_t ensure_events(nnv_plan& p, bool timing) {
     const size_t n = p.layers.size();
-    if (p.ev.size() != 3 * n + 3) {                                // + fork, join(copy), join(transform)
-        p.ev.resize(3 * n + 3, nullptr);
-        for (size_t i = 0; i < 3 * n + 3; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming));
+    if (p.ev.size() != 3 * n + 6) {                                // + fork, join(copy), join(transform), 3 transform groups
+        p.ev.resize(3 * n + 6, nullptr);
+        for (size_t i = 0; i < 3 * n + 6; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming));
     }
-    if (timing && p.tev.size() != 6 * n + 1) {
-        p.tev.resize(6 * n + 1, nullptr);
-        for (size_t i = 0; i < 6 * n + 1; ++i) NNV_CUDA(cudaEventCreate(&p.tev[i]));
+    if (timing && p.tev.size() != 6 * n + 7) {                     // + start / end of the 3 transform groups
+        p.tev.resize(6 * n + 7, nullptr);
+        for (size_t i = 0; i < 6 * n + 7; ++i) NNV_CUDA(cudaEventCreate(&p.tev[i]));
     }
     return NNV_OK;
 }
@@ -66,6 +67,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     if (tm) std::memset(timings, 0, sizeof(nnv_timing_t) * n);
     NNV_TRY(gemm_tc_init());
 
+    const bool grouped = resident && depth == 0 && !std::getenv("NNV_DEBUG_NO_GROUP");
+    std::vector<cudaEvent_t> group_event(n, nullptr);
+
     // Everything the pass puts on the streams: fork from s_exec, the per-layer operations, join back.
     auto enqueue = [&]() -> nnv_status_t {
     if (tm) NNV_CUDA(cudaEventRecord(p->tev[0], s_exec));
@@ -82,6 +86,38 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     }
     NNV_TRY(launch_chw_to_hwc(in_chw, (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, s_exec));
 
+    // Weights resident and no staging limit: nothing orders the transforms, so they are issued as up
+    // to three multi-layer launches of growing size (the first ~1 MB of raw weights so that execution
+    // can start at once, the next ~8 MB, then all the rest) instead of one small launch per layer.
+    if (grouped) {
+        std::vector<XformDesc> descs[3];
+        uint64_t first_bytes = 0;
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p->layers[i];
+            if (L.op != NNV_OP_CONV) continue;
+            const nnv_choice_t ch = choices[i];
+            if (!variant_has_transform(ch.variant) || ch.cached) continue;
+            XformDesc d{};
+            d.src = (const uint8_t*)weights + L.w_off;
+            d.dst = base + A.xf_off[i];
+            d.K = L.K; d.C = L.C; d.Cp = p->geom[i].Cp; d.RS = L.R * L.S; d.Qp = p->geom[i].Qp;
+            d.bf16 = ch.math == NNV_MATH_BF16;
+            const int m = wino_m(ch.variant);
+            d.kind = m == 2 ? XF_WINO2 : m == 4 ? XF_WINO4 : m == 6 ? XF_WINO6 : (d.RS == 1 ? XF_PACK1X1 : XF_PACK);
+            const int g = first_bytes < (1u << 20) ? 0 : first_bytes < (9u << 20) ? 1 : 2;
+            first_bytes += raw_weight_bytes(L);
+            descs[g].push_back(d);
+            group_event[i] = p->ev[3 * n + 3 + g];
+        }
+        for (int g = 0; g < 3; ++g) {
+            if (descs[g].empty()) continue;
+            if (tm) NNV_CUDA(cudaEventRecord(p->tev[6 * n + 1 + 2 * g], s_xform));
+            NNV_TRY(launch_transform_batch(descs[g].data(), (int)descs[g].size(), s_xform));
+            if (tm) NNV_CUDA(cudaEventRecord(p->tev[6 * n + 2 + 2 * g], s_xform));
+            NNV_CUDA(cudaEventRecord(p->ev[3 * n + 3 + g], s_xform));
+        }
+    }
+
     std::vector<int> conv_ids;
     for (int i = 0; i < n; ++i) {
         const nnv_layer_desc_t& L = p->layers[i];
@@ -97,10 +133,10 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         const nnv_choice_t ch = choices[i];
         const int j = (int)conv_ids.size();
         conv_ids.push_back(i);
-        const int slot = j % depth;
-        const uint8_t* raw = base + A.raw_slot0 + (uint64_t)slot * A.raw_slot_bytes;
-        const uint8_t* bias = raw + A.raw_bias_off;
-        const uint8_t* xf = base + A.xf_slot0 + (uint64_t)slot * A.xf_slot_bytes;
+        const int slot = depth ? j % depth : 0;
+        const uint8_t* raw = depth ? base + A.raw_slot0 + (uint64_t)slot * A.raw_slot_bytes : base + A.raw_off[i];
+        const uint8_t* bias = depth ? raw + A.raw_bias_off : base + A.bias_off[i];
+        const uint8_t* xf = depth ? base + A.xf_slot0 + (uint64_t)slot * A.xf_slot_bytes : base + A.xf_off[i];
         const bool has_xf = variant_has_transform(ch.variant);
         const bool cached = has_xf && ch.cached;
         const uint64_t rbytes = raw_weight_bytes(L), tbytes = transformed_bytes(*p, i, ch.variant, ch.math);
@@ -113,7 +149,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (cached) xf = (const uint8_t*)cached_blob + coff[i];
         } else {
             // read: the staging slot is free once the layer that used it last has executed
-            if (j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
+            if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
             if (cached) {
                 NNV_CUDA(cudaMemcpyAsync((void*)xf, (const uint8_t*)cached_blob + coff[i], tbytes, cudaMemcpyHostToDevice, s_copy));
@@ -132,9 +168,11 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         }
 
         // transform
-        if (has_xf && !cached) {
+        if (grouped) {
+            if (has_xf && !cached) ready = group_event[i];
+        } else if (has_xf && !cached) {
             if (ready) NNV_CUDA(cudaStreamWaitEvent(s_xform, ready, 0));
-            else if (j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
+            else if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
             NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, (void*)xf, s_xform));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
@@ -230,7 +268,11 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                 NNV_TRY(stamp(TEV(i, 0), &timings[i].h2d_start_ns));
                 NNV_TRY(stamp(TEV(i, 1), &timings[i].h2d_end_ns));
             }
-            if (timings[i].xform_bytes) {
+            if (timings[i].xform_bytes && grouped) {             // the interval of the layer's multi-layer launch
+                const int g = group_event[i] == p->ev[3 * n + 3] ? 0 : group_event[i] == p->ev[3 * n + 4] ? 1 : 2;
+                NNV_TRY(stamp(p->tev[6 * n + 1 + 2 * g], &timings[i].xform_start_ns));
+                NNV_TRY(stamp(p->tev[6 * n + 2 + 2 * g], &timings[i].xform_end_ns));
+            } else if (timings[i].xform_bytes) {
                 NNV_TRY(stamp(TEV(i, 2), &timings[i].xform_start_ns));
                 NNV_TRY(stamp(TEV(i, 3), &timings[i].xform_end_ns));
             }
@@ -254,7 +296,7 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
                           void* d_arena, uint64_t arena_bytes, void* s_copy, void* s_xform, void* s_exec,
                           int32_t depth, nnv_timing_t* timings) {
     NNV_REQUIRE(p && choices && h_weights && h_input && h_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(depth >= 0 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 0..%d", depth, p->opts.max_depth);
     NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
     NNV_REQUIRE(s_copy != s_xform && s_copy != s_exec && s_xform != s_exec, NNV_ERR_INVALID_ARG,
                 "the three streams must be distinct");
@@ -267,7 +309,7 @@ nnv_status_t nnv_resident_run(nnv_plan_t* p, const nnv_choice_t* choices, const 
                               void* d_arena, uint64_t arena_bytes, void* s_xform, void* s_exec, int32_t depth,
                               nnv_timing_t* timings) {
     NNV_REQUIRE(p && choices && d_weights && d_input && d_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(depth >= 0 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 0..%d", depth, p->opts.max_depth);
     NNV_REQUIRE(aligned256(d_arena) && aligned256(d_input) && aligned256(d_output), NNV_ERR_INVALID_ARG,
                 "device pointers must be 256-byte aligned");
     NNV_REQUIRE(s_xform != s_exec, NNV_ERR_INVALID_ARG, "the two streams must be distinct");

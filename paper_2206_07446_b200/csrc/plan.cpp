@@ -152,11 +152,23 @@ nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int de
     }
     const nnv_layer_desc_t& Ln = p.layers[n - 1];
     a.out_chw = take(4ull * p.geom[n - 1].P * Ln.K);
-    a.raw_bias_off = align_up(max_raw ? max_raw : 1, 1024);
-    a.raw_slot_bytes = a.raw_bias_off + align_up(max_bias ? max_bias : 1, 1024);
-    a.raw_slot0 = take(a.raw_slot_bytes * depth);
-    a.xf_slot_bytes = align_up(max_xf ? max_xf : 1, 1024);
-    a.xf_slot0 = take(a.xf_slot_bytes * depth);
+    if (depth == 0) {
+        // no staging limit: every conv layer owns a raw (weights + bias) and a transformed buffer
+        a.raw_off.assign(n, 0); a.bias_off.assign(n, 0); a.xf_off.assign(n, 0);
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p.layers[i];
+            if (L.op != NNV_OP_CONV) continue;
+            a.raw_off[i] = take(raw_weight_bytes(L));
+            a.bias_off[i] = take(4ull * L.K);
+            a.xf_off[i] = take(transformed_bytes(p, i, choices[i].variant, choices[i].math));
+        }
+    } else {
+        a.raw_bias_off = align_up(max_raw ? max_raw : 1, 1024);
+        a.raw_slot_bytes = a.raw_bias_off + align_up(max_bias ? max_bias : 1, 1024);
+        a.raw_slot0 = take(a.raw_slot_bytes * depth);
+        a.xf_slot_bytes = align_up(max_xf ? max_xf : 1, 1024);
+        a.xf_slot0 = take(a.xf_slot_bytes * depth);
+    }
     a.ws_bytes = align_up(max_ws ? max_ws : 1, 1024);
     a.ws_off = take(a.ws_bytes);
     a.total = pos;
@@ -322,7 +334,7 @@ nnv_status_t nnv_exec_workspace_bytes(const nnv_plan_t* p, int32_t layer, int32_
 
 nnv_status_t nnv_arena_bytes(const nnv_plan_t* p, const nnv_choice_t* choices, int32_t depth, uint64_t* bytes) {
     NNV_REQUIRE(p && choices && bytes, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(depth >= 1 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 1..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(depth >= 0 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 0..%d", depth, p->opts.max_depth);
     ArenaLayout a;
     NNV_TRY(layout_arena(*p, choices, depth, &a));
     *bytes = a.total;

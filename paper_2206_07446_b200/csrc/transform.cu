@@ -79,13 +79,11 @@ constexpr int FT_THREADS = 256;
 // 32*NF consecutive elements of the plane.  With C == Cp the block's raw filters are one
 // contiguous range, staged through shared memory with 128-bit loads.
 template <int M_, typename OutT, int NF>
-__global__ void __launch_bounds__(FT_THREADS)
-filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp) {
-    pdl_enter();
+__device__ __forceinline__ void filter_transform_block(const float* __restrict__ g, OutT* __restrict__ U, int K, int C,
+                                                       int Cp, unsigned block, float* sg) {
     constexpr int A = WinoG<M_>::A;
-    __shared__ __align__(16) float sg[FT_THREADS * NF * 9];
     const long long F = (long long)K * Cp;                      // padded filter count = plane size
-    const long long f_block = (long long)blockIdx.x * (FT_THREADS * NF);
+    const long long f_block = (long long)block * (FT_THREADS * NF);
     const long long f0 = f_block + (long long)threadIdx.x * NF;
     const bool contiguous = (C == Cp);
 
@@ -149,6 +147,16 @@ filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K
     }
 }
 
+constexpr int XF_SMEM_FLOATS = 8192;                            // 32 KB staging buffer shared by all transform kernels
+
+template <int M_, typename OutT, int NF>
+__global__ void __launch_bounds__(FT_THREADS)
+filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp) {
+    pdl_enter();
+    __shared__ __align__(16) float sg[XF_SMEM_FLOATS];
+    filter_transform_block<M_, OutT, NF>(g, U, K, C, Cp, blockIdx.x, sg);
+}
+
 template <int M_, typename OutT>
 static nnv_status_t launch_ft(const float* g, void* U, int K, int C, int Cp, cudaStream_t st) {
     constexpr int NF = 2;
@@ -185,57 +193,175 @@ template <> __device__ inline float cvt_out<float>(float v) { return round_tf32(
 template <> __device__ inline __nv_bfloat16 cvt_out<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 constexpr int PACK_THREADS = 256;
-constexpr int PACK_SMEM_FLOATS = 8192;
+constexpr int PACK_SMEM_FLOATS = XF_SMEM_FLOATS;
+constexpr int PACK1X1_PER_BLOCK = PACK_THREADS * 8;             // elements of P one block of pack1x1 writes
 
-// One block per output channel k.  The row W[k][c][rs] (contiguous) is staged through shared
-// memory in channel chunks and written back as P[k][rs*C + c]: a transpose of the (c, rs)
-// index pair, coalesced on both sides; the pad q in [R*S*C, Qp) is written as +0.
+template <typename OutT> __device__ __forceinline__ void store4(OutT* p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(p) = make_float4(round_tf32(a), round_tf32(b), round_tf32(c), round_tf32(d));
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float a, float b, float c, float d) {
+    __nv_bfloat162 x = __floats2bfloat162_rn(a, b), y = __floats2bfloat162_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&x);
+    u.y = *reinterpret_cast<uint32_t*>(&y);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+
+// Repack of R*S > 1 filters.  Work unit = (output channel k, chunk of CH input channels): CH*RS
+// contiguous raw floats in, RS segments of CH consecutive elements out -- a transpose of the
+// (c, rs) index pair.  One WARP owns a unit and stages it in its private slice of shared memory
+// (only __syncwarp between its coalesced loads and its coalesced stores), so the eight warps of
+// a block stream independently and many loads stay in flight.  CH = 32 (128-byte store segments)
+// while 32*RS floats fit the slice, else 8.  The pad q in [R*S*C, Qp) is written as +0 by the
+// unit of the row's last chunk.
+constexpr int PACK_WARPS = PACK_THREADS / 32;
+constexpr int PACK_SLICE = PACK_SMEM_FLOATS / PACK_WARPS;        // floats of shared memory per warp
+
+__host__ __device__ inline int pack_ch(int RS) { return 32 * RS <= PACK_SLICE ? 32 : 8; }
+__host__ __device__ inline int pack_units_per_row(int C, int RS) { return (C + pack_ch(RS) - 1) / pack_ch(RS); }
+
 template <typename OutT>
-__global__ void __launch_bounds__(PACK_THREADS)
-pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int C, int RS, int Qp) {
-    pdl_enter();
-    __shared__ float sw[PACK_SMEM_FLOATS];
-    const int k = blockIdx.x;
-    const long long Q = (long long)C * RS;
-    const float* src = w + (long long)k * Q;
+__device__ __forceinline__ void pack_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp,
+                                           unsigned block, float* smem) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int CH = pack_ch(RS), upr = pack_units_per_row(C, RS);
+    const long long unit = (long long)block * PACK_WARPS + warp;
+    if (unit >= (long long)K * upr) return;
+    const int k = (int)(unit / upr), c0 = (int)(unit - (long long)k * upr) * CH;
+    const int cc = min(CH, C - c0), n = cc * RS;
+    float* sw = smem + warp * PACK_SLICE;
+    const float* src = w + ((long long)k * C + c0) * RS;
     OutT* dst = P + (long long)k * Qp;
-    const int CC = PACK_SMEM_FLOATS / RS;                      // channels per chunk
-    for (int c0 = 0; c0 < C; c0 += CC) {
-        const int cc = min(CC, C - c0);
-        const int n = cc * RS;
-        for (int i = threadIdx.x; i < n; i += PACK_THREADS) sw[i] = __ldg(src + (long long)c0 * RS + i);
-        __syncthreads();
-        for (int i = threadIdx.x; i < n; i += PACK_THREADS) {
+    for (int i = lane; i < n; i += 32) sw[i] = __ldg(src + i);
+    __syncwarp();
+    if (CH == 32) {
+        for (int rs = 0; rs < RS; ++rs)
+            if (lane < cc) dst[(long long)rs * C + c0 + lane] = cvt_out<OutT>(sw[lane * RS + rs]);
+    } else {
+        for (int i = lane; i < n; i += 32) {
             const int rs = i / cc, c = i - rs * cc;
             dst[(long long)rs * C + c0 + c] = cvt_out<OutT>(sw[c * RS + rs]);
         }
-        __syncthreads();
     }
-    for (int q = (int)Q + threadIdx.x; q < Qp; q += PACK_THREADS) dst[q] = cvt_out<OutT>(0.f);
+    if (c0 + cc == C)
+        for (int q = C * RS + lane; q < Qp; q += 32) dst[q] = cvt_out<OutT>(0.f);
 }
 
-// 1x1 filters: the repack is a row-padded copy (and conversion).
+// 1x1 filters: the repack is a row-padded copy (and conversion); one block writes
+// PACK1X1_PER_BLOCK consecutive elements of P.
+template <typename OutT>
+__device__ __forceinline__ void pack1x1_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp,
+                                              unsigned block) {
+    const long long n = (long long)K * Qp;
+    const long long base = (long long)block * PACK1X1_PER_BLOCK;
+    if (C == Qp) {                                              // no padding: a straight conversion copy, 4 at a time
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const long long i = base + ((long long)u * PACK_THREADS + threadIdx.x) * 4;
+            if (i < n) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(w + i));
+                store4<OutT>(P + i, v.x, v.y, v.z, v.w);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const long long i = base + (long long)u * PACK_THREADS + threadIdx.x;
+            if (i < n) {
+                const int k = (int)(i / Qp), q = (int)(i - (long long)k * Qp);
+                P[i] = cvt_out<OutT>(q < C ? __ldg(w + (long long)k * C + q) : 0.f);
+            }
+        }
+    }
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(PACK_THREADS)
+pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp) {
+    pdl_enter();
+    __shared__ __align__(16) float sw[PACK_SMEM_FLOATS];
+    pack_block<OutT>(w, P, K, C, RS, Qp, blockIdx.x, sw);
+}
+
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
 pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp) {
     pdl_enter();
-    const long long n = (long long)K * Qp;
-    for (long long i = (long long)blockIdx.x * PACK_THREADS + threadIdx.x; i < n; i += (long long)gridDim.x * PACK_THREADS) {
-        const int k = (int)(i / Qp), q = (int)(i - (long long)k * Qp);
-        P[i] = cvt_out<OutT>(q < C ? __ldg(w + (long long)k * C + q) : 0.f);
+    pack1x1_block<OutT>(w, P, K, C, Qp, blockIdx.x);
+}
+
+// ---- many layers in one launch ----------------------------------------------------------------
+// Block b belongs to the descriptor whose [block0, block0 + blocks) range holds it and does there
+// exactly what the single-layer kernels do.  A batch of small layers then costs one launch and
+// presents the memory system with one large stream of work.
+__global__ void __launch_bounds__(FT_THREADS)
+multi_transform_kernel(const __grid_constant__ XformBatch batch) {
+    pdl_enter();
+    __shared__ __align__(16) float smem[XF_SMEM_FLOATS];
+    // Persistent blocks walk the virtual block list with a grid stride: the grid is capped at a few
+    // blocks per SM so that the latency-critical execution kernels running beside this one always
+    // find room (shared memory, block slots) on every SM.
+    for (unsigned vb = blockIdx.x; vb < (unsigned)batch.total_blocks; vb += gridDim.x) {
+        int di = 0;
+        for (int i = 1; i < batch.n; ++i)
+            if (vb >= (unsigned)batch.d[i].block0) di = i;
+        const XformDesc& d = batch.d[di];
+        const unsigned lb = vb - (unsigned)d.block0;
+        const float* src = static_cast<const float*>(d.src);
+        switch (d.kind * 2 + d.bf16) {
+            case XF_PACK * 2: pack_block<float>(src, (float*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem); break;
+            case XF_PACK * 2 + 1: pack_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem); break;
+            case XF_PACK1X1 * 2: pack1x1_block<float>(src, (float*)d.dst, d.K, d.C, d.Qp, lb); break;
+            case XF_PACK1X1 * 2 + 1: pack1x1_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Qp, lb); break;
+            case XF_WINO2 * 2: filter_transform_block<2, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 2>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO4 * 2: filter_transform_block<4, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO6 * 2: filter_transform_block<6, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            default: break;
+        }
+        __syncthreads();                                        // the staging buffer is reused by the next virtual block
     }
+}
+
+int xform_blocks(const XformDesc& d) {
+    switch (d.kind) {
+        case XF_PACK: return (int)(((long long)d.K * pack_units_per_row(d.C, d.RS) + PACK_WARPS - 1) / PACK_WARPS);
+        case XF_PACK1X1: return (int)(((long long)d.K * d.Qp + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
+        default: return (int)(((long long)d.K * d.Cp + FT_THREADS * 2 - 1) / (FT_THREADS * 2));
+    }
+}
+
+nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st) {
+    for (int i0 = 0; i0 < n; i0 += XF_BATCH_MAX) {
+        XformBatch b;
+        b.n = std::min(XF_BATCH_MAX, n - i0);
+        int blocks = 0;
+        for (int i = 0; i < b.n; ++i) {
+            b.d[i] = descs[i0 + i];
+            NNV_REQUIRE(b.d[i].kind != XF_PACK || 8 * b.d[i].RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED,
+                        "filter window of %d taps is too large to repack", b.d[i].RS);
+            b.d[i].block0 = blocks;
+            blocks += xform_blocks(b.d[i]);
+        }
+        b.total_blocks = blocks;
+        NNV_LAUNCH((multi_transform_kernel), blocks, FT_THREADS, 0, st, b);
+        NNV_CUDA(cudaGetLastError());
+    }
+    return NNV_OK;
 }
 
 nnv_status_t launch_pack(bool bf16, const float* w, void* P, int K, int C, int RS, int Qp, cudaStream_t st) {
     if (RS == 1) {
         const long long n = (long long)K * Qp;
-        const unsigned grid = (unsigned)std::min<long long>((n + PACK_THREADS - 1) / PACK_THREADS, 148 * 16);
+        const unsigned grid = (unsigned)((n + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
         if (bf16) NNV_LAUNCH((pack1x1_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, Qp);
         else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp);
     } else {
-        NNV_REQUIRE(RS <= PACK_SMEM_FLOATS, NNV_ERR_UNSUPPORTED, "filter window of %d taps is too large to repack", RS);
-        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), K, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, C, RS, Qp);
-        else NNV_LAUNCH((pack_kernel<float>), K, PACK_THREADS, 0, st, w, (float*)P, C, RS, Qp);
+        NNV_REQUIRE(8 * RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED, "filter window of %d taps is too large to repack", RS);
+        const unsigned grid = (unsigned)(((long long)K * pack_units_per_row(C, RS) + PACK_WARPS - 1) / PACK_WARPS);
+        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, RS, Qp);
+        else NNV_LAUNCH((pack_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, RS, Qp);
     }
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;

@@ -36,7 +36,9 @@ class Model:
         self.h_weights = _pinned_bytes(np.ascontiguousarray(blob_u8))
         self.w_bytes = int(blob_u8.size)
         self.w_off, self.b_off = list(w_off), list(b_off)
-        self.streams = [torch.cuda.Stream() for _ in range(3)]
+        # copy, transform, execute; execution is latency-critical, so its blocks get scheduled ahead of
+        # the bandwidth-heavy transforms that run beside it
+        self.streams = [torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream(priority=-1)]
         L0, Ln = layers[0], layers[-1]
         self.h_input = torch.empty((1, L0["C"], L0["H"], L0["W"]), dtype=torch.float32).pin_memory()
         oh, ow = self.out_hw(len(layers) - 1)

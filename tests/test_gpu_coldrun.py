@@ -98,6 +98,47 @@ def test_resident_run_equals_cold_run_bitwise():
         assert all(t["h2d_bytes"] == 0 for t in tm)
 
 
+def test_depth_zero_and_grouped_transforms_give_the_same_bits():
+    """depth 0 (own buffers per layer, no staging waits; in the resident run the transforms become two
+    multi-layer launches) changes scheduling only."""
+    for layers, seed in ((wl.tiny_net(), 8), (wl.cfg2_resnet18(), 0)):
+        model, ws, bs, x = _model(layers, seed=seed)
+        ch = _choices(model, [nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+        y1, _ = model.cold_run(x, ch, depth=1)
+        y0, tm0 = model.cold_run(x, ch, depth=0, want_timings=True)
+        yr, tmr = model.resident_run(x, ch, depth=0, want_timings=True)
+        yg, _ = model.resident_run(x, ch, depth=0)            # graph replay path
+        assert np.array_equal(y1.view(np.uint32), y0.view(np.uint32))
+        assert np.array_equal(y1.view(np.uint32), yr.view(np.uint32))
+        assert np.array_equal(y1.view(np.uint32), yg.view(np.uint32))
+        groups = {(t["xform_start_ns"], t["xform_end_ns"]) for t in tmr if t["xform_bytes"]}
+        assert 1 <= len(groups) <= 3                           # three multi-layer launches at most
+
+
+def test_transform_all_equals_per_layer_transforms():
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers)
+    model.to_device()
+    for prefer, math in (([nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32),
+                         ([nb.VAR_WINO_F2, nb.VAR_IM2COL], nb.MATH_BF16), ([nb.VAR_WINO_F6, nb.VAR_IM2COL], nb.MATH_TF32)):
+        ch = _choices(model, prefer, math)
+        offs, total = nb.nnv_transformed_layout(model.plan, ch)
+        out = harness.dev_bytes(total)
+        nb.nnv_transform_all(model.plan, ch, model.d_weights, model.w_bytes, out, total, torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        for i, c in enumerate(ch):
+            if c is None or c[0] in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE):
+                continue
+            tb = nb.nnv_transformed_bytes(model.plan, i, c[0], c[1])
+            one = harness.dev_bytes(tb)
+            L = layers[i]
+            rb = 4 * L["K"] * L["C"] * L["R"] * L["S"]
+            nb.nnv_transform_weights(model.plan, i, c[0], c[1], model.d_weights[model.w_off[i]:model.w_off[i] + rb], one,
+                                     torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            assert torch.equal(out[offs[i]:offs[i] + tb], one[:tb]), (i, c)
+
+
 def test_cached_bypass_gives_identical_result():
     """Reading cached post-transform weights and skipping the transform changes nothing in the output."""
     layers = wl.tiny_net()
@@ -142,5 +183,5 @@ def test_arena_too_small_and_bad_depth():
     assert e.value.status == 4
     with pytest.raises(nb.NnvError) as e:
         nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
-                        model.arena, need, model.streams[0], model.streams[1], model.streams[2], 0)
+                        model.arena, need, model.streams[0], model.streams[1], model.streams[2], -1)
     assert e.value.status == 1
