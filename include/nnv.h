@@ -179,6 +179,50 @@ nnv_status_t nnv_filter_candidates(const nnv_plan_t* plan, int32_t layer,
 nnv_status_t nnv_select_kernels(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs,
                                 int32_t allow_cached, nnv_choice_t* out);
 
+/* ---- scheduling (integer, exact; host only) -------------------------------------------------- */
+
+/* Cold latency of one assignment (the paper's Eq. (1)-(2), Section 3.2): the end
+ * of the last execution when queue 0 runs every execution in layer order plus the
+ * preparation (read + transform, or read of cached weights) of the conv layers
+ * with queue_of = 0, each directly before its execution, and queues 1..n_little
+ * run the other preparations in layer order.  An execution starts when queue 0 is
+ * free, its preparation has ended and the layers in0/in1 have executed.  All
+ * arrays are host arrays with one entry per layer; prep entries and queue_of of
+ * pool layers are ignored.  prep_big_ns is the preparation time on queue 0,
+ * prep_little_ns on any other queue.  n_little in 1..64; a conv layer's queue
+ * outside 0..n_little -> NNV_ERR_INVALID_ARG. */
+nnv_status_t nnv_simulate(const nnv_plan_t* plan, const uint64_t* prep_little_ns, const uint64_t* prep_big_ns,
+                          const uint64_t* exec_ns, const int32_t* queue_of, int32_t n_little,
+                          uint64_t* t_cold_ns);
+
+/* The body of the paper's Algorithm 1 for one kernel combination.  B starts as
+ * the first conv layer.  The preparations outside B are dealt round-robin to the
+ * little queues and balanced: while the longest and shortest queue differ by more
+ * than eps_ns, every operation of the longest (longest first) that is shorter
+ * than half the current gap moves to the shortest.  While the longest little
+ * queue outlasts queue 0 (preparations of B + all executions) by more than
+ * eps_ns, the first layer outside B whose big + little preparation time is below
+ * that gap joins B and the little queues are dealt again.  Writes the queue of
+ * every layer's preparation (-1 for pool layers) and the resulting nnv_simulate
+ * value.  Same argument rules as nnv_simulate. */
+nnv_status_t nnv_schedule_queues(const nnv_plan_t* plan, const uint64_t* prep_little_ns,
+                                 const uint64_t* prep_big_ns, const uint64_t* exec_ns, int32_t n_little,
+                                 uint64_t eps_ns, int32_t* queue_of, uint64_t* t_cold_ns);
+
+/* The whole of Algorithm 1: over the combinations of each conv layer's
+ * nnv_filter_candidates survivors, the one whose nnv_schedule_queues latency is
+ * least.  An option's little-queue preparation time is its prep, its queue-0 time
+ * prep * big_pct / 100 (rounded down).  pool_ns: execution time of the pool
+ * layers (NULL = 0).  Up to combo_limit combinations are tried exhaustively (last
+ * layer varying fastest; a tie keeps the earlier one); beyond that, coordinate
+ * descent from nnv_select_kernels' choice: layer by layer, adopt the first
+ * survivor in (variant, math, cached) order that strictly lowers the latency,
+ * until a sweep changes nothing (at most 8 sweeps).  out / queue_of: one entry per
+ * layer (pool layers {-1,-1,0} / -1).  Errors as nnv_select_kernels. */
+nnv_status_t nnv_schedule(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                          const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
+                          uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns);
+
 /* ---- single operations (asynchronous on `stream`) ------------------------------------------ */
 
 /* Weights transformation (the paper's Section 2 stage, Figure 3): Winograd

@@ -14,15 +14,15 @@ All times are unsigned integers (nanoseconds); every comparison is exact.
 
 Reading of Algorithm 1 used here (the listing is ambiguous about which statements the outer while encloses
 and about the bookkeeping of s; this is the reading, in the listing's order):
-  line 3     B = {first conv layer}; queue 0 = p_1 and all executions.
-  line 12    the preparations not in B go to queues 1..M round-robin in layer order.
-  lines 13-19  while max - min of the little-queue totals exceeds eps: sort the longest queue's operations
+  start      B = {first conv layer}; queue 0 = p_1 and all executions.
+  spread     the preparations not in B go to queues 1..M round-robin in layer order.
+  balance    while max - min of the little-queue totals exceeds eps: sort the longest queue's operations
              by time, descending, and move to the shortest queue every operation whose time is below half
              the current gap, updating the totals after each move; stop when a pass moves nothing.
-  lines 6-11 while the longest little queue exceeds queue 0's total by more than eps: take the first layer
-             (in layer order) not in B with t_big + t_little < gap, add it to B, and redo lines 12-19;
-             stop when no layer qualifies.
-  line 21    T_cold = makespan of the resulting queues.
+  grow B     while the longest little queue exceeds queue 0's total by more than eps: take the first layer
+             (in layer order) not in B with t_big + t_little < gap, add it to B, and redo spread and
+             balance; stop when no layer qualifies.
+  result     T_cold = makespan of the resulting queues.
 Within queue 0 a layer's preparation sits directly before its execution; little queues keep layer order.
 """
 
@@ -62,7 +62,7 @@ def simulate(layers, prep_little, prep_big, exec_t, queue_of, n_little):
 
 
 def balance_little(items, n_little, eps):
-    """Lines 12-19: round-robin start, then move operations from the longest to the shortest queue.
+    """The spread and balance steps: round-robin start, then move operations from the longest to the shortest queue.
 
     items: list of (layer, time) in layer order.  Returns {layer: queue in 1..n_little}.
     """
@@ -127,7 +127,7 @@ def option_times(opt, big_pct):
 
 
 def search(layers, options, n_little, eps, big_pct=100, exhaustive_limit=4096, pool_t=None):
-    """The outer loop of Algorithm 1 (lines 2 and 22) over the filtered candidates.
+    """The outer loop of Algorithm 1 over the filtered candidates.
 
     options: per layer, the list of surviving (rank, prep, exec) options in rank order (None for non-conv
     layers; pool_t gives their execution time).  With at most `exhaustive_limit` combinations every one is

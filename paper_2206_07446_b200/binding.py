@@ -72,6 +72,9 @@ _SIGS = {
     "nnv_cached_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
     "nnv_filter_candidates": [_vp, _i32, _P(Cost), _i32, _i32, _P(Choice), _i32, _P(_i32)],
     "nnv_select_kernels": [_vp, _P(Cost), _i32, _i32, _P(Choice)],
+    "nnv_simulate": [_vp, _P(_u64), _P(_u64), _P(_u64), _P(_i32), _i32, _P(_u64)],
+    "nnv_schedule_queues": [_vp, _P(_u64), _P(_u64), _P(_u64), _i32, _u64, _P(_i32), _P(_u64)],
+    "nnv_schedule": [_vp, _P(Cost), _i32, _i32, _P(_u64), _i32, _u64, _i32, _u64, _P(Choice), _P(_i32), _P(_u64)],
     "nnv_transform_weights": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
     "nnv_transformed_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
     "nnv_transform_all": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp],
@@ -235,6 +238,41 @@ def nnv_select_kernels(plan, costs, allow_cached):
     out = (Choice * plan.n)()
     _check(_lib.nnv_select_kernels(plan.handle, _costs_array(costs), len(costs), int(allow_cached), out))
     return [None if out[i].variant < 0 else (out[i].variant, out[i].math, out[i].cached) for i in range(plan.n)]
+
+
+def _u64_array(plan, values):
+    if len(values) != plan.n:
+        raise ValueError("one entry per layer expected")
+    return (_u64 * plan.n)(*[int(v) for v in values])
+
+
+def nnv_simulate(plan, prep_little_ns, prep_big_ns, exec_ns, queue_of, n_little):
+    if len(queue_of) != plan.n:
+        raise ValueError("one entry per layer expected")
+    t = _u64(0)
+    _check(_lib.nnv_simulate(plan.handle, _u64_array(plan, prep_little_ns), _u64_array(plan, prep_big_ns),
+                             _u64_array(plan, exec_ns), (_i32 * plan.n)(*[int(q) for q in queue_of]), n_little,
+                             ctypes.byref(t)))
+    return int(t.value)
+
+
+def nnv_schedule_queues(plan, prep_little_ns, prep_big_ns, exec_ns, n_little, eps_ns=0):
+    q = (_i32 * plan.n)()
+    t = _u64(0)
+    _check(_lib.nnv_schedule_queues(plan.handle, _u64_array(plan, prep_little_ns), _u64_array(plan, prep_big_ns),
+                                    _u64_array(plan, exec_ns), n_little, int(eps_ns), q, ctypes.byref(t)))
+    return [int(v) for v in q], int(t.value)
+
+
+def nnv_schedule(plan, costs, allow_cached, n_little, eps_ns=0, big_pct=100, combo_limit=4096, pool_ns=None):
+    out = (Choice * plan.n)()
+    q = (_i32 * plan.n)()
+    t = _u64(0)
+    pool = _u64_array(plan, pool_ns) if pool_ns is not None else None
+    _check(_lib.nnv_schedule(plan.handle, _costs_array(costs), len(costs), int(allow_cached), pool, n_little,
+                             int(eps_ns), int(big_pct), int(combo_limit), out, q, ctypes.byref(t)))
+    choices = [None if out[i].variant < 0 else (out[i].variant, out[i].math, out[i].cached) for i in range(plan.n)]
+    return choices, [int(v) for v in q], int(t.value)
 
 
 def nnv_transform_weights(plan, layer, variant, math, d_raw, d_out, stream=None):

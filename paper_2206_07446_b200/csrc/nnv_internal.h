@@ -151,6 +151,15 @@ uint64_t exec_ws_bytes(const nnv_plan& p, int layer, int variant, int math);
 uint64_t raw_weight_bytes(const nnv_layer_desc_t& L);
 uint64_t exec_flops(const nnv_plan& p, int layer, int variant);
 nnv_status_t check_choice(const nnv_plan& p, int layer, int variant, int math);
+// One way to run a layer: a kernel (variant, math), raw or cached weights, and its integer costs.
+struct Option {
+    int variant, math, cached;
+    uint64_t prep, exec;
+};
+// Options of `layer` from the cost table, and the candidate filter over them (rank order out).
+nnv_status_t gather_options(const nnv_plan& p, int layer, const nnv_cost_t* costs, int n_costs, int allow_cached,
+                            std::vector<Option>* opts);
+void pareto(const std::vector<Option>& in, std::vector<Option>* out);
 nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int depth, ArenaLayout* out);
 
 // ---- kernel launchers (device TUs) ----------------------------------------------------------

@@ -177,17 +177,13 @@ nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int de
 }
 
 // ---- selection ------------------------------------------------------------------------------
-struct Option {
-    int variant, math, cached;
-    uint64_t prep, exec;
-};
 static inline bool rank_less(const Option& a, const Option& b) {
     if (a.variant != b.variant) return a.variant < b.variant;
     if (a.math != b.math) return a.math < b.math;
     return a.cached < b.cached;
 }
 
-static nnv_status_t gather_options(const nnv_plan& p, int layer, const nnv_cost_t* costs, int n_costs,
+nnv_status_t gather_options(const nnv_plan& p, int layer, const nnv_cost_t* costs, int n_costs,
                                    int allow_cached, std::vector<Option>* opts) {
     for (int i = 0; i < n_costs; ++i) {
         const nnv_cost_t& c = costs[i];
@@ -202,7 +198,7 @@ static nnv_status_t gather_options(const nnv_plan& p, int layer, const nnv_cost_
     return NNV_OK;
 }
 
-static void pareto(const std::vector<Option>& in, std::vector<Option>* out) {
+void pareto(const std::vector<Option>& in, std::vector<Option>* out) {
     for (size_t i = 0; i < in.size(); ++i) {
         const Option& o = in[i];
         bool drop = false;
