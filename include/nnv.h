@@ -189,7 +189,7 @@ nnv_status_t nnv_select_kernels(const nnv_plan_t* plan, const nnv_cost_t* costs,
  * free, its preparation has ended and the layers in0/in1 have executed.  All
  * arrays are host arrays with one entry per layer; prep entries and queue_of of
  * pool layers are ignored.  prep_big_ns is the preparation time on queue 0,
- * prep_little_ns on any other queue.  n_little in 1..64; a conv layer's queue
+ * prep_little_ns on any other queue.  n_little in 1..NNV_MAX_QUEUES; a conv layer's queue
  * outside 0..n_little -> NNV_ERR_INVALID_ARG. */
 nnv_status_t nnv_simulate(const nnv_plan_t* plan, const uint64_t* prep_little_ns, const uint64_t* prep_big_ns,
                           const uint64_t* exec_ns, const int32_t* queue_of, int32_t n_little,
@@ -314,6 +314,27 @@ nnv_status_t nnv_cold_run(nnv_plan_t* plan, const nnv_choice_t* choices,
                           void* d_arena, uint64_t arena_bytes,
                           void* s_copy, void* s_xform, void* s_exec,
                           int32_t depth, nnv_timing_t* timings);
+
+/* One cold inference on the queues Algorithm 1 produced.  queue_of (one entry
+ * per layer, as written by nnv_schedule / nnv_schedule_queues) names the queue of
+ * every conv layer's bundled preparation -- the copy of its raw (or cached)
+ * weights followed by the transform, if any, on ONE stream: queue 0 is the
+ * execution stream streams[0], where the preparation sits directly before the
+ * layer's execution (the paper's big cores taking over preparation work); queue
+ * j >= 1 is streams[j] (its little cores), which runs its preparations in layer
+ * order and never waits for execution.  streams: n_little + 1 distinct CUDA
+ * streams, n_little in 1..NNV_MAX_QUEUES.  The arena is the depth-0 one
+ * (nnv_arena_bytes with depth 0).  Other arguments, results and errors as
+ * nnv_cold_run; the output is bit-identical to nnv_cold_run's for the same
+ * choices.  Synchronises every stream before returning. */
+#define NNV_MAX_QUEUES 16
+nnv_status_t nnv_cold_run_queues(nnv_plan_t* plan, const nnv_choice_t* choices,
+                                 const int32_t* queue_of, int32_t n_little,
+                                 const void* h_weights, uint64_t w_bytes,
+                                 const void* h_cached, uint64_t c_bytes,
+                                 const float* h_input, float* h_output,
+                                 void* d_arena, uint64_t arena_bytes,
+                                 void* const* streams, nnv_timing_t* timings);
 
 /* The same pass with the read stage already done (the paper's Tables 1 and 2
  * separate reading from transformation and execution; this call measures the

@@ -84,6 +84,7 @@ _SIGS = {
     "nnv_chw_to_hwc": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_hwc_to_chw": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_cold_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing)],
+    "nnv_cold_run_queues": [_vp, _P(Choice), _P(_i32), _i32, _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _P(_vp), _P(Timing)],
     "nnv_resident_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _i32, _P(Timing)],
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
@@ -325,6 +326,20 @@ def nnv_cold_run(plan, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, 
     _check(_lib.nnv_cold_run(plan.handle, _choices_array(plan, choices), _ptr(h_weights), int(w_bytes),
                              _ptr(h_cached), int(c_bytes), _ptr(h_input), _ptr(h_output), _ptr(d_arena),
                              int(arena_bytes), _stream(s_copy), _stream(s_xform), _stream(s_exec), int(depth), tarr))
+    return _timings_list(tarr)
+
+
+def nnv_cold_run_queues(plan, choices, queue_of, n_little, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output,
+                        d_arena, arena_bytes, streams, want_timings=False):
+    """streams: n_little + 1 streams, [0] = execution.  Returns per-layer timing dicts when want_timings."""
+    if len(queue_of) != plan.n or len(streams) != n_little + 1:
+        raise ValueError("queue_of needs one entry per layer and streams n_little + 1 entries")
+    tarr = (Timing * plan.n)() if want_timings else None
+    sarr = (_vp * (n_little + 1))(*[_stream(s) for s in streams])
+    _check(_lib.nnv_cold_run_queues(plan.handle, _choices_array(plan, choices),
+                                    (_i32 * plan.n)(*[int(q) for q in queue_of]), int(n_little), _ptr(h_weights),
+                                    int(w_bytes), _ptr(h_cached), int(c_bytes), _ptr(h_input), _ptr(h_output),
+                                    _ptr(d_arena), int(arena_bytes), sarr, tarr))
     return _timings_list(tarr)
 
 

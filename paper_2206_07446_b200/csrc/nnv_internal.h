@@ -110,9 +110,10 @@ struct GraphKey {
     uint64_t w_bytes = 0;
     int depth = 0;
     bool resident = false;
+    std::vector<int32_t> queues;          // preparation queue per layer (scheduled runs), else empty
     bool operator==(const GraphKey& o) const {
         if (ptrs != o.ptrs || w_bytes != o.w_bytes || depth != o.depth || resident != o.resident ||
-            choices.size() != o.choices.size())
+            queues != o.queues || choices.size() != o.choices.size())
             return false;
         for (size_t i = 0; i < choices.size(); ++i)
             if (choices[i].variant != o.choices[i].variant || choices[i].math != o.choices[i].math ||

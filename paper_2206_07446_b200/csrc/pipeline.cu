@@ -13,9 +13,10 @@ nnv_status_t do_pool(const nnv_plan& p, int layer, const void* d_in, void* d_out
 
 static nnv_status_t ensure_events(nnv_plan& p, bool timing) {
     const size_t n = p.layers.size();
-    if (p.ev.size() != 3 * n + 6) {                                // + fork, join(copy), join(transform), 3 transform groups
-        p.ev.resize(3 * n + 6, nullptr);
-        for (size_t i = 0; i < 3 * n + 6; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming));
+    const size_t ne = 3 * n + 6 + NNV_MAX_QUEUES;                   // + fork, join(copy), join(transform), 3 transform groups, queue joins
+    if (p.ev.size() != ne) {
+        p.ev.resize(ne, nullptr);
+        for (size_t i = 0; i < ne; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming));
     }
     if (timing && p.tev.size() != 6 * n + 7) {                     // + start / end of the 3 transform groups
         p.tev.resize(6 * n + 7, nullptr);
@@ -36,8 +37,10 @@ namespace nnv {
 static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const void* weights, uint64_t w_bytes,
                               const void* cached_blob, uint64_t c_bytes, const float* input, float* output,
                               void* d_arena, uint64_t arena_bytes, cudaStream_t s_copy, cudaStream_t s_xform,
-                              cudaStream_t s_exec, int depth, nnv_timing_t* timings, bool resident) {
+                              cudaStream_t s_exec, int depth, nnv_timing_t* timings, bool resident,
+                              const int32_t* queue_of = nullptr, const cudaStream_t* s_prep = nullptr, int n_little = 0) {
     const int n = (int)p->layers.size();
+    const bool queued = queue_of != nullptr;        // preparations follow a schedule: queue 0 = s_exec, j = s_prep[j-1]
     ArenaLayout A;
     NNV_TRY(layout_arena(*p, choices, depth, &A));
     NNV_REQUIRE(arena_bytes >= A.total, NNV_ERR_WORKSPACE_TOO_SMALL, "arena needs %llu bytes, got %llu",
@@ -74,8 +77,12 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     auto enqueue = [&]() -> nnv_status_t {
     if (tm) NNV_CUDA(cudaEventRecord(p->tev[0], s_exec));
     NNV_CUDA(cudaEventRecord(p->ev[3 * n], s_exec));
-    if (!resident) NNV_CUDA(cudaStreamWaitEvent(s_copy, p->ev[3 * n], 0));
-    NNV_CUDA(cudaStreamWaitEvent(s_xform, p->ev[3 * n], 0));
+    if (queued) {
+        for (int j = 0; j < n_little; ++j) NNV_CUDA(cudaStreamWaitEvent(s_prep[j], p->ev[3 * n], 0));
+    } else {
+        if (!resident) NNV_CUDA(cudaStreamWaitEvent(s_copy, p->ev[3 * n], 0));
+        NNV_CUDA(cudaStreamWaitEvent(s_xform, p->ev[3 * n], 0));
+    }
 
     // model input: NCHW -> device NHWC, on the execution stream
     const nnv_layer_desc_t& L0 = p->layers[0];
@@ -143,7 +150,32 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         cudaEvent_t ready = nullptr;
         uint64_t copied = 0;
 
-        if (resident) {
+        if (queued) {
+            // the layer's bundled preparation (read, then transform) on the queue the schedule gave it
+            cudaStream_t ps = queue_of[i] == 0 ? s_exec : s_prep[queue_of[i] - 1];
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), ps));
+            if (cached) {
+                NNV_CUDA(cudaMemcpyAsync((void*)xf, (const uint8_t*)cached_blob + coff[i], tbytes, cudaMemcpyHostToDevice, ps));
+                copied += tbytes;
+            } else {
+                NNV_CUDA(cudaMemcpyAsync((void*)raw, (const uint8_t*)weights + L.w_off, rbytes, cudaMemcpyHostToDevice, ps));
+                copied += rbytes;
+            }
+            if (L.has_bias) {
+                NNV_CUDA(cudaMemcpyAsync((void*)bias, (const uint8_t*)weights + L.b_off, 4ull * L.K, cudaMemcpyHostToDevice, ps));
+                copied += 4ull * L.K;
+            }
+            if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), ps));
+            if (has_xf && !cached) {
+                if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), ps));
+                NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, (void*)xf, ps));
+                if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), ps));
+            }
+            if (ps != s_exec) {
+                NNV_CUDA(cudaEventRecord(EV(i, 1), ps));
+                ready = EV(i, 1);
+            }
+        } else if (resident) {
             raw = (const uint8_t*)weights + L.w_off;
             bias = (const uint8_t*)weights + L.b_off;
             if (cached) xf = (const uint8_t*)cached_blob + coff[i];
@@ -168,7 +200,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         }
 
         // transform
-        if (grouped) {
+        if (queued) {
+            // done above, inside the bundled preparation
+        } else if (grouped) {
             if (has_xf && !cached) ready = group_event[i];
         } else if (has_xf && !cached) {
             if (ready) NNV_CUDA(cudaStreamWaitEvent(s_xform, ready, 0));
@@ -202,12 +236,19 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     float* out_chw = resident ? output : (float*)(base + A.out_chw);
     NNV_TRY(launch_hwc_to_chw((const float*)(base + A.act_off[n - 1]), out_chw, Ln.K, gn.OH, gn.OW, s_exec));
     if (!resident) NNV_CUDA(cudaMemcpyAsync(output, out_chw, 4ull * gn.P * Ln.K, cudaMemcpyDeviceToHost, s_exec));
-    if (!resident) {
-        NNV_CUDA(cudaEventRecord(p->ev[3 * n + 1], s_copy));
-        NNV_CUDA(cudaStreamWaitEvent(s_exec, p->ev[3 * n + 1], 0));
+    if (queued) {
+        for (int j = 0; j < n_little; ++j) {
+            NNV_CUDA(cudaEventRecord(p->ev[3 * n + 6 + j], s_prep[j]));
+            NNV_CUDA(cudaStreamWaitEvent(s_exec, p->ev[3 * n + 6 + j], 0));
+        }
+    } else {
+        if (!resident) {
+            NNV_CUDA(cudaEventRecord(p->ev[3 * n + 1], s_copy));
+            NNV_CUDA(cudaStreamWaitEvent(s_exec, p->ev[3 * n + 1], 0));
+        }
+        NNV_CUDA(cudaEventRecord(p->ev[3 * n + 2], s_xform));
+        NNV_CUDA(cudaStreamWaitEvent(s_exec, p->ev[3 * n + 2], 0));
     }
-    NNV_CUDA(cudaEventRecord(p->ev[3 * n + 2], s_xform));
-    NNV_CUDA(cudaStreamWaitEvent(s_exec, p->ev[3 * n + 2], 0));
     NNV_TRY(enqueue_status_read(p->h_status, s_exec));
     return NNV_OK;
     };  // enqueue
@@ -219,6 +260,10 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     key.choices.assign(choices, choices + n);
     key.ptrs = {weights, cached_blob, input, output, d_arena};
     key.w_bytes = w_bytes; key.depth = depth; key.resident = resident;
+    if (queued) {
+        key.queues.assign(queue_of, queue_of + n);
+        key.queues.push_back(n_little);
+    }
     CachedGraph* cg = nullptr;
     if (!tm && p->opts.use_graphs) {
         for (CachedGraph& g : p->graphs)
@@ -264,7 +309,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             NNV_TRY(stamp(TEV(i, 4), &timings[i].exec_start_ns));
             NNV_TRY(stamp(TEV(i, 5), &timings[i].exec_end_ns));
             if (L.op != NNV_OP_CONV) continue;
-            if (!resident) {
+            if (!resident || queued) {
                 NNV_TRY(stamp(TEV(i, 0), &timings[i].h2d_start_ns));
                 NNV_TRY(stamp(TEV(i, 1), &timings[i].h2d_end_ns));
             }
@@ -302,6 +347,29 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
                 "the three streams must be distinct");
     return run_model(p, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena, arena_bytes,
                      (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings, false);
+}
+
+nnv_status_t nnv_cold_run_queues(nnv_plan_t* p, const nnv_choice_t* choices, const int32_t* queue_of, int32_t n_little,
+                                 const void* h_weights, uint64_t w_bytes, const void* h_cached, uint64_t c_bytes,
+                                 const float* h_input, float* h_output, void* d_arena, uint64_t arena_bytes,
+                                 void* const* streams, nnv_timing_t* timings) {
+    NNV_REQUIRE(p && choices && queue_of && h_weights && h_input && h_output && d_arena && streams, NNV_ERR_INVALID_ARG,
+                "null argument");
+    NNV_REQUIRE(n_little >= 1 && n_little <= NNV_MAX_QUEUES, NNV_ERR_INVALID_ARG, "n_little %d outside 1..%d", n_little,
+                NNV_MAX_QUEUES);
+    NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
+    cudaStream_t prep[NNV_MAX_QUEUES];
+    for (int j = 0; j <= n_little; ++j) {
+        for (int k = 0; k < j; ++k)
+            NNV_REQUIRE(streams[j] != streams[k], NNV_ERR_INVALID_ARG, "the streams must be distinct");
+        if (j) prep[j - 1] = (cudaStream_t)streams[j];
+    }
+    for (int i = 0; i < (int)p->layers.size(); ++i)
+        if (p->layers[i].op == NNV_OP_CONV)
+            NNV_REQUIRE(queue_of[i] >= 0 && queue_of[i] <= n_little, NNV_ERR_INVALID_ARG,
+                        "layer %d: queue %d outside 0..%d", i, queue_of[i], n_little);
+    return run_model(p, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena, arena_bytes,
+                     nullptr, nullptr, (cudaStream_t)streams[0], 0, timings, false, queue_of, prep, n_little);
 }
 
 nnv_status_t nnv_resident_run(nnv_plan_t* p, const nnv_choice_t* choices, const void* d_weights, uint64_t w_bytes,

@@ -200,7 +200,7 @@ extern "C" {
 nnv_status_t nnv_simulate(const nnv_plan_t* p, const uint64_t* prep_little_ns, const uint64_t* prep_big_ns,
                           const uint64_t* exec_ns, const int32_t* queue_of, int32_t n_little, uint64_t* t_cold_ns) {
     NNV_REQUIRE(p && prep_little_ns && prep_big_ns && exec_ns && queue_of && t_cold_ns, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(n_little >= 1 && n_little <= 64, NNV_ERR_INVALID_ARG, "n_little %d outside 1..64", n_little);
+    NNV_REQUIRE(n_little >= 1 && n_little <= NNV_MAX_QUEUES, NNV_ERR_INVALID_ARG, "n_little %d outside 1..%d", n_little, NNV_MAX_QUEUES);
     NNV_TRY(check_queues(*p, queue_of, n_little));
     *t_cold_ns = makespan(*p, prep_little_ns, prep_big_ns, exec_ns, queue_of, n_little);
     return NNV_OK;
@@ -210,7 +210,7 @@ nnv_status_t nnv_schedule_queues(const nnv_plan_t* p, const uint64_t* prep_littl
                                  const uint64_t* exec_ns, int32_t n_little, uint64_t eps_ns, int32_t* queue_of,
                                  uint64_t* t_cold_ns) {
     NNV_REQUIRE(p && prep_little_ns && prep_big_ns && exec_ns && queue_of && t_cold_ns, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(n_little >= 1 && n_little <= 64, NNV_ERR_INVALID_ARG, "n_little %d outside 1..64", n_little);
+    NNV_REQUIRE(n_little >= 1 && n_little <= NNV_MAX_QUEUES, NNV_ERR_INVALID_ARG, "n_little %d outside 1..%d", n_little, NNV_MAX_QUEUES);
     std::vector<int32_t> q;
     *t_cold_ns = schedule_queues(*p, prep_little_ns, prep_big_ns, exec_ns, n_little, eps_ns, &q);
     std::copy(q.begin(), q.end(), queue_of);
@@ -221,7 +221,7 @@ nnv_status_t nnv_schedule(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t 
                           const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
                           uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns) {
     NNV_REQUIRE(p && costs && out && queue_of && t_cold_ns, NNV_ERR_INVALID_ARG, "null argument");
-    NNV_REQUIRE(n_little >= 1 && n_little <= 64, NNV_ERR_INVALID_ARG, "n_little %d outside 1..64", n_little);
+    NNV_REQUIRE(n_little >= 1 && n_little <= NNV_MAX_QUEUES, NNV_ERR_INVALID_ARG, "n_little %d outside 1..%d", n_little, NNV_MAX_QUEUES);
     NNV_REQUIRE(big_pct >= 0 && big_pct <= 1000, NNV_ERR_INVALID_ARG, "big_pct %d outside 0..1000", big_pct);
     const int n = (int)p->layers.size();
     std::vector<std::vector<Option>> options(n);

@@ -111,6 +111,56 @@ class Model:
                              self.streams[0], self.streams[1], self.streams[2], depth, want_timings)
         return self.h_output.numpy().copy(), tm
 
+    def prep_streams(self, n_little):
+        """Execution stream + n_little preparation streams for nnv_cold_run_queues (created once)."""
+        extra = getattr(self, "_prep_streams", [])
+        while len(extra) < n_little:
+            extra.append(torch.cuda.Stream())
+        self._prep_streams = extra
+        return [self.streams[2]] + extra[:n_little]
+
+    def cold_run_queues(self, x_nchw, choices, queue_of, n_little, want_timings=False, poison=True):
+        """One cold inference on the queues Algorithm 1 produced (nnv_cold_run_queues)."""
+        self.h_input.copy_(torch.from_numpy(np.ascontiguousarray(x_nchw, dtype=np.float32)).reshape(self.h_input.shape))
+        need = self.ensure_arena(choices, 0)
+        if poison:
+            self.arena.fill_(0xFF)
+            torch.cuda.synchronize()
+        tm = nb.nnv_cold_run_queues(self.plan, choices, queue_of, n_little, self.h_weights, self.w_bytes,
+                                    self.h_cached, self.c_bytes, self.h_input, self.h_output, self.arena, need,
+                                    self.prep_streams(n_little), want_timings)
+        return self.h_output.numpy().copy(), tm
+
+    def schedule(self, x_nchw, costs, n_little, allow_cached=1, rounds=2, eps_pct=1, big_pct=100, combo_limit=4096):
+        """Algorithm 1 with its calibration step: schedule from the cost table, run the schedule once with
+        per-operation timings, overwrite the chosen kernels' costs with what they took while the other
+        queues were busy, and schedule again (`rounds` times).  eps is eps_pct percent of the summed
+        execution time of the per-layer choice.  Returns (choices, queue_of, predicted ns, costs used)."""
+        costs = [dict(c) for c in costs]
+        base = nb.nnv_select_kernels(self.plan, costs, allow_cached)
+        rows = {(c["layer"], c["variant"], c["math"]): c for c in costs}
+        eps = sum(rows[(i,) + ch[:2]]["exec_ns"] for i, ch in enumerate(base) if ch is not None) * eps_pct // 100
+        out = None
+        for r in range(rounds + 1):
+            out = nb.nnv_schedule(self.plan, costs, allow_cached, n_little, eps, big_pct, combo_limit)
+            if r == rounds:
+                break
+            choices, queue_of, _ = out
+            if any(c is not None and c[2] for c in choices):
+                self.build_cached_blob(choices)
+            _, tm = self.cold_run_queues(x_nchw, choices, queue_of, n_little, want_timings=True, poison=False)
+            for i, ch in enumerate(choices):
+                if ch is None:
+                    continue
+                row, t = rows[(i,) + ch[:2]], tm[i]
+                row["exec_ns"] = t["exec_end_ns"] - t["exec_start_ns"]
+                if ch[2]:
+                    row["h2d_cached_ns"] = t["h2d_end_ns"] - t["h2d_start_ns"]
+                else:
+                    row["h2d_raw_ns"] = t["h2d_end_ns"] - t["h2d_start_ns"]
+                    row["xform_ns"] = t["xform_end_ns"] - t["xform_start_ns"]
+        return out[0], out[1], out[2], costs
+
     def to_device(self):
         """Device copies of the weight blob, the cached blob (if built) and I/O buffers for nnv_resident_run."""
         self.d_weights = dev_bytes(self.w_bytes, fill=None)

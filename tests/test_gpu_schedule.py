@@ -1,0 +1,115 @@
+"""GPU: cold runs on the queues of Algorithm 1 (nnv_cold_run_queues): same bits as the three-stream run for
+every queue assignment, stamps that obey the queue model, and the profile -> schedule -> run loop."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from oracle import model as omodel
+from oracle import scheduler as osch
+from oracle import selection as osel
+from paper_2206_07446_b200 import binding as nb
+from paper_2206_07446_b200 import harness
+from gpu_util import rel_l2
+
+pytestmark = pytest.mark.gpu
+
+PREFER = [nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL]
+
+
+def _model(layers, seed=0, use_graphs=1):
+    ws, bs = wl.make_weights(layers, seed=seed)
+    x = wl.make_input(layers, seed=seed)
+    return harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=use_graphs), ws, bs, x
+
+
+@pytest.mark.parametrize("use_graphs", [0, 1])
+def test_queue_runs_give_the_bits_of_the_three_stream_run(use_graphs):
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers, use_graphs=use_graphs)
+    ch = model.default_choices(prefer=PREFER, math=nb.MATH_TF32)
+    want, _ = model.cold_run(x, ch, depth=2)
+    conv = [i for i, L in enumerate(layers) if L["op"] == wl.OP_CONV]
+    rng = np.random.default_rng(1)
+    for n_little in (1, 2, 4):
+        assigns = [
+            [0 if L["op"] == wl.OP_CONV else -1 for L in layers],                         # everything on queue 0
+            [1 + conv.index(i) % n_little if i in conv else -1 for i in range(len(layers))],
+            [int(rng.integers(0, n_little + 1)) if i in conv else -1 for i in range(len(layers))],
+        ]
+        for q in assigns:
+            for rep in range(2):                # the second call replays the recorded graph when graphs are on
+                y, _ = model.cold_run_queues(x, ch, q, n_little)
+                assert np.array_equal(y.view(np.uint32), want.view(np.uint32)), (n_little, q, rep)
+
+
+def test_queue_run_with_cached_choices_and_stamps():
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers, seed=2)
+    ch = model.default_choices(prefer=PREFER, math=nb.MATH_TF32)
+    ch = [c if c is None or not osel.has_transform(c[0]) or i % 3 else (c[0], c[1], 1) for i, c in enumerate(ch)]
+    model.build_cached_blob(ch)
+    want, _ = model.cold_run(x, ch, depth=3)
+    conv = [i for i, L in enumerate(layers) if L["op"] == wl.OP_CONV]
+    n_little = 2
+    q = [(-1 if i not in conv else (0 if conv.index(i) % 3 == 0 else 1 + conv.index(i) % 2)) for i in range(len(layers))]
+    y, tm = model.cold_run_queues(x, ch, q, n_little, want_timings=True)
+    assert np.array_equal(y.view(np.uint32), want.view(np.uint32))
+    slack = 2000
+    last_end = {}
+    for i in conv:
+        t = tm[i]
+        prep_end = t["xform_end_ns"] if t["xform_bytes"] else t["h2d_end_ns"]
+        assert t["exec_start_ns"] + slack >= prep_end                       # execution after its preparation
+        if t["xform_bytes"]:
+            assert t["xform_start_ns"] + slack >= t["h2d_end_ns"]           # bundled: read, then transform
+        for src in (layers[i]["in0"], layers[i]["in1"]):
+            if src >= 0:
+                assert t["exec_start_ns"] + slack >= tm[src]["exec_end_ns"]
+        if q[i] in last_end:                                                # one operation per queue at a time
+            assert t["h2d_start_ns"] + slack >= last_end[q[i]]
+        last_end[q[i]] = prep_end if q[i] else t["exec_end_ns"]
+        if q[i] == 0 and layers[i]["in0"] >= 0:                             # queue-0 preparations sit between executions
+            assert t["h2d_start_ns"] + slack >= tm[i - 1]["exec_end_ns"]
+        assert (t["choice"][2] == 1) == bool(ch[i][2])
+
+
+def test_profile_schedule_run():
+    """Profile, run Algorithm 1 (library == oracle on the measured table), execute its queues: the output
+    matches the oracle model and the three-stream run of the same choices bit for bit."""
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=5)
+    costs = model.profile(x, reps=3)
+    for n_little, big_pct in ((1, 100), (2, 80)):
+        got = nb.nnv_schedule(model.plan, costs, 1, n_little, 0, big_pct, 4096)
+        options = [None if L["op"] != wl.OP_CONV else
+                   osel.pareto_filter(osel.options_from_costs([c for c in costs if c["layer"] == i], 1))
+                   for i, L in enumerate(layers)]
+        want = osch.search(layers, options, n_little, 0, big_pct=big_pct, exhaustive_limit=4096)
+        assert got[0] == want[0] and got[1] == want[1] and got[2] == want[2]
+    choices, queue_of, t_pred, used = model.schedule(x, costs, 2, rounds=2)
+    assert t_pred > 0 and len(used) == len(costs)
+    if any(c is not None and c[2] for c in choices):
+        model.build_cached_blob(choices)
+    y, _ = model.cold_run_queues(x, choices, queue_of, 2)
+    y3, _ = model.cold_run(x, choices, depth=0)
+    assert np.array_equal(y.view(np.uint32), y3.view(np.uint32))
+    acts = omodel.run_model(layers, ws, bs, x)
+    assert rel_l2(y[0], acts[-1]) <= 2e-2
+
+
+def test_queue_run_argument_errors():
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=1)
+    ch = model.default_choices(prefer=PREFER, math=nb.MATH_TF32)
+    q = [0 if L["op"] == wl.OP_CONV else -1 for L in layers]
+    need = model.ensure_arena(ch, 0)
+    st = model.prep_streams(2)
+    args = (model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output, model.arena)
+    with pytest.raises(nb.NnvError):                                        # queue index outside 0..n_little
+        nb.nnv_cold_run_queues(model.plan, ch, [3 if v == 0 else v for v in q], 2, *args, need, st)
+    with pytest.raises(nb.NnvError):                                        # the same stream twice
+        nb.nnv_cold_run_queues(model.plan, ch, q, 2, *args, need, [st[0], st[1], st[1]])
+    with pytest.raises(nb.NnvError):                                        # arena too small
+        nb.nnv_cold_run_queues(model.plan, ch, q, 2, *args, need - 256, st)
+    y, _ = model.cold_run_queues(x, ch, q, 2)                               # the plan still runs afterwards
+    assert np.isfinite(y).all()
