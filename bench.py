@@ -7,6 +7,8 @@ profiled cost table, then for every conv layer the weights are read (host -> HBM
 
   value   cold ms with weights and input already resident in HBM (transform + exec only)
   e2e     cold ms through nnv_cold_run with pinned HOST weights / input / output (H2D, D2H inside)
+  algorithm1  the same end-to-end step on the queues the paper's Algorithm 1 produces (nnv_schedule +
+          calibration, nnv_cold_run_queues), reported beside e2e
 
 Run `python bench.py` (1 GPU) or under torch.distributed.run with --gpus N (independent replicas,
 the path does not shard).  `--impl reference` times the CPU oracle instead.
@@ -44,6 +46,7 @@ def parse():
     ap.add_argument("--cpu-passes", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="enqueue every call eagerly instead of replaying a recorded CUDA graph")
+    ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run reported beside e2e (0 = skip)")
     ap.add_argument("--save-costs", default=None, help="write the profiled cost table (JSON) to this file")
     ap.add_argument("--load-costs", default=None, help="use a cost table saved earlier instead of profiling (e.g. under a profiler)")
     return ap.parse_args()
@@ -297,6 +300,45 @@ def run_ours(args):
     e2e = reduce_max(sum(cold_ms) / len(cold_ms))
     e2e_wall = reduce_max(1e3 * sum(wall) / len(wall))
 
+    # ---- Algorithm 1: schedule (with calibration under overlap), then the same end-to-end step on its queues
+    alg1 = None
+    if args.queues > 0:
+        ch_s, q_s, t_pred, _ = model.schedule(x, costs, args.queues, allow_cached=1, rounds=2, eps_pct=1,
+                                              combo_limit=4096)
+        if any(c is not None and c[2] for c in ch_s):
+            model.build_cached_blob(ch_s)
+        need_s = model.ensure_arena(ch_s, 0)
+        st_s = model.prep_streams(args.queues)
+
+        def step_sched(k, timed):
+            flush.fill_(k & 0xFF)
+            torch.cuda.synchronize()
+            if timed:
+                ev0[k].record(s_exec)
+                for s in st_s[1:]:
+                    s.wait_event(ev0[k])
+            nb.nnv_cold_run_queues(model.plan, ch_s, q_s, args.queues, model.h_weights, model.w_bytes, model.h_cached,
+                                   model.c_bytes, model.h_input, model.h_output, model.arena, need_s, st_s)
+            if timed:
+                ev1[k].record(s_exec)
+
+        for k in range(args.warmup):
+            step_sched(k, False)
+        barrier()
+        for k in range(args.steps):
+            step_sched(k, True)
+        barrier()
+        sched_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
+        alg1 = {"n_little": args.queues, "e2e_ms": reduce_max(sum(sched_ms) / len(sched_ms)),
+                "predicted_ms": t_pred / 1e6, "calibration_factors": getattr(model, "calibration", None),
+                "preps_on_queue0": sum(1 for q in q_s if q == 0),
+                "choices_differing_from_per_layer_argmin": sum(1 for a, b in zip(ch_s, choices_cold) if a != b),
+                "parity_rel_l2_end_to_end": None}
+        y_s = model.h_output.numpy().copy()
+        if any(c is not None and c[2] for c in choices_cold):
+            model.build_cached_blob(choices_cold)
+        model.arena.fill_(0xFF)
+
     # ---- per-kernel durations for the roofline (same resident steps, with per-operation events) --
     xf = {}          # layer -> [ns]
     ex = {}
@@ -418,6 +460,7 @@ def run_ours(args):
         "roofline": roof,
         "roofline_transform": xroof,
         "transform_all": xall,
+        "algorithm1": alg1,
         "breakdown": {"sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3, "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
                       "choices_resident": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_res],
                       "choices_cold": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_cold]},
@@ -451,6 +494,8 @@ def run_ours(args):
         ref = omodel.run_model(layers, ws, bs, x)[-1]
         den = float(np.sqrt(np.sum(ref * ref)))
         line["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_gpu[0] - ref) ** 2)) / den)
+        if alg1:
+            alg1["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_s[0] - ref) ** 2)) / den)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

@@ -20,4 +20,9 @@ Parity pins (tests/test_oracle_*.py, all CPU):
   selection.*              the paper's Table 2 worked example; brute-force enumeration
                            on random small integer tables
   conv.maxpool/gavgpool    closed forms on ramps / constants
+  scheduler.simulate       hand-computed makespans; an independent unit-time tick simulator
+                           on random layer graphs
+  scheduler.schedule/search  hand examples; fixed point of the balancing loop; bounded by
+                           brute force over all queue assignments and by queue 0's own load;
+                           exhaustive search no worse than any single combination
 """

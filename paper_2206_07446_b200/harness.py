@@ -133,33 +133,44 @@ class Model:
 
     def schedule(self, x_nchw, costs, n_little, allow_cached=1, rounds=2, eps_pct=1, big_pct=100, combo_limit=4096):
         """Algorithm 1 with its calibration step: schedule from the cost table, run the schedule once with
-        per-operation timings, overwrite the chosen kernels' costs with what they took while the other
-        queues were busy, and schedule again (`rounds` times).  eps is eps_pct percent of the summed
-        execution time of the per-layer choice.  Returns (choices, queue_of, predicted ns, costs used)."""
-        costs = [dict(c) for c in costs]
-        base = nb.nnv_select_kernels(self.plan, costs, allow_cached)
-        rows = {(c["layer"], c["variant"], c["math"]): c for c in costs}
-        eps = sum(rows[(i,) + ch[:2]]["exec_ns"] for i, ch in enumerate(base) if ch is not None) * eps_pct // 100
+        per-operation timings, and rescale the table by how much slower each kind of operation (read,
+        transform, execution) ran while the other queues were busy than it did alone -- the queues share
+        one host link and one GPU, so co-running operations slow each other down; then schedule again
+        (`rounds` times).  Every option of a kind gets the same factor, so that options that were not
+        run are not favoured over the calibrated ones.  eps is eps_pct percent of the summed execution
+        time of the per-layer choice.  Returns (choices, queue_of, predicted ns, calibrated costs)."""
+        table = [dict(c) for c in costs]
+        base = nb.nnv_select_kernels(self.plan, table, allow_cached)
+        iso = {(c["layer"], c["variant"], c["math"]): c for c in costs}
+        eps = sum(iso[(i,) + ch[:2]]["exec_ns"] for i, ch in enumerate(base) if ch is not None) * eps_pct // 100
         out = None
         for r in range(rounds + 1):
-            out = nb.nnv_schedule(self.plan, costs, allow_cached, n_little, eps, big_pct, combo_limit)
+            out = nb.nnv_schedule(self.plan, table, allow_cached, n_little, eps, big_pct, combo_limit)
             if r == rounds:
                 break
             choices, queue_of, _ = out
             if any(c is not None and c[2] for c in choices):
                 self.build_cached_blob(choices)
+            self.cold_run_queues(x_nchw, choices, queue_of, n_little, poison=False)          # warm
             _, tm = self.cold_run_queues(x_nchw, choices, queue_of, n_little, want_timings=True, poison=False)
+            got = dict(h2d=0, xform=0, exec=0)
+            alone = dict(h2d=0, xform=0, exec=0)
             for i, ch in enumerate(choices):
                 if ch is None:
                     continue
-                row, t = rows[(i,) + ch[:2]], tm[i]
-                row["exec_ns"] = t["exec_end_ns"] - t["exec_start_ns"]
-                if ch[2]:
-                    row["h2d_cached_ns"] = t["h2d_end_ns"] - t["h2d_start_ns"]
-                else:
-                    row["h2d_raw_ns"] = t["h2d_end_ns"] - t["h2d_start_ns"]
-                    row["xform_ns"] = t["xform_end_ns"] - t["xform_start_ns"]
-        return out[0], out[1], out[2], costs
+                row, t = iso[(i,) + ch[:2]], tm[i]
+                got["exec"] += t["exec_end_ns"] - t["exec_start_ns"]
+                alone["exec"] += row["exec_ns"]
+                got["h2d"] += t["h2d_end_ns"] - t["h2d_start_ns"]
+                alone["h2d"] += row["h2d_cached_ns"] if ch[2] else row["h2d_raw_ns"]
+                if not ch[2]:
+                    got["xform"] += t["xform_end_ns"] - t["xform_start_ns"]
+                    alone["xform"] += row["xform_ns"]
+            f = {k: (got[k] / alone[k] if alone[k] else 1.0) for k in got}
+            self.calibration = f
+            table = [dict(c, h2d_raw_ns=int(c["h2d_raw_ns"] * f["h2d"]), h2d_cached_ns=int(c["h2d_cached_ns"] * f["h2d"]),
+                          xform_ns=int(c["xform_ns"] * f["xform"]), exec_ns=int(c["exec_ns"] * f["exec"])) for c in costs]
+        return out[0], out[1], out[2], table
 
     def to_device(self):
         """Device copies of the weight blob, the cached blob (if built) and I/O buffers for nnv_resident_run."""
