@@ -18,7 +18,8 @@ def needs_build():
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, "nnv_internal.h"), os.path.join(ROOT, "include", "nnv.h")]
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
+    deps = sources() + headers + [os.path.join(ROOT, "include", "nnv.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -1,0 +1,286 @@
+// Tensor-core 3x3 / stride 1 / pad 1 convolution as an implicit GEMM whose A operand keeps its
+// halo in shared memory.  Included by gemm_tc.cu (inside namespace nnv, after the PTX helpers).
+//
+// The plain implicit GEMM fetches one 128-pixel x 32-channel tile of the activation per filter tap:
+// nine fetches of mostly the same pixels.  Here one CTA owns an output patch of TH x 8 pixels
+// (TH = 16 or 32, i.e. one or two 128-row MMA tiles) and, per block of 32 input channels, fetches
+// the patch's halo only three times -- once per horizontal tap offset s, as a (TH + 2) x 8 pixel
+// box.  Inside such a box a vertical tap offset r is a whole number of 8-pixel rows, that is
+// r x 1024 bytes of shared memory, which is exactly one 8-row group of the 128-byte-swizzled
+// K-major layout: the MMA for tap (r, s) reads box s through a descriptor whose start address is
+// moved down by r groups.  Every tile base stays 1024-byte aligned, so the swizzle phase of the
+// TMA's writes and of the MMA's reads agree.  Activation bytes from L2 drop from 9 x 16 KB to
+// 3 x (TH + 2) KB per channel block and MMA tile, and with TH = 32 the two MMA tiles share every
+// weight tile.
+//
+// Output pixel (oh0 + g, ow0 + px) of MMA tile mt is TMEM lane / MMA row 8 * (g - 16 * mt) + px.
+// Pixels outside the image are zero-filled by the TMA on the way in and skipped on the way out.
+//
+// Warp roles and the bounded waits are those of gemm_tc_kernel; there are two rings here, one of
+// activation boxes (reused by three taps each) and one of weight tiles (one tap each).
+#pragma once
+
+struct ConvDev {
+    float* D;
+    const float* bias;
+    const float* addend;
+    int C, H, W, K;                 // input channels, image (input = output grid), output channels
+    int BN, MT, act, tmem_cols, splits, na, nb, cblk, tiles_w;
+};
+
+constexpr int CONV_MAX_NA = 4, CONV_MAX_NB = 8;
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ConvDev g) {
+    extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int BN = g.BN, MT = g.MT, NA = g.na, NB = g.nb;
+    const uint32_t a_slot_bytes = (uint32_t)(16 * MT + 2) * 1024u;
+    const uint32_t b_slot_bytes = (uint32_t)BN * BK_BYTES;
+    const uint32_t a_ring = sbase, b_ring = sbase + NA * a_slot_bytes;
+    const uint32_t bars = b_ring + NB * b_slot_bytes;
+    auto a_full = [&](int s) { return bars + 8u * s; };
+    auto a_empty = [&](int s) { return bars + 8u * (CONV_MAX_NA + s); };
+    auto b_full = [&](int s) { return bars + 8u * (2 * CONV_MAX_NA + s); };
+    auto b_empty = [&](int s) { return bars + 8u * (2 * CONV_MAX_NA + CONV_MAX_NB + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB);
+    const uint32_t holder = tmem_full_bar + 8u;
+    volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int splits = g.splits, sp = (int)blockIdx.z;       // the cluster spans grid z: one K split per CTA
+    const int tile_h = (int)blockIdx.x / g.tiles_w, tile_w = (int)blockIdx.x - tile_h * g.tiles_w;
+    const int oh0 = tile_h * 16 * MT, ow0 = tile_w * 8, n0 = blockIdx.y * BN;
+    const int cb0 = (int)(((long long)g.cblk * sp) / splits);
+    const int ncb = (int)(((long long)g.cblk * (sp + 1)) / splits) - cb0;
+
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+        for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
+        mbar_init(tmem_full_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"((uint32_t)g.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *holder_ptr;
+    pdl_wait();                                               // set-up above overlaps the previous kernel's tail
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int ia = 0, ib = 0;                               // boxes / weight tiles issued so far
+            for (int cbi = 0; cbi < ncb && ok; ++cbi) {
+                const int c0 = (cb0 + cbi) * 32;
+                for (int s = 0; s < 3 && ok; ++s) {
+                    const int sa = ia % NA;
+                    ok = mbar_wait(a_empty(sa), ((ia / NA) & 1) ^ 1u);
+                    if (!ok) break;
+                    mbar_expect_tx(a_full(sa), a_slot_bytes);
+                    tma_load_3d(a_ring + sa * a_slot_bytes, &tmA, c0, ow0 + s - 1, oh0 - 1, a_full(sa));
+                    ++ia;
+                    for (int r = 0; r < 3; ++r) {
+                        const int sb = ib % NB;
+                        ok = mbar_wait(b_empty(sb), ((ib / NB) & 1) ^ 1u);
+                        if (!ok) break;
+                        mbar_expect_tx(b_full(sb), b_slot_bytes);
+                        tma_load_3d(b_ring + sb * b_slot_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, b_full(sb));
+                        ++ib;
+                    }
+                }
+            }
+            if (!ok) {
+                atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let loads already in flight land
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // instruction descriptor: fp32 accumulate, TF32 operands, both K-major, N = BN, M = 128
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            int ia = 0, ib = 0;
+            for (int cbi = 0; cbi < ncb && ok; ++cbi) {
+                for (int s = 0; s < 3 && ok; ++s) {
+                    const int sa = ia % NA;
+                    ok = mbar_wait(a_full(sa), (ia / NA) & 1);
+                    if (!ok) break;
+                    const uint32_t a_box = a_ring + sa * a_slot_bytes;
+                    for (int r = 0; r < 3; ++r) {
+                        const int sb = ib % NB;
+                        ok = mbar_wait(b_full(sb), (ib / NB) & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t bdesc = make_smem_desc(b_ring + sb * b_slot_bytes);
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const uint64_t adesc = make_smem_desc(a_box + (uint32_t)(mt * 16 + r) * 1024u);
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk)     // 4 MMAs of 32 bytes of K each
+                                umma<false>(tmem_base + (uint32_t)(mt * BN), adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2),
+                                            idesc, (cbi | s | r | kk) ? 1u : 0u);
+                        }
+                        umma_commit(b_empty(sb));
+                        ++ib;
+                    }
+                    if (ok) umma_commit(a_empty(sa));
+                    ++ia;
+                }
+            }
+            if (ok) umma_commit(tmem_full_bar);
+            else atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        }
+    } else {
+        const bool ok = mbar_wait(tmem_full_bar, 0);
+        tc_fence_after();
+        const int quarter = warp & 3;                         // TMEM lanes this warp may read
+        const int row = quarter * 32 + lane;                  // MMA row = 8 * (patch row) + (patch column)
+        if (!ok) {
+            if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        } else if (splits == 1) {
+            // Each warp turns its 32 accumulator rows (one pixel per lane) into pixel-contiguous
+            // stores through a private 32 x 32 staging tile (row pitch 36 words; both rings are idle
+            // by now): lane = pixel on the way in, 8 lanes x 16 bytes = 128 contiguous bytes of one
+            // pixel on the way out, so every global access covers whole 128-byte lines.
+            const bool vec = ((g.K & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
+                             (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
+                             (!g.bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+            const uint32_t stage = sbase + (uint32_t)quarter * (32u * 36u * 4u);
+            const int sub = lane >> 3, cc = (lane & 7) * 4;       // row within a group of four, first column
+            for (int mt = 0; mt < MT; ++mt) {
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        if (c0 + half * 16 < BN) {                // warp-uniform
+                            uint32_t r[16];
+                            tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mt * BN + c0 + half * 16), r);
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(stage + (uint32_t)(lane * 36 + half * 16 + j) * 4u),
+                                             "r"(r[j]), "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]) : "memory");
+                        }
+                    }
+                    __syncwarp();
+                    const int n = n0 + c0 + cc;
+                    const bool col_ok = (c0 + cc < BN) && (n < g.K);
+                    float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (vec && col_ok && g.bias) bb = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+#pragma unroll 2
+                    for (int it = 0; it < 8; ++it) {
+                        const int rl = it * 4 + sub, mrow = quarter * 32 + rl;
+                        const int oh = oh0 + mt * 16 + (mrow >> 3), ow = ow0 + (mrow & 7);
+                        if (!col_ok || oh >= g.H || ow >= g.W) continue;
+                        float4 v;
+                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                     : "r"(stage + (uint32_t)(rl * 36 + cc) * 4u));
+                        const long long off = ((long long)oh * g.W + ow) * g.K + n;
+                        if (vec) {
+                            v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                            if (g.addend) {
+                                const float4 aa = __ldg(reinterpret_cast<const float4*>(g.addend + off));
+                                v.x += aa.x; v.y += aa.y; v.z += aa.z; v.w += aa.w;
+                            }
+                            v.x = act_fn(v.x, g.act); v.y = act_fn(v.y, g.act); v.z = act_fn(v.z, g.act); v.w = act_fn(v.w, g.act);
+                            *reinterpret_cast<float4*>(g.D + off) = v;
+                        } else {
+                            const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if (n + j < g.K) {
+                                    float t = vv[j];
+                                    if (g.bias) t += __ldg(g.bias + n + j);
+                                    if (g.addend) t += __ldg(g.addend + off + j);
+                                    g.D[off + j] = act_fn(t, g.act);
+                                }
+                            }
+                        }
+                    }
+                    __syncwarp();                                 // the staging tile is rewritten by the next chunk
+                }
+            }
+        } else {
+            // park this CTA's partial tiles in its own shared memory (both rings are idle by now):
+            // P[mt * 128 + row][col], row pitch BN + 4 words
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint32_t prow = sbase + (uint32_t)(mt * 128 + row) * (uint32_t)(BN + 4) * 4u;
+                for (int c0 = 0; c0 < BN; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mt * BN + c0), r);
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4)
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (uint32_t)(c0 + j) * 4u), "r"(r[j]),
+                                     "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]) : "memory");
+                }
+            }
+        }
+    }
+    __syncwarp();
+    if (splits > 1) {
+        // Split-K write-out, as in gemm_tc_kernel: CTA `sp` sums its share of the 128 * MT rows over
+        // the cluster through distributed shared memory in rank order, then applies the epilogue.
+        cluster_sync_all();
+        if (warp >= 2 && g_device_status == 0) {
+            const int t = (int)threadIdx.x - 64;
+            const int rows_per = (BM * MT) / splits, r0 = sp * rows_per;
+            const int c4n = BN / 4;
+            const bool vec = ((g.K & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
+                             (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
+                             (!g.bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+            const int total = rows_per * c4n;
+#pragma unroll 1
+            for (int idx = t; idx < total; idx += 128) {
+                const int rq = idx / c4n;
+                const int rr = r0 + rq, cc = (idx - rq * c4n) * 4;
+                const uint32_t local = sbase + ((uint32_t)rr * (uint32_t)(BN + 4) + (uint32_t)cc) * 4u;
+                float4 v[8];
+#pragma unroll
+                for (int rk = 0; rk < 8; ++rk) {
+                    if (rk < splits) {
+                        uint32_t remote;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rk));
+                        asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v[rk].x), "=f"(v[rk].y), "=f"(v[rk].z), "=f"(v[rk].w) : "r"(remote));
+                    }
+                }
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int rk = 0; rk < 8; ++rk)
+                    if (rk < splits) { acc.x += v[rk].x; acc.y += v[rk].y; acc.z += v[rk].z; acc.w += v[rk].w; }
+                const int mt = rr >> 7, mrow = rr & 127;
+                const int oh = oh0 + mt * 16 + (mrow >> 3), ow = ow0 + (mrow & 7), n = n0 + cc;
+                if (oh >= g.H || ow >= g.W || n >= g.K) continue;
+                const long long pix = (long long)oh * g.W + ow;
+                float* drow = g.D + pix * g.K;
+                const float* arow = g.addend ? g.addend + pix * g.K : nullptr;
+                float vv[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (vec || n + j < g.K) {
+                        if (g.bias) vv[j] += __ldg(g.bias + n + j);
+                        if (arow) vv[j] += __ldg(arow + n + j);
+                        vv[j] = act_fn(vv[j], g.act);
+                    }
+                }
+                if (vec) {
+                    *reinterpret_cast<float4*>(drow + n) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (n + j < g.K) drow[n + j] = vv[j];
+                }
+            }
+        }
+        cluster_sync_all();                                   // nobody leaves while its tiles may still be read
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
+    }
+}

@@ -520,6 +520,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
+#include "conv3x3_tc.cuh"
+
 // ---- host side --------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 PFN_cuTensorMapEncodeIm2col_v12000 g_encode_im2col = nullptr;
@@ -578,6 +580,79 @@ nnv_status_t encode_im2col_operand(CUtensorMap* map, const void* base, int C, in
     return NNV_OK;
 }
 
+// 3-D tiled map over an NHWC fp32 activation {C, W, H}: boxes of 32 channels x 8 pixels x `box_h`
+// rows (the halo boxes of conv3x3_tc_kernel); coordinates outside the image read as zero.
+nnv_status_t encode_halo_operand(CUtensorMap* map, const void* base, int C, int H, int W, int box_h) {
+    NNV_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0 && (C % 4) == 0, NNV_ERR_INVALID_ARG,
+                "activation must be 16-byte aligned with C a multiple of 4");
+    cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H};
+    cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)W * C * 4};
+    cuuint32_t box[3] = {32, 8, (cuuint32_t)box_h};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (halo boxes) failed with code %d", (int)r);
+    return NNV_OK;
+}
+
+// Tiling of conv3x3_tc_kernel for one layer.
+struct ConvTiling { int MT, BN, splits, na, nb, tmem_cols; size_t smem; };
+
+size_t conv_smem_bytes(int MT, int BN, int na, int nb) {
+    return (size_t)1024 + (size_t)na * (16 * MT + 2) * 1024 + (size_t)nb * BN * BK_BYTES + 8 * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 2);
+}
+
+// Fills in ring depths (unless given), shared-memory size and TMEM columns; false if the tiling does
+// not fit (shared memory, or room to park the partial tiles of a K split).
+bool finish_conv_tiling(ConvTiling* t) {
+    const size_t park = t->splits > 1 ? (size_t)t->MT * BM * (t->BN + 4) * 4 : 0;
+    auto rings = [&] { return (size_t)t->na * (16 * t->MT + 2) * 1024 + (size_t)t->nb * t->BN * BK_BYTES; };
+    if (t->na <= 0 || t->nb <= 0) {
+        t->na = 2; t->nb = 3;
+        while (rings() < park && t->nb < CONV_MAX_NB) ++t->nb;      // deeper rings only to make room for the parked tiles
+        while (rings() < park && t->na < CONV_MAX_NA) ++t->na;
+    }
+    t->smem = conv_smem_bytes(t->MT, t->BN, t->na, t->nb);
+    t->tmem_cols = 32;
+    while (t->tmem_cols < t->MT * t->BN) t->tmem_cols *= 2;
+    return t->smem <= 200u * 1024u && rings() >= park;
+}
+
+// Measured on B200 (sweeps over tilings, ring depths and K splits at the 3x3 shapes of the VGG / ResNet
+// configurations, L2 flushed before each launch): the kernel runs best with one MMA tile per CTA,
+// channel tiles of 128, shallow rings (two or three CTAs then share an SM, and one CTA's fill and
+// write-out overlap another's MMAs) and enough K splits for ~1.5 CTAs per SM; all CTAs should be
+// resident at once (a second, mostly empty wave costs as much as the first), so the box ring drops
+// to one slot when that makes them fit.  Layers with fewer than four channel blocks and fewer than
+// two patches per SM, and layers too small to give every SM a CTA even with 8 splits, stay on the
+// plain implicit GEMM, which is faster there.
+bool pick_conv_tiling(int C, int H, int W, int N, ConvTiling* out) {
+    const int cblk = ceil_div(C, 32);
+    ConvTiling t{};
+    t.MT = 1;
+    t.BN = std::min(128, ceil_div(N, 16) * 16);
+    const long long tiles = (long long)ceil_div(H, 16) * ceil_div(W, 8) * ceil_div(N, t.BN);
+    int max_sp = 1;
+    while (max_sp * 2 <= std::min(8, cblk)) max_sp *= 2;
+    if (tiles * max_sp < 148 || (cblk < 4 && tiles < 296)) return false;
+    t.splits = 1;
+    while (t.splits < max_sp && tiles * t.splits < 224) t.splits *= 2;
+    const long long ctas = tiles * t.splits;
+    bool found = false;
+    const int rings[2][2] = {{2, 3}, {1, 3}};
+    for (int i = 0; i < 2 && !found; ++i) {
+        ConvTiling c = t;
+        c.na = rings[i][0]; c.nb = rings[i][1];
+        if (!finish_conv_tiling(&c)) continue;
+        const int occ = std::max(1, std::min((int)(227u * 1024u / (c.smem + 1024)), 512 / c.tmem_cols));
+        if (ctas <= 148ll * occ) { t = c; found = true; }
+    }
+    if (!found) { t.na = 0; t.nb = 0; found = finish_conv_tiling(&t); }
+    if (found) *out = t;
+    return found;
+}
+
 std::once_flag g_attr_once;
 
 }  // namespace
@@ -588,7 +663,25 @@ nnv_status_t gemm_tc_init() {
         cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     });
+    return NNV_OK;
+}
+
+static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 16 * ct.MT + 2));
+    NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, ct.BN));
+    ConvDev g;
+    g.D = a.D; g.bias = a.bias; g.addend = a.addend;
+    g.C = a.ic.C; g.H = a.ic.H; g.W = a.ic.W; g.K = a.N;
+    g.BN = ct.BN; g.MT = ct.MT; g.act = a.act; g.tmem_cols = ct.tmem_cols; g.splits = ct.splits; g.na = ct.na; g.nb = ct.nb;
+    g.cblk = ceil_div(a.ic.C, 32); g.tiles_w = ceil_div(a.ic.W, 8);
+    NNV_REQUIRE(a.ldd == a.N, NNV_ERR_INVALID_ARG, "the 3x3 kernel writes a dense NHWC output");
+    dim3 grid(ceil_div(a.ic.H, 16 * ct.MT) * g.tiles_w, ceil_div(a.N, ct.BN), ct.splits);
+    NNV_REQUIRE(grid.y <= 65535, NNV_ERR_UNSUPPORTED, "convolution grid too large");
+    (void)launch_pdl_cluster(conv3x3_tc_kernel, grid, dim3(GEMM_THREADS), ct.smem, st, ct.splits, tmA, tmB, g);
+    NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
 
@@ -624,6 +717,26 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         int fb = 0, fs = 0;
         if (std::sscanf(e, "%d,%d", &fb, &fs) == 2 && fb >= 16 && fb <= 128 && fb % 16 == 0 && fs >= 1 && fs <= 8 &&
             (fs & (fs - 1)) == 0 && fs <= nkb_all) { BN = fb; splits = fs; }
+    }
+    // A 3x3 / stride 1 / pad 1 layer large enough to fill the GPU runs on the halo-resident kernel,
+    // which moves fewer operand bytes through L2 and shared memory.
+    if (a.ic.on && a.mode == GEMM_TF32 && a.batch == 1 && a.ic.R == 3 && a.ic.S == 3 && a.ic.stride == 1 && a.ic.pad == 1 &&
+        (a.ic.C % 32) == 0) {
+        ConvTiling ct;
+        bool use = pick_conv_tiling(a.ic.C, a.ic.H, a.ic.W, a.N, &ct);
+        if (const char* e = std::getenv("NNV_DEBUG_CONV3X3")) {     // debug only: "off", or "MT,BN,splits[,boxes,weight tiles]"
+            ConvTiling f{};
+            if (e[0] == 'o') {
+                use = false;
+            } else if (std::sscanf(e, "%d,%d,%d,%d,%d", &f.MT, &f.BN, &f.splits, &f.na, &f.nb) >= 3 && (f.MT == 1 || f.MT == 2) &&
+                       f.BN >= 16 && f.BN <= 128 && f.BN % 16 == 0 && f.splits >= 1 && f.splits <= 8 &&
+                       (f.splits & (f.splits - 1)) == 0 && f.splits <= ceil_div(a.ic.C, 32) && f.na <= CONV_MAX_NA &&
+                       f.nb <= CONV_MAX_NB && finish_conv_tiling(&f)) {
+                ct = f;
+                use = true;
+            }
+        }
+        if (use) return launch_conv3x3_tc(a, ct, st);
     }
     int tmem_cols = 32;
     while (tmem_cols < BN) tmem_cols *= 2;

@@ -1,0 +1,72 @@
+"""GPU parity of the halo-resident 3x3 tensor-core kernel: every tiling it can take (one or two MMA
+tiles per CTA, several channel-tile widths, K splits over a thread-block cluster) against the fp64
+direct-convolution oracle, and against the plain implicit GEMM that it replaces."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import model as omodel
+from paper_2206_07446_b200 import binding as nb
+from gpu_util import TOL, rel_l2, run_conv
+
+pytestmark = pytest.mark.gpu
+
+ENV = "NNV_DEBUG_CONV3X3"          # debug override read by the library at every launch
+
+
+def _run(L, x, w, b, add, setting):
+    old = os.environ.get(ENV)
+    if setting is None:
+        os.environ.pop(ENV, None)
+    else:
+        os.environ[ENV] = setting
+    try:
+        plan = nb.Plan([L], [0], [0])
+        return run_conv(plan, 0, L, nb.VAR_IM2COL, nb.MATH_TF32, x, w, b, add)
+    finally:
+        if old is None:
+            os.environ.pop(ENV, None)
+        else:
+            os.environ[ENV] = old
+
+
+@pytest.mark.parametrize("shape", [
+    # C, K, H, W, bias/addend/act
+    (64, 64, 56, 56, False),         # config 1 / ResNet stage 1
+    (32, 48, 40, 30, True),          # ragged: H % 16 != 0, W % 8 != 0, K = 48, epilogue terms
+    (128, 128, 28, 28, True),        # four channel blocks: K splits 2 and 4
+    (96, 40, 19, 21, False),         # K = 40 (not a multiple of 16), three channel blocks
+    (256, 20, 17, 9, True),          # K = 20: scalar epilogue stores; eight channel blocks: split 8
+])
+def test_every_tiling_matches_the_oracle(shape):
+    C, K, H, W, epi = shape
+    L = dict(op=0, C=C, K=K, R=3, S=3, stride=1, pad=1, groups=1, H=H, W=W, in0=-1, in1=-1, act=2 if epi else 1,
+             has_bias=1 if epi else 0)
+    rng = np.random.default_rng([7] + list(shape[:4]))
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((K, C, 3, 3)) * np.sqrt(2.0 / (C * 9))).astype(np.float32)
+    b = rng.uniform(-1, 1, K).astype(np.float32) if epi else None
+    add = rng.uniform(-1, 1, (K, H, W)).astype(np.float32) if epi else None
+    ref = omodel.run_layer(L, x, w, b, add)
+    plain = _run(L, x, w, b, add, "off")
+    assert rel_l2(plain, ref) <= TOL[nb.MATH_TF32]
+    bn_full = min(128, -(-K // 16) * 16)
+    cblk = C // 32
+    ran = 0
+    for mt in (1, 2):
+        for bn in sorted({bn_full, 16, min(bn_full, 64)}):
+            for sp in (1, 2, 4, 8):
+                if sp > cblk:
+                    continue
+                y = _run(L, x, w, b, add, "%d,%d,%d" % (mt, bn, sp))
+                assert np.all(np.isfinite(y)), (mt, bn, sp)
+                err = rel_l2(y, ref)
+                assert err <= TOL[nb.MATH_TF32], (mt, bn, sp, err)
+                # same products, other summation order than the plain kernel: fp32 rounding apart only
+                assert rel_l2(y, plain) <= 1e-5, (mt, bn, sp, rel_l2(y, plain))
+                ran += 1
+    assert ran >= 4
+    # whatever the library picks by itself is one of the two kernels above
+    auto = _run(L, x, w, b, add, None)
+    assert rel_l2(auto, ref) <= TOL[nb.MATH_TF32]
