@@ -194,7 +194,7 @@ template <> __device__ inline __nv_bfloat16 cvt_out<__nv_bfloat16>(float v) { re
 
 constexpr int PACK_THREADS = 256;
 constexpr int PACK_SMEM_FLOATS = XF_SMEM_FLOATS;
-constexpr int PACK1X1_PER_BLOCK = PACK_THREADS * 8;             // elements of P one block of pack1x1 writes
+constexpr int PACK1X1_PER_BLOCK = PACK_THREADS * 16;            // elements of P one block of pack1x1 writes
 
 template <typename OutT> __device__ __forceinline__ void store4(OutT* p, float a, float b, float c, float d);
 template <> __device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
@@ -221,9 +221,44 @@ constexpr int PACK_SLICE = PACK_SMEM_FLOATS / PACK_WARPS;        // floats of sh
 __host__ __device__ inline int pack_ch(int RS) { return 32 * RS <= PACK_SLICE ? 32 : 8; }
 __host__ __device__ inline int pack_units_per_row(int C, int RS) { return (C + pack_ch(RS) - 1) / pack_ch(RS); }
 
+// Fast repack for the common case C % 64 == 0 (then R*S*C needs no padding): a block stages a
+// contiguous range of PACK_NF filters (k, c pairs; PACK_NF * RS floats) with 128-bit loads, as the
+// filter transform does, and writes the transposed (rs, c) order with 128-bit stores -- consecutive
+// threads write consecutive 16-byte words of one (k, rs) segment.
+constexpr int PACK_NF = 512;
+__host__ __device__ inline bool pack_fast(int C, int RS) {
+    return RS > 1 && (C % 64) == 0 && PACK_NF * RS <= PACK_SMEM_FLOATS && (C >= PACK_NF ? C % PACK_NF == 0 : PACK_NF % C == 0);
+}
+
+template <typename OutT>
+__device__ __forceinline__ void pack_fast_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS,
+                                                int Qp, unsigned block, float* sg) {
+    const long long F = (long long)K * C;
+    const long long f_block = (long long)block * PACK_NF;
+    const int nf = (int)min((long long)PACK_NF, F - f_block);    // multiple of 64
+    const float4* src = reinterpret_cast<const float4*>(w + f_block * RS);
+    float4* dst = reinterpret_cast<float4*>(sg);
+    const int nv = nf * RS / 4;
+    for (int i = threadIdx.x; i < nv; i += PACK_THREADS) dst[i] = __ldg(src + i);
+    __syncthreads();
+    const int Cb = min(C, PACK_NF);                               // channels of one k row inside this block
+    const int c4n = Cb / 4, per_k = RS * c4n;
+    const int k0 = (int)(f_block / C), cbase = (int)(f_block - (long long)k0 * C);
+    for (int i = threadIdx.x; i < nv; i += PACK_THREADS) {
+        const int kl = i / per_k, r = i - kl * per_k;
+        const int rs = r / c4n, c = (r - rs * c4n) * 4;
+        const float* s = sg + ((kl * Cb + c) * RS + rs);
+        store4<OutT>(P + (long long)(k0 + kl) * Qp + (long long)rs * C + cbase + c, s[0], s[RS], s[2 * RS], s[3 * RS]);
+    }
+}
+
 template <typename OutT>
 __device__ __forceinline__ void pack_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp,
                                            unsigned block, float* smem) {
+    if (pack_fast(C, RS)) {
+        pack_fast_block<OutT>(w, P, K, C, RS, Qp, block, smem);
+        return;
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int CH = pack_ch(RS), upr = pack_units_per_row(C, RS);
     const long long unit = (long long)block * PACK_WARPS + warp;
@@ -256,17 +291,20 @@ __device__ __forceinline__ void pack1x1_block(const float* __restrict__ w, OutT*
     const long long n = (long long)K * Qp;
     const long long base = (long long)block * PACK1X1_PER_BLOCK;
     if (C == Qp) {                                              // no padding: a straight conversion copy, 4 at a time
+        float4 v[4];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < 4; ++u) {                             // all loads first: four 16-byte requests in flight per thread
             const long long i = base + ((long long)u * PACK_THREADS + threadIdx.x) * 4;
-            if (i < n) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(w + i));
-                store4<OutT>(P + i, v.x, v.y, v.z, v.w);
-            }
+            if (i < n) v[u] = __ldg(reinterpret_cast<const float4*>(w + i));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long i = base + ((long long)u * PACK_THREADS + threadIdx.x) * 4;
+            if (i < n) store4<OutT>(P + i, v[u].x, v[u].y, v[u].z, v[u].w);
         }
     } else {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 16; ++u) {
             const long long i = base + (long long)u * PACK_THREADS + threadIdx.x;
             if (i < n) {
                 const int k = (int)(i / Qp), q = (int)(i - (long long)k * Qp);
@@ -294,59 +332,86 @@ pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, 
 // ---- many layers in one launch ----------------------------------------------------------------
 // Block b belongs to the descriptor whose [block0, block0 + blocks) range holds it and does there
 // exactly what the single-layer kernels do.  A batch of small layers then costs one launch and
-// presents the memory system with one large stream of work.
+// presents the memory system with one large stream of work.  The kernel is instantiated per group
+// of transform kinds (repacks / F(2,3) and F(4,3) / F(6,3)) so that the register allocation, and with
+// it the number of resident warps, is that of the group's own code and not of the largest transform.
+enum { XG_PACK = 0, XG_WINO_SMALL = 1, XG_WINO6 = 2, XG_COUNT = 3 };
+__host__ __device__ inline int xform_group(int kind) {
+    return kind == XF_WINO6 ? XG_WINO6 : (kind == XF_WINO2 || kind == XF_WINO4) ? XG_WINO_SMALL : XG_PACK;
+}
+
+template <int GROUP>
 __global__ void __launch_bounds__(FT_THREADS)
 multi_transform_kernel(const __grid_constant__ XformBatch batch) {
     pdl_enter();
     __shared__ __align__(16) float smem[XF_SMEM_FLOATS];
-    // Persistent blocks walk the virtual block list with a grid stride: the grid is capped at a few
-    // blocks per SM so that the latency-critical execution kernels running beside this one always
-    // find room (shared memory, block slots) on every SM.
-    for (unsigned vb = blockIdx.x; vb < (unsigned)batch.total_blocks; vb += gridDim.x) {
-        int di = 0;
-        for (int i = 1; i < batch.n; ++i)
-            if (vb >= (unsigned)batch.d[i].block0) di = i;
-        const XformDesc& d = batch.d[di];
-        const unsigned lb = vb - (unsigned)d.block0;
-        const float* src = static_cast<const float*>(d.src);
+    const unsigned vb = blockIdx.x;
+    int di = 0;
+    for (int i = 1; i < batch.n; ++i)
+        if (vb >= (unsigned)batch.d[i].block0) di = i;
+    const XformDesc& d = batch.d[di];
+    const unsigned lb = vb - (unsigned)d.block0;
+    const float* src = static_cast<const float*>(d.src);
+    if constexpr (GROUP == XG_PACK) {
         switch (d.kind * 2 + d.bf16) {
             case XF_PACK * 2: pack_block<float>(src, (float*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem); break;
             case XF_PACK * 2 + 1: pack_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem); break;
             case XF_PACK1X1 * 2: pack1x1_block<float>(src, (float*)d.dst, d.K, d.C, d.Qp, lb); break;
             case XF_PACK1X1 * 2 + 1: pack1x1_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Qp, lb); break;
+            default: break;
+        }
+    } else if constexpr (GROUP == XG_WINO_SMALL) {
+        switch (d.kind * 2 + d.bf16) {
             case XF_WINO2 * 2: filter_transform_block<2, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
             case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 2>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
             case XF_WINO4 * 2: filter_transform_block<4, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
-            case XF_WINO6 * 2: filter_transform_block<6, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
             default: break;
         }
-        __syncthreads();                                        // the staging buffer is reused by the next virtual block
+    } else {
+        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem);
     }
+}
+
+static long long pack_blocks(int K, int C, int RS) {
+    if (pack_fast(C, RS)) return ((long long)K * C + PACK_NF - 1) / PACK_NF;
+    return ((long long)K * pack_units_per_row(C, RS) + PACK_WARPS - 1) / PACK_WARPS;
 }
 
 int xform_blocks(const XformDesc& d) {
     switch (d.kind) {
-        case XF_PACK: return (int)(((long long)d.K * pack_units_per_row(d.C, d.RS) + PACK_WARPS - 1) / PACK_WARPS);
+        case XF_PACK: return (int)pack_blocks(d.K, d.C, d.RS);
         case XF_PACK1X1: return (int)(((long long)d.K * d.Qp + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
         default: return (int)(((long long)d.K * d.Cp + FT_THREADS * 2 - 1) / (FT_THREADS * 2));
     }
 }
 
 nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st) {
-    for (int i0 = 0; i0 < n; i0 += XF_BATCH_MAX) {
+    for (int grp = 0; grp < XG_COUNT; ++grp) {
         XformBatch b;
-        b.n = std::min(XF_BATCH_MAX, n - i0);
+        b.n = 0;
         int blocks = 0;
-        for (int i = 0; i < b.n; ++i) {
-            b.d[i] = descs[i0 + i];
-            NNV_REQUIRE(b.d[i].kind != XF_PACK || 8 * b.d[i].RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED,
-                        "filter window of %d taps is too large to repack", b.d[i].RS);
-            b.d[i].block0 = blocks;
-            blocks += xform_blocks(b.d[i]);
+        auto flush = [&]() -> nnv_status_t {
+            if (b.n == 0) return NNV_OK;
+            b.total_blocks = blocks;
+            if (grp == XG_PACK) NNV_LAUNCH((multi_transform_kernel<XG_PACK>), blocks, FT_THREADS, 0, st, b);
+            else if (grp == XG_WINO_SMALL) NNV_LAUNCH((multi_transform_kernel<XG_WINO_SMALL>), blocks, FT_THREADS, 0, st, b);
+            else NNV_LAUNCH((multi_transform_kernel<XG_WINO6>), blocks, FT_THREADS, 0, st, b);
+            NNV_CUDA(cudaGetLastError());
+            b.n = 0;
+            blocks = 0;
+            return NNV_OK;
+        };
+        for (int i = 0; i < n; ++i) {
+            if (xform_group(descs[i].kind) != grp) continue;
+            XformDesc d = descs[i];
+            NNV_REQUIRE(d.kind != XF_PACK || 8 * d.RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED,
+                        "filter window of %d taps is too large to repack", d.RS);
+            d.block0 = blocks;
+            blocks += xform_blocks(d);
+            b.d[b.n++] = d;
+            if (b.n == XF_BATCH_MAX) NNV_TRY(flush());
         }
-        b.total_blocks = blocks;
-        NNV_LAUNCH((multi_transform_kernel), blocks, FT_THREADS, 0, st, b);
-        NNV_CUDA(cudaGetLastError());
+        NNV_TRY(flush());
     }
     return NNV_OK;
 }
@@ -359,7 +424,7 @@ nnv_status_t launch_pack(bool bf16, const float* w, void* P, int K, int C, int R
         else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp);
     } else {
         NNV_REQUIRE(8 * RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED, "filter window of %d taps is too large to repack", RS);
-        const unsigned grid = (unsigned)(((long long)K * pack_units_per_row(C, RS) + PACK_WARPS - 1) / PACK_WARPS);
+        const unsigned grid = (unsigned)pack_blocks(K, C, RS);
         if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, RS, Qp);
         else NNV_LAUNCH((pack_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, RS, Qp);
     }

@@ -4,6 +4,7 @@
   python -m paper_2206_07446_b200.sweep transform-sweep
   python -m paper_2206_07446_b200.sweep conv --variant wino_f4 --C 64 --K 64 --H 56
   python -m paper_2206_07446_b200.sweep conv-sweep
+  python -m paper_2206_07446_b200.sweep transform-all --config cfg2_resnet18 --prefer wino_f4
 
 Each line of output is one JSON record with the algorithmic bytes / flops of the operation, the
 median duration and the achieved rate.  Weights and inputs are seeded random tensors created on
@@ -91,9 +92,57 @@ def time_conv(variant, math, C, K, R, stride, H, W, groups=1, reps=20, flush=Non
                 H=H, W=W, groups=groups, direct_flops=flops, us=med, us_min=best, direct_tflops=flops / med / 1e6)
 
 
+def time_transform_all(config, prefer, math, reps=20, flush=None):
+    """Every layer's weight transform of one configuration in a single nnv_transform_all launch
+    (run from the repository root: the layer shapes come from the top-level `workloads` module).
+    Layers take the first eligible variant of `prefer`, then gemm1x1 / im2col."""
+    import workloads as wl
+    layers = wl.CONFIGS[config]()
+    w_off, b_off, w_bytes = _offsets(layers)
+    plan = nb.Plan(layers, w_off, b_off)
+    choices = []
+    for i, L in enumerate(layers):
+        if L["op"] != nb.OP_CONV:
+            choices.append(None)
+            continue
+        el = nb.nnv_eligible(plan, i)
+        v = next((c for c in prefer + [nb.VAR_GEMM1X1, nb.VAR_IM2COL] if c in el), None)
+        if v is None:
+            v = nb.VAR_DEPTHWISE if nb.VAR_DEPTHWISE in el else el[0]
+        m = nb.MATH_FP32 if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else (nb.MATH_TF32 if v in (nb.VAR_WINO_F4, nb.VAR_WINO_F6) else math)
+        choices.append((v, m, 0))
+    d_w = _rand(w_bytes // 4 + 64, 0.05)
+    offs, total = nb.nnv_transformed_layout(plan, choices)
+    d_out = _buf(total)
+    med, best = _time(lambda st: nb.nnv_transform_all(plan, choices, d_w, w_bytes, d_out, total, st), reps, flush)
+    raw = sum(4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"] for L, c in zip(layers, choices)
+              if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
+    out = sum(nb.nnv_transformed_bytes(plan, i, c[0], c[1]) for i, c in enumerate(choices)
+              if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
+    # the same bytes moved by a plain device copy, timed the same way: the ceiling of this measurement
+    half = (raw + out) // 2
+    a, b = _buf(half), _buf(half)
+    cmed, _ = _time(lambda st: b.copy_(a, non_blocking=True), reps, flush)
+    return dict(op="transform-all", config=config, prefer=[nb.VARIANT_NAMES[v] for v in prefer], math=nb.MATH_NAMES[math],
+                bytes=raw + out, us=med, us_min=best, gbs=(raw + out) / med / 1e3, copy_same_bytes_us=cmed,
+                copy_gbs=2 * half / cmed / 1e3)
+
+
+def _offsets(layers):
+    """Byte offsets of each layer's weights in a dense blob (256-byte aligned), no biases."""
+    w_off, pos = [], 0
+    for L in layers:
+        w_off.append(pos)
+        if L["op"] == nb.OP_CONV:
+            pos += (4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"] + 255) // 256 * 256
+    return w_off, [0] * len(layers), pos
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["transform", "transform-sweep", "conv", "conv-sweep"])
+    ap.add_argument("what", choices=["transform", "transform-sweep", "conv", "conv-sweep", "transform-all"])
+    ap.add_argument("--config", default="cfg2_resnet18")
+    ap.add_argument("--prefer", default="", help="comma-separated variants tried first per layer (transform-all)")
     ap.add_argument("--m", type=int, default=4)
     ap.add_argument("--variant", default="wino_f4", choices=nb.VARIANT_NAMES)
     ap.add_argument("--math", default="tf32", choices=nb.MATH_NAMES)
@@ -118,6 +167,9 @@ def main():
         for n in (64, 256, 512, 1024):
             print(json.dumps(time_transform(nb.VAR_IM2COL, nb.MATH_TF32, n, n, 3, a.reps, flush)), flush=True)
             print(json.dumps(time_transform(nb.VAR_IM2COL, nb.MATH_BF16, n, n, 3, a.reps, flush)), flush=True)
+    elif a.what == "transform-all":
+        prefer = [nb.VARIANT_NAMES.index(v) for v in a.prefer.split(",") if v]
+        print(json.dumps(time_transform_all(a.config, prefer, math, a.reps, flush)))
     elif a.what == "conv":
         v = nb.VARIANT_NAMES.index(a.variant)
         print(json.dumps(time_conv(v, math, a.C, a.K, a.R, a.stride, a.H, a.H, a.groups, a.reps, flush)))
