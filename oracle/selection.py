@@ -116,3 +116,44 @@ def select_kernels(layers, costs, allow_cached):
             raise ValueError("no cost rows for layer %d" % i)
         out.append(choose(options_from_costs(rows, allow_cached))[0])
     return out
+
+
+def choose_warm(rows):
+    """Of one layer's cost rows, the kernel with the least execution time; ties -> lowest (variant, math).
+
+    Warm inference has every weight prepared already, so only the execution column counts: this is
+    the paper's K_warm (its Section 3.5, "the kernels with the fastest warm inference")."""
+    best = None
+    for r in sorted(rows, key=lambda r: (int(r["variant"]), int(r["math"]))):
+        if best is None or int(r["exec_ns"]) < int(best["exec_ns"]):
+            best = r
+    return (int(best["variant"]), int(best["math"]))
+
+
+def select_warm(layers, costs):
+    """K_warm per conv layer as (variant, math, prepared): prepared = 1 when the kernel reads
+    transformed weights (they stay resident after the first inference), 0 when it reads raw ones."""
+    out = []
+    for i, L in enumerate(layers):
+        if L["op"] != 0:
+            out.append(None)
+            continue
+        rows = [r for r in costs if int(r["layer"]) == i]
+        if not rows:
+            raise ValueError("no cost rows for layer %d" % i)
+        v, m = choose_warm(rows)
+        out.append((v, m, 1 if has_transform(v) else 0))
+    return out
+
+
+def switch_set(k_cold, k_warm):
+    """Layers of K_warm - K_cold (Section 3.5): their warm kernel differs from the cold one, so its
+    weights are still to be prepared (read, transformed) while or after the cold inference runs.
+    A warm kernel without a transform needs no preparation beyond the raw weights."""
+    out = []
+    for i, (c, w) in enumerate(zip(k_cold, k_warm)):
+        if c is None or w is None:
+            continue
+        if (c[0], c[1]) != (w[0], w[1]) and has_transform(w[0]):
+            out.append(i)
+    return out

@@ -94,3 +94,50 @@ def test_select_kernels_over_layers():
              dict(layer=2, variant=sel.DEPTHWISE, math=sel.FP32, h2d_raw_ns=1, xform_ns=0, h2d_cached_ns=1, exec_ns=5)]
     assert sel.select_kernels(layers, costs, True) == [(sel.WINO_F2, sel.TF32, 1), None, (sel.DEPTHWISE, sel.FP32, 0)]
     assert sel.select_kernels(layers, costs, False) == [(sel.DIRECT, sel.FP32, 0), None, (sel.DEPTHWISE, sel.FP32, 0)]
+
+
+def test_table2_warm_kernel_and_switch_set():
+    """Table 2's execution column: the fastest-executing kernel is winograd-pack4 (2.98 ms), while the cold
+    choice is the unpacked Winograd from the cache (7.49 ms) or, without caching, the untransformed 3x3s1
+    kernel (8.71 ms): K_warm differs from K_cold in both modes, the situation Section 3.5 describes."""
+    names = [r[0] for r in _table2()]
+    rows = [dict(layer=0, variant=i, math=0, h2d_raw_ns=rr, xform_ns=wt, h2d_cached_ns=rc, exec_ns=ex)
+            for i, (name, rr, wt, rc, ex) in enumerate(_table2())]
+    v, m = sel.choose_warm(rows)
+    assert names[v] == "3x3s1-winograd-pack4" and rows[v]["exec_ns"] == 2980
+    assert min(r["exec_ns"] for r in rows) == 2980
+    cold_cached = sel.choose(_table2_options(True))[0]
+    cold_raw = sel.choose(_table2_options(False))[0]
+    assert (cold_cached[0], cold_cached[1]) != (v, m) and (cold_raw[0], cold_raw[1]) != (v, m)
+
+
+def test_warm_selection_and_switch_set_properties():
+    """Brute force on random tables: K_warm minimises the summed execution time over all combinations;
+    the switch set is empty iff the kernels agree (or the warm kernel has no transform)."""
+    rng = np.random.default_rng(21)
+    layer = dict(op=0, C=8, K=8, R=3, S=3, stride=1, pad=1, groups=1)
+    kernels = [(sel.DIRECT, sel.FP32), (sel.IM2COL, sel.TF32), (sel.IM2COL, sel.BF16), (sel.WINO_F2, sel.TF32),
+               (sel.WINO_F4, sel.TF32)]
+    for _ in range(100):
+        n = int(rng.integers(1, 4))
+        layers = [layer] * n
+        costs = []
+        for i in range(n):
+            for (v, m) in kernels:
+                costs.append(dict(layer=i, variant=v, math=m, h2d_raw_ns=int(rng.integers(1, 9)),
+                                  xform_ns=0 if v == sel.DIRECT else int(rng.integers(0, 9)),
+                                  h2d_cached_ns=int(rng.integers(1, 9)), exec_ns=int(rng.integers(1, 6))))
+        warm = sel.select_warm(layers, costs)
+        ex = {(c["layer"], c["variant"], c["math"]): c["exec_ns"] for c in costs}
+        total = sum(ex[(i, w[0], w[1])] for i, w in enumerate(warm))
+        for combo in itertools.product(kernels, repeat=n):
+            assert total <= sum(ex[(i, k[0], k[1])] for i, k in enumerate(combo))
+        for i, w in enumerate(warm):                      # ties go to the lowest (variant, math)
+            assert (w[0], w[1]) == min(k for k in kernels if ex[(i, k[0], k[1])] == ex[(i, w[0], w[1])])
+            assert w[2] == (0 if w[0] == sel.DIRECT else 1)
+        cold = sel.select_kernels(layers, costs, True)
+        sw = sel.switch_set(cold, warm)
+        for i in range(n):
+            differs = (cold[i][0], cold[i][1]) != (warm[i][0], warm[i][1])
+            assert (i in sw) == (differs and warm[i][0] != sel.DIRECT)
+        assert sel.switch_set(warm, warm) == []
