@@ -47,6 +47,7 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="enqueue every call eagerly instead of replaying a recorded CUDA graph")
     ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run reported beside e2e (0 = skip)")
+    ap.add_argument("--continuous-reps", type=int, default=20, help="cold + warm sequences timed for the kernel-switching report (0 = skip)")
     ap.add_argument("--save-costs", default=None, help="write the profiled cost table (JSON) to this file")
     ap.add_argument("--load-costs", default=None, help="use a cost table saved earlier instead of profiling (e.g. under a profiler)")
     return ap.parse_args()
@@ -339,6 +340,46 @@ def run_ours(args):
             model.build_cached_blob(choices_cold)
         model.arena.fill_(0xFF)
 
+    # ---- continuous mode (the paper's Section 3.5): cold inference with K_cold that leaves K_warm prepared,
+    # then warm inferences; latency of the 1st, 2nd and later inferences, end to end from host buffers
+    cont = None
+    if args.continuous_reps > 0:
+        warm = nb.nnv_select_warm(model.plan, costs)
+        cold_c = nb.nnv_select_kernels(model.plan, costs, 1)
+        if any(c is not None and c[2] for c in cold_c):
+            model.build_cached_blob(cold_c)
+        need_c = max(model.ensure_arena(cold_c, 0), model.ensure_arena(warm, 0))
+        wbytes = nb.nnv_warm_bytes(model.plan, warm, model.w_bytes)
+        d_warm = harness.dev_bytes(wbytes)
+        seq = [[], [], [], []]
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        for k in range(args.continuous_reps + 2):
+            flush.fill_(k & 0xFF)
+            torch.cuda.synchronize()
+            evs[0].record(s_exec)
+            s_copy.wait_event(evs[0])
+            s_xform.wait_event(evs[0])
+            nb.nnv_cold_run_continuous(model.plan, cold_c, warm, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes,
+                                       model.h_input, model.h_output, model.arena, need_c, d_warm, wbytes, s_copy, s_xform, s_exec)
+            evs[1].record(s_exec)
+            for j in range(3):
+                nb.nnv_warm_run(model.plan, warm, d_warm, wbytes, model.w_bytes, model.h_input, model.h_output, model.arena,
+                                need_c, s_xform, s_exec)
+                evs[2 + j].record(s_exec)
+            torch.cuda.synchronize()
+            if k >= 2:
+                for j in range(4):
+                    seq[j].append(evs[j].elapsed_time(evs[j + 1]))
+        y_w = model.h_output.numpy().copy()
+        cont = {"first_cold_ms": reduce_max(statistics.mean(seq[0])), "second_ms": reduce_max(statistics.mean(seq[1])),
+                "third_ms": reduce_max(statistics.mean(seq[2])), "fourth_ms": reduce_max(statistics.mean(seq[3])),
+                "switched_layers": len(nb.nnv_switch_set(model.plan, cold_c, warm)), "warm_buffer_bytes": int(wbytes),
+                "parity_rel_l2_end_to_end": None}
+        del d_warm
+        if any(c is not None and c[2] for c in choices_cold):
+            model.build_cached_blob(choices_cold)
+        model.arena.fill_(0xFF)
+
     # ---- per-kernel durations for the roofline (same resident steps, with per-operation events) --
     xf = {}          # layer -> [ns]
     ex = {}
@@ -461,6 +502,7 @@ def run_ours(args):
         "roofline_transform": xroof,
         "transform_all": xall,
         "algorithm1": alg1,
+        "continuous": cont,
         "breakdown": {"sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3, "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
                       "choices_resident": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_res],
                       "choices_cold": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_cold]},
@@ -496,6 +538,8 @@ def run_ours(args):
         line["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_gpu[0] - ref) ** 2)) / den)
         if alg1:
             alg1["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_s[0] - ref) ** 2)) / den)
+        if cont:
+            cont["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_w[0] - ref) ** 2)) / den)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

@@ -179,6 +179,21 @@ nnv_status_t nnv_filter_candidates(const nnv_plan_t* plan, int32_t layer,
 nnv_status_t nnv_select_kernels(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs,
                                 int32_t allow_cached, nnv_choice_t* out);
 
+/* The warm kernel set K_warm of the paper's Section 3.5: per conv layer the
+ * (variant, math) with the least exec_ns among its cost rows -- with every
+ * weight already prepared only execution counts; ties go to the lowest
+ * (variant, math).  out[i].cached = 1 when that kernel reads transformed weights
+ * (which then stay resident), 0 when it reads raw ones; pool layers {-1,-1,0}.
+ * Errors as nnv_select_kernels. */
+nnv_status_t nnv_select_warm(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs,
+                             nnv_choice_t* out);
+
+/* K_warm - K_cold (Section 3.5): the layers whose warm kernel differs from the
+ * cold one in (variant, math) and has a transform -- the weights that remain to
+ * be prepared once the cold inference has what it needs.  Ascending layer order. */
+nnv_status_t nnv_switch_set(const nnv_plan_t* plan, const nnv_choice_t* cold, const nnv_choice_t* warm,
+                            int32_t* layers_out, int32_t cap, int32_t* n_out);
+
 /* ---- scheduling (integer, exact; host only) -------------------------------------------------- */
 
 /* Cold latency of one assignment (the paper's Eq. (1)-(2), Section 3.2): the end
@@ -351,6 +366,40 @@ nnv_status_t nnv_resident_run(nnv_plan_t* plan, const nnv_choice_t* choices,
                               void* d_arena, uint64_t arena_bytes,
                               void* s_xform, void* s_exec,
                               int32_t depth, nnv_timing_t* timings);
+
+/* Continuous mode (the paper's Section 3.5: a cold inference that will be
+ * followed by more).  nnv_cold_run_continuous is nnv_cold_run with depth 0 for
+ * the kernels `cold`, except that what it prepares stays: raw weights and biases
+ * are read into d_warm (same offsets as in the host blob), and a layer whose cold
+ * kernel is also its warm kernel writes its transformed weights into d_warm's
+ * transformed region (nnv_cached_layout order, after the raw copy rounded up to
+ * 1 KiB).  For the layers of nnv_switch_set(cold, warm) -- and for warm kernels
+ * that need raw weights the cold run did not read -- the read and the warm
+ * kernel's transform are queued on s_copy / s_xform BEHIND everything the cold
+ * inference needs, so they use the time those streams would idle while the last
+ * layers execute.  The call returns when h_output holds the cold result; these
+ * preparations may still be running.  nnv_warm_run then executes K_warm from
+ * d_warm (input and output on the host, nothing else crosses the link); the
+ * first call after nnv_cold_run_continuous makes each layer wait for its own
+ * preparation, i.e. the rest is pipelined into the second inference; later
+ * calls wait for nothing and replay a recorded graph.
+ *   d_warm: nnv_warm_bytes() bytes of device memory, the caller's, kept for as
+ *           long as warm runs follow.  warm[i].cached is ignored.
+ *   Results are bit-identical to nnv_cold_run with the same kernels. */
+nnv_status_t nnv_warm_bytes(const nnv_plan_t* plan, const nnv_choice_t* warm, uint64_t w_bytes, uint64_t* bytes);
+nnv_status_t nnv_cold_run_continuous(nnv_plan_t* plan, const nnv_choice_t* cold, const nnv_choice_t* warm,
+                                     const void* h_weights, uint64_t w_bytes,
+                                     const void* h_cached, uint64_t c_bytes,
+                                     const float* h_input, float* h_output,
+                                     void* d_arena, uint64_t arena_bytes,
+                                     void* d_warm, uint64_t warm_bytes,
+                                     void* s_copy, void* s_xform, void* s_exec,
+                                     nnv_timing_t* timings);
+nnv_status_t nnv_warm_run(nnv_plan_t* plan, const nnv_choice_t* warm,
+                          const void* d_warm, uint64_t warm_bytes, uint64_t w_bytes,
+                          const float* h_input, float* h_output,
+                          void* d_arena, uint64_t arena_bytes,
+                          void* s_xform, void* s_exec, nnv_timing_t* timings);
 
 /* Device address, inside the arena of the most recent nnv_cold_run on this
  * plan, of layer `layer`'s NHWC fp32 output (valid until the arena is reused). */

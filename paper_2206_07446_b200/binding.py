@@ -72,6 +72,8 @@ _SIGS = {
     "nnv_cached_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
     "nnv_filter_candidates": [_vp, _i32, _P(Cost), _i32, _i32, _P(Choice), _i32, _P(_i32)],
     "nnv_select_kernels": [_vp, _P(Cost), _i32, _i32, _P(Choice)],
+    "nnv_select_warm": [_vp, _P(Cost), _i32, _P(Choice)],
+    "nnv_switch_set": [_vp, _P(Choice), _P(Choice), _P(_i32), _i32, _P(_i32)],
     "nnv_simulate": [_vp, _P(_u64), _P(_u64), _P(_u64), _P(_i32), _i32, _P(_u64)],
     "nnv_schedule_queues": [_vp, _P(_u64), _P(_u64), _P(_u64), _i32, _u64, _P(_i32), _P(_u64)],
     "nnv_schedule": [_vp, _P(Cost), _i32, _i32, _P(_u64), _i32, _u64, _i32, _u64, _P(Choice), _P(_i32), _P(_u64)],
@@ -86,6 +88,10 @@ _SIGS = {
     "nnv_cold_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing)],
     "nnv_cold_run_queues": [_vp, _P(Choice), _P(_i32), _i32, _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _P(_vp), _P(Timing)],
     "nnv_resident_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _i32, _P(Timing)],
+    "nnv_warm_bytes": [_vp, _P(Choice), _u64, _P(_u64)],
+    "nnv_cold_run_continuous": [_vp, _P(Choice), _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _u64, _vp, _vp, _vp,
+                                _P(Timing)],
+    "nnv_warm_run": [_vp, _P(Choice), _vp, _u64, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _P(Timing)],
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
     "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
@@ -241,6 +247,22 @@ def nnv_select_kernels(plan, costs, allow_cached):
     return [None if out[i].variant < 0 else (out[i].variant, out[i].math, out[i].cached) for i in range(plan.n)]
 
 
+def nnv_select_warm(plan, costs):
+    """K_warm: per conv layer the kernel with the least execution time, as (variant, math, prepared)."""
+    out = (Choice * plan.n)()
+    _check(_lib.nnv_select_warm(plan.handle, _costs_array(costs), len(costs), out))
+    return [None if out[i].variant < 0 else (out[i].variant, out[i].math, out[i].cached) for i in range(plan.n)]
+
+
+def nnv_switch_set(plan, cold, warm):
+    """Layers of K_warm - K_cold."""
+    out = (_i32 * max(1, plan.n))()
+    n = _i32(0)
+    _check(_lib.nnv_switch_set(plan.handle, _choices_array(plan, cold), _choices_array(plan, warm), out, plan.n,
+                               ctypes.byref(n)))
+    return [int(out[i]) for i in range(n.value)]
+
+
 def _u64_array(plan, values):
     if len(values) != plan.n:
         raise ValueError("one entry per layer expected")
@@ -340,6 +362,31 @@ def nnv_cold_run_queues(plan, choices, queue_of, n_little, h_weights, w_bytes, h
                                     (_i32 * plan.n)(*[int(q) for q in queue_of]), int(n_little), _ptr(h_weights),
                                     int(w_bytes), _ptr(h_cached), int(c_bytes), _ptr(h_input), _ptr(h_output),
                                     _ptr(d_arena), int(arena_bytes), sarr, tarr))
+    return _timings_list(tarr)
+
+
+def nnv_warm_bytes(plan, warm, w_bytes):
+    b = _u64(0)
+    _check(_lib.nnv_warm_bytes(plan.handle, _choices_array(plan, warm), int(w_bytes), ctypes.byref(b)))
+    return int(b.value)
+
+
+def nnv_cold_run_continuous(plan, cold, warm, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena,
+                            arena_bytes, d_warm, warm_bytes, s_copy, s_xform, s_exec, want_timings=False):
+    tarr = (Timing * plan.n)() if want_timings else None
+    _check(_lib.nnv_cold_run_continuous(plan.handle, _choices_array(plan, cold), _choices_array(plan, warm),
+                                        _ptr(h_weights), int(w_bytes), _ptr(h_cached), int(c_bytes), _ptr(h_input),
+                                        _ptr(h_output), _ptr(d_arena), int(arena_bytes), _ptr(d_warm), int(warm_bytes),
+                                        _stream(s_copy), _stream(s_xform), _stream(s_exec), tarr))
+    return _timings_list(tarr)
+
+
+def nnv_warm_run(plan, warm, d_warm, warm_bytes, w_bytes, h_input, h_output, d_arena, arena_bytes, s_xform, s_exec,
+                 want_timings=False):
+    tarr = (Timing * plan.n)() if want_timings else None
+    _check(_lib.nnv_warm_run(plan.handle, _choices_array(plan, warm), _ptr(d_warm), int(warm_bytes), int(w_bytes),
+                             _ptr(h_input), _ptr(h_output), _ptr(d_arena), int(arena_bytes), _stream(s_xform),
+                             _stream(s_exec), tarr))
     return _timings_list(tarr)
 
 

@@ -110,9 +110,10 @@ struct GraphKey {
     uint64_t w_bytes = 0;
     int depth = 0;
     bool resident = false;
+    bool host_io = false;
     std::vector<int32_t> queues;          // preparation queue per layer (scheduled runs), else empty
     bool operator==(const GraphKey& o) const {
-        if (ptrs != o.ptrs || w_bytes != o.w_bytes || depth != o.depth || resident != o.resident ||
+        if (ptrs != o.ptrs || w_bytes != o.w_bytes || depth != o.depth || resident != o.resident || host_io != o.host_io ||
             queues != o.queues || choices.size() != o.choices.size())
             return false;
         for (size_t i = 0; i < choices.size(); ++i)
@@ -139,6 +140,8 @@ struct nnv_plan {
     const void* last_arena = nullptr;
     std::vector<nnv::CachedGraph> graphs;   // recorded passes, one per distinct argument set
     int* h_status = nullptr;              // pinned host word the device status is copied into
+    std::vector<cudaEvent_t> warm_ev;     // continuous mode: layer i's warm weights are prepared
+    bool warm_pending = false;            // warm preparations may still be running (first warm run waits)
 };
 
 namespace nnv {

@@ -34,13 +34,27 @@ namespace nnv {
 
 // One pass over the layer list.  `resident` = the read stage is already done: weights, cached
 // blob, input and output are device buffers and nothing crosses the host link.
+// Continuous mode (the paper's Section 3.5): where the warm kernel set K_warm is to be left behind.
+// d_warm holds a copy of the raw weight blob (same offsets as the host blob) followed, at
+// xf_region, by the transformed weights of K_warm laid out by nnv_cached_layout().
+struct WarmCtx {
+    const nnv_choice_t* warm;
+    uint8_t* d_warm;
+    uint64_t xf_region;
+    std::vector<uint64_t> woff;
+};
+
+static bool same_kernel(const nnv_choice_t& a, const nnv_choice_t& b) { return a.variant == b.variant && a.math == b.math; }
+
 static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const void* weights, uint64_t w_bytes,
                               const void* cached_blob, uint64_t c_bytes, const float* input, float* output,
                               void* d_arena, uint64_t arena_bytes, cudaStream_t s_copy, cudaStream_t s_xform,
                               cudaStream_t s_exec, int depth, nnv_timing_t* timings, bool resident,
-                              const int32_t* queue_of = nullptr, const cudaStream_t* s_prep = nullptr, int n_little = 0) {
+                              const int32_t* queue_of = nullptr, const cudaStream_t* s_prep = nullptr, int n_little = 0,
+                              int io_host = -1, const WarmCtx* wc = nullptr, bool wait_warm = false) {
     const int n = (int)p->layers.size();
     const bool queued = queue_of != nullptr;        // preparations follow a schedule: queue 0 = s_exec, j = s_prep[j-1]
+    const bool host_io = io_host < 0 ? !resident : io_host != 0;   // input / output are host buffers
     ArenaLayout A;
     NNV_TRY(layout_arena(*p, choices, depth, &A));
     NNV_REQUIRE(arena_bytes >= A.total, NNV_ERR_WORKSPACE_TOO_SMALL, "arena needs %llu bytes, got %llu",
@@ -59,6 +73,10 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                     NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the weight blob", i);
     }
     NNV_TRY(ensure_events(*p, timings != nullptr));
+    if (wc && p->warm_ev.size() != (size_t)n) {
+        p->warm_ev.assign(n, nullptr);
+        for (int i = 0; i < n; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p->warm_ev[i], cudaEventDisableTiming));
+    }
     if (!p->h_status) NNV_CUDA(cudaHostAlloc((void**)&p->h_status, sizeof(int), cudaHostAllocDefault));
     p->last_layout = A;
     p->last_arena = d_arena;
@@ -87,7 +105,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // model input: NCHW -> device NHWC, on the execution stream
     const nnv_layer_desc_t& L0 = p->layers[0];
     const float* in_chw = input;
-    if (!resident) {
+    if (host_io) {
         NNV_CUDA(cudaMemcpyAsync(base + A.in_chw, input, 4ull * L0.C * L0.H * L0.W, cudaMemcpyHostToDevice, s_exec));
         in_chw = (const float*)(base + A.in_chw);
     }
@@ -147,6 +165,13 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         const bool has_xf = variant_has_transform(ch.variant);
         const bool cached = has_xf && ch.cached;
         const uint64_t rbytes = raw_weight_bytes(L), tbytes = transformed_bytes(*p, i, ch.variant, ch.math);
+        if (wc) {
+            // raw weights and biases are read straight into the copy that stays; a kernel that is also
+            // the warm one writes its transformed weights where the warm runs will look for them
+            raw = wc->d_warm + L.w_off;
+            bias = wc->d_warm + L.b_off;
+            if (has_xf && same_kernel(ch, wc->warm[i])) xf = wc->d_warm + wc->xf_region + wc->woff[i];
+        }
         cudaEvent_t ready = nullptr;
         uint64_t copied = 0;
 
@@ -216,6 +241,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
 
         // execute
         if (ready) NNV_CUDA(cudaStreamWaitEvent(s_exec, ready, 0));
+        if (wait_warm && i < (int)p->warm_ev.size() && p->warm_ev[i]) NNV_CUDA(cudaStreamWaitEvent(s_exec, p->warm_ev[i], 0));
         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), s_exec));
         const void* add = L.in1 >= 0 ? base + A.act_off[L.in1] : nullptr;
         NNV_TRY(do_exec(*p, i, ch.variant, ch.math, in, add, has_xf ? xf : raw, L.has_bias ? bias : nullptr, out,
@@ -233,9 +259,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // last layer's output: device NHWC -> NCHW
     const nnv_layer_desc_t& Ln = p->layers[n - 1];
     const LayerGeom& gn = p->geom[n - 1];
-    float* out_chw = resident ? output : (float*)(base + A.out_chw);
+    float* out_chw = host_io ? (float*)(base + A.out_chw) : output;
     NNV_TRY(launch_hwc_to_chw((const float*)(base + A.act_off[n - 1]), out_chw, Ln.K, gn.OH, gn.OW, s_exec));
-    if (!resident) NNV_CUDA(cudaMemcpyAsync(output, out_chw, 4ull * gn.P * Ln.K, cudaMemcpyDeviceToHost, s_exec));
+    if (host_io) NNV_CUDA(cudaMemcpyAsync(output, out_chw, 4ull * gn.P * Ln.K, cudaMemcpyDeviceToHost, s_exec));
     if (queued) {
         for (int j = 0; j < n_little; ++j) {
             NNV_CUDA(cudaEventRecord(p->ev[3 * n + 6 + j], s_prep[j]));
@@ -250,6 +276,36 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         NNV_CUDA(cudaStreamWaitEvent(s_exec, p->ev[3 * n + 2], 0));
     }
     NNV_TRY(enqueue_status_read(p->h_status, s_exec));
+    if (wc) {
+        // K_warm - K_cold: behind everything the cold inference needs (the streams are idle from here
+        // on, and s_exec no longer waits for them), read what was not read yet and transform it with
+        // the warm kernel.  The first warm run waits for warm_ev[i] before executing layer i.
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p->layers[i];
+            if (L.op != NNV_OP_CONV) continue;
+            const nnv_choice_t ch = choices[i], wm = wc->warm[i];
+            const bool cold_read_raw = !(variant_has_transform(ch.variant) && ch.cached);
+            const bool warm_xf = variant_has_transform(wm.variant);
+            if (same_kernel(ch, wm) || (cold_read_raw && !warm_xf)) continue;     // nothing left to prepare
+            uint8_t* raw = wc->d_warm + L.w_off;
+            if (!cold_read_raw) {
+                NNV_CUDA(cudaMemcpyAsync(raw, (const uint8_t*)weights + L.w_off, raw_weight_bytes(L), cudaMemcpyHostToDevice, s_copy));
+                NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
+            }
+            cudaEvent_t done = EV(i, 0);
+            if (warm_xf) {
+                NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(i, 0), 0));
+                NNV_TRY(do_transform(*p, i, wm.variant, wm.math, raw, wc->d_warm + wc->xf_region + wc->woff[i], s_xform));
+                NNV_CUDA(cudaEventRecord(p->warm_ev[i], s_xform));
+                done = p->warm_ev[i];
+            } else {
+                NNV_CUDA(cudaEventRecord(p->warm_ev[i], s_copy));
+                done = p->warm_ev[i];
+            }
+            (void)done;
+            p->warm_pending = true;
+        }
+    }
     return NNV_OK;
     };  // enqueue
 
@@ -259,13 +315,13 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     GraphKey key;
     key.choices.assign(choices, choices + n);
     key.ptrs = {weights, cached_blob, input, output, d_arena};
-    key.w_bytes = w_bytes; key.depth = depth; key.resident = resident;
+    key.w_bytes = w_bytes; key.depth = depth; key.resident = resident; key.host_io = host_io;
     if (queued) {
         key.queues.assign(queue_of, queue_of + n);
         key.queues.push_back(n_little);
     }
     CachedGraph* cg = nullptr;
-    if (!tm && p->opts.use_graphs) {
+    if (!tm && p->opts.use_graphs && !wc && !wait_warm) {
         for (CachedGraph& g : p->graphs)
             if (g.key == key) { cg = &g; break; }
         if (!cg) {
@@ -383,6 +439,77 @@ nnv_status_t nnv_resident_run(nnv_plan_t* p, const nnv_choice_t* choices, const 
     NNV_REQUIRE(s_xform != s_exec, NNV_ERR_INVALID_ARG, "the two streams must be distinct");
     return run_model(p, choices, d_weights, w_bytes, d_cached, c_bytes, d_input, d_output, d_arena, arena_bytes,
                      nullptr, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings, true);
+}
+
+// ---- continuous mode: cold inference that leaves K_warm behind, then warm inferences ----------
+namespace {
+// Warm choices with the `cached` flag normalised: kernels with a transform read the prepared copy.
+nnv_status_t warm_layout(const nnv_plan& p, const nnv_choice_t* warm, uint64_t w_bytes, std::vector<nnv_choice_t>* norm,
+                         std::vector<uint64_t>* woff, uint64_t* xf_region, uint64_t* total) {
+    const int n = (int)p.layers.size();
+    norm->assign(warm, warm + n);
+    for (int i = 0; i < n; ++i) {
+        if (p.layers[i].op != NNV_OP_CONV) continue;
+        NNV_TRY(check_choice(p, i, warm[i].variant, warm[i].math));
+        (*norm)[i].cached = variant_has_transform(warm[i].variant) ? 1 : 0;
+    }
+    woff->assign(n, 0);
+    uint64_t xf_total = 0;
+    NNV_TRY(nnv_cached_layout(&p, norm->data(), woff->data(), &xf_total));
+    *xf_region = align_up(w_bytes, 1024);
+    *total = *xf_region + xf_total;
+    return NNV_OK;
+}
+}  // namespace
+
+nnv_status_t nnv_warm_bytes(const nnv_plan_t* p, const nnv_choice_t* warm, uint64_t w_bytes, uint64_t* bytes) {
+    NNV_REQUIRE(p && warm && bytes, NNV_ERR_INVALID_ARG, "null argument");
+    std::vector<nnv_choice_t> norm;
+    std::vector<uint64_t> woff;
+    uint64_t region = 0;
+    return warm_layout(*p, warm, w_bytes, &norm, &woff, &region, bytes);
+}
+
+nnv_status_t nnv_cold_run_continuous(nnv_plan_t* p, const nnv_choice_t* cold, const nnv_choice_t* warm,
+                                     const void* h_weights, uint64_t w_bytes, const void* h_cached, uint64_t c_bytes,
+                                     const float* h_input, float* h_output, void* d_arena, uint64_t arena_bytes,
+                                     void* d_warm, uint64_t warm_bytes, void* s_copy, void* s_xform, void* s_exec,
+                                     nnv_timing_t* timings) {
+    NNV_REQUIRE(p && cold && warm && h_weights && h_input && h_output && d_arena && d_warm, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(aligned256(d_arena) && aligned256(d_warm), NNV_ERR_INVALID_ARG, "device buffers must be 256-byte aligned");
+    NNV_REQUIRE(s_copy != s_xform && s_copy != s_exec && s_xform != s_exec, NNV_ERR_INVALID_ARG,
+                "the three streams must be distinct");
+    WarmCtx wc;
+    std::vector<nnv_choice_t> norm;
+    uint64_t need = 0;
+    NNV_TRY(warm_layout(*p, warm, w_bytes, &norm, &wc.woff, &wc.xf_region, &need));
+    NNV_REQUIRE(warm_bytes >= need, NNV_ERR_WORKSPACE_TOO_SMALL, "warm buffer needs %llu bytes, got %llu",
+                (unsigned long long)need, (unsigned long long)warm_bytes);
+    wc.warm = norm.data();
+    wc.d_warm = (uint8_t*)d_warm;
+    return run_model(p, cold, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena, arena_bytes,
+                     (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, 0, timings, false, nullptr, nullptr, 0,
+                     -1, &wc, false);
+}
+
+nnv_status_t nnv_warm_run(nnv_plan_t* p, const nnv_choice_t* warm, const void* d_warm, uint64_t warm_bytes, uint64_t w_bytes,
+                          const float* h_input, float* h_output, void* d_arena, uint64_t arena_bytes, void* s_xform,
+                          void* s_exec, nnv_timing_t* timings) {
+    NNV_REQUIRE(p && warm && d_warm && h_input && h_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(aligned256(d_arena) && aligned256(d_warm), NNV_ERR_INVALID_ARG, "device buffers must be 256-byte aligned");
+    NNV_REQUIRE(s_xform != s_exec, NNV_ERR_INVALID_ARG, "the two streams must be distinct");
+    std::vector<nnv_choice_t> norm;
+    std::vector<uint64_t> woff;
+    uint64_t region = 0, need = 0;
+    NNV_TRY(warm_layout(*p, warm, w_bytes, &norm, &woff, &region, &need));
+    NNV_REQUIRE(warm_bytes >= need, NNV_ERR_WORKSPACE_TOO_SMALL, "warm buffer needs %llu bytes, got %llu",
+                (unsigned long long)need, (unsigned long long)warm_bytes);
+    const bool wait = p->warm_pending;
+    const nnv_status_t rc = run_model(p, norm.data(), d_warm, w_bytes, (const uint8_t*)d_warm + region, need - region, h_input,
+                                      h_output, d_arena, arena_bytes, nullptr, (cudaStream_t)s_xform, (cudaStream_t)s_exec, 0,
+                                      timings, true, nullptr, nullptr, 0, 1, nullptr, wait);
+    if (rc == NNV_OK) p->warm_pending = false;       // every preparation this run waited for has finished
+    return rc;
 }
 
 nnv_status_t nnv_layer_output(const nnv_plan_t* p, int32_t layer, const void** d_ptr, uint64_t* bytes) {

@@ -294,6 +294,8 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* p) {
     if (!p) return NNV_OK;
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     for (cudaEvent_t e : p->tev) cudaEventDestroy(e);
+    for (cudaEvent_t e : p->warm_ev)
+        if (e) cudaEventDestroy(e);
     if (p->h_status) cudaFreeHost(p->h_status);
     for (nnv::CachedGraph& g : p->graphs)
         if (g.exec) cudaGraphExecDestroy(g.exec);
@@ -383,6 +385,37 @@ nnv_status_t nnv_select_kernels(const nnv_plan_t* p, const nnv_cost_t* costs, in
             if (!best || o.prep + o.exec < best->prep + best->exec) best = &o;
         out[i] = nnv_choice_t{best->variant, best->math, best->cached};
     }
+    return NNV_OK;
+}
+
+nnv_status_t nnv_select_warm(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, nnv_choice_t* out) {
+    NNV_REQUIRE(p && costs && out, NNV_ERR_INVALID_ARG, "null argument");
+    for (int i = 0; i < (int)p->layers.size(); ++i) {
+        out[i] = nnv_choice_t{-1, -1, 0};
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        std::vector<Option> opts;
+        NNV_TRY(gather_options(*p, i, costs, n_costs, 0, &opts));     // raw arms only: one option per kernel, rank order
+        NNV_REQUIRE(!opts.empty(), NNV_ERR_STATE, "no cost rows for conv layer %d", i);
+        const Option* best = nullptr;
+        for (const Option& o : opts)
+            if (!best || o.exec < best->exec) best = &o;             // first minimum wins ties
+        out[i] = nnv_choice_t{best->variant, best->math, variant_has_transform(best->variant) ? 1 : 0};
+    }
+    return NNV_OK;
+}
+
+nnv_status_t nnv_switch_set(const nnv_plan_t* p, const nnv_choice_t* cold, const nnv_choice_t* warm, int32_t* layers_out,
+                            int32_t cap, int32_t* n_out) {
+    NNV_REQUIRE(p && cold && warm && layers_out && n_out, NNV_ERR_INVALID_ARG, "null argument");
+    int cnt = 0;
+    for (int i = 0; i < (int)p->layers.size(); ++i) {
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        if (cold[i].variant == warm[i].variant && cold[i].math == warm[i].math) continue;
+        if (!variant_has_transform(warm[i].variant)) continue;
+        NNV_REQUIRE(cnt < cap, NNV_ERR_INVALID_ARG, "output capacity %d too small", cap);
+        layers_out[cnt++] = i;
+    }
+    *n_out = cnt;
     return NNV_OK;
 }
 

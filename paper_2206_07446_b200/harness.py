@@ -172,6 +172,29 @@ class Model:
                           xform_ns=int(c["xform_ns"] * f["xform"]), exec_ns=int(c["exec_ns"] * f["exec"])) for c in costs]
         return out[0], out[1], out[2], table
 
+    def cold_run_continuous(self, x_nchw, cold, warm, want_timings=False):
+        """Cold inference with kernels `cold` that leaves the kernels `warm` prepared in a device buffer
+        (nnv_cold_run_continuous); returns (output NCHW numpy, timings)."""
+        self.h_input.copy_(torch.from_numpy(np.ascontiguousarray(x_nchw, dtype=np.float32)).reshape(self.h_input.shape))
+        need = self.ensure_arena(cold, 0)
+        need = max(need, self.ensure_arena(warm, 0))
+        self.warm_bytes = nb.nnv_warm_bytes(self.plan, warm, self.w_bytes)
+        if getattr(self, "d_warm", None) is None or self.d_warm.numel() < self.warm_bytes:
+            self.d_warm = dev_bytes(self.warm_bytes)
+        torch.cuda.synchronize()
+        tm = nb.nnv_cold_run_continuous(self.plan, cold, warm, self.h_weights, self.w_bytes, self.h_cached, self.c_bytes,
+                                        self.h_input, self.h_output, self.arena, self.arena.numel(), self.d_warm, self.warm_bytes,
+                                        self.streams[0], self.streams[1], self.streams[2], want_timings)
+        return self.h_output.numpy().copy(), tm
+
+    def warm_run(self, x_nchw, warm, want_timings=False):
+        """One warm inference from the buffer a continuous cold run left behind (nnv_warm_run)."""
+        if x_nchw is not None:
+            self.h_input.copy_(torch.from_numpy(np.ascontiguousarray(x_nchw, dtype=np.float32)).reshape(self.h_input.shape))
+        tm = nb.nnv_warm_run(self.plan, warm, self.d_warm, self.warm_bytes, self.w_bytes, self.h_input, self.h_output,
+                             self.arena, self.arena.numel(), self.streams[1], self.streams[2], want_timings)
+        return self.h_output.numpy().copy(), tm
+
     def to_device(self):
         """Device copies of the weight blob, the cached blob (if built) and I/O buffers for nnv_resident_run."""
         self.d_weights = dev_bytes(self.w_bytes, fill=None)

@@ -95,6 +95,21 @@ def test_selection_matches_oracle_bit_exact(seed):
             assert nb.nnv_filter_candidates(plan, i, costs, allow) == want
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_warm_selection_and_switch_set_match_oracle(seed):
+    """K_warm (least execution time) and K_warm - K_cold, exactly as the oracle has them."""
+    rng = np.random.default_rng(100 + seed)
+    layers = [wl.tiny_net, wl.cfg2_resnet18, wl.cfg3_mobilenetv2][seed % 3]()
+    plan = _plan(layers)
+    costs = _random_costs(layers, rng, hi=6 if seed % 2 else 10 ** 9)
+    warm = nb.nnv_select_warm(plan, costs)
+    assert warm == osel.select_warm(layers, costs)
+    for allow in (0, 1):
+        cold = nb.nnv_select_kernels(plan, costs, allow)
+        assert nb.nnv_switch_set(plan, cold, warm) == osel.switch_set(cold, warm)
+    assert nb.nnv_switch_set(plan, warm, warm) == []
+
+
 def test_selection_on_paper_table2_shaped_costs():
     """The paper's Table 2 numbers mapped onto this library's variants for a 64->192 3x3 layer:
     winograd-pack4 -> WINO_F6/TF32, winograd -> WINO_F4/TF32, sgemm-pack4 -> IM2COL/TF32, 3x3s1 -> DIRECT."""
@@ -112,6 +127,10 @@ def test_selection_on_paper_table2_shaped_costs():
     assert nb.nnv_select_kernels(plan, costs, 1) == [(nb.VAR_WINO_F4, 1, 1)]       # cached winograd: 7.49 ms
     assert nb.nnv_select_kernels(plan, costs, 0) == [(nb.VAR_DIRECT, 0, 0)]        # raw only: 3x3s1, 8.71 ms
     assert nb.nnv_filter_candidates(plan, 0, costs, 1) == [(nb.VAR_DIRECT, 0, 0), (nb.VAR_WINO_F4, 1, 1), (nb.VAR_WINO_F6, 1, 1)]
+    # warm inference: winograd-pack4 executes fastest (2.98 ms), so K_warm differs from both cold choices
+    warm = nb.nnv_select_warm(plan, costs)
+    assert warm == [(nb.VAR_WINO_F6, 1, 1)]
+    assert nb.nnv_switch_set(plan, nb.nnv_select_kernels(plan, costs, 1), warm) == [0]
 
 
 def test_plan_validation_errors():
