@@ -48,6 +48,7 @@ def parse():
     ap.add_argument("--no-graphs", action="store_true", help="enqueue every call eagerly instead of replaying a recorded CUDA graph")
     ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run reported beside e2e (0 = skip)")
     ap.add_argument("--continuous-reps", type=int, default=20, help="cold + warm sequences timed for the kernel-switching report (0 = skip)")
+    ap.add_argument("--file-reps", type=int, default=20, help="cold runs fed from a model file on local storage (0 = skip)")
     ap.add_argument("--save-costs", default=None, help="write the profiled cost table (JSON) to this file")
     ap.add_argument("--load-costs", default=None, help="use a cost table saved earlier instead of profiling (e.g. under a profiler)")
     return ap.parse_args()
@@ -380,6 +381,39 @@ def run_ours(args):
             model.build_cached_blob(choices_cold)
         model.arena.fill_(0xFF)
 
+    # ---- storage stage: the same end-to-end step with the weights read from a model file (page cache
+    # dropped before every run), the paper's "weights reading" in front of copy / transform / execution
+    storage = None
+    if args.file_reps > 0:
+        path = os.path.join(tempfile.gettempdir(), "nnv_bench_%d_%d.nnv" % (os.getpid(), rank))
+        try:
+            model.write_model_file(path, choices_cold)
+            cache = nb.CacheFile(path)
+            ts, rd_ns, rd_b = [], [], []
+            for k in range(args.file_reps + 2):
+                flush.fill_(k & 0xFF)
+                torch.cuda.synchronize()
+                cache.drop_pages()
+                evs2 = [torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)]
+                evs2[0].record(s_exec)
+                s_copy.wait_event(evs2[0])
+                s_xform.wait_event(evs2[0])
+                _, _, ns, nbytes = model.cold_run_file(None, choices_cold, cache, depth=args.cold_depth, drop_pages=False)
+                evs2[1].record(s_exec)
+                evs2[1].synchronize()
+                if k >= 2:
+                    ts.append(evs2[0].elapsed_time(evs2[1])); rd_ns.append(ns); rd_b.append(nbytes)
+            raw_total = sum(4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"] for L in layers if L["op"] == wl.OP_CONV)
+            storage = {"e2e_from_file_ms": reduce_max(statistics.mean(ts)), "file_bytes": int(cache.file_bytes),
+                       "raw_weight_bytes": int(raw_total), "cached_blob_bytes": int(cache.c_bytes),
+                       "bytes_read_per_step": int(rd_b[-1]), "reader_gbs": rd_b[-1] / statistics.mean(rd_ns),
+                       "page_cache": "posix_fadvise DONTNEED before every run (best effort)"}
+            cache.close()
+        finally:
+            if os.path.exists(path):
+                os.unlink(path)
+        model.arena.fill_(0xFF)
+
     # ---- per-kernel durations for the roofline (same resident steps, with per-operation events) --
     xf = {}          # layer -> [ns]
     ex = {}
@@ -503,6 +537,7 @@ def run_ours(args):
         "transform_all": xall,
         "algorithm1": alg1,
         "continuous": cont,
+        "storage": storage,
         "breakdown": {"sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3, "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
                       "choices_resident": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_res],
                       "choices_cold": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_cold]},

@@ -58,6 +58,7 @@ typedef enum {
 } nnv_status_t;
 
 typedef struct nnv_plan nnv_plan_t;   /* opaque; created by nnv_plan_create */
+typedef struct nnv_cache nnv_cache_t; /* opaque; an open model file, created by nnv_cache_open */
 
 typedef enum { NNV_OP_CONV = 0, NNV_OP_MAXPOOL = 1, NNV_OP_GAVGPOOL = 2 } nnv_op_t;
 
@@ -400,6 +401,70 @@ nnv_status_t nnv_warm_run(nnv_plan_t* plan, const nnv_choice_t* warm,
                           const float* h_input, float* h_output,
                           void* d_arena, uint64_t arena_bytes,
                           void* s_xform, void* s_exec, nnv_timing_t* timings);
+
+/* ---- model file: what the decision stage leaves in storage ----------------------------------- */
+
+/* The paper's decision stage writes a kernel scheduling plan and the
+ * post-transformed weights to storage (its Sections 3 and 3.1.2; Table 4 counts
+ * the storage overhead); the cold inference starts by reading weights from
+ * there (Section 2, "weights reading").  The paper prints no file layout; this
+ * library's is (all integers little-endian):
+ *   header, 64 bytes: 8 bytes magic "NNV12WC\0", u32 version = 1, u32 n_layers,
+ *       u64 w_bytes, u64 c_bytes, u64 raw_off = round_up(64 + 88 n_layers, 4096),
+ *       u64 cached_off = raw_off + round_up(w_bytes, 4096), u32 n_little, u32 0,
+ *       u64 FNV-1a (64 bit) of the two tables;
+ *   layer table, 72 bytes per layer: nnv_layer_desc_t as declared above;
+ *   plan table, 16 bytes per layer: i32 variant, math, cached, queue
+ *       (-1, -1, 0, -1 for pool layers; queue -1 when no schedule is stored);
+ *   zero padding; the raw weight blob at raw_off; zero padding; the cached blob
+ *   (nnv_cached_layout of the stored choices) at cached_off; zero padding to a
+ *   multiple of 4096.
+ * nnv_cache_write creates / replaces `path` from host buffers and fsyncs it.
+ * queue_of / n_little: a schedule from nnv_schedule, or NULL / 0.  h_cached may be
+ * NULL when no stored choice has cached = 1.  I/O failures -> NNV_ERR_STATE. */
+nnv_status_t nnv_cache_write(const char* path, const nnv_plan_t* plan, const nnv_choice_t* choices,
+                             const int32_t* queue_of, int32_t n_little,
+                             const void* h_weights, uint64_t w_bytes,
+                             const void* h_cached, uint64_t c_bytes);
+
+/* Open a model file and check it: magic, version, offsets against the file
+ * size, table hash (anything wrong -> NNV_ERR_INVALID_ARG; cannot open / read
+ * -> NNV_ERR_STATE).  The blobs are not read.  Close with nnv_cache_close. */
+nnv_status_t nnv_cache_open(const char* path, nnv_cache_t** out);
+nnv_status_t nnv_cache_close(nnv_cache_t* cache);
+/* Sizes stored in the header; any output pointer may be NULL. */
+nnv_status_t nnv_cache_info(const nnv_cache_t* cache, int32_t* n_layers, uint64_t* w_bytes, uint64_t* c_bytes,
+                            int32_t* n_little, uint64_t* file_bytes);
+/* The stored layer descriptors, choices and (if queue_of != NULL) queues; cap = entries per array. */
+nnv_status_t nnv_cache_read_plan(const nnv_cache_t* cache, nnv_layer_desc_t* layers, nnv_choice_t* choices,
+                                 int32_t* queue_of, int32_t cap);
+/* Read the whole raw blob (and, if h_cached != NULL, the cached blob) into host buffers. */
+nnv_status_t nnv_cache_read_blobs(const nnv_cache_t* cache, void* h_weights, uint64_t w_cap,
+                                  void* h_cached, uint64_t c_cap);
+/* Ask the operating system to drop the file's pages from its cache
+ * (posix_fadvise DONTNEED), so that the next reads come from the device again:
+ * the paper clears caches before each cold run.  Best effort. */
+nnv_status_t nnv_cache_drop_pages(const nnv_cache_t* cache);
+
+/* nnv_cold_run with the weights still in storage: a reader thread walks the
+ * layers in order and reads, from the open model file into the PINNED staging
+ * buffers, exactly the bytes each layer's choice consumes (its cached blob entry
+ * if cached = 1, else its raw weights; its bias), and each layer's host->device
+ * copy is issued as soon as its bytes have arrived -- storage -> host memory
+ * becomes a fourth pipeline stage in front of copy, transform and execution.
+ *   h_stage_weights: pinned, >= the file's w_bytes; h_stage_cached: pinned, >= the
+ *       cached bytes these choices read, or NULL if none is cached.
+ *   Layers read with cached = 1 must be stored in the file with the same kernel
+ *       and at the same cached-blob offset, else NNV_ERR_INVALID_ARG.
+ *   read_ns / read_bytes (nullable): wall time the reader took and bytes it read.
+ * Everything else as nnv_cold_run; the result is bit-identical to it. */
+nnv_status_t nnv_cold_run_file(nnv_plan_t* plan, const nnv_choice_t* choices, const nnv_cache_t* cache,
+                               void* h_stage_weights, uint64_t stage_w_bytes,
+                               void* h_stage_cached, uint64_t stage_c_bytes,
+                               const float* h_input, float* h_output,
+                               void* d_arena, uint64_t arena_bytes,
+                               void* s_copy, void* s_xform, void* s_exec, int32_t depth,
+                               nnv_timing_t* timings, uint64_t* read_ns, uint64_t* read_bytes);
 
 /* Device address, inside the arena of the most recent nnv_cold_run on this
  * plan, of layer `layer`'s NHWC fp32 output (valid until the arena is reused). */

@@ -92,6 +92,15 @@ _SIGS = {
     "nnv_cold_run_continuous": [_vp, _P(Choice), _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _u64, _vp, _vp, _vp,
                                 _P(Timing)],
     "nnv_warm_run": [_vp, _P(Choice), _vp, _u64, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _P(Timing)],
+    "nnv_cache_write": [ctypes.c_char_p, _vp, _P(Choice), _P(_i32), _i32, _vp, _u64, _vp, _u64],
+    "nnv_cache_open": [ctypes.c_char_p, _P(_vp)],
+    "nnv_cache_close": [_vp],
+    "nnv_cache_info": [_vp, _P(_i32), _P(_u64), _P(_u64), _P(_i32), _P(_u64)],
+    "nnv_cache_read_plan": [_vp, _P(LayerDesc), _P(Choice), _P(_i32), _i32],
+    "nnv_cache_read_blobs": [_vp, _vp, _u64, _vp, _u64],
+    "nnv_cache_drop_pages": [_vp],
+    "nnv_cold_run_file": [_vp, _P(Choice), _vp, _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing),
+                          _P(_u64), _P(_u64)],
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
     "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
@@ -388,6 +397,63 @@ def nnv_warm_run(plan, warm, d_warm, warm_bytes, w_bytes, h_input, h_output, d_a
                              _ptr(h_input), _ptr(h_output), _ptr(d_arena), int(arena_bytes), _stream(s_xform),
                              _stream(s_exec), tarr))
     return _timings_list(tarr)
+
+
+def nnv_cache_write(path, plan, choices, queue_of, n_little, h_weights, w_bytes, h_cached, c_bytes):
+    q = None if queue_of is None else (_i32 * plan.n)(*[int(v) for v in queue_of])
+    _check(_lib.nnv_cache_write(os.fsencode(path), plan.handle, _choices_array(plan, choices), q, int(n_little),
+                                _ptr(h_weights), int(w_bytes), _ptr(h_cached), int(c_bytes)))
+
+
+class CacheFile:
+    """An open model file (nnv_cache_t*)."""
+
+    def __init__(self, path):
+        h = _vp()
+        _check(_lib.nnv_cache_open(os.fsencode(path), ctypes.byref(h)))
+        self.handle = h
+        n, w, c, nl, fb = _i32(0), _u64(0), _u64(0), _i32(0), _u64(0)
+        _check(_lib.nnv_cache_info(h, ctypes.byref(n), ctypes.byref(w), ctypes.byref(c), ctypes.byref(nl), ctypes.byref(fb)))
+        self.n_layers, self.w_bytes, self.c_bytes, self.n_little, self.file_bytes = n.value, w.value, c.value, nl.value, fb.value
+
+    def read_plan(self):
+        """(layer dicts, choices, queue_of) as stored."""
+        n = self.n_layers
+        layers, choices, queues = (LayerDesc * n)(), (Choice * n)(), (_i32 * n)()
+        _check(_lib.nnv_cache_read_plan(self.handle, layers, choices, queues, n))
+        ls = [{f: int(getattr(layers[i], f)) for f, _ in LayerDesc._fields_} for i in range(n)]
+        cs = [None if choices[i].variant < 0 else (choices[i].variant, choices[i].math, choices[i].cached) for i in range(n)]
+        return ls, cs, [int(q) for q in queues]
+
+    def read_blobs(self, h_weights, h_cached=None):
+        _check(_lib.nnv_cache_read_blobs(self.handle, _ptr(h_weights), int(self.w_bytes), _ptr(h_cached),
+                                         int(self.c_bytes if h_cached is not None else 0)))
+
+    def drop_pages(self):
+        _check(_lib.nnv_cache_drop_pages(self.handle))
+
+    def close(self):
+        if self.handle:
+            _lib.nnv_cache_close(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def nnv_cold_run_file(plan, choices, cache, h_stage_weights, stage_w_bytes, h_stage_cached, stage_c_bytes, h_input, h_output,
+                      d_arena, arena_bytes, s_copy, s_xform, s_exec, depth, want_timings=False):
+    """Returns (timings or None, reader nanoseconds, bytes read from the file)."""
+    tarr = (Timing * plan.n)() if want_timings else None
+    ns, nbytes = _u64(0), _u64(0)
+    _check(_lib.nnv_cold_run_file(plan.handle, _choices_array(plan, choices), cache.handle, _ptr(h_stage_weights),
+                                  int(stage_w_bytes), _ptr(h_stage_cached), int(stage_c_bytes), _ptr(h_input), _ptr(h_output),
+                                  _ptr(d_arena), int(arena_bytes), _stream(s_copy), _stream(s_xform), _stream(s_exec),
+                                  int(depth), tarr, ctypes.byref(ns), ctypes.byref(nbytes)))
+    return _timings_list(tarr), int(ns.value), int(nbytes.value)
 
 
 def _timings_list(tarr):

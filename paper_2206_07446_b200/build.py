@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnnv.so")
-SOURCES = ["plan.cpp", "scheduler.cpp", "transform.cu", "exec_kernels.cu", "gemm_tc.cu", "exec.cu", "pipeline.cu", "noalloc.cu"]
+SOURCES = ["plan.cpp", "scheduler.cpp", "cachefile.cpp", "transform.cu", "exec_kernels.cu", "gemm_tc.cu", "exec.cu", "pipeline.cu", "noalloc.cu"]
 
 
 def sources():

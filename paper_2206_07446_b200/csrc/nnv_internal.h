@@ -9,6 +9,8 @@
 
 #include "nnv.h"
 
+struct nnv_cache;
+
 namespace nnv {
 
 // ---- error plumbing -------------------------------------------------------------------------
@@ -22,6 +24,13 @@ nnv_status_t fail(nnv_status_t code, const char* fmt, ...);
         cudaError_t e__ = (call);                                                          \
         if (e__ != cudaSuccess)                                                            \
             return ::nnv::fail(NNV_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+#define NNV_REQUIRE_OR(cond, cleanup, code, ...)            \
+    do {                                                    \
+        if (!(cond)) {                                      \
+            cleanup;                                        \
+            return ::nnv::fail((code), __VA_ARGS__);        \
+        }                                                   \
     } while (0)
 #define NNV_TRY(call)                         \
     do {                                      \
@@ -229,6 +238,11 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
 // One-time host set-up of the GEMM (driver entry point, shared-memory attributes); call before
 // stream capture.
 nnv_status_t gemm_tc_init();
+
+// Model file (cachefile.cpp): exact-range read, and where the two blobs sit in the file.
+nnv_status_t cache_read_range(const nnv_cache* c, uint64_t off, void* dst, uint64_t n);
+void cache_geometry(const nnv_cache* c, uint64_t* raw_off, uint64_t* cached_off, uint64_t* w_bytes, uint64_t* c_bytes,
+                    const nnv_choice_t** file_choices, int* n_layers);
 
 nnv_status_t read_device_status(int32_t* code);
 // Enqueue a copy of the device status word into pinned host memory on `st` (no synchronisation).

@@ -1,7 +1,13 @@
 // Whole-model cold run (three-stream layer pipeline) and per-operation profiling.
 #include <algorithm>
+#include <atomic>
+#include <chrono>
+#include <condition_variable>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
+#include <mutex>
+#include <thread>
 
 #include "nnv_internal.h"
 
@@ -51,7 +57,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                               void* d_arena, uint64_t arena_bytes, cudaStream_t s_copy, cudaStream_t s_xform,
                               cudaStream_t s_exec, int depth, nnv_timing_t* timings, bool resident,
                               const int32_t* queue_of = nullptr, const cudaStream_t* s_prep = nullptr, int n_little = 0,
-                              int io_host = -1, const WarmCtx* wc = nullptr, bool wait_warm = false) {
+                              int io_host = -1, const WarmCtx* wc = nullptr, bool wait_warm = false,
+                              const std::function<nnv_status_t(int)>* before_read = nullptr) {
     const int n = (int)p->layers.size();
     const bool queued = queue_of != nullptr;        // preparations follow a schedule: queue 0 = s_exec, j = s_prep[j-1]
     const bool host_io = io_host < 0 ? !resident : io_host != 0;   // input / output are host buffers
@@ -178,6 +185,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         if (queued) {
             // the layer's bundled preparation (read, then transform) on the queue the schedule gave it
             cudaStream_t ps = queue_of[i] == 0 ? s_exec : s_prep[queue_of[i] - 1];
+            if (before_read) NNV_TRY((*before_read)(i));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), ps));
             if (cached) {
                 NNV_CUDA(cudaMemcpyAsync((void*)xf, (const uint8_t*)cached_blob + coff[i], tbytes, cudaMemcpyHostToDevice, ps));
@@ -207,6 +215,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         } else {
             // read: the staging slot is free once the layer that used it last has executed
             if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
+            if (before_read) NNV_TRY((*before_read)(i));         // the layer's bytes have arrived from storage
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
             if (cached) {
                 NNV_CUDA(cudaMemcpyAsync((void*)xf, (const uint8_t*)cached_blob + coff[i], tbytes, cudaMemcpyHostToDevice, s_copy));
@@ -321,7 +330,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         key.queues.push_back(n_little);
     }
     CachedGraph* cg = nullptr;
-    if (!tm && p->opts.use_graphs && !wc && !wait_warm) {
+    if (!tm && p->opts.use_graphs && !wc && !wait_warm && !before_read) {
         for (CachedGraph& g : p->graphs)
             if (g.key == key) { cg = &g; break; }
         if (!cg) {
@@ -510,6 +519,109 @@ nnv_status_t nnv_warm_run(nnv_plan_t* p, const nnv_choice_t* warm, const void* d
                                       timings, true, nullptr, nullptr, 0, 1, nullptr, wait);
     if (rc == NNV_OK) p->warm_pending = false;       // every preparation this run waited for has finished
     return rc;
+}
+
+// ---- cold run fed from the model file: storage -> pinned memory as a fourth pipeline stage -----
+nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const nnv_cache_t* cache, void* h_stage_weights,
+                               uint64_t stage_w_bytes, void* h_stage_cached, uint64_t stage_c_bytes, const float* h_input,
+                               float* h_output, void* d_arena, uint64_t arena_bytes, void* s_copy, void* s_xform, void* s_exec,
+                               int32_t depth, nnv_timing_t* timings, uint64_t* read_ns, uint64_t* read_bytes) {
+    NNV_REQUIRE(p && choices && cache && h_stage_weights && h_input && h_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(depth >= 0 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 0..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(aligned256(d_arena), NNV_ERR_INVALID_ARG, "arena must be 256-byte aligned");
+    NNV_REQUIRE(s_copy != s_xform && s_copy != s_exec && s_xform != s_exec, NNV_ERR_INVALID_ARG,
+                "the three streams must be distinct");
+    const int n = (int)p->layers.size();
+    uint64_t raw_off, cached_off, w_bytes, c_bytes;
+    const nnv_choice_t* file_choices;
+    int file_n;
+    cache_geometry(cache, &raw_off, &cached_off, &w_bytes, &c_bytes, &file_choices, &file_n);
+    NNV_REQUIRE(file_n == n, NNV_ERR_INVALID_ARG, "the file describes %d layers, the plan %d", file_n, n);
+    NNV_REQUIRE(stage_w_bytes >= w_bytes, NNV_ERR_WORKSPACE_TOO_SMALL, "weight staging needs %llu bytes", (unsigned long long)w_bytes);
+    std::vector<uint64_t> coff(n), fcoff(n);
+    uint64_t ctotal = 0, fctotal = 0;
+    NNV_TRY(nnv_cached_layout(p, choices, coff.data(), &ctotal));
+    if (ctotal) {
+        // the cached blob in the file was laid out for the file's own choices: the layers read from it
+        // must sit where this run's choices expect them
+        NNV_TRY(nnv_cached_layout(p, file_choices, fcoff.data(), &fctotal));
+        NNV_REQUIRE(h_stage_cached && stage_c_bytes >= ctotal && c_bytes >= ctotal, NNV_ERR_INVALID_ARG,
+                    "the cached blob (file %llu bytes, staging %llu) is smaller than the %llu bytes these choices read",
+                    (unsigned long long)c_bytes, (unsigned long long)stage_c_bytes, (unsigned long long)ctotal);
+        for (int i = 0; i < n; ++i) {
+            if (p->layers[i].op != NNV_OP_CONV || !(variant_has_transform(choices[i].variant) && choices[i].cached)) continue;
+            NNV_REQUIRE(file_choices[i].cached && file_choices[i].variant == choices[i].variant && file_choices[i].math == choices[i].math &&
+                            fcoff[i] == coff[i],
+                        NNV_ERR_INVALID_ARG, "layer %d: the file holds no cached weights for this kernel at the expected place", i);
+        }
+    }
+
+    // Reader thread: layer by layer, the bytes the layer's choice reads (cached blob entry, or raw
+    // weights; the bias) from the file into the pinned staging buffers, at the blobs' own offsets.
+    std::vector<int> ready(n, 0);
+    std::mutex mu;
+    std::condition_variable cv;
+    std::atomic<bool> stop{false};
+    nnv_status_t reader_rc = NNV_OK;
+    std::string reader_err;
+    uint64_t bytes_read = 0, ns_read = 0;
+    std::thread reader([&] {
+        const auto t0 = std::chrono::steady_clock::now();
+        for (int i = 0; i < n && !stop.load(); ++i) {
+            const nnv_layer_desc_t& L = p->layers[i];
+            nnv_status_t rc = NNV_OK;
+            if (L.op == NNV_OP_CONV) {
+                const nnv_choice_t ch = choices[i];
+                if (variant_has_transform(ch.variant) && ch.cached) {
+                    const uint64_t tb = transformed_bytes(*p, i, ch.variant, ch.math);
+                    rc = cache_read_range(cache, cached_off + coff[i], (uint8_t*)h_stage_cached + coff[i], tb);
+                    bytes_read += tb;
+                } else {
+                    rc = cache_read_range(cache, raw_off + L.w_off, (uint8_t*)h_stage_weights + L.w_off, raw_weight_bytes(L));
+                    bytes_read += raw_weight_bytes(L);
+                }
+                if (rc == NNV_OK && L.has_bias) {
+                    rc = cache_read_range(cache, raw_off + L.b_off, (uint8_t*)h_stage_weights + L.b_off, 4ull * L.K);
+                    bytes_read += 4ull * L.K;
+                }
+            }
+            std::lock_guard<std::mutex> lk(mu);
+            if (rc != NNV_OK) {
+                reader_rc = rc;
+                reader_err = nnv_last_error();
+                ready[i] = -1;
+                cv.notify_all();
+                return;
+            }
+            ready[i] = 1;
+            cv.notify_all();
+        }
+        ns_read = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+    });
+    const std::function<nnv_status_t(int)> gate = [&](int i) -> nnv_status_t {
+        std::unique_lock<std::mutex> lk(mu);
+        cv.wait(lk, [&] { return ready[i] != 0 || reader_rc != NNV_OK; });
+        if (reader_rc != NNV_OK) return fail(reader_rc, "%s", reader_err.c_str());
+        return NNV_OK;
+    };
+    for (int i = 0; i < n; ++i)
+        if (p->layers[i].op == NNV_OP_CONV)
+            NNV_REQUIRE_OR(p->layers[i].w_off + raw_weight_bytes(p->layers[i]) <= w_bytes, { stop = true; reader.join(); },
+                           NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the file's raw blob", i);
+    const nnv_status_t rc = run_model(p, choices, h_stage_weights, w_bytes, h_stage_cached, stage_c_bytes, h_input, h_output, d_arena,
+                                      arena_bytes, (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings,
+                                      false, nullptr, nullptr, 0, -1, nullptr, false, &gate);
+    stop = true;
+    reader.join();
+    if (rc != NNV_OK) {
+        cudaStreamSynchronize((cudaStream_t)s_copy);            // nothing of the failed pass may still touch the staging buffers
+        cudaStreamSynchronize((cudaStream_t)s_xform);
+        cudaStreamSynchronize((cudaStream_t)s_exec);
+        return rc;
+    }
+    if (read_ns) *read_ns = ns_read;
+    if (read_bytes) *read_bytes = bytes_read;
+    return NNV_OK;
 }
 
 nnv_status_t nnv_layer_output(const nnv_plan_t* p, int32_t layer, const void** d_ptr, uint64_t* bytes) {

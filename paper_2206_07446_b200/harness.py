@@ -195,6 +195,31 @@ class Model:
                              self.arena, self.arena.numel(), self.streams[1], self.streams[2], want_timings)
         return self.h_output.numpy().copy(), tm
 
+    def write_model_file(self, path, choices, queue_of=None, n_little=0):
+        """Store the plan, the raw weights and (for choices with cached = 1) the cached blob in a model file."""
+        if any(c is not None and c[2] for c in choices):
+            self.build_cached_blob(choices)
+        nb.nnv_cache_write(path, self.plan, choices, queue_of, n_little, self.h_weights, self.w_bytes,
+                           self.h_cached if self.c_bytes else None, self.c_bytes)
+
+    def cold_run_file(self, x_nchw, choices, cache, depth=2, want_timings=False, drop_pages=True):
+        """One cold inference whose weights come from an open model file (nnv_cold_run_file) through pinned
+        staging buffers of this object; returns (output NCHW numpy, timings, reader ns, bytes read)."""
+        if x_nchw is not None:
+            self.h_input.copy_(torch.from_numpy(np.ascontiguousarray(x_nchw, dtype=np.float32)).reshape(self.h_input.shape))
+        if getattr(self, "h_stage_w", None) is None or self.h_stage_w.numel() < cache.w_bytes:
+            self.h_stage_w = torch.empty(max(1, cache.w_bytes), dtype=torch.uint8).pin_memory()
+        if getattr(self, "h_stage_c", None) is None or self.h_stage_c.numel() < max(1, cache.c_bytes):
+            self.h_stage_c = torch.empty(max(1, cache.c_bytes), dtype=torch.uint8).pin_memory()
+        need = self.ensure_arena(choices, depth)
+        if drop_pages:
+            cache.drop_pages()
+        tm, ns, nbytes = nb.nnv_cold_run_file(self.plan, choices, cache, self.h_stage_w, self.h_stage_w.numel(),
+                                              self.h_stage_c if cache.c_bytes else None, self.h_stage_c.numel() if cache.c_bytes else 0,
+                                              self.h_input, self.h_output, self.arena, need,
+                                              self.streams[0], self.streams[1], self.streams[2], depth, want_timings)
+        return self.h_output.numpy().copy(), tm, ns, nbytes
+
     def to_device(self):
         """Device copies of the weight blob, the cached blob (if built) and I/O buffers for nnv_resident_run."""
         self.d_weights = dev_bytes(self.w_bytes, fill=None)
