@@ -242,13 +242,26 @@ __device__ __forceinline__ void pack_fast_block(const float* __restrict__ w, Out
     for (int i = threadIdx.x; i < nv; i += PACK_THREADS) dst[i] = __ldg(src + i);
     __syncthreads();
     const int Cb = min(C, PACK_NF);                               // channels of one k row inside this block
-    const int c4n = Cb / 4, per_k = RS * c4n;
     const int k0 = (int)(f_block / C), cbase = (int)(f_block - (long long)k0 * C);
-    for (int i = threadIdx.x; i < nv; i += PACK_THREADS) {
-        const int kl = i / per_k, r = i - kl * per_k;
-        const int rs = r / c4n, c = (r - rs * c4n) * 4;
-        const float* s = sg + ((kl * Cb + c) * RS + rs);
-        store4<OutT>(P + (long long)(k0 + kl) * Qp + (long long)rs * C + cbase + c, s[0], s[RS], s[2 * RS], s[3 * RS]);
+    // Write-out.  A row is one (k, rs) pair: Cb consecutive output elements.  A warp takes four
+    // consecutive rows x 32 channels: lane = 8 * (row in the group) + (16-byte word of the chunk).
+    // Each lane gathers its four channels from the staged (c, rs) order; the 32 addresses of one
+    // such gather differ by 36 words along the chunk and by 1 word along the rows, i.e. they fall
+    // in 32 different banks.  Each group of eight lanes stores 128 contiguous bytes.
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nch = Cb >> 5;                                      // 32-channel chunks per row (a power of two)
+    const int rows = (nf / Cb) * RS;
+    const int items = ((rows + 3) >> 2) * nch;
+    const int sub = lane >> 3, c = (lane & 7) * 4;
+    const int nch_log = __ffs(nch) - 1;
+    for (int item = warp; item < items; item += PACK_WARPS) {
+        const int g = item >> nch_log, ch = item & (nch - 1);
+        const int row = 4 * g + sub;
+        if (row >= rows) continue;
+        const int kl = row / RS, rs = row - kl * RS;
+        const int cc = ch * 32 + c;
+        const float* s = sg + ((kl * Cb + cc) * RS + rs);
+        store4<OutT>(P + (long long)(k0 + kl) * Qp + (long long)rs * C + cbase + cc, s[0], s[RS], s[2 * RS], s[3 * RS]);
     }
 }
 

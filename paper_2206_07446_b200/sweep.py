@@ -1,6 +1,6 @@
 """Per-kernel timing sweeps through the C ABI (CUDA events, L2 flushed between repetitions).
 
-  python -m paper_2206_07446_b200.sweep transform --m 4 --C 512 --K 512
+  python -m paper_2206_07446_b200.sweep transform --m 4 --C 512 --K 512      (--m 0: GEMM repack)
   python -m paper_2206_07446_b200.sweep transform-sweep
   python -m paper_2206_07446_b200.sweep conv --variant wino_f4 --C 64 --K 64 --H 56
   python -m paper_2206_07446_b200.sweep conv-sweep
@@ -158,7 +158,7 @@ def main():
     flush = None if a.no_flush else torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     math = nb.MATH_NAMES.index(a.math)
     if a.what == "transform":
-        v = WINO[a.m] if a.R == 3 else nb.VAR_IM2COL
+        v = WINO[a.m] if (a.R == 3 and a.m in WINO) else nb.VAR_IM2COL      # --m 0: the repack of a 3x3 layer
         print(json.dumps(time_transform(v, math, a.C, a.K, a.R, a.reps, flush)))
     elif a.what == "transform-sweep":
         for m in (2, 4, 6):
