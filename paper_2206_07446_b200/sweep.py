@@ -175,7 +175,8 @@ def main():
         print(json.dumps(time_conv(v, math, a.C, a.K, a.R, a.stride, a.H, a.H, a.groups, a.reps, flush)))
     else:
         shapes = [(64, 64, 3, 1, 56), (128, 128, 3, 1, 28), (256, 256, 3, 1, 14), (512, 512, 3, 1, 7),
-                  (64, 64, 3, 1, 224), (128, 128, 3, 1, 112), (256, 256, 3, 1, 56), (512, 512, 3, 1, 28)]
+                  (64, 64, 3, 1, 224), (128, 128, 3, 1, 112), (256, 256, 3, 1, 56), (512, 512, 3, 1, 28),
+                  (256, 256, 3, 1, 112), (256, 256, 3, 1, 224), (512, 512, 3, 1, 112)]   # beyond the configurations: the asymptote
         for (C, K, R, s, H) in shapes:
             for v, m in ((nb.VAR_DIRECT, 0), (nb.VAR_IM2COL, 1), (nb.VAR_IM2COL, 2), (nb.VAR_WINO_F2, 1),
                          (nb.VAR_WINO_F2, 2), (nb.VAR_WINO_F4, 1), (nb.VAR_WINO_F6, 1)):
