@@ -29,6 +29,8 @@ sys.path.insert(0, ROOT)
 
 import workloads as wl  # noqa: E402
 
+NCU_GEMM_TRAFFIC_BYTES = {("cfg2_resnet18", "tf32"): 3351634}   # profiles/gemm_tc_cfg2_dram_traffic.md
+
 METRIC = "cold_inference_ms_batch1"
 UNIT = "ms"
 
@@ -492,7 +494,11 @@ def run_ours(args):
                 "frac": gfl / gns / 1e3 / tf32_peak}
         hbm = {"bound": "hbm", "achieved": gby / gns, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gby / gns / peaks["hbm_gbs"]}
         roof = dict(hbm if t_hbm >= t_tensor else tens)           # the binding roofline of these launches
-        roof.update({"kernel": "gemm_tc_kernel", "traffic": None,
+        # DRAM bytes per GEMM launch from one ncu capture of this command's timed steps (dram__bytes_read.sum +
+        # dram__bytes_write.sum averaged over the gemm_tc_kernel launches of a step; profiles/ has the command).
+        # Valid for the kernels as they were when it was taken; other workloads have none.
+        traffic = NCU_GEMM_TRAFFIC_BYTES.get((args.config, args.math))
+        roof.update({"kernel": "gemm_tc_kernel (conv3x3_tc_kernel for the layers that take it)", "traffic": traffic,
                      "peak_source": peaks["source"] + (" HBM copy" if t_hbm >= t_tensor else " bf16 burst x 0.5 (tf32:bf16 nominal ratio)"),
                      "other_roofline": tens if t_hbm >= t_tensor else hbm,
                      "launches_per_step": len(single), "flops_per_step": gfl, "bytes_per_step": gby,
