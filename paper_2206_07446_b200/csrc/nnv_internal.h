@@ -149,6 +149,7 @@ struct nnv_plan {
     const void* last_arena = nullptr;
     std::vector<nnv::CachedGraph> graphs;   // recorded passes, one per distinct argument set
     int* h_status = nullptr;              // pinned host word the device status is copied into
+    cudaStream_t s_side = nullptr;        // the plan's own stream for residual-branch layers (created on first use)
     std::vector<cudaEvent_t> warm_ev;     // continuous mode: layer i's warm weights are prepared
     bool warm_pending = false;            // warm preparations may still be running (first warm run waits)
 };

@@ -19,7 +19,7 @@ nnv_status_t do_pool(const nnv_plan& p, int layer, const void* d_in, void* d_out
 
 static nnv_status_t ensure_events(nnv_plan& p, bool timing) {
     const size_t n = p.layers.size();
-    const size_t ne = 3 * n + 6 + NNV_MAX_QUEUES;                   // + fork, join(copy), join(transform), 3 transform groups, queue joins
+    const size_t ne = 3 * n + 8 + NNV_MAX_QUEUES;                   // + fork, join(copy), join(transform), 3 transform groups, queue joins, input ready, side join
     if (p.ev.size() != ne) {
         p.ev.resize(ne, nullptr);
         for (size_t i = 0; i < ne; ++i) NNV_CUDA(cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming));
@@ -95,6 +95,31 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     if (tm) std::memset(timings, 0, sizeof(nnv_timing_t) * n);
     NNV_TRY(gemm_tc_init());
 
+    // Residual-branch layers (a conv whose output is only ever the addend of a later layer, e.g. the
+    // 1x1 downsample of a ResNet block) run on a side stream of the plan's own, beside the main
+    // branch, when they need no execution scratch (the one scratch buffer belongs to s_exec).
+    std::vector<char> on_side(n, 0);
+    bool any_side = false;
+    if (!queued && !std::getenv("NNV_DEBUG_NO_SIDE")) {
+        for (int i = 0; i < n; ++i) {
+            if (p->layers[i].op != NNV_OP_CONV || exec_ws_bytes(*p, i, choices[i].variant, choices[i].math) != 0) continue;
+            bool as_input = false, as_addend = false;
+            for (int j = i + 1; j < n; ++j) {
+                as_input = as_input || p->layers[j].in0 == i;
+                as_addend = as_addend || p->layers[j].in1 == i;
+            }
+            on_side[i] = (as_addend && !as_input && i != n - 1) ? 1 : 0;
+            any_side = any_side || on_side[i];
+        }
+    }
+    if (any_side && !p->s_side) {
+        int prio = 0;
+        NNV_CUDA(cudaStreamGetPriority(s_exec, &prio));
+        NNV_CUDA(cudaStreamCreateWithPriority(&p->s_side, cudaStreamNonBlocking, prio));
+    }
+    cudaStream_t s_side = p->s_side;
+    const cudaEvent_t ev_input = p->ev[3 * n + 6 + NNV_MAX_QUEUES], ev_side_join = p->ev[3 * n + 7 + NNV_MAX_QUEUES];
+
     const bool grouped = resident && depth == 0 && !std::getenv("NNV_DEBUG_NO_GROUP");
     std::vector<cudaEvent_t> group_event(n, nullptr);
 
@@ -117,6 +142,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         in_chw = (const float*)(base + A.in_chw);
     }
     NNV_TRY(launch_chw_to_hwc(in_chw, (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, s_exec));
+    if (any_side) NNV_CUDA(cudaEventRecord(ev_input, s_exec));
 
     // Weights resident and no staging limit: nothing orders the transforms, so they are issued as up
     // to three multi-layer launches of growing size (the first ~1 MB of raw weights so that execution
@@ -155,6 +181,11 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         const nnv_layer_desc_t& L = p->layers[i];
         const void* in = L.in0 < 0 ? base + A.in_hwc : base + A.act_off[L.in0];
         void* out = base + A.act_off[i];
+        // order this layer after its producers when they ran on the other execution stream
+        cudaStream_t se = on_side[i] ? s_side : s_exec;
+        for (int prod : {L.in0, L.in1})
+            if (prod >= 0 && on_side[prod] != on_side[i]) NNV_CUDA(cudaStreamWaitEvent(se, EV(prod, 2), 0));
+        if (on_side[i] && L.in0 < 0) NNV_CUDA(cudaStreamWaitEvent(se, ev_input, 0));
         if (L.op != NNV_OP_CONV) {
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), s_exec));
             NNV_TRY(do_pool(*p, i, in, out, s_exec));
@@ -249,14 +280,14 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         }
 
         // execute
-        if (ready) NNV_CUDA(cudaStreamWaitEvent(s_exec, ready, 0));
-        if (wait_warm && i < (int)p->warm_ev.size() && p->warm_ev[i]) NNV_CUDA(cudaStreamWaitEvent(s_exec, p->warm_ev[i], 0));
-        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), s_exec));
+        if (ready) NNV_CUDA(cudaStreamWaitEvent(se, ready, 0));
+        if (wait_warm && i < (int)p->warm_ev.size() && p->warm_ev[i]) NNV_CUDA(cudaStreamWaitEvent(se, p->warm_ev[i], 0));
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), se));
         const void* add = L.in1 >= 0 ? base + A.act_off[L.in1] : nullptr;
         NNV_TRY(do_exec(*p, i, ch.variant, ch.math, in, add, has_xf ? xf : raw, L.has_bias ? bias : nullptr, out,
-                        base + A.ws_off, A.ws_bytes, s_exec));
-        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 5), s_exec));
-        NNV_CUDA(cudaEventRecord(EV(i, 2), s_exec));
+                        base + A.ws_off, A.ws_bytes, se));
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 5), se));
+        NNV_CUDA(cudaEventRecord(EV(i, 2), se));
         if (tm) {
             timings[i].h2d_bytes = copied;
             timings[i].xform_bytes = (has_xf && !cached) ? rbytes + tbytes : 0;
@@ -265,6 +296,10 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         }
     }
 
+    if (any_side) {                                           // the side stream rejoins the execution stream
+        NNV_CUDA(cudaEventRecord(ev_side_join, s_side));
+        NNV_CUDA(cudaStreamWaitEvent(s_exec, ev_side_join, 0));
+    }
     // last layer's output: device NHWC -> NCHW
     const nnv_layer_desc_t& Ln = p->layers[n - 1];
     const LayerGeom& gn = p->geom[n - 1];

@@ -297,6 +297,7 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* p) {
     for (cudaEvent_t e : p->warm_ev)
         if (e) cudaEventDestroy(e);
     if (p->h_status) cudaFreeHost(p->h_status);
+    if (p->s_side) cudaStreamDestroy(p->s_side);
     for (nnv::CachedGraph& g : p->graphs)
         if (g.exec) cudaGraphExecDestroy(g.exec);
     delete p;

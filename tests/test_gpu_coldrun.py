@@ -185,3 +185,30 @@ def test_arena_too_small_and_bad_depth():
         nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
                         model.arena, need, model.streams[0], model.streams[1], model.streams[2], -1)
     assert e.value.status == 1
+
+
+def test_residual_branch_layers_on_the_side_stream():
+    """ResNet-18-shaped: the 1x1 downsample convs run on the plan's side stream beside the main branch.  Same
+    result bit for bit as with everything on the execution stream, and every consumer of a side layer
+    starts after that layer has ended."""
+    import os
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers)
+    ch = _choices(model, [nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    side = [i for i, L in enumerate(layers) if L["op"] == wl.OP_CONV and any(M["in1"] == i for M in layers)
+            and not any(M["in0"] == i for M in layers)]
+    assert len(side) == 3
+    y_side, tm = model.cold_run(x, ch, depth=0, want_timings=True)
+    for i in side:
+        for j, M in enumerate(layers):
+            if M["in1"] == i:
+                assert tm[j]["exec_start_ns"] >= tm[i]["exec_end_ns"], (i, j)
+        assert tm[i]["exec_start_ns"] >= tm[layers[i]["in0"]]["exec_end_ns"]
+    os.environ["NNV_DEBUG_NO_SIDE"] = "1"
+    try:
+        y_main, _ = model.cold_run(x, ch, depth=0, want_timings=True)
+    finally:
+        del os.environ["NNV_DEBUG_NO_SIDE"]
+    assert np.array_equal(y_side, y_main)
+    y_graph, _ = model.cold_run(x, ch, depth=0)
+    assert np.array_equal(y_graph, y_side)
