@@ -76,23 +76,22 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
-            int ia = 0, ib = 0;                               // boxes / weight tiles issued so far
+            int sa = 0, sb = 0;                               // ring slots and their phases, carried along (no divisions:
+            uint32_t pa = 0, pb = 0;                          // every instruction of this single-thread loop is latency)
             for (int cbi = 0; cbi < ncb && ok; ++cbi) {
                 const int c0 = (cb0 + cbi) * 32;
                 for (int s = 0; s < 3 && ok; ++s) {
-                    const int sa = ia % NA;
-                    ok = mbar_wait(a_empty(sa), ((ia / NA) & 1) ^ 1u);
+                    ok = mbar_wait(a_empty(sa), pa ^ 1u);
                     if (!ok) break;
                     mbar_expect_tx(a_full(sa), a_slot_bytes);
                     tma_load_3d(a_ring + sa * a_slot_bytes, &tmA, c0, ow0 + s - 1, oh0 - 1, a_full(sa));
-                    ++ia;
+                    if (++sa == NA) { sa = 0; pa ^= 1u; }
                     for (int r = 0; r < 3; ++r) {
-                        const int sb = ib % NB;
-                        ok = mbar_wait(b_empty(sb), ((ib / NB) & 1) ^ 1u);
+                        ok = mbar_wait(b_empty(sb), pb ^ 1u);
                         if (!ok) break;
                         mbar_expect_tx(b_full(sb), b_slot_bytes);
                         tma_load_3d(b_ring + sb * b_slot_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, b_full(sb));
-                        ++ib;
+                        if (++sb == NB) { sb = 0; pb ^= 1u; }
                     }
                 }
             }
@@ -106,16 +105,15 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             // instruction descriptor: fp32 accumulate, TF32 operands, both K-major, N = BN, M = 128
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             bool ok = true;
-            int ia = 0, ib = 0;
+            int sa = 0, sb = 0;
+            uint32_t pa = 0, pb = 0;
             for (int cbi = 0; cbi < ncb && ok; ++cbi) {
                 for (int s = 0; s < 3 && ok; ++s) {
-                    const int sa = ia % NA;
-                    ok = mbar_wait(a_full(sa), (ia / NA) & 1);
+                    ok = mbar_wait(a_full(sa), pa);
                     if (!ok) break;
                     const uint32_t a_box = a_ring + sa * a_slot_bytes;
                     for (int r = 0; r < 3; ++r) {
-                        const int sb = ib % NB;
-                        ok = mbar_wait(b_full(sb), (ib / NB) & 1);
+                        ok = mbar_wait(b_full(sb), pb);
                         if (!ok) break;
                         tc_fence_after();
                         const uint64_t bdesc = make_smem_desc(b_ring + sb * b_slot_bytes);
@@ -127,10 +125,10 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                                             idesc, (cbi | s | r | kk) ? 1u : 0u);
                         }
                         umma_commit(b_empty(sb));
-                        ++ib;
+                        if (++sb == NB) { sb = 0; pb ^= 1u; }
                     }
                     if (ok) umma_commit(a_empty(sa));
-                    ++ia;
+                    if (++sa == NA) { sa = 0; pa ^= 1u; }
                 }
             }
             if (ok) umma_commit(tmem_full_bar);

@@ -275,10 +275,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"((uint32_t)g.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // One K block: operand tiles of iteration `it` into ring slot it % STAGES.
-    auto issue_stage = [&](int it) {
+    // One K block: operand tiles of iteration `it` into ring slot `s` (= it mod STAGES; the loops carry
+    // slot and phase along instead of dividing: STAGES is a run-time value and these single-thread
+    // loops are latency-bound, every instruction in them is on the critical path).
+    auto issue_stage = [&](int it, int s) {
         const int kb = kb0 + it;
-        const int s = it % STAGES;
         mbar_expect_tx(full_bar(s), tma_bytes);
         const uint32_t a_dst = sbase + s * stage_bytes;
         if (g.ic_on) {
@@ -300,7 +301,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int prefill = g.prefill ? (nkb < STAGES ? nkb : STAGES) : 0;
     if (warp == 0 && lane == 0) {
         pdl_wait();
-        for (int it = 0; it < prefill; ++it) issue_stage(it);
+        for (int it = 0; it < prefill; ++it) issue_stage(it, it);
     }
     tc_fence_before();
     __syncthreads();
@@ -312,12 +313,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
+            int s = prefill == STAGES ? 0 : prefill;
+            uint32_t ph = prefill == STAGES ? 1u : 0u;
             for (int it = prefill; it < nkb && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
                 ok = mbar_wait(empty_bar(s), ph ^ 1u);
                 if (!ok) break;
-                issue_stage(it);
+                issue_stage(it, s);
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
             if (!ok) {
                 atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
@@ -330,9 +332,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t fmt = (MODE == 0) ? 2u : 1u;
             const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             bool ok = true;
-            for (int it = 0; it < nkb; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < nkb; ++it, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
                 ok = mbar_wait(MODE == 2 ? conv_bar(s) : full_bar(s), ph);
                 if (!ok) break;
                 tc_fence_after();
@@ -369,9 +371,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if constexpr (MODE == 2) {
             // warps 2-5 first convert every staged fp32 tile into its bf16 hi / lo tiles
             const int idx = (int)threadIdx.x - 64;              // 0..127: one row of A (and of B) each
-            for (int it = 0; it < nkb; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < nkb; ++it, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
                 ok = mbar_wait(full_bar(s), ph);
                 if (!ok) break;
                 const uint32_t a_src = sbase + s * stage_bytes;
