@@ -52,8 +52,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int splits = g.splits, sp = (int)blockIdx.z;       // the cluster spans grid z: one K split per CTA
     const int tile_h = (int)blockIdx.x / g.tiles_w, tile_w = (int)blockIdx.x - tile_h * g.tiles_w;
     const int oh0 = tile_h * 16 * MT, ow0 = tile_w * 8, n0 = blockIdx.y * BN;
-    const int cb0 = (int)(((long long)g.cblk * sp) / splits);
-    const int ncb = (int)(((long long)g.cblk * (sp + 1)) / splits) - cb0;
+    const int cb0 = (g.cblk * sp) / splits;
+    const int ncb = (g.cblk * (sp + 1)) / splits - cb0;
 
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");

@@ -257,8 +257,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int sp = (int)blockIdx.z % splits, b = (int)blockIdx.z / splits;
     const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
     const int nkb_all = g.ic_on ? g.Kd : (g.Kd + BKE - 1) / BKE;  // implicit mode: Kd already counts K blocks
-    const int kb0 = (int)(((long long)nkb_all * sp) / splits);
-    const int nkb = (int)(((long long)nkb_all * (sp + 1)) / splits) - kb0;
+    const int kb0 = (nkb_all * sp) / splits;                  // K blocks number a few thousand at most: 32-bit is enough
+    const int nkb = (nkb_all * (sp + 1)) / splits - kb0;
 
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
@@ -278,18 +278,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // One K block: operand tiles of iteration `it` into ring slot `s` (= it mod STAGES; the loops carry
     // slot and phase along instead of dividing: STAGES is a run-time value and these single-thread
     // loops are latency-bound, every instruction in them is on the critical path).
+    // Implicit mode: K runs over (filter tap, channel block).  The tile's first output pixel and the K
+    // position of the next block are kept as running values: the producer issues blocks in order, and a
+    // division per block would sit on the latency path of the very first loads.
+    int ic_w0 = 0, ic_h0 = 0, ic_cb = 0, ic_fs = 0, ic_fr = 0, ic_tap = 0;
+    if (g.ic_on) {
+        const int p0 = m0 / g.ic_OW, q0 = m0 - p0 * g.ic_OW;
+        ic_w0 = q0 * g.ic_stride - g.ic_pad;
+        ic_h0 = p0 * g.ic_stride - g.ic_pad;
+        ic_tap = kb0 / g.ic_cblk;
+        ic_cb = kb0 - ic_tap * g.ic_cblk;
+        ic_fr = ic_tap / g.ic_S;
+        ic_fs = ic_tap - ic_fr * g.ic_S;
+    }
     auto issue_stage = [&](int it, int s) {
         const int kb = kb0 + it;
         mbar_expect_tx(full_bar(s), tma_bytes);
         const uint32_t a_dst = sbase + s * stage_bytes;
         if (g.ic_on) {
-            // K runs over (filter tap, channel block): A comes straight from the activation
-            const int tap = kb / g.ic_cblk, cb = kb - tap * g.ic_cblk;
-            const int fr = tap / g.ic_S, fs = tap - fr * g.ic_S;
-            const int p0 = m0 / g.ic_OW, q0 = m0 - p0 * g.ic_OW;
-            tma_load_im2col_4d(a_dst, &tmA, cb * BKE, q0 * g.ic_stride - g.ic_pad, p0 * g.ic_stride - g.ic_pad, 0,
-                               (uint16_t)fs, (uint16_t)fr, full_bar(s));
-            tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, tap * g.ic_C + cb * BKE, n0, b, full_bar(s));
+            // A comes straight from the activation: block `kb` is channel block ic_cb of tap (ic_fr, ic_fs)
+            tma_load_im2col_4d(a_dst, &tmA, ic_cb * BKE, ic_w0, ic_h0, 0, (uint16_t)ic_fs, (uint16_t)ic_fr, full_bar(s));
+            tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, ic_tap * g.ic_C + ic_cb * BKE, n0, b, full_bar(s));
+            if (++ic_cb == g.ic_cblk) {
+                ic_cb = 0; ++ic_tap;
+                if (++ic_fs == g.ic_S) { ic_fs = 0; ++ic_fr; }
+            }
         } else {
             tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
             tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
