@@ -322,6 +322,9 @@ nnv_status_t nnv_hwc_to_chw(const float* d_in, float* d_out, int32_t C, int32_t 
  *              receives the LAST layer's output.
  *   d_arena:   nnv_arena_bytes() bytes of device memory.
  *   timings:   NULL, or n entries filled from CUDA events (adds event records).
+ * At depth 0, when the weights' copy time is estimated to exceed the execution
+ * time, consecutive layers whose host and arena ranges line up are read by one
+ * copy of up to ~1 MB (the per-layer timings then share that copy's interval).
  * A conv layer whose output is only ever the residual addend of a later layer
  * and which needs no execution scratch runs on a fourth stream that the plan
  * creates and owns, beside the main branch; the result is the same bit for bit.

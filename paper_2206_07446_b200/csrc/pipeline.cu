@@ -120,6 +120,57 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     cudaStream_t s_side = p->s_side;
     const cudaEvent_t ev_input = p->ev[3 * n + 6 + NNV_MAX_QUEUES], ev_side_join = p->ev[3 * n + 7 + NNV_MAX_QUEUES];
 
+    // Host-to-device copies cost ~8 us each before the first byte moves, so at depth 0 (where the arena
+    // mirrors the host blobs' layouts) consecutive layers whose source and destination ranges line up are
+    // read by ONE copy of up to ~1 MB; all layers of such a chunk become ready when it lands.
+    struct CopyChunk { const uint8_t* src; uint8_t* dst; uint64_t bytes; int first, last; };
+    std::vector<CopyChunk> chunks;
+    std::vector<int> chunk_of(n, -1);
+    bool merge = !resident && !queued && depth == 0 && !wc && !std::getenv("NNV_DEBUG_NO_MERGE");
+    if (merge) {
+        // Coarser copies make layers ready later (a layer waits for its whole chunk), which only pays when
+        // the link, not execution, is what the run waits for: rough estimate, bytes at 50 GB/s against
+        // 8 us per layer (measured: ResNet / VGG shapes gain 2-4 %, a MobileNetV2 shape loses 14 %).
+        uint64_t bytes = 0;
+        int convs = 0;
+        for (int i = 0; i < n; ++i) {
+            if (p->layers[i].op != NNV_OP_CONV) continue;
+            ++convs;
+            const nnv_choice_t ch = choices[i];
+            bytes += (variant_has_transform(ch.variant) && ch.cached) ? transformed_bytes(*p, i, ch.variant, ch.math)
+                                                                       : raw_weight_bytes(p->layers[i]);
+        }
+        merge = (double)bytes / 50e3 > 8.0 * convs;              // us
+    }
+    if (merge) {
+        constexpr uint64_t kTarget = 1u << 20, kMaxGap = 4096;
+        int cur_kind = -1;
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p->layers[i];
+            if (L.op != NNV_OP_CONV) continue;
+            const nnv_choice_t ch = choices[i];
+            const bool cached = variant_has_transform(ch.variant) && ch.cached;
+            const uint8_t* src = cached ? (const uint8_t*)cached_blob + coff[i] : (const uint8_t*)weights + L.w_off;
+            uint8_t* dst = (uint8_t*)d_arena + (cached ? A.xf_off[i] : A.raw_off[i]);
+            const uint64_t len = cached ? transformed_bytes(*p, i, ch.variant, ch.math) : raw_weight_bytes(L);
+            bool joined = false;
+            if (!chunks.empty() && cur_kind == (int)cached) {
+                CopyChunk& c = chunks.back();
+                if (src >= c.src + c.bytes && (uint64_t)(src - (c.src + c.bytes)) <= kMaxGap && src - c.src == dst - c.dst &&
+                    c.bytes < kTarget) {
+                    c.bytes = (uint64_t)(src - c.src) + len;
+                    c.last = i;
+                    joined = true;
+                }
+            }
+            if (!joined) {
+                chunks.push_back(CopyChunk{src, dst, len, i, i});
+                cur_kind = (int)cached;
+            }
+            chunk_of[i] = (int)chunks.size() - 1;
+        }
+    }
+
     const bool grouped = resident && depth == 0 && !std::getenv("NNV_DEBUG_NO_GROUP");
     std::vector<cudaEvent_t> group_event(n, nullptr);
 
@@ -246,6 +297,25 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         } else {
             // read: the staging slot is free once the layer that used it last has executed
             if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
+            if (merge) {
+                const CopyChunk& c = chunks[chunk_of[i]];
+                if (c.first == i) {                             // the chunk's one copy, issued with its first layer
+                    for (int k = c.first; k <= c.last; ++k)
+                        if (before_read && p->layers[k].op == NNV_OP_CONV) NNV_TRY((*before_read)(k));
+                    if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
+                    NNV_CUDA(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, s_copy));
+                    for (int k = c.first; k <= c.last; ++k) {
+                        const nnv_layer_desc_t& Lk = p->layers[k];
+                        if (Lk.op == NNV_OP_CONV && Lk.has_bias)
+                            NNV_CUDA(cudaMemcpyAsync(base + A.bias_off[k], (const uint8_t*)weights + Lk.b_off, 4ull * Lk.K,
+                                                     cudaMemcpyHostToDevice, s_copy));
+                    }
+                    if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
+                    NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
+                }
+                copied += (cached ? tbytes : rbytes) + (L.has_bias ? 4ull * L.K : 0);
+                ready = EV(c.first, 0);
+            } else {
             if (before_read) NNV_TRY((*before_read)(i));         // the layer's bytes have arrived from storage
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
             if (cached) {
@@ -262,6 +332,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
             NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
             ready = EV(i, 0);
+            }
         }
 
         // transform
@@ -410,8 +481,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             NNV_TRY(stamp(TEV(i, 5), &timings[i].exec_end_ns));
             if (L.op != NNV_OP_CONV) continue;
             if (!resident || queued) {
-                NNV_TRY(stamp(TEV(i, 0), &timings[i].h2d_start_ns));
-                NNV_TRY(stamp(TEV(i, 1), &timings[i].h2d_end_ns));
+                const int hi = (merge && chunk_of[i] >= 0) ? chunks[chunk_of[i]].first : i;   // a merged copy's interval
+                NNV_TRY(stamp(TEV(hi, 0), &timings[i].h2d_start_ns));
+                NNV_TRY(stamp(TEV(hi, 1), &timings[i].h2d_end_ns));
             }
             if (timings[i].xform_bytes && grouped) {             // the interval of the layer's multi-layer launch
                 const int g = group_event[i] == p->ev[3 * n + 3] ? 0 : group_event[i] == p->ev[3 * n + 4] ? 1 : 2;

@@ -154,13 +154,30 @@ nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int de
     a.out_chw = take(4ull * p.geom[n - 1].P * Ln.K);
     if (depth == 0) {
         // no staging limit: every conv layer owns a raw (weights + bias) and a transformed buffer
+        // The raw buffers mirror the host weight blob (same distances between layers) and the
+        // transformed buffers of layers read from the cached blob mirror that blob, so that one copy can
+        // serve several consecutive layers.
         a.raw_off.assign(n, 0); a.bias_off.assign(n, 0); a.xf_off.assign(n, 0);
+        uint64_t lo = ~0ull, hi = 0;
         for (int i = 0; i < n; ++i) {
             const nnv_layer_desc_t& L = p.layers[i];
             if (L.op != NNV_OP_CONV) continue;
-            a.raw_off[i] = take(raw_weight_bytes(L));
-            a.bias_off[i] = take(4ull * L.K);
-            a.xf_off[i] = take(transformed_bytes(p, i, choices[i].variant, choices[i].math));
+            lo = std::min<uint64_t>(lo, L.w_off); hi = std::max<uint64_t>(hi, L.w_off + raw_weight_bytes(L));
+            if (L.has_bias) { lo = std::min<uint64_t>(lo, L.b_off); hi = std::max<uint64_t>(hi, L.b_off + 4ull * L.K); }
+        }
+        if (lo > hi) lo = hi = 0;
+        const uint64_t raw_region = take(hi - lo);
+        std::vector<uint64_t> coff(n, 0);
+        uint64_t ctotal = 0;
+        NNV_TRY(nnv_cached_layout(&p, choices, coff.data(), &ctotal));
+        const uint64_t cached_region = take(ctotal);
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& L = p.layers[i];
+            if (L.op != NNV_OP_CONV) continue;
+            a.raw_off[i] = raw_region + (L.w_off - lo);
+            a.bias_off[i] = L.has_bias ? raw_region + (L.b_off - lo) : raw_region;
+            const bool cached = variant_has_transform(choices[i].variant) && choices[i].cached;
+            a.xf_off[i] = cached ? cached_region + coff[i] : take(transformed_bytes(p, i, choices[i].variant, choices[i].math));
         }
     } else {
         a.raw_bias_off = align_up(max_raw ? max_raw : 1, 1024);

@@ -212,3 +212,28 @@ def test_residual_branch_layers_on_the_side_stream():
     assert np.array_equal(y_side, y_main)
     y_graph, _ = model.cold_run(x, ch, depth=0)
     assert np.array_equal(y_graph, y_side)
+
+
+def test_merged_copies_at_depth_zero():
+    """ResNet-18-shaped, depth 0: consecutive layers whose host and device ranges line up are read by one copy.
+    Same result bit for bit as with one copy per layer; layers of one chunk report the same copy interval, the
+    byte counts stay per layer, and no layer executes before its chunk has landed."""
+    import os
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers)
+    ch = _choices(model, [nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    y_merged, tm = model.cold_run(x, ch, depth=0, want_timings=True)
+    convs = [i for i, L in enumerate(layers) if L["op"] == wl.OP_CONV]
+    intervals = {(tm[i]["h2d_start_ns"], tm[i]["h2d_end_ns"]) for i in convs}
+    assert len(intervals) < len(convs)                     # some layers share a copy
+    for i in convs:
+        L = layers[i]
+        assert tm[i]["h2d_bytes"] == 4 * L["K"] * L["C"] * L["R"] * L["S"]
+        assert tm[i]["exec_start_ns"] >= tm[i]["h2d_end_ns"]
+    os.environ["NNV_DEBUG_NO_MERGE"] = "1"
+    try:
+        y_single, tm1 = model.cold_run(x, ch, depth=0, want_timings=True)
+    finally:
+        del os.environ["NNV_DEBUG_NO_MERGE"]
+    assert len({(tm1[i]["h2d_start_ns"], tm1[i]["h2d_end_ns"]) for i in convs}) == len(convs)
+    assert np.array_equal(y_merged, y_single)
