@@ -46,6 +46,41 @@ im2col_kernel(const float* __restrict__ x, OutT* __restrict__ col, int C, int H,
     }
 }
 
+// The same matrix for small reductions (R*S*C up to IM2COL_TABLE entries: network stems with C = 3).  The
+// (r, s, c) of every column q is worked out once per block into a shared-memory table; a warp then writes one
+// pixel's row at a time, lane = q, so the inner loop has no division and the stores are contiguous.
+constexpr int IM2COL_TABLE = 1024;
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+im2col_table_kernel(const float* __restrict__ x, OutT* __restrict__ col, int C, int H, int W, int R, int S, int stride,
+                    int pad, int OH, int OW, int Qp) {
+    pdl_enter();
+    __shared__ int tab[IM2COL_TABLE];                           // (r << 20) | (s << 10) | c, or -1 for the zero padding q >= Q
+    const int Q = R * S * C;
+    for (int q = threadIdx.x; q < Qp; q += 256) {
+        const int rs = q / C, c = q - rs * C;
+        const int r = rs / S, sx = rs - r * S;
+        tab[q] = q < Q ? ((r << 20) | (sx << 10) | c) : -1;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int P = OH * OW;
+    for (int p = blockIdx.x * 8 + warp; p < P; p += gridDim.x * 8) {
+        const int oh = p / OW, ow = p - oh * OW;
+        const int ih0 = oh * stride - pad, iw0 = ow * stride - pad;
+        OutT* dst = col + (long long)p * Qp;
+        for (int q = lane; q < Qp; q += 32) {
+            const int e = tab[q];
+            float v = 0.f;
+            if (e >= 0) {
+                const int ih = ih0 + (e >> 20), iw = iw0 + ((e >> 10) & 1023);
+                if (ih >= 0 && ih < H && iw >= 0 && iw < W) v = __ldg(x + ((long long)ih * W + iw) * C + (e & 1023));
+            }
+            dst[q] = to_out<OutT>(sizeof(OutT) == 4 ? round_tf32(v) : v);
+        }
+    }
+}
+
 // Four consecutive q per thread; valid when C % 4 == 0 (a quad never straddles a filter tap).
 template <typename OutT>
 __global__ void __launch_bounds__(256)
@@ -87,6 +122,10 @@ nnv_status_t launch_im2col(bool bf16, const float* x, void* col, int C, int H, i
     if (vec) {
         if (bf16) NNV_LAUNCH((im2col_vec4_kernel<__nv_bfloat16>), grid, 256, 0, st, x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
         else NNV_LAUNCH((im2col_vec4_kernel<float>), grid, 256, 0, st, x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
+    } else if (Qp <= IM2COL_TABLE && C < 1024 && R < 1024 && S < 1024) {
+        const unsigned g2 = (unsigned)std::min<long long>(((long long)OH * OW + 7) / 8, 148ll * 16);
+        if (bf16) NNV_LAUNCH((im2col_table_kernel<__nv_bfloat16>), g2, 256, 0, st, x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
+        else NNV_LAUNCH((im2col_table_kernel<float>), g2, 256, 0, st, x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
     } else {
         if (bf16) NNV_LAUNCH((im2col_kernel<__nv_bfloat16>), grid, 256, 0, st, x, (__nv_bfloat16*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
         else NNV_LAUNCH((im2col_kernel<float>), grid, 256, 0, st, x, (float*)col, C, H, W, R, S, stride, pad, OH, OW, Qp);
