@@ -14,7 +14,8 @@
  *   - Plain C types only.  Pointers prefixed h_ are HOST pointers, d_ are DEVICE
  *     pointers.  Streams are cudaStream_t / CUstream handles passed as void*.
  *   - The caller owns every device buffer, host blob and stream.  The library owns
- *     only nnv_plan_t (host memory, plus CUDA events created lazily) and allocates
+ *     only nnv_plan_t (host memory, plus CUDA events, recorded graphs and one
+ *     side stream created lazily) and nnv_cache_t (an open model file), and allocates
  *     NO device memory; nnv_cold_run and nnv_profile sub-allocate from the arena
  *     the caller passes.
  *   - Device pointers must be 256-byte aligned unless stated otherwise.
