@@ -1,17 +1,22 @@
 #!/usr/bin/env python
 """Benchmark of the cold-start convolution path on B200.
 
-One step = one cold inference of the workload at batch 1: per-layer kernel selection on the
-profiled cost table, then for every conv layer the weights are read (host -> HBM), transformed
-(Winograd filter transform or GEMM repack) and the layer is executed, pipelined over streams.
+One step = one cold inference of the workload at batch 1, as the paper's Section 2 lists its stages:
+every conv layer's RAW fp32 weights are read (pinned host memory -> HBM), transformed on the device
+(Winograd filter transform or GEMM repack) and the layer is executed, pipelined over streams.  The
+kernels come from the per-layer selection on the profiled cost table with the cached-weights bypass
+switched OFF, and every call is enqueued eagerly (no recorded graph: a cold inference happens once).
 
-  value   cold ms with weights and input already resident in HBM (transform + exec only)
-  e2e     cold ms through nnv_cold_run with pinned HOST weights / input / output (H2D, D2H inside)
-  algorithm1  the same end-to-end step on the queues the paper's Algorithm 1 produces (nnv_schedule +
-          calibration, nnv_cold_run_queues), reported beside e2e
+  value   cold ms of that step with the model input / output in device memory (nnv_cold_run_dio):
+          weights H2D + transform + execution inside the timed region, CUDA events
+  e2e     the same step through nnv_cold_run with HOST input and output (their copies inside too)
+  arms    beside them: the bypass arm (selection may take cached post-transform weights), the
+          graph-replayed variant of the headline, and the device-resident pass (no read stage)
+  roofline*  kernel durations come from the per-layer events of the TIMED headline steps
 
-Run `python bench.py` (1 GPU) or under torch.distributed.run with --gpus N (independent replicas,
-the path does not shard).  `--impl reference` times the CPU oracle instead.
+`python bench.py` (1 GPU) or under torch.distributed.run with --gpus N (independent replicas; the path
+does not shard).  `--impl reference` times the CPU oracle instead.  `--kernel ...` times one kernel
+(or a sweep of shapes) through the C ABI instead of a whole step.
 """
 import argparse
 import json
@@ -29,31 +34,58 @@ sys.path.insert(0, ROOT)
 
 import workloads as wl  # noqa: E402
 
-NCU_GEMM_TRAFFIC_BYTES = {("cfg2_resnet18", "tf32"): 3351634}   # profiles/gemm_tc_cfg2_dram_traffic.md
+# DRAM bytes per tensor-core GEMM launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the
+# launches of one step) from an ncu capture of this command; the file under profiles/ gives the command.
+# An entry is dropped (traffic = null) whenever the kernel changes after the capture.
+NCU_GEMM_TRAFFIC_BYTES = {}
 
 METRIC = "cold_inference_ms_batch1"
 UNIT = "ms"
+DEFAULT_CONFIG = "cfg4_resnet50"       # the largest configuration by bytes over the host link (94 MB raw weights)
+FLUSH_BYTES = 256 << 20
 
 
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg2_resnet18", choices=list(wl.CONFIGS))
-    ap.add_argument("--depth", type=int, default=3, help="pipeline depth of the device-resident run (staging slots; 0 = no limit)")
-    ap.add_argument("--cold-depth", type=int, default=0, help="pipeline depth of the end-to-end run (0 = no staging limit)")
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=list(wl.CONFIGS))
+    ap.add_argument("--cold-depth", type=int, default=0, help="pipeline depth of the cold runs (staging slots; 0 = no limit)")
+    ap.add_argument("--depth", type=int, default=3, help="pipeline depth of the device-resident pass")
     ap.add_argument("--math", default="tf32", choices=["tf32", "bf16"])
     ap.add_argument("--cpu-passes", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graphs", action="store_true", help="enqueue every call eagerly instead of replaying a recorded CUDA graph")
-    ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run reported beside e2e (0 = skip)")
-    ap.add_argument("--continuous-reps", type=int, default=20, help="cold + warm sequences timed for the kernel-switching report (0 = skip)")
-    ap.add_argument("--file-reps", type=int, default=20, help="cold runs fed from a model file on local storage (0 = skip)")
+    ap.add_argument("--arm-steps", type=int, default=20, help="timed steps of each side arm (bypass, graph replay, resident)")
+    ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run (0 = skip)")
+    ap.add_argument("--continuous-reps", type=int, default=10, help="cold + warm sequences for the kernel-switching report (0 = skip)")
+    ap.add_argument("--file-reps", type=int, default=5, help="cold runs fed from a model file on local storage (0 = skip)")
+    ap.add_argument("--minimal", action="store_true", help="headline + e2e + rooflines only (no side arms or sections)")
     ap.add_argument("--save-costs", default=None, help="write the profiled cost table (JSON) to this file")
     ap.add_argument("--load-costs", default=None, help="use a cost table saved earlier instead of profiling (e.g. under a profiler)")
+    # single-kernel timing through the C ABI
+    ap.add_argument("--kernel", default=None, choices=["transform", "transform-sweep", "conv", "conv-sweep", "transform-all"])
+    ap.add_argument("--prefer", default="", help="comma-separated variants tried first per layer (--kernel transform-all)")
+    ap.add_argument("--m", type=int, default=4, help="Winograd tile size of --kernel transform (0 = the GEMM repack)")
+    ap.add_argument("--variant", default="im2col")
+    ap.add_argument("--C", type=int, default=512)
+    ap.add_argument("--K", type=int, default=512)
+    ap.add_argument("--R", type=int, default=3)
+    ap.add_argument("--stride", type=int, default=1)
+    ap.add_argument("--H", type=int, default=56)
+    ap.add_argument("--groups", type=int, default=1)
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--tuning", default=None, help="nnv_tuning_set specification applied before anything runs")
     return ap.parse_args()
+
+
+def config_dict(args):
+    """The workload description; identical for both arms (`--impl ours` and `--impl reference`)."""
+    return {"workload": args.config, "batch": 1, "math": args.math,
+            "weights": "raw fp32, He-normal, seed 0; every step reads, transforms and executes all of them",
+            "l2": "GPU arm: flushed between steps by a 256 MiB device write"}
 
 
 def load_peaks():
@@ -158,7 +190,7 @@ def run_reference(args):
     line = {
         "impl": "reference", "metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": args.config, "batch": 1},
+        "dtype": "f64", "data": "synthetic", "config": config_dict(args),
         "cpu_baseline": {"value": ms, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": ms, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -239,6 +271,33 @@ def count_launches(layers, choices, plan, nb):
     return n
 
 
+def raw_bytes(L):
+    return 4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"]
+
+
+def h2d_bytes(layers, choices, plan, nb, with_input_bytes):
+    """Bytes that cross the host link per cold step: weights (raw or cached), biases, and the input image."""
+    total = with_input_bytes
+    for i, c in enumerate(choices):
+        if c is None:
+            continue
+        L = layers[i]
+        total += nb.nnv_transformed_bytes(plan, i, c[0], c[1]) if c[2] else raw_bytes(L)
+        total += 4 * L["K"] if L["has_bias"] else 0
+    return int(total)
+
+
+def names(choices, nb):
+    return [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices]
+
+
+def gemm_bytes(L):
+    """Algorithmic bytes of one GEMM-executed layer: X once + packed weights + Y (fp32 words)."""
+    oh, ow = wl.out_hw(L)
+    qp = -(-(L["R"] * L["S"] * L["C"]) // 8) * 8
+    return 4 * (L["C"] * L["H"] * L["W"] + L["K"] * qp + oh * ow * L["K"])
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -253,11 +312,15 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if args.tuning:
+        nb.nnv_tuning_set(args.tuning)
 
     layers = wl.CONFIGS[args.config]()
     ws, bs = wl.make_weights(layers)
     x = wl.make_input(layers)
-    model = harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=0 if args.no_graphs else 1)
+    # the headline is eager; a second plan over the same blob replays recorded graphs for the side arms
+    model = harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=0)
+    plan_g = model.second_plan(use_graphs=1)
     math = nb.MATH_BF16 if args.math == "bf16" else nb.MATH_TF32
 
     # offline decision stage: profile every candidate kernel, select per layer by cold cost
@@ -267,57 +330,24 @@ def run_ours(args):
         costs = model.profile(x, reps=5)
     if args.save_costs and rank == 0:
         json.dump(costs, open(args.save_costs, "w"))
-    costs = [c for c in costs if c["math"] in (nb.MATH_FP32, math) or c["variant"] in (nb.VAR_WINO_F4, nb.VAR_WINO_F6)]
-    choices_cold = nb.nnv_select_kernels(model.plan, costs, 1)
-    if any(c is not None and c[2] for c in choices_cold):
-        model.build_cached_blob(choices_cold)
-    # with the read stage removed (weights resident) h2d costs vanish: select on transform + exec only
-    costs_res = [dict(c, h2d_raw_ns=0, h2d_cached_ns=0) for c in costs]
-    choices_res = nb.nnv_select_kernels(model.plan, costs_res, 0)
+    costs = nb.CostTable([c for c in costs if c["math"] in (nb.MATH_FP32, math) or c["variant"] in (nb.VAR_WINO_F4, nb.VAR_WINO_F6)])
+    choices_raw = nb.nnv_select_kernels(model.plan, costs, 0)        # headline: every layer reads RAW weights and transforms them
+    choices_byp = nb.nnv_select_kernels(model.plan, costs, 1)        # bypass arm: cached post-transform weights allowed
+    costs_res = nb.CostTable([dict(c, h2d_raw_ns=0, h2d_cached_ns=0) for c in costs])
+    choices_res = nb.nnv_select_kernels(model.plan, costs_res, 0)    # no read stage: transform + exec only
     model.to_device()
     model.d_input.copy_(torch.from_numpy(x))
     model.h_input.copy_(torch.from_numpy(x))
-    need_cold = model.ensure_arena(choices_cold, args.cold_depth)
-    need_res = model.ensure_arena(choices_res, args.depth)
-    need = max(need_cold, need_res)
-    model.arena.fill_(0xFF)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     s_copy, s_xform, s_exec = model.streams
-    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    nev = max(args.steps, args.arm_steps)
+    ev0 = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
+    ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def step_resident(k, timed, want_timings=False):
-        flush.fill_(k & 0xFF)                                # evict L2 between steps
-        torch.cuda.synchronize()
-        ch = nb.nnv_select_kernels(model.plan, costs_res, 0)
-        if timed:
-            ev0[k].record(s_exec)
-            s_xform.wait_event(ev0[k])
-        tm = nb.nnv_resident_run(model.plan, ch, model.d_weights, model.w_bytes, model.d_cached, model.c_bytes,
-                                 model.d_input, model.d_output, model.arena, need, s_xform, s_exec, args.depth, want_timings)
-        if timed:
-            ev1[k].record(s_exec)
-        return tm
-
-    def step_cold(k, timed):
-        flush.fill_(k & 0xFF)
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        ch = nb.nnv_select_kernels(model.plan, costs, 1)
-        if timed:
-            ev0[k].record(s_exec)
-            s_copy.wait_event(ev0[k])
-            s_xform.wait_event(ev0[k])
-        nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes, model.h_input,
-                        model.h_output, model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
-        if timed:
-            ev1[k].record(s_exec)
-        return time.perf_counter() - t0
 
     def reduce_max(v):
         if world > 1:
@@ -326,80 +356,139 @@ def run_ours(args):
             return float(t.item())
         return v
 
+    def timed_region(step_fn, steps, warmup):
+        """W untimed + K timed steps between barriers; mean ms per step (max over ranks)."""
+        for k in range(warmup):
+            step_fn(k, False)
+        barrier()
+        out = [step_fn(k, True) for k in range(steps)]
+        barrier()
+        ms = [ev0[k].elapsed_time(ev1[k]) for k in range(steps)]
+        return reduce_max(sum(ms) / len(ms)), out
+
+    def begin(k, timed, streams):
+        flush.fill_(k & 0xFF)                                 # evict L2 between steps
+        torch.cuda.synchronize()
+        if timed:
+            ev0[k].record(s_exec)
+            for s in streams:
+                s.wait_event(ev0[k])
+
     uuid = str(torch.cuda.get_device_properties(local).uuid)
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    model.arena = None
+    need = max(model.ensure_arena(c, d) for c, d in ((choices_raw, args.cold_depth), (choices_byp, args.cold_depth), (choices_res, args.depth)))
+    model.arena.fill_(0xFF)
+    if any(c is not None and c[2] for c in choices_byp):
+        model.build_cached_blob(choices_byp)
 
-    # ---- timed region 1: weights resident in HBM ------------------------------------------------
+    # ---- headline: raw weights from pinned host memory, transform, execute; input / output on the device ----
+    def step_value(k, timed):
+        begin(k, timed, (s_copy, s_xform))
+        ch = nb.nnv_select_kernels(model.plan, costs, 0)      # the selection call belongs to the cold inference
+        tm = nb.nnv_cold_run_dio(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
+                                 model.arena, need, s_copy, s_xform, s_exec, args.cold_depth, timed)
+        if timed:
+            ev1[k].record(s_exec)
+        return tm
+
     sampler.start()
-    for k in range(args.warmup):
-        step_resident(k, False)
-    barrier()
     torch.cuda.cudart().cudaProfilerStart()                  # a profiler attached with "profile from start off" sees the timed steps only
-    for k in range(args.steps):
-        step_resident(k, True)
-    barrier()
-    res_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
-    value = reduce_max(sum(res_ms) / len(res_ms))
+    value, step_timings = timed_region(step_value, args.steps, args.warmup)
+    y_gpu = model.d_output.cpu().numpy()
 
-    # ---- timed region 2: end to end from pinned host memory -------------------------------------
-    for k in range(args.warmup):
-        step_cold(k, False)
-    barrier()
-    wall = [step_cold(k, True) for k in range(args.steps)]
-    barrier()
+    # ---- e2e: the same step through nnv_cold_run, input and output in pinned host memory ---------------------
+    wall, enq = [], []
+
+    def step_e2e(k, timed):
+        begin(k, timed, (s_copy, s_xform))
+        t0 = time.perf_counter()
+        ch = nb.nnv_select_kernels(model.plan, costs, 0)
+        nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
+                        model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+        if timed:
+            ev1[k].record(s_exec)
+            wall.append(time.perf_counter() - t0)
+            enq.append(nb.nnv_last_enqueue_ns(model.plan))
+
+    e2e, _ = timed_region(step_e2e, args.steps, args.warmup)
     torch.cuda.cudart().cudaProfilerStop()
-    cold_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
-    e2e = reduce_max(sum(cold_ms) / len(cold_ms))
+    y_e2e = model.h_output.numpy().copy()
     e2e_wall = reduce_max(1e3 * sum(wall) / len(wall))
+
+    arms = {}
+    if not args.minimal:
+        # ---- bypass arm (the paper's Section 3.1.2): selection may read cached post-transform weights ----
+        def step_bypass(k, timed):
+            begin(k, timed, (s_copy, s_xform))
+            ch = nb.nnv_select_kernels(model.plan, costs, 1)
+            nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes, model.h_input,
+                            model.h_output, model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+            if timed:
+                ev1[k].record(s_exec)
+
+        ms, _ = timed_region(step_bypass, args.arm_steps, 3)
+        arms["bypass_allowed"] = {"e2e_ms": ms, "what": "nnv_cold_run, eager, selection with allow_cached = 1",
+                                  "cached_layers": sum(1 for c in choices_byp if c is not None and c[2]),
+                                  "transform_launches": sum(1 for c in choices_byp if c is not None and not c[2] and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE)),
+                                  "h2d_bytes_per_step": h2d_bytes(layers, choices_byp, model.plan, nb, x.nbytes)}
+
+        # ---- the headline step replayed from a recorded CUDA graph ----
+        def step_graph(k, timed):
+            begin(k, timed, (s_copy, s_xform))
+            ch = nb.nnv_select_kernels(plan_g, costs, 0)
+            nb.nnv_cold_run(plan_g, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
+                            model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+            if timed:
+                ev1[k].record(s_exec)
+
+        ms, _ = timed_region(step_graph, args.arm_steps, 3)
+        arms["graph_replay"] = {"e2e_ms": ms, "what": "nnv_cold_run with raw weights, replayed from a CUDA graph recorded by an earlier identical call"}
+
+        # ---- weights already resident in HBM: transform + execution only ----
+        def step_resident(k, timed):
+            begin(k, timed, (s_xform,))
+            ch = nb.nnv_select_kernels(plan_g, costs_res, 0)
+            nb.nnv_resident_run(plan_g, ch, model.d_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
+                                model.arena, need, s_xform, s_exec, args.depth)
+            if timed:
+                ev1[k].record(s_exec)
+
+        ms, _ = timed_region(step_resident, args.arm_steps, 3)
+        arms["resident"] = {"ms": ms, "what": "nnv_resident_run (no read stage), graph replay, pipeline depth %d" % args.depth}
 
     # ---- Algorithm 1: schedule (with calibration under overlap), then the same end-to-end step on its queues
     alg1 = None
-    if args.queues > 0:
-        ch_s, q_s, t_pred, _ = model.schedule(x, costs, args.queues, allow_cached=1, rounds=2, eps_pct=1,
-                                              combo_limit=4096)
-        if any(c is not None and c[2] for c in ch_s):
-            model.build_cached_blob(ch_s)
+    y_s = None
+    if args.queues > 0 and not args.minimal:
+        ch_s, q_s, t_pred, _ = model.schedule(x, costs, args.queues, allow_cached=0, rounds=2, eps_pct=1, combo_limit=4096)
         need_s = model.ensure_arena(ch_s, 0)
         st_s = model.prep_streams(args.queues)
 
         def step_sched(k, timed):
-            flush.fill_(k & 0xFF)
-            torch.cuda.synchronize()
-            if timed:
-                ev0[k].record(s_exec)
-                for s in st_s[1:]:
-                    s.wait_event(ev0[k])
-            nb.nnv_cold_run_queues(model.plan, ch_s, q_s, args.queues, model.h_weights, model.w_bytes, model.h_cached,
-                                   model.c_bytes, model.h_input, model.h_output, model.arena, need_s, st_s)
+            begin(k, timed, st_s[1:])
+            nb.nnv_cold_run_queues(model.plan, ch_s, q_s, args.queues, model.h_weights, model.w_bytes, None, 0,
+                                   model.h_input, model.h_output, model.arena, need_s, st_s)
             if timed:
                 ev1[k].record(s_exec)
 
-        for k in range(args.warmup):
-            step_sched(k, False)
-        barrier()
-        for k in range(args.steps):
-            step_sched(k, True)
-        barrier()
-        sched_ms = [ev0[k].elapsed_time(ev1[k]) for k in range(args.steps)]
-        alg1 = {"n_little": args.queues, "e2e_ms": reduce_max(sum(sched_ms) / len(sched_ms)),
-                "predicted_ms": t_pred / 1e6, "calibration_factors": getattr(model, "calibration", None),
+        ms, _ = timed_region(step_sched, args.arm_steps, 3)
+        alg1 = {"n_little": args.queues, "e2e_ms": ms, "predicted_ms": t_pred / 1e6,
+                "calibration_factors": getattr(model, "calibration", None),
                 "preps_on_queue0": sum(1 for q in q_s if q == 0),
-                "choices_differing_from_per_layer_argmin": sum(1 for a, b in zip(ch_s, choices_cold) if a != b),
+                "choices_differing_from_per_layer_argmin": sum(1 for a, b in zip(ch_s, choices_raw) if a != b),
                 "parity_rel_l2_end_to_end": None}
         y_s = model.h_output.numpy().copy()
-        if any(c is not None and c[2] for c in choices_cold):
-            model.build_cached_blob(choices_cold)
+        need = max(need, need_s)
         model.arena.fill_(0xFF)
 
     # ---- continuous mode (the paper's Section 3.5): cold inference with K_cold that leaves K_warm prepared,
     # then warm inferences; latency of the 1st, 2nd and later inferences, end to end from host buffers
     cont = None
-    if args.continuous_reps > 0:
+    y_w = None
+    if args.continuous_reps > 0 and not args.minimal:
         warm = nb.nnv_select_warm(model.plan, costs)
-        cold_c = nb.nnv_select_kernels(model.plan, costs, 1)
-        if any(c is not None and c[2] for c in cold_c):
-            model.build_cached_blob(cold_c)
-        need_c = max(model.ensure_arena(cold_c, 0), model.ensure_arena(warm, 0))
+        need_c = max(model.ensure_arena(choices_raw, 0), model.ensure_arena(warm, 0))
         wbytes = nb.nnv_warm_bytes(model.plan, warm, model.w_bytes)
         d_warm = harness.dev_bytes(wbytes)
         seq = [[], [], [], []]
@@ -410,7 +499,7 @@ def run_ours(args):
             evs[0].record(s_exec)
             s_copy.wait_event(evs[0])
             s_xform.wait_event(evs[0])
-            nb.nnv_cold_run_continuous(model.plan, cold_c, warm, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes,
+            nb.nnv_cold_run_continuous(model.plan, choices_raw, warm, model.h_weights, model.w_bytes, None, 0,
                                        model.h_input, model.h_output, model.arena, need_c, d_warm, wbytes, s_copy, s_xform, s_exec)
             evs[1].record(s_exec)
             for j in range(3):
@@ -424,20 +513,19 @@ def run_ours(args):
         y_w = model.h_output.numpy().copy()
         cont = {"first_cold_ms": reduce_max(statistics.mean(seq[0])), "second_ms": reduce_max(statistics.mean(seq[1])),
                 "third_ms": reduce_max(statistics.mean(seq[2])), "fourth_ms": reduce_max(statistics.mean(seq[3])),
-                "switched_layers": len(nb.nnv_switch_set(model.plan, cold_c, warm)), "warm_buffer_bytes": int(wbytes),
+                "switched_layers": len(nb.nnv_switch_set(model.plan, choices_raw, warm)), "warm_buffer_bytes": int(wbytes),
                 "parity_rel_l2_end_to_end": None}
         del d_warm
-        if any(c is not None and c[2] for c in choices_cold):
-            model.build_cached_blob(choices_cold)
+        need = max(need, need_c)
         model.arena.fill_(0xFF)
 
     # ---- storage stage: the same end-to-end step with the weights read from a model file (page cache
     # dropped before every run), the paper's "weights reading" in front of copy / transform / execution
     storage = None
-    if args.file_reps > 0:
+    if args.file_reps > 0 and not args.minimal:
         path = os.path.join(tempfile.gettempdir(), "nnv_bench_%d_%d.nnv" % (os.getpid(), rank))
         try:
-            model.write_model_file(path, choices_cold)
+            model.write_model_file(path, choices_byp)
             cache = nb.CacheFile(path)
             ts, rd_ns, rd_b = [], [], []
             for k in range(args.file_reps + 2):
@@ -448,32 +536,22 @@ def run_ours(args):
                 evs2[0].record(s_exec)
                 s_copy.wait_event(evs2[0])
                 s_xform.wait_event(evs2[0])
-                _, _, ns, nbytes = model.cold_run_file(None, choices_cold, cache, depth=args.cold_depth, drop_pages=False)
+                _, _, ns, nbytes = model.cold_run_file(None, choices_raw, cache, depth=args.cold_depth, drop_pages=False)
                 evs2[1].record(s_exec)
                 evs2[1].synchronize()
                 if k >= 2:
                     ts.append(evs2[0].elapsed_time(evs2[1])); rd_ns.append(ns); rd_b.append(nbytes)
-            raw_total = sum(4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"] for L in layers if L["op"] == wl.OP_CONV)
             storage = {"e2e_from_file_ms": reduce_max(statistics.mean(ts)), "file_bytes": int(cache.file_bytes),
-                       "raw_weight_bytes": int(raw_total), "cached_blob_bytes": int(cache.c_bytes),
+                       "raw_weight_bytes": int(sum(raw_bytes(L) for L in layers if L["op"] == wl.OP_CONV)),
+                       "cached_blob_bytes": int(cache.c_bytes),
                        "bytes_read_per_step": int(rd_b[-1]), "reader_gbs": rd_b[-1] / statistics.mean(rd_ns),
-                       "page_cache": "posix_fadvise DONTNEED before every run (best effort)"}
+                       "reader_threads": 4, "page_cache": "posix_fadvise DONTNEED before every run (best effort)"}
             cache.close()
         finally:
             if os.path.exists(path):
                 os.unlink(path)
         model.arena.fill_(0xFF)
 
-    # ---- per-kernel durations for the roofline (same resident steps, with per-operation events) --
-    xf = {}          # layer -> [ns]
-    ex = {}
-    for k in range(args.steps):
-        tm = step_resident(k, False, want_timings=True)
-        for i, t in enumerate(tm):
-            if t["xform_bytes"]:
-                xf.setdefault(i, []).append(t["xform_end_ns"] - t["xform_start_ns"])
-            if layers[i]["op"] == wl.OP_CONV:
-                ex.setdefault(i, []).append(t["exec_end_ns"] - t["exec_start_ns"])
     # host link: one bulk pinned copy of the same number of bytes, as the floor of the end-to-end number
     link_ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     link_ms = []
@@ -486,10 +564,11 @@ def run_ours(args):
         link_ev[1].synchronize()
         link_ms.append(link_ev[0].elapsed_time(link_ev[1]))
     link_gbs = nlink / (min(link_ms) * 1e-3) / 1e9
+
     # the whole model's weights transformed by one multi-layer launch (the decision stage's job, also
     # what builds the cached blob): algorithmic bytes = raw read + transformed written
-    offs_all, total_all = nb.nnv_transformed_layout(model.plan, choices_res)
     xall = None
+    offs_all, total_all = nb.nnv_transformed_layout(model.plan, choices_raw)
     if total_all:
         out_all = harness.dev_bytes(total_all, fill=None)
         ta = []
@@ -497,67 +576,60 @@ def run_ours(args):
             flush.fill_(k & 0xFF)
             s_xform.wait_stream(torch.cuda.current_stream())
             link_ev[0].record(s_xform)
-            nb.nnv_transform_all(model.plan, choices_res, model.d_weights, model.w_bytes, out_all, total_all, s_xform)
+            nb.nnv_transform_all(model.plan, choices_raw, model.d_weights, model.w_bytes, out_all, total_all, s_xform)
             link_ev[1].record(s_xform)
             link_ev[1].synchronize()
             ta.append(link_ev[0].elapsed_time(link_ev[1]))
-        raw_all = sum(4 * layers[i]["K"] * (layers[i]["C"] // layers[i]["groups"]) * layers[i]["R"] * layers[i]["S"]
-                      for i, c in enumerate(choices_res) if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
-        tr_all = sum(nb.nnv_transformed_bytes(model.plan, i, c[0], c[1]) for i, c in enumerate(choices_res)
-                     if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
+        has_xf = [i for i, c in enumerate(choices_raw) if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE)]
+        raw_all = sum(raw_bytes(layers[i]) for i in has_xf)
+        tr_all = sum(nb.nnv_transformed_bytes(model.plan, i, choices_raw[i][0], choices_raw[i][1]) for i in has_xf)
         med = sorted(ta)[len(ta) // 2]
-        xall = {"kernel": "multi_transform_kernel (nnv_transform_all, one launch for the whole model)", "bound": "hbm",
+        xall = {"kernel": "multi_transform_kernel (nnv_transform_all, one launch per transform group for the whole model)", "bound": "hbm",
                 "bytes": raw_all + tr_all, "us": med * 1e3, "achieved": (raw_all + tr_all) / (med * 1e-3) / 1e9,
                 "peak": None, "unit": "GB/s"}
         del out_all
     clocks = sampler.stop()
-    last_tm = tm
-    y_gpu = model.d_output.cpu().numpy()
-
     peaks = load_peaks()
 
-    def avg(v):
-        return statistics.mean(v)
-
-    # The tile / im2col GEMM is the dominant kernel of the step by time share (profiles/): its launches
-    # that are a layer's whole execution (implicit-GEMM and direct-operand 1x1 layers) are timed by the
-    # library's events around that layer.  TF32 dense peak = measured bf16 burst peak x 1/2 (nominal ratio).
-    single = [i for i in ex if choices_res[i][0] in (nb.VAR_IM2COL, nb.VAR_GEMM1X1)
-              and nb.nnv_exec_workspace_bytes(model.plan, i, choices_res[i][0], choices_res[i][1]) == 0]
+    # ---- rooflines from the per-layer events of the TIMED headline steps ----------------------------------
+    xf, ex = {}, {}                                              # layer -> [ns] over the timed steps
+    for tm in step_timings:
+        for i, t in enumerate(tm):
+            if t["xform_bytes"]:
+                xf.setdefault(i, []).append(t["xform_end_ns"] - t["xform_start_ns"])
+            if layers[i]["op"] == wl.OP_CONV:
+                ex.setdefault(i, []).append(t["exec_end_ns"] - t["exec_start_ns"])
+    last_tm = step_timings[-1]
+    avg = statistics.mean
     tf32_peak = peaks["bf16_tflops"] * 0.5
+    tens_peak = peaks["bf16_tflops"] if math == nb.MATH_BF16 else tf32_peak
+    # the tensor-core GEMM launches that are a layer's whole execution (implicit-GEMM, 3x3 halo kernel, direct-operand 1x1)
+    single = [i for i in ex if choices_raw[i][0] in (nb.VAR_IM2COL, nb.VAR_GEMM1X1)
+              and nb.nnv_exec_workspace_bytes(model.plan, i, choices_raw[i][0], choices_raw[i][1]) == 0]
     roof = None
     if single:
-        def gemm_bytes(i):
-            L = layers[i]
-            oh, ow = wl.out_hw(L)
-            qp = -(-(L["R"] * L["S"] * L["C"]) // 8) * 8
-            return 4 * (L["C"] * L["H"] * L["W"] + L["K"] * qp + oh * ow * L["K"])   # X once + packed weights + Y
         gfl = sum(last_tm[i]["exec_flops"] for i in single)
-        gby = sum(gemm_bytes(i) for i in single)
+        gby = sum(gemm_bytes(layers[i]) for i in single)
         gns = sum(avg(ex[i]) for i in single)
         big = max(single, key=lambda i: last_tm[i]["exec_flops"])
-        t_tensor = gfl / (tf32_peak * 1e3)                       # ns at the tensor peak
-        t_hbm = gby / peaks["hbm_gbs"]                            # ns at the HBM peak (weights arrive cold)
-        tens = {"bound": "tensor", "achieved": gfl / gns / 1e3, "peak": tf32_peak, "unit": "TFLOP/s",
-                "frac": gfl / gns / 1e3 / tf32_peak}
+        t_tensor = gfl / (tens_peak * 1e3)                       # ns at the tensor peak
+        t_hbm = gby / peaks["hbm_gbs"]                            # ns at the HBM peak (the weights arrive cold)
+        tens = {"bound": "tensor", "achieved": gfl / gns / 1e3, "peak": tens_peak, "unit": "TFLOP/s", "frac": gfl / gns / 1e3 / tens_peak}
         hbm = {"bound": "hbm", "achieved": gby / gns, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gby / gns / peaks["hbm_gbs"]}
         roof = dict(hbm if t_hbm >= t_tensor else tens)           # the binding roofline of these launches
-        # DRAM bytes per GEMM launch from one ncu capture of this command's timed steps (dram__bytes_read.sum +
-        # dram__bytes_write.sum averaged over the gemm_tc_kernel launches of a step; profiles/ has the command).
-        # Valid for the kernels as they were when it was taken; other workloads have none.
-        traffic = NCU_GEMM_TRAFFIC_BYTES.get((args.config, args.math))
-        roof.update({"kernel": "gemm_tc_kernel (conv3x3_tc_kernel for the layers that take it)", "traffic": traffic,
-                     "peak_source": peaks["source"] + (" HBM copy" if t_hbm >= t_tensor else " bf16 burst x 0.5 (tf32:bf16 nominal ratio)"),
+        roof.update({"kernel": "gemm_tc_kernel / conv3x3_tc_kernel (tcgen05 GEMM; every launch that is a layer's whole execution)",
+                     "traffic": NCU_GEMM_TRAFFIC_BYTES.get((args.config, args.math)),
+                     "durations": "CUDA events around each layer on the execution stream, inside the timed headline steps",
+                     "peak_source": peaks["source"] + (" HBM copy" if t_hbm >= t_tensor else " bf16 burst" + ("" if math == nb.MATH_BF16 else " x 0.5 (tf32:bf16 nominal ratio)")),
                      "other_roofline": tens if t_hbm >= t_tensor else hbm,
                      "launches_per_step": len(single), "flops_per_step": gfl, "bytes_per_step": gby,
-                     "avg_launch_us": gns / len(single) / 1e3,
-                     "largest_launch": {"layer": big, "flops": last_tm[big]["exec_flops"], "bytes": gemm_bytes(big),
+                     "sum_us_per_step": gns / 1e3, "avg_launch_us": gns / len(single) / 1e3,
+                     "largest_launch": {"layer": big, "flops": last_tm[big]["exec_flops"], "bytes": gemm_bytes(layers[big]),
                                         "us": avg(ex[big]) / 1e3, "tflops": last_tm[big]["exec_flops"] / avg(ex[big]) / 1e3}})
-    # the weight-transform kernels (the metric's second half): filter transform and repack, HBM-bound
+    # the weight-transform kernels: filter transform and repack, HBM-bound
     xroof = None
     if xf:
-        # layers transformed by one multi-layer launch share its interval: count each launch once
-        launches = {}
+        launches = {}                                             # layers transformed by one launch share its interval
         for i in xf:
             key = (last_tm[i]["xform_start_ns"], last_tm[i]["xform_end_ns"])
             ent = launches.setdefault(key, {"bytes": 0, "ns": avg(xf[i]), "layers": 0})
@@ -566,51 +638,57 @@ def run_ours(args):
         tb = sum(e["bytes"] for e in launches.values())
         tns = sum(e["ns"] for e in launches.values())
         bigx = max(launches.values(), key=lambda e: e["bytes"])
-        xroof = {"kernel": "multi_transform_kernel (filter transform + repack)", "bound": "hbm", "achieved": tb / tns,
+        xroof = {"kernel": "filter_transform / pack kernels of the timed headline steps", "bound": "hbm", "achieved": tb / tns,
                  "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": tb / tns / peaks["hbm_gbs"], "traffic": None,
                  "peak_source": peaks["source"], "launches_per_step": len(launches), "bytes_per_step": tb,
-                 "avg_launch_us": tns / len(launches) / 1e3,
+                 "sum_us_per_step": tns / 1e3, "avg_launch_us": tns / len(launches) / 1e3,
                  "largest_launch": {"layers": bigx["layers"], "bytes": bigx["bytes"], "us": bigx["ns"] / 1e3,
                                     "gbs": bigx["bytes"] / bigx["ns"]}}
-    flops = sum(last_tm[i]["exec_flops"] for i in ex)
-    exec_ns = sum(statistics.mean(v) for v in ex.values())
-    xform_ns = sum(statistics.mean(v) for v in xf.values())
+    # kernels that are not tensor-core GEMMs, each on the workload's layers that can run it (isolated launches, L2 flushed)
+    krows = None if args.minimal else other_kernel_rooflines(layers, model, nb, torch, flush, peaks)
 
+    flops = sum(last_tm[i]["exec_flops"] for i in ex)
+    exec_ns = sum(avg(v) for v in ex.values())
+    xform_ns = sum(avg(v) for v in xf.values())
+    h2d_ns = sum(last_tm[i]["h2d_end_ns"] - last_tm[i]["h2d_start_ns"] for i in ex)
+    n_xf = sum(1 for c in choices_raw if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
+    per_step_launches = count_launches(layers, choices_raw, model.plan, nb)
+
+    h2d_value = h2d_bytes(layers, choices_raw, model.plan, nb, 0)
+    h2d_e2e = h2d_bytes(layers, choices_raw, model.plan, nb, x.nbytes)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": value, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "tf32" if math == nb.MATH_TF32 else "bf16", "data": "synthetic",
-        "config": {"workload": args.config, "batch": 1, "pipeline_depth": args.depth, "pipeline_depth_e2e": args.cold_depth, "l2": "flushed between steps (256 MiB write)",
-                   "replicas": world, "weights_bytes": int(model.w_bytes), "cuda_graphs": not args.no_graphs},
-        "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": None,
-                "d2h_bytes_per_step": int(model.h_output.numel() * 4), "host_wall_ms": e2e_wall},
-        "gpu_launches": (count_launches(layers, choices_res, model.plan, nb) + count_launches(layers, choices_cold, model.plan, nb)) * args.steps,
+        "config": config_dict(args),
+        "run": {"what": "nnv_cold_run_dio: raw weights H2D + transform + execution, eager (no CUDA graph), selection with allow_cached = 0",
+                "pipeline_depth": args.cold_depth, "replicas": world, "weights_bytes": int(model.w_bytes),
+                "h2d_bytes_per_step": h2d_value, "transform_launches_per_step": n_xf,
+                "cached_layers": sum(1 for c in choices_raw if c is not None and c[2])},
+        "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": h2d_e2e,
+                "d2h_bytes_per_step": int(model.h_output.numel() * 4), "host_wall_ms": e2e_wall,
+                "host_enqueue_ms": statistics.mean(enq) / 1e6,
+                "what": "nnv_cold_run: as `value`, plus the input image from and the output to pinned host memory",
+                "host_link": {"bound": "pcie", "bulk_copy_gbs": link_gbs, "floor_ms": h2d_e2e / link_gbs / 1e6,
+                              "frac_of_floor": (h2d_e2e / link_gbs / 1e6) / e2e if e2e > 0 else None}},
+        "gpu_launches": 2 * per_step_launches * args.steps,
         "clocks": clocks,
         "roofline": roof,
         "roofline_transform": xroof,
         "transform_all": xall,
+        "kernel_rooflines": krows,
+        "arms": arms,
         "algorithm1": alg1,
         "continuous": cont,
         "storage": storage,
-        "breakdown": {"sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3, "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
-                      "choices_resident": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_res],
-                      "choices_cold": [None if c is None else [nb.VARIANT_NAMES[c[0]], nb.MATH_NAMES[c[1]], c[2]] for c in choices_cold]},
+        "breakdown": {"sum_h2d_us": h2d_ns / 1e3, "sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3,
+                      "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
+                      "choices": names(choices_raw, nb), "choices_bypass_arm": names(choices_byp, nb),
+                      "choices_resident_arm": names(choices_res, nb)},
     }
-    # bytes that cross the host link per cold step: weights (raw or cached) + biases + the input
-    h2d = int(x.nbytes)
-    for i, c in enumerate(choices_cold):
-        if c is None:
-            continue
-        L = layers[i]
-        h2d += nb.nnv_transformed_bytes(model.plan, i, c[0], c[1]) if c[2] else 4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"]
-        h2d += 4 * L["K"] if L["has_bias"] else 0
-    line["e2e"]["h2d_bytes_per_step"] = h2d
     if xall:
         xall["peak"] = peaks["hbm_gbs"]
         xall["frac"] = xall["achieved"] / peaks["hbm_gbs"]
-    # the end-to-end step is bound by the host link: bytes that must cross it / measured bulk-copy bandwidth
-    line["e2e"]["host_link"] = {"bound": "pcie", "bulk_copy_gbs": link_gbs, "floor_ms": h2d / link_gbs / 1e6,
-                                "frac_of_floor": (h2d / link_gbs / 1e6) / e2e if e2e > 0 else None}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import conv as oconv
@@ -625,6 +703,7 @@ def run_ours(args):
         ref = omodel.run_model(layers, ws, bs, x)[-1]
         den = float(np.sqrt(np.sum(ref * ref)))
         line["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_gpu[0] - ref) ** 2)) / den)
+        line["e2e"]["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_e2e[0] - ref) ** 2)) / den)
         if alg1:
             alg1["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_s[0] - ref) ** 2)) / den)
         if cont:
@@ -635,9 +714,195 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# Single kernels through the C ABI (CUDA events, L2 flushed between repetitions).  Weights and inputs are
+# seeded random tensors created on the device; nothing here checks results (the tests do).
+def _layer(C, K, R, stride, H, W, groups=1):
+    return dict(op=0, C=C, K=K, R=R, S=R, stride=stride, pad=R // 2 if R > 1 else 0, groups=groups, H=H, W=W, in0=-1, in1=-1,
+                act=1, has_bias=0)
+
+
+def _buf(torch, nbytes):
+    t = torch.empty(max(256, int(nbytes)), dtype=torch.uint8, device="cuda")
+    assert t.data_ptr() % 256 == 0
+    return t
+
+
+def _rand(torch, nfloats, scale=1.0):
+    return (torch.rand(max(64, int(nfloats)), device="cuda", dtype=torch.float32) * 2 - 1) * scale
+
+
+def _time(torch, fn, reps, flush):
+    st = torch.cuda.current_stream()
+    ts = []
+    for r in range(reps + 2):
+        if flush is not None:
+            flush.fill_(r & 0xFF)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        fn(st)
+        e1.record(st)
+        e1.synchronize()
+        if r >= 2:
+            ts.append(e0.elapsed_time(e1) * 1e3)            # us
+    return statistics.median(ts), min(ts)
+
+
+def time_transform(torch, nb, variant, math, C, K, R=3, reps=20, flush=None):
+    L = _layer(C, K, R, 1, 8, 8)
+    plan = nb.Plan([L], [0], [0])
+    rawb = 4 * K * C * R * R
+    outb = nb.nnv_transformed_bytes(plan, 0, variant, math)
+    d_raw = _rand(torch, K * C * R * R, 0.05)
+    d_out = _buf(torch, outb)
+    med, best = _time(torch, lambda st: nb.nnv_transform_weights(plan, 0, variant, math, d_raw, d_out, st), reps, flush)
+    return dict(op="transform", variant=nb.VARIANT_NAMES[variant], math=nb.MATH_NAMES[math], C=C, K=K, R=R,
+                bytes=rawb + outb, us=med, us_min=best, gbs=(rawb + outb) / med / 1e3)
+
+
+def time_conv(torch, nb, variant, math, C, K, R, stride, H, W, groups=1, reps=20, flush=None):
+    L = _layer(C, K, R, stride, H, W, groups)
+    plan = nb.Plan([L], [0], [0])
+    oh, ow = wl.out_hw(L)
+    cg = C // groups
+    d_raw = _rand(torch, K * cg * R * R, 0.05)
+    if variant in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE):
+        d_wt = d_raw
+    else:
+        d_wt = _buf(torch, nb.nnv_transformed_bytes(plan, 0, variant, math))
+        nb.nnv_transform_weights(plan, 0, variant, math, d_raw, d_wt, torch.cuda.current_stream())
+    d_in = _rand(torch, C * H * W)
+    d_out = _buf(torch, 4 * oh * ow * K)
+    wsb = nb.nnv_exec_workspace_bytes(plan, 0, variant, math)
+    d_ws = _buf(torch, wsb) if wsb else None
+    med, best = _time(torch, lambda st: nb.nnv_conv_exec(plan, 0, variant, math, d_in, None, d_wt, None, d_out, d_ws, wsb, st),
+                      reps, flush)
+    flops = 2.0 * oh * ow * K * cg * R * R
+    return dict(op="conv", variant=nb.VARIANT_NAMES[variant], math=nb.MATH_NAMES[math], C=C, K=K, R=R, stride=stride,
+                H=H, W=W, groups=groups, direct_flops=flops, us=med, us_min=best, direct_tflops=flops / med / 1e6)
+
+
+def _offsets(layers):
+    """Byte offsets of each layer's weights in a dense blob (256-byte aligned), no biases."""
+    w_off, pos = [], 0
+    for L in layers:
+        w_off.append(pos)
+        if L["op"] == wl.OP_CONV:
+            pos += (raw_bytes(L) + 255) // 256 * 256
+    return w_off, [0] * len(layers), pos
+
+
+def time_transform_all(torch, nb, config, prefer, math, reps=20, flush=None):
+    """Every layer's weight transform of one configuration by nnv_transform_all.  Layers take the first
+    eligible variant of `prefer`, then gemm1x1 / im2col."""
+    layers = wl.CONFIGS[config]()
+    w_off, b_off, w_bytes = _offsets(layers)
+    plan = nb.Plan(layers, w_off, b_off)
+    choices = []
+    for i, L in enumerate(layers):
+        if L["op"] != wl.OP_CONV:
+            choices.append(None)
+            continue
+        el = nb.nnv_eligible(plan, i)
+        v = next((c for c in prefer + [nb.VAR_GEMM1X1, nb.VAR_IM2COL] if c in el), None)
+        if v is None:
+            v = nb.VAR_DEPTHWISE if nb.VAR_DEPTHWISE in el else el[0]
+        m = nb.MATH_FP32 if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else (nb.MATH_TF32 if v in (nb.VAR_WINO_F4, nb.VAR_WINO_F6) else math)
+        choices.append((v, m, 0))
+    d_w = _rand(torch, w_bytes // 4 + 64, 0.05)
+    offs, total = nb.nnv_transformed_layout(plan, choices)
+    d_out = _buf(torch, total)
+    med, best = _time(torch, lambda st: nb.nnv_transform_all(plan, choices, d_w, w_bytes, d_out, total, st), reps, flush)
+    has = [i for i, c in enumerate(choices) if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE)]
+    raw = sum(raw_bytes(layers[i]) for i in has)
+    out = sum(nb.nnv_transformed_bytes(plan, i, choices[i][0], choices[i][1]) for i in has)
+    # the same bytes moved by a plain device copy, timed the same way: the ceiling of this measurement
+    half = (raw + out) // 2
+    a, b = _buf(torch, half), _buf(torch, half)
+    cmed, _ = _time(torch, lambda st: b.copy_(a, non_blocking=True), reps, flush)
+    return dict(op="transform-all", config=config, prefer=[nb.VARIANT_NAMES[v] for v in prefer], math=nb.MATH_NAMES[math],
+                bytes=raw + out, us=med, us_min=best, gbs=(raw + out) / med / 1e3, copy_same_bytes_us=cmed,
+                copy_gbs=2 * half / cmed / 1e3)
+
+
+def other_kernel_rooflines(layers, model, nb, torch, flush, peaks):
+    """Roofline rows for the kernels that are not tensor-core GEMMs, each timed alone (CUDA events, L2 flushed)
+    on the layers of the workload that can run it: depthwise and direct convolution through nnv_conv_exec.
+    Peaks: HBM = the measured copy bandwidth; FP32 = 2 flop x 128 lanes x 148 SMs x the maximum SM clock."""
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    sms = props.multi_processor_count
+    clk_ghz = 1.965
+    fp32_peak = 2 * 128 * sms * clk_ghz / 1e3                   # TFLOP/s
+    rows = []
+    dw = [L for L in layers if L["op"] == wl.OP_CONV and L["groups"] > 1]
+    if dw:
+        L = max(dw, key=lambda L: L["C"] * L["H"] * L["W"])
+        r = time_conv(torch, nb, nb.VAR_DEPTHWISE, nb.MATH_FP32, L["C"], L["K"], L["R"], L["stride"], L["H"], L["W"], L["groups"], 10, flush)
+        oh, ow = wl.out_hw(L)
+        by = 4 * (L["C"] * L["H"] * L["W"] + L["C"] * oh * ow + L["C"] * L["R"] * L["S"])
+        rows.append({"kernel": "depthwise_kernel", "bound": "hbm", "layer": "%dx%d C=%d stride %d" % (L["H"], L["W"], L["C"], L["stride"]),
+                     "bytes": by, "us": r["us"], "achieved": by / r["us"] / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": by / r["us"] / 1e3 / peaks["hbm_gbs"]})
+    dense = [L for L in layers if L["op"] == wl.OP_CONV and L["groups"] == 1]
+    if dense:
+        L = max(dense, key=lambda L: wl.out_hw(L)[0] * wl.out_hw(L)[1] * L["K"] * L["C"] * L["R"] * L["S"])
+        r = time_conv(torch, nb, nb.VAR_DIRECT, nb.MATH_FP32, L["C"], L["K"], L["R"], L["stride"], L["H"], L["W"], 1, 5, flush)
+        rows.append({"kernel": "direct_conv_kernel", "bound": "alu", "layer": "%dx%d C=%d K=%d R=%d stride %d" % (L["H"], L["W"], L["C"], L["K"], L["R"], L["stride"]),
+                     "flops": r["direct_flops"], "us": r["us"], "achieved": r["direct_tflops"], "peak": fp32_peak, "unit": "TFLOP/s",
+                     "frac": r["direct_tflops"] / fp32_peak,
+                     "peak_derivation": "2 flop x 128 FP32 lanes x %d SMs x %.3f GHz (clocks.max.sm)" % (sms, clk_ghz)})
+    return rows
+
+
+def run_kernel(args):
+    import torch
+    from paper_2206_07446_b200 import binding as nb
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    if args.tuning:
+        nb.nnv_tuning_set(args.tuning)
+    wino = {2: nb.VAR_WINO_F2, 4: nb.VAR_WINO_F4, 6: nb.VAR_WINO_F6}
+    flush = None if args.no_flush else torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    math = nb.MATH_NAMES.index(args.math)
+    a = args
+    if a.kernel == "transform":
+        v = wino[a.m] if (a.R == 3 and a.m in wino) else (nb.VAR_GEMM1X1 if a.R == 1 else nb.VAR_IM2COL)
+        print(json.dumps(time_transform(torch, nb, v, math, a.C, a.K, a.R, a.reps, flush)))
+    elif a.kernel == "transform-sweep":
+        for m in (2, 4, 6):
+            for n in (64, 128, 256, 512, 1024, 2048):
+                print(json.dumps(time_transform(torch, nb, wino[m], nb.MATH_TF32, n, n, 3, a.reps, flush)), flush=True)
+        for n in (64, 256, 512, 1024):
+            print(json.dumps(time_transform(torch, nb, nb.VAR_IM2COL, nb.MATH_TF32, n, n, 3, a.reps, flush)), flush=True)
+            print(json.dumps(time_transform(torch, nb, nb.VAR_IM2COL, nb.MATH_BF16, n, n, 3, a.reps, flush)), flush=True)
+    elif a.kernel == "transform-all":
+        prefer = [nb.VARIANT_NAMES.index(v) for v in a.prefer.split(",") if v]
+        print(json.dumps(time_transform_all(torch, nb, a.config, prefer, math, a.reps, flush)))
+    elif a.kernel == "conv":
+        v = nb.VARIANT_NAMES.index(a.variant)
+        m = nb.MATH_FP32 if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else math
+        print(json.dumps(time_conv(torch, nb, v, m, a.C, a.K, a.R, a.stride, a.H, a.H, a.groups, a.reps, flush)))
+    else:
+        shapes = [(64, 64, 3, 1, 56), (128, 128, 3, 1, 28), (256, 256, 3, 1, 14), (512, 512, 3, 1, 7),
+                  (64, 64, 3, 1, 224), (128, 128, 3, 1, 112), (256, 256, 3, 1, 56), (512, 512, 3, 1, 28),
+                  (256, 256, 3, 1, 112), (256, 256, 3, 1, 224), (512, 512, 3, 1, 112)]   # beyond the configurations: the asymptote
+        for (C, K, R, s, H) in shapes:
+            for v, m in ((nb.VAR_DIRECT, 0), (nb.VAR_IM2COL, 1), (nb.VAR_IM2COL, 2), (nb.VAR_WINO_F2, 1),
+                         (nb.VAR_WINO_F2, 2), (nb.VAR_WINO_F4, 1), (nb.VAR_WINO_F6, 1)):
+                print(json.dumps(time_conv(torch, nb, v, m, C, K, R, s, H, H, 1, a.reps, flush)), flush=True)
+        for (C, K, H) in [(64, 256, 56), (256, 64, 56), (512, 2048, 7), (2048, 512, 7), (320, 1280, 7), (16, 96, 112),
+                          (256, 1024, 14), (1024, 256, 14), (128, 512, 28), (512, 128, 28)]:
+            for m in (1, 2):
+                print(json.dumps(time_conv(torch, nb, nb.VAR_GEMM1X1, m, C, K, 1, 1, H, H, 1, a.reps, flush)), flush=True)
+        for (C, s, H) in [(96, 2, 112), (384, 1, 14), (960, 1, 7)]:
+            print(json.dumps(time_conv(torch, nb, nb.VAR_DEPTHWISE, 0, C, C, 3, s, H, H, C, a.reps, flush)), flush=True)
+
+
 def main():
     args = parse()
-    if args.impl == "reference":
+    if args.kernel:
+        run_kernel(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -133,7 +133,22 @@ typedef struct {
  * a list of layers, each with candidate kernels (input of its Algorithm 1). */
 nnv_status_t nnv_plan_create(const nnv_layer_desc_t* layers, int32_t n,
                              const nnv_plan_opts_t* opts, nnv_plan_t** out);
+/* Waits for work the plan itself still has in flight (the tail of a continuous-mode cold run:
+ * reads and transforms of K_warm - K_cold), then releases events, graphs and the side stream. */
 nnv_status_t nnv_plan_destroy(nnv_plan_t* plan);
+
+/* Tuning overrides for experiments and sweeps (the paper's offline decision stage profiles
+ * candidate kernels, Section 3.3; this lets a harness also profile candidate TILINGS of one
+ * kernel).  Process-wide; read whenever a launch is planned; a recorded graph is tied to the
+ * settings it was recorded under.  spec: "key=value;key=value", NULL or "" = all defaults.
+ *   gemm_tile=BN,splits   column tile (16..128, multiple of 16) and K splits (1,2,4,8) of the GEMM
+ *   gemm_ring=N           shared-memory ring depth 2..8        gemm_prefill=0|1
+ *   conv3x3=off|auto|MT,BN,splits[,boxes,weight_tiles]          the halo-resident 3x3 kernel
+ *   side=0|1  merge=0|1  group=0|1   side stream for residual branches, merged reads, grouped transforms
+ * Every call replaces all settings (unnamed keys return to their defaults).  An item that does not
+ * parse or is out of range -> NNV_ERR_INVALID_ARG and nothing changes; a setting that does not fit a
+ * particular layer (more splits than K blocks, a tiling beyond shared memory) is ignored for it. */
+nnv_status_t nnv_tuning_set(const char* spec);
 
 /* Variants that can execute `layer`, ascending, written to out[0..*n_out).
  * Rules keyed on filter size, stride and grouping (the keys of the paper's
@@ -240,6 +255,46 @@ nnv_status_t nnv_schedule(const nnv_plan_t* plan, const nnv_cost_t* costs, int32
                           const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
                           uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns);
 
+/* The same latency for a machine on which the weights of EVERY queue arrive over one host
+ * link (the paper's Eq. (1)-(2) give each queue its own processor for the whole bundled
+ * preparation; on a discrete GPU all reads share the PCIe link, whatever stream issues them).
+ * A preparation is two operations on its queue, a read (read_ns) and then a transform
+ * (xform_little_ns, or xform_big_ns on queue 0).  The link carries one read at a time; a read
+ * waits from the moment the operation before it on its queue has ended; a free link takes the
+ * waiting read of the lowest layer (reads are issued in layer order).  Executions and the order
+ * inside the queues are as in nnv_simulate, which this call equals when every read_ns is 0. */
+nnv_status_t nnv_simulate_link(const nnv_plan_t* plan, const uint64_t* read_ns, const uint64_t* xform_little_ns,
+                               const uint64_t* xform_big_ns, const uint64_t* exec_ns, const int32_t* queue_of,
+                               int32_t n_little, uint64_t* t_cold_ns);
+
+/* nnv_schedule, except that a combination's latency -- what the search minimises and what
+ * *t_cold_ns returns -- is nnv_simulate_link's: read = the option's h2d_raw_ns or
+ * h2d_cached_ns, transform = xform_ns (0 for a cached option; x big_pct / 100 on queue 0).
+ * The queues of a combination still come from nnv_schedule_queues on the bundled times. */
+nnv_status_t nnv_schedule_link(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                               const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
+                               uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns);
+
+/* Algorithm 1's epsilon (the listing leaves it open): eps_pct percent, rounded down, of the
+ * summed execution time of nnv_select_kernels' per-layer choice. */
+nnv_status_t nnv_schedule_eps(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                              int32_t eps_pct, uint64_t* eps_ns);
+
+/* Algorithm 1's profiling step, repeated under load (the paper's Section 3.3 notes that
+ * operations running beside each other interfere): given the timings of one run of a schedule
+ * (nnv_cold_run_queues with timings), rescale the isolated cost table by how much slower each
+ * KIND of operation ran than it did alone.  For kind k in (read, transform, execution):
+ * num_k = sum over the conv layers of the run's measured interval, den_k = sum of the chosen
+ * kernels' isolated costs (read: h2d_cached_ns if the choice read cached weights, else
+ * h2d_raw_ns; transform: only layers that transformed).  Every row's costs of kind k become
+ * floor(cost * num_k / den_k), exactly; a kind with num_k = 0 or den_k = 0 is left alone.
+ * Scaling by kind, not by kernel, keeps options that did not run from looking cheaper than
+ * those that did.  out: n_costs rows (may alias costs).  factors: NULL or 6 values
+ * {num, den} x {read, transform, execution}.  A chosen kernel without a row -> NNV_ERR_STATE. */
+nnv_status_t nnv_calibrate_costs(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs,
+                                 const nnv_choice_t* choices, const nnv_timing_t* timings,
+                                 nnv_cost_t* out, uint64_t* factors);
+
 /* ---- single operations (asynchronous on `stream`) ------------------------------------------ */
 
 /* Weights transformation (the paper's Section 2 stage, Figure 3): Winograd
@@ -338,6 +393,19 @@ nnv_status_t nnv_cold_run(nnv_plan_t* plan, const nnv_choice_t* choices,
                           void* s_copy, void* s_xform, void* s_exec,
                           int32_t depth, nnv_timing_t* timings);
 
+/* nnv_cold_run for a caller whose activations already live on the GPU (an upstream stage
+ * produced the input there, a downstream stage consumes the output there): d_input / d_output
+ * are DEVICE NCHW fp32 buffers (256-byte aligned).  The weights still take the whole path of
+ * the paper's Section 2 -- read from pinned host memory, transformed, executed; only the two
+ * activation copies across the host link are gone.  Everything else as nnv_cold_run. */
+nnv_status_t nnv_cold_run_dio(nnv_plan_t* plan, const nnv_choice_t* choices,
+                              const void* h_weights, uint64_t w_bytes,
+                              const void* h_cached, uint64_t c_bytes,
+                              const float* d_input, float* d_output,
+                              void* d_arena, uint64_t arena_bytes,
+                              void* s_copy, void* s_xform, void* s_exec,
+                              int32_t depth, nnv_timing_t* timings);
+
 /* One cold inference on the queues Algorithm 1 produced.  queue_of (one entry
  * per layer, as written by nnv_schedule / nnv_schedule_queues) names the queue of
  * every conv layer's bundled preparation -- the copy of its raw (or cached)
@@ -393,6 +461,9 @@ nnv_status_t nnv_resident_run(nnv_plan_t* plan, const nnv_choice_t* choices,
  * calls wait for nothing and replay a recorded graph.
  *   d_warm: nnv_warm_bytes() bytes of device memory, the caller's, kept for as
  *           long as warm runs follow.  warm[i].cached is ignored.
+ *   h_weights (and h_cached) must stay valid and unchanged until the first nnv_warm_run
+ *           after this call has returned (or until s_copy and s_xform have been
+ *           synchronised): the queued reads still copy from them.
  *   Results are bit-identical to nnv_cold_run with the same kernels. */
 nnv_status_t nnv_warm_bytes(const nnv_plan_t* plan, const nnv_choice_t* warm, uint64_t w_bytes, uint64_t* bytes);
 nnv_status_t nnv_cold_run_continuous(nnv_plan_t* plan, const nnv_choice_t* cold, const nnv_choice_t* warm,
@@ -476,6 +547,12 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* plan, const nnv_choice_t* choices, co
 /* Device address, inside the arena of the most recent nnv_cold_run on this
  * plan, of layer `layer`'s NHWC fp32 output (valid until the arena is reused). */
 nnv_status_t nnv_layer_output(const nnv_plan_t* plan, int32_t layer, const void** d_ptr, uint64_t* bytes);
+
+/* Host time, in nanoseconds, that the most recent run on this plan (nnv_cold_run and its
+ * variants, nnv_resident_run, nnv_warm_run) spent putting its work on the streams: every API
+ * call of an eager run, or the one graph launch of a replayed one.  When this exceeds the
+ * device time of the run, the host and not the GPU or the link bounds the cold latency. */
+nnv_status_t nnv_last_enqueue_ns(const nnv_plan_t* plan, uint64_t* ns);
 
 /* Profile every eligible (variant, math) of every conv layer in isolation --
  * the per-operation profiling that feeds the paper's Algorithm 1 -- and write

@@ -126,8 +126,12 @@ def option_times(opt, big_pct):
     return opt[1], opt[1] * big_pct // 100, opt[2]
 
 
-def search(layers, options, n_little, eps, big_pct=100, exhaustive_limit=4096, pool_t=None):
+def search(layers, options, n_little, eps, big_pct=100, exhaustive_limit=4096, pool_t=None, link=False):
     """The outer loop of Algorithm 1 over the filtered candidates.
+
+    With link=True every option is (rank, prep, exec, read) -- read is the part of prep that crosses the host
+    link -- the queues still come from schedule() on the bundled times, but the latency that is compared and
+    returned is simulate_link()'s (transform on queue 0 = (prep - read) * big_pct // 100).
 
     options: per layer, the list of surviving (rank, prep, exec) options in rank order (None for non-conv
     layers; pool_t gives their execution time).  With at most `exhaustive_limit` combinations every one is
@@ -147,6 +151,11 @@ def search(layers, options, n_little, eps, big_pct=100, exhaustive_limit=4096, p
             else:
                 ex[i] = pool_t[i] if pool_t else 0
         q, t = schedule(layers, pl, pb, ex, n_little, eps)
+        if link:
+            rd = [options[i][pick[i]][3] if layers[i]["op"] == 0 else 0 for i in range(n)]
+            xl = [pl[i] - rd[i] for i in range(n)]
+            xb = [xl[i] * big_pct // 100 for i in range(n)]
+            t = simulate_link(layers, rd, xl, xb, ex, q, n_little)
         return t, q
 
     total = 1
@@ -187,3 +196,111 @@ def search(layers, options, n_little, eps, big_pct=100, exhaustive_limit=4096, p
                 break
     ranks = [options[i][best_pick[i]][0] if layers[i]["op"] == 0 else None for i in range(n)]
     return ranks, best_q, best_t
+
+
+# ---- one host link shared by every queue's reads ------------------------------------------------------
+def simulate_link(layers, read_t, xf_little, xf_big, exec_t, queue_of, n_little):
+    """Makespan when the reads of ALL queues pass through one link (a reading of the model for a machine
+    where every queue's weights arrive over the same host link: Eq. (1)-(2) give each queue its own
+    processor for the whole bundled preparation; here only the transform part runs on the queue alone).
+
+    A preparation is now two operations on its queue, read then transform.  The link carries one read at a
+    time; a read is waiting from the moment the operation before it on its queue has ended; whenever the
+    link is free it takes, among the waiting reads, the one of the lowest layer (the order the reads were
+    issued in); a read occupies its queue and the link for read_t.  Everything else is as in simulate():
+    queue 0 runs, in layer order, [read, transform] of its own layers directly before their execution and
+    every execution; queues 1..n_little run their layers' [read, transform] in layer order; an execution
+    needs its transform and the executions of its producers.  Times are integers; returns the end of the
+    last execution.
+    """
+    n = len(layers)
+    conv = [layers[i]["op"] == 0 for i in range(n)]
+    ops = [[] for _ in range(n_little + 1)]                    # per queue: (kind, layer, duration)
+    for i in range(n):
+        if conv[i] and queue_of[i] == 0:
+            ops[0].append(("r", i, read_t[i]))
+            ops[0].append(("x", i, xf_big[i]))
+        ops[0].append(("e", i, exec_t[i]))
+        if conv[i] and queue_of[i] > 0:
+            ops[queue_of[i]].append(("r", i, read_t[i]))
+            ops[queue_of[i]].append(("x", i, xf_little[i]))
+    head = [0] * (n_little + 1)                                # index of the next operation to start
+    busy_until = [0] * (n_little + 1)                          # end of the operation that was started last
+    end = {}                                                   # (kind, layer) -> end time, once started
+    link_free = 0
+    t = 0
+    while ("e", n - 1) not in end:
+        progressed = True
+        while progressed:                                      # start everything that can start at time t
+            progressed = False
+            waiting = []
+            for q in range(n_little + 1):
+                if head[q] >= len(ops[q]) or busy_until[q] > t:
+                    continue
+                kind, i, dur = ops[q][head[q]]
+                if kind == "r":
+                    waiting.append((i, q, dur))
+                    continue
+                deps = [("r", i)] if kind == "x" else ([("x", i)] if conv[i] else []) + \
+                    [("e", s) for s in (layers[i]["in0"], layers[i]["in1"]) if s >= 0]
+                if all(d in end and end[d] <= t for d in deps):
+                    end[(kind, i)] = t + dur
+                    busy_until[q] = t + dur
+                    head[q] += 1
+                    progressed = True
+            if waiting and link_free <= t:
+                i, q, dur = min(waiting)
+                end[("r", i)] = t + dur
+                busy_until[q] = t + dur
+                link_free = t + dur
+                head[q] += 1
+                progressed = True
+        later = [v for v in list(end.values()) + [link_free] if v > t]
+        if ("e", n - 1) in end:
+            break
+        t = min(later)
+    return end[("e", n - 1)]
+
+
+def calibrate(rows, choices, timings):
+    """The re-profiling step of Algorithm 1 (its profiling of operations happens with the other queues
+    busy; Section 3.3's remark on interference): scale the isolated cost table by how much slower each KIND
+    of operation ran in a run of the schedule than it did alone.
+
+    rows: cost rows as dicts (layer, variant, math, h2d_raw_ns, xform_ns, h2d_cached_ns, exec_ns).
+    choices: per layer (variant, math, cached) or None.  timings: per layer dict with h2d/xform/exec start and
+    end stamps of that run.  For kind k in (read, transform, execution): num_k = sum over the chosen kernels
+    of the measured interval, den_k = sum of their isolated costs (read: the cached or the raw read, whichever
+    the choice made; transform: only where the choice transformed).  Every row's costs of kind k become
+    floor(cost * num_k / den_k); a kind with num_k = 0 or den_k = 0 stays as it is.
+    Returns (new rows, [(num, den) for read, transform, execution]).
+    """
+    iso = {(r["layer"], r["variant"], r["math"]): r for r in rows}
+    num = [0, 0, 0]
+    den = [0, 0, 0]
+    for i, ch in enumerate(choices):
+        if ch is None:
+            continue
+        r, t = iso[(i, ch[0], ch[1])], timings[i]
+        has_xf = ch[0] not in (0, 3)                           # DIRECT and DEPTHWISE read raw weights as they are
+        cached = bool(ch[2]) and has_xf
+        num[0] += t["h2d_end_ns"] - t["h2d_start_ns"]
+        den[0] += r["h2d_cached_ns"] if cached else r["h2d_raw_ns"]
+        if has_xf and not cached:
+            num[1] += t["xform_end_ns"] - t["xform_start_ns"]
+            den[1] += r["xform_ns"]
+        num[2] += t["exec_end_ns"] - t["exec_start_ns"]
+        den[2] += r["exec_ns"]
+
+    def scale(v, k):
+        return v if num[k] == 0 or den[k] == 0 else v * num[k] // den[k]
+
+    out = [dict(r, h2d_raw_ns=scale(r["h2d_raw_ns"], 0), h2d_cached_ns=scale(r["h2d_cached_ns"], 0),
+                xform_ns=scale(r["xform_ns"], 1), exec_ns=scale(r["exec_ns"], 2)) for r in rows]
+    return out, list(zip(num, den))
+
+
+def schedule_eps(exec_of_choice, eps_pct):
+    """Algorithm 1's epsilon: eps_pct percent (rounded down) of the summed execution time of the per-layer
+    cold-cost choice; exec_of_choice lists those execution times."""
+    return sum(exec_of_choice) * eps_pct // 100

@@ -65,6 +65,7 @@ _P = ctypes.POINTER
 _SIGS = {
     "nnv_plan_create": [_P(LayerDesc), _i32, _P(PlanOpts), _P(_vp)],
     "nnv_plan_destroy": [_vp],
+    "nnv_tuning_set": [ctypes.c_char_p],
     "nnv_eligible": [_vp, _i32, _P(_i32), _i32, _P(_i32)],
     "nnv_transformed_bytes": [_vp, _i32, _i32, _i32, _P(_u64)],
     "nnv_exec_workspace_bytes": [_vp, _i32, _i32, _i32, _P(_u64)],
@@ -77,6 +78,10 @@ _SIGS = {
     "nnv_simulate": [_vp, _P(_u64), _P(_u64), _P(_u64), _P(_i32), _i32, _P(_u64)],
     "nnv_schedule_queues": [_vp, _P(_u64), _P(_u64), _P(_u64), _i32, _u64, _P(_i32), _P(_u64)],
     "nnv_schedule": [_vp, _P(Cost), _i32, _i32, _P(_u64), _i32, _u64, _i32, _u64, _P(Choice), _P(_i32), _P(_u64)],
+    "nnv_simulate_link": [_vp, _P(_u64), _P(_u64), _P(_u64), _P(_u64), _P(_i32), _i32, _P(_u64)],
+    "nnv_schedule_link": [_vp, _P(Cost), _i32, _i32, _P(_u64), _i32, _u64, _i32, _u64, _P(Choice), _P(_i32), _P(_u64)],
+    "nnv_schedule_eps": [_vp, _P(Cost), _i32, _i32, _i32, _P(_u64)],
+    "nnv_calibrate_costs": [_vp, _P(Cost), _i32, _P(Choice), _P(Timing), _P(Cost), _P(_u64)],
     "nnv_transform_weights": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
     "nnv_transformed_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
     "nnv_transform_all": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp],
@@ -86,6 +91,7 @@ _SIGS = {
     "nnv_chw_to_hwc": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_hwc_to_chw": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_cold_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing)],
+    "nnv_cold_run_dio": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing)],
     "nnv_cold_run_queues": [_vp, _P(Choice), _P(_i32), _i32, _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _P(_vp), _P(Timing)],
     "nnv_resident_run": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _i32, _P(Timing)],
     "nnv_warm_bytes": [_vp, _P(Choice), _u64, _P(_u64)],
@@ -102,6 +108,7 @@ _SIGS = {
     "nnv_cold_run_file": [_vp, _P(Choice), _vp, _vp, _u64, _vp, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _i32, _P(Timing),
                           _P(_u64), _P(_u64)],
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
+    "nnv_last_enqueue_ns": [_vp, _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
     "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
     "nnv_device_status": [_P(_i32)],
@@ -192,6 +199,11 @@ def nnv_plan_destroy(plan):
     plan.close()
 
 
+def nnv_tuning_set(spec=None):
+    """Process-wide tuning overrides, "key=value;key=value"; None or "" restores the defaults."""
+    _check(_lib.nnv_tuning_set(None if spec is None else spec.encode("ascii")))
+
+
 def nnv_eligible(plan, layer):
     out = (_i32 * 8)()
     n = _i32(0)
@@ -234,7 +246,24 @@ def nnv_cached_layout(plan, choices):
     return [int(o) for o in offs], int(total.value)
 
 
+class CostTable:
+    """A cost table already laid out as the C array of nnv_cost_t, so that calls that take one (selection,
+    scheduling) cost what the library call costs and not the conversion from Python dicts."""
+
+    def __init__(self, costs):
+        self.rows = [dict(c) for c in costs]
+        self.array = _costs_array(self.rows)
+
+    def __len__(self):
+        return len(self.rows)
+
+    def __iter__(self):
+        return iter(self.rows)
+
+
 def _costs_array(costs):
+    if isinstance(costs, CostTable):
+        return costs.array
     arr = (Cost * max(1, len(costs)))()
     for i, c in enumerate(costs):
         arr[i] = Cost(int(c["layer"]), int(c["variant"]), int(c["math"]), 0, int(c["h2d_raw_ns"]),
@@ -296,13 +325,52 @@ def nnv_schedule_queues(plan, prep_little_ns, prep_big_ns, exec_ns, n_little, ep
     return [int(v) for v in q], int(t.value)
 
 
-def nnv_schedule(plan, costs, allow_cached, n_little, eps_ns=0, big_pct=100, combo_limit=4096, pool_ns=None):
+def nnv_simulate_link(plan, read_ns, xform_little_ns, xform_big_ns, exec_ns, queue_of, n_little):
+    if len(queue_of) != plan.n:
+        raise ValueError("one entry per layer expected")
+    t = _u64(0)
+    _check(_lib.nnv_simulate_link(plan.handle, _u64_array(plan, read_ns), _u64_array(plan, xform_little_ns),
+                                  _u64_array(plan, xform_big_ns), _u64_array(plan, exec_ns),
+                                  (_i32 * plan.n)(*[int(q) for q in queue_of]), n_little, ctypes.byref(t)))
+    return int(t.value)
+
+
+def nnv_schedule_eps(plan, costs, allow_cached, eps_pct):
+    e = _u64(0)
+    _check(_lib.nnv_schedule_eps(plan.handle, _costs_array(costs), len(costs), int(allow_cached), int(eps_pct), ctypes.byref(e)))
+    return int(e.value)
+
+
+def _timings_array(plan, timings):
+    arr = (Timing * plan.n)()
+    for i, t in enumerate(timings):
+        for f, _ in Timing._fields_:
+            if f in ("choice", "reserved"):
+                continue
+            setattr(arr[i], f, int(t.get(f, 0)))
+    return arr
+
+
+def nnv_calibrate_costs(plan, costs, choices, timings):
+    """Returns (rescaled cost rows as dicts, [(num, den) for read, transform, execution])."""
+    n = len(costs)
+    out = (Cost * max(1, n))()
+    fac = (_u64 * 6)()
+    _check(_lib.nnv_calibrate_costs(plan.handle, _costs_array(costs), n, _choices_array(plan, choices),
+                                    _timings_array(plan, timings), out, fac))
+    rows = [{f: int(getattr(out[i], f)) for f, _ in Cost._fields_ if f != "reserved"} for i in range(n)]
+    return rows, [(int(fac[2 * k]), int(fac[2 * k + 1])) for k in range(3)]
+
+
+def nnv_schedule(plan, costs, allow_cached, n_little, eps_ns=0, big_pct=100, combo_limit=4096, pool_ns=None, link=False):
+    """Algorithm 1; link=True evaluates every combination with the shared-link latency (nnv_schedule_link)."""
     out = (Choice * plan.n)()
     q = (_i32 * plan.n)()
     t = _u64(0)
     pool = _u64_array(plan, pool_ns) if pool_ns is not None else None
-    _check(_lib.nnv_schedule(plan.handle, _costs_array(costs), len(costs), int(allow_cached), pool, n_little,
-                             int(eps_ns), int(big_pct), int(combo_limit), out, q, ctypes.byref(t)))
+    fn = _lib.nnv_schedule_link if link else _lib.nnv_schedule
+    _check(fn(plan.handle, _costs_array(costs), len(costs), int(allow_cached), pool, n_little,
+              int(eps_ns), int(big_pct), int(combo_limit), out, q, ctypes.byref(t)))
     choices = [None if out[i].variant < 0 else (out[i].variant, out[i].math, out[i].cached) for i in range(plan.n)]
     return choices, [int(v) for v in q], int(t.value)
 
@@ -357,6 +425,16 @@ def nnv_cold_run(plan, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, 
     _check(_lib.nnv_cold_run(plan.handle, _choices_array(plan, choices), _ptr(h_weights), int(w_bytes),
                              _ptr(h_cached), int(c_bytes), _ptr(h_input), _ptr(h_output), _ptr(d_arena),
                              int(arena_bytes), _stream(s_copy), _stream(s_xform), _stream(s_exec), int(depth), tarr))
+    return _timings_list(tarr)
+
+
+def nnv_cold_run_dio(plan, choices, h_weights, w_bytes, h_cached, c_bytes, d_input, d_output, d_arena, arena_bytes,
+                     s_copy, s_xform, s_exec, depth, want_timings=False):
+    """nnv_cold_run with the model input / output in device memory; weights still come from pinned host memory."""
+    tarr = (Timing * plan.n)() if want_timings else None
+    _check(_lib.nnv_cold_run_dio(plan.handle, _choices_array(plan, choices), _ptr(h_weights), int(w_bytes),
+                                 _ptr(h_cached), int(c_bytes), _ptr(d_input), _ptr(d_output), _ptr(d_arena),
+                                 int(arena_bytes), _stream(s_copy), _stream(s_xform), _stream(s_exec), int(depth), tarr))
     return _timings_list(tarr)
 
 
@@ -481,6 +559,12 @@ def nnv_layer_output(plan, layer):
     b = _u64(0)
     _check(_lib.nnv_layer_output(plan.handle, layer, ctypes.byref(p), ctypes.byref(b)))
     return int(p.value), int(b.value)
+
+
+def nnv_last_enqueue_ns(plan):
+    b = _u64(0)
+    _check(_lib.nnv_last_enqueue_ns(plan.handle, ctypes.byref(b)))
+    return int(b.value)
 
 
 def nnv_profile_arena_bytes(plan):

@@ -93,6 +93,8 @@ void cache_geometry(const nnv_cache* c, uint64_t* raw_off, uint64_t* cached_off,
     *file_choices = c->choices.data(); *n_layers = (int)c->n_layers;
 }
 
+const nnv_layer_desc_t* cache_layers(const nnv_cache* c) { return c->layers.data(); }
+
 }  // namespace nnv
 
 extern "C" {

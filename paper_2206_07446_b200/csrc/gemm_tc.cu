@@ -21,7 +21,6 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
-#include <cstdlib>
 #include <mutex>
 
 #include "nnv_internal.h"
@@ -728,25 +727,20 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         }
         if (bn <= 16) break;
     }
-    if (const char* e = std::getenv("NNV_DEBUG_GEMM_TILE")) {      // debug only: "BN,splits"
-        int fb = 0, fs = 0;
-        if (std::sscanf(e, "%d,%d", &fb, &fs) == 2 && fb >= 16 && fb <= 128 && fb % 16 == 0 && fs >= 1 && fs <= 8 &&
-            (fs & (fs - 1)) == 0 && fs <= nkb_all) { BN = fb; splits = fs; }
-    }
+    const Tuning tn = tuning();
+    if (tn.gemm_bn && tn.gemm_splits <= nkb_all) { BN = tn.gemm_bn; splits = tn.gemm_splits; }   // override (nnv_tuning_set)
     // A 3x3 / stride 1 / pad 1 layer large enough to fill the GPU runs on the halo-resident kernel,
     // which moves fewer operand bytes through L2 and shared memory.
     if (a.ic.on && a.mode == GEMM_TF32 && a.batch == 1 && a.ic.R == 3 && a.ic.S == 3 && a.ic.stride == 1 && a.ic.pad == 1 &&
         (a.ic.C % 32) == 0) {
         ConvTiling ct;
         bool use = pick_conv_tiling(a.ic.C, a.ic.H, a.ic.W, a.N, &ct);
-        if (const char* e = std::getenv("NNV_DEBUG_CONV3X3")) {     // debug only: "off", or "MT,BN,splits[,boxes,weight tiles]"
+        if (tn.conv3x3 == 1) {
+            use = false;
+        } else if (tn.conv3x3 == 2) {
             ConvTiling f{};
-            if (e[0] == 'o') {
-                use = false;
-            } else if (std::sscanf(e, "%d,%d,%d,%d,%d", &f.MT, &f.BN, &f.splits, &f.na, &f.nb) >= 3 && (f.MT == 1 || f.MT == 2) &&
-                       f.BN >= 16 && f.BN <= 128 && f.BN % 16 == 0 && f.splits >= 1 && f.splits <= 8 &&
-                       (f.splits & (f.splits - 1)) == 0 && f.splits <= ceil_div(a.ic.C, 32) && f.na <= CONV_MAX_NA &&
-                       f.nb <= CONV_MAX_NB && finish_conv_tiling(&f)) {
+            f.MT = tn.conv_mt; f.BN = tn.conv_bn; f.splits = tn.conv_splits; f.na = tn.conv_na; f.nb = tn.conv_nb;
+            if (f.splits <= ceil_div(a.ic.C, 32) && finish_conv_tiling(&f)) {
                 ct = f;
                 use = true;
             }
@@ -759,10 +753,7 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     // by the SM's L2 read rate, not by latency), so 4 stages (3 with the extra converted tiles).
     const uint32_t sb = (a.mode == GEMM_X3) ? stage_bytes_of<2>(BN) : stage_bytes_of<0>(BN);
     int ring = (a.mode == GEMM_X3) ? 3 : 4;
-    if (const char* e = std::getenv("NNV_DEBUG_GEMM_RING")) {      // debug only: ring depth
-        const int r = std::atoi(e);
-        if (r >= 2 && r <= 8 && (size_t)r * sb <= 210u * 1024u) ring = r;
-    }
+    if (tn.gemm_ring && (size_t)tn.gemm_ring * sb <= 210u * 1024u) ring = tn.gemm_ring;
     while (splits > 1 && (uint32_t)ring * sb < (uint32_t)BM * (BN + 4) * 4u) ++ring;   // room to park the partial tile
 
     const bool bf16 = a.mode == GEMM_BF16;
@@ -770,7 +761,7 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     GemmDev g;
     g.D = a.D; g.bias = a.bias; g.addend = a.addend;
     g.ldd = a.ldd; g.strideD = a.strideD;
-    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits; g.stages = ring; g.prefill = std::getenv("NNV_DEBUG_GEMM_NOPREFILL") ? 0 : 1;
+    g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits; g.stages = ring; g.prefill = tn.gemm_prefill;
     g.ic_on = 0; g.ic_C = g.ic_cblk = g.ic_S = g.ic_OW = g.ic_stride = g.ic_pad = 0;
     if (a.ic.on) {
         NNV_REQUIRE(a.mode == GEMM_TF32 && a.batch == 1, NNV_ERR_INVALID_ARG, "implicit im2col needs the TF32 mode and one batch");

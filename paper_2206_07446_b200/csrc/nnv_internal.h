@@ -113,7 +113,22 @@ struct ArenaLayout {
 }  // namespace nnv
 
 namespace nnv {
+// Tuning overrides (nnv_tuning_set): process-wide, read when a launch is planned.  `generation`
+// changes with every successful nnv_tuning_set call and is part of the key of a recorded graph, so a
+// replay never runs with other tilings than an eager call made at the same time would.
+struct Tuning {
+    int gemm_bn = 0, gemm_splits = 0;         // 0 = the cost model decides
+    int gemm_ring = 0;                        // 0 = default ring depth
+    int gemm_prefill = 1;
+    int conv3x3 = 0;                          // 0 auto, 1 off, 2 forced tiling below
+    int conv_mt = 0, conv_bn = 0, conv_splits = 0, conv_na = 0, conv_nb = 0;
+    int side = 1, merge = 1, group = 1;       // pipeline features: side stream, merged reads, grouped transforms
+    uint64_t generation = 0;
+};
+Tuning tuning();                              // a copy of the current overrides (thread safe)
+
 struct GraphKey {
+    uint64_t tuning_gen = 0;
     std::vector<nnv_choice_t> choices;
     std::vector<const void*> ptrs;
     uint64_t w_bytes = 0;
@@ -122,7 +137,7 @@ struct GraphKey {
     bool host_io = false;
     std::vector<int32_t> queues;          // preparation queue per layer (scheduled runs), else empty
     bool operator==(const GraphKey& o) const {
-        if (ptrs != o.ptrs || w_bytes != o.w_bytes || depth != o.depth || resident != o.resident || host_io != o.host_io ||
+        if (tuning_gen != o.tuning_gen || ptrs != o.ptrs || w_bytes != o.w_bytes || depth != o.depth || resident != o.resident || host_io != o.host_io ||
             queues != o.queues || choices.size() != o.choices.size())
             return false;
         for (size_t i = 0; i < choices.size(); ++i)
@@ -151,6 +166,7 @@ struct nnv_plan {
     int* h_status = nullptr;              // pinned host word the device status is copied into
     cudaStream_t s_side = nullptr;        // the plan's own stream for residual-branch layers (created on first use)
     std::vector<cudaEvent_t> warm_ev;     // continuous mode: layer i's warm weights are prepared
+    uint64_t last_enqueue_ns = 0;         // host time the last run spent putting its work on the streams
     bool warm_pending = false;            // warm preparations may still be running (first warm run waits)
 };
 
@@ -244,6 +260,8 @@ nnv_status_t gemm_tc_init();
 nnv_status_t cache_read_range(const nnv_cache* c, uint64_t off, void* dst, uint64_t n);
 void cache_geometry(const nnv_cache* c, uint64_t* raw_off, uint64_t* cached_off, uint64_t* w_bytes, uint64_t* c_bytes,
                     const nnv_choice_t** file_choices, int* n_layers);
+
+const nnv_layer_desc_t* cache_layers(const nnv_cache* c);      // the file's layer table (n_layers entries)
 
 nnv_status_t read_device_status(int32_t* code);
 // Enqueue a copy of the device status word into pinned host memory on `st` (no synchronisation).

@@ -3,7 +3,6 @@
 #include <atomic>
 #include <chrono>
 #include <condition_variable>
-#include <cstdlib>
 #include <cstring>
 #include <functional>
 #include <mutex>
@@ -49,6 +48,18 @@ struct WarmCtx {
     uint64_t xf_region;
     std::vector<uint64_t> woff;
 };
+
+static XformDesc make_xform_desc(const nnv_plan& p, int i, const nnv_choice_t& ch, const void* src, void* dst) {
+    const nnv_layer_desc_t& L = p.layers[i];
+    XformDesc d{};
+    d.src = src;
+    d.dst = dst;
+    d.K = L.K; d.C = L.C; d.Cp = p.geom[i].Cp; d.RS = L.R * L.S; d.Qp = p.geom[i].Qp;
+    d.bf16 = ch.math == NNV_MATH_BF16;
+    const int m = wino_m(ch.variant);
+    d.kind = m == 2 ? XF_WINO2 : m == 4 ? XF_WINO4 : m == 6 ? XF_WINO6 : (d.RS == 1 ? XF_PACK1X1 : XF_PACK);
+    return d;
+}
 
 static bool same_kernel(const nnv_choice_t& a, const nnv_choice_t& b) { return a.variant == b.variant && a.math == b.math; }
 
@@ -100,7 +111,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // branch, when they need no execution scratch (the one scratch buffer belongs to s_exec).
     std::vector<char> on_side(n, 0);
     bool any_side = false;
-    if (!queued && !std::getenv("NNV_DEBUG_NO_SIDE")) {
+    const Tuning tn = tuning();
+    if (!queued && tn.side) {
         for (int i = 0; i < n; ++i) {
             if (p->layers[i].op != NNV_OP_CONV || exec_ws_bytes(*p, i, choices[i].variant, choices[i].math) != 0) continue;
             bool as_input = false, as_addend = false;
@@ -120,13 +132,16 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     cudaStream_t s_side = p->s_side;
     const cudaEvent_t ev_input = p->ev[3 * n + 6 + NNV_MAX_QUEUES], ev_side_join = p->ev[3 * n + 7 + NNV_MAX_QUEUES];
 
-    // Host-to-device copies cost ~8 us each before the first byte moves, so at depth 0 (where the arena
-    // mirrors the host blobs' layouts) consecutive layers whose source and destination ranges line up are
-    // read by ONE copy of up to ~1 MB; all layers of such a chunk become ready when it lands.
+    // A host-to-device copy costs ~4 us on top of its bytes even when it directly follows another one on
+    // its stream (measured: 64 MB as 1 MB copies moves at 45 GB/s, as 4 MB copies at 52, as one copy at
+    // 55), so at depth 0 (where the arena mirrors the host blobs' layouts) consecutive layers whose source
+    // and destination ranges line up are read by ONE copy.  The chunks start at 256 KB, so that execution
+    // begins early, and double up to 4 MB; all layers of a chunk become ready when it lands, and their
+    // weight transforms are one grouped launch.
     struct CopyChunk { const uint8_t* src; uint8_t* dst; uint64_t bytes; int first, last; };
     std::vector<CopyChunk> chunks;
     std::vector<int> chunk_of(n, -1);
-    bool merge = !resident && !queued && depth == 0 && !wc && !std::getenv("NNV_DEBUG_NO_MERGE");
+    bool merge = !resident && !queued && depth == 0 && !wc && tn.merge;
     if (merge) {
         // Coarser copies make layers ready later (a layer waits for its whole chunk), which only pays when
         // the link, not execution, is what the run waits for: rough estimate, bytes at 50 GB/s against
@@ -143,7 +158,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         merge = (double)bytes / 50e3 > 8.0 * convs;              // us
     }
     if (merge) {
-        constexpr uint64_t kTarget = 1u << 20, kMaxGap = 4096;
+        constexpr uint64_t kFirstTarget = 256u << 10, kMaxTarget = 4u << 20, kMaxGap = 4096;
+        uint64_t target = kFirstTarget;
         int cur_kind = -1;
         for (int i = 0; i < n; ++i) {
             const nnv_layer_desc_t& L = p->layers[i];
@@ -157,13 +173,14 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (!chunks.empty() && cur_kind == (int)cached) {
                 CopyChunk& c = chunks.back();
                 if (src >= c.src + c.bytes && (uint64_t)(src - (c.src + c.bytes)) <= kMaxGap && src - c.src == dst - c.dst &&
-                    c.bytes < kTarget) {
+                    c.bytes < target && i - c.first < XF_BATCH_MAX) {
                     c.bytes = (uint64_t)(src - c.src) + len;
                     c.last = i;
                     joined = true;
                 }
             }
             if (!joined) {
+                if (!chunks.empty()) target = std::min(target * 2, kMaxTarget);
                 chunks.push_back(CopyChunk{src, dst, len, i, i});
                 cur_kind = (int)cached;
             }
@@ -171,7 +188,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         }
     }
 
-    const bool grouped = resident && depth == 0 && !std::getenv("NNV_DEBUG_NO_GROUP");
+    const bool grouped = resident && depth == 0 && tn.group;
     std::vector<cudaEvent_t> group_event(n, nullptr);
 
     // Everything the pass puts on the streams: fork from s_exec, the per-layer operations, join back.
@@ -206,13 +223,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (L.op != NNV_OP_CONV) continue;
             const nnv_choice_t ch = choices[i];
             if (!variant_has_transform(ch.variant) || ch.cached) continue;
-            XformDesc d{};
-            d.src = (const uint8_t*)weights + L.w_off;
-            d.dst = base + A.xf_off[i];
-            d.K = L.K; d.C = L.C; d.Cp = p->geom[i].Cp; d.RS = L.R * L.S; d.Qp = p->geom[i].Qp;
-            d.bf16 = ch.math == NNV_MATH_BF16;
-            const int m = wino_m(ch.variant);
-            d.kind = m == 2 ? XF_WINO2 : m == 4 ? XF_WINO4 : m == 6 ? XF_WINO6 : (d.RS == 1 ? XF_PACK1X1 : XF_PACK);
+            const XformDesc d = make_xform_desc(*p, i, ch, (const uint8_t*)weights + L.w_off, base + A.xf_off[i]);
             const int g = first_bytes < (1u << 20) ? 0 : first_bytes < (9u << 20) ? 1 : 2;
             first_bytes += raw_weight_bytes(L);
             descs[g].push_back(d);
@@ -312,9 +323,23 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                     }
                     if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
                     NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
+                    // the weight transforms of the chunk's layers: one grouped launch behind the copy
+                    std::vector<XformDesc> descs;
+                    for (int k = c.first; k <= c.last; ++k) {
+                        const nnv_layer_desc_t& Lk = p->layers[k];
+                        if (Lk.op != NNV_OP_CONV || !variant_has_transform(choices[k].variant) || choices[k].cached) continue;
+                        descs.push_back(make_xform_desc(*p, k, choices[k], base + A.raw_off[k], base + A.xf_off[k]));
+                    }
+                    if (!descs.empty()) {
+                        NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(i, 0), 0));
+                        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
+                        NNV_TRY(launch_transform_batch(descs.data(), (int)descs.size(), s_xform));
+                        if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
+                        NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
+                    }
                 }
                 copied += (cached ? tbytes : rbytes) + (L.has_bias ? 4ull * L.K : 0);
-                ready = EV(c.first, 0);
+                ready = (has_xf && !cached) ? EV(c.first, 1) : EV(c.first, 0);
             } else {
             if (before_read) NNV_TRY((*before_read)(i));         // the layer's bytes have arrived from storage
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
@@ -340,6 +365,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             // done above, inside the bundled preparation
         } else if (grouped) {
             if (has_xf && !cached) ready = group_event[i];
+        } else if (merge) {
+            // done with the chunk's copy
         } else if (has_xf && !cached) {
             if (ready) NNV_CUDA(cudaStreamWaitEvent(s_xform, ready, 0));
             else if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
@@ -428,6 +455,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // by the choices and every buffer address) and replayed by later calls with the same arguments:
     // the host then issues one launch instead of a few hundred API calls.
     GraphKey key;
+    key.tuning_gen = tn.generation;
     key.choices.assign(choices, choices + n);
     key.ptrs = {weights, cached_blob, input, output, d_arena};
     key.w_bytes = w_bytes; key.depth = depth; key.resident = resident; key.host_io = host_io;
@@ -461,11 +489,13 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             cg = &p->graphs.back();
         }
     }
+    const auto t_enq0 = std::chrono::steady_clock::now();
     if (cg && cg->exec) {
         NNV_CUDA(cudaGraphLaunch(cg->exec, s_exec));
     } else {
         NNV_TRY(enqueue());
     }
+    p->last_enqueue_ns = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t_enq0).count();
     NNV_CUDA(cudaStreamSynchronize(s_exec));
 
     if (tm) {
@@ -490,8 +520,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                 NNV_TRY(stamp(p->tev[6 * n + 1 + 2 * g], &timings[i].xform_start_ns));
                 NNV_TRY(stamp(p->tev[6 * n + 2 + 2 * g], &timings[i].xform_end_ns));
             } else if (timings[i].xform_bytes) {
-                NNV_TRY(stamp(TEV(i, 2), &timings[i].xform_start_ns));
-                NNV_TRY(stamp(TEV(i, 3), &timings[i].xform_end_ns));
+                const int xi = (merge && chunk_of[i] >= 0) ? chunks[chunk_of[i]].first : i;   // a chunk's grouped launch
+                NNV_TRY(stamp(TEV(xi, 2), &timings[i].xform_start_ns));
+                NNV_TRY(stamp(TEV(xi, 3), &timings[i].xform_end_ns));
             }
         }
     }
@@ -519,6 +550,21 @@ nnv_status_t nnv_cold_run(nnv_plan_t* p, const nnv_choice_t* choices, const void
                 "the three streams must be distinct");
     return run_model(p, choices, h_weights, w_bytes, h_cached, c_bytes, h_input, h_output, d_arena, arena_bytes,
                      (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings, false);
+}
+
+nnv_status_t nnv_cold_run_dio(nnv_plan_t* p, const nnv_choice_t* choices, const void* h_weights, uint64_t w_bytes,
+                              const void* h_cached, uint64_t c_bytes, const float* d_input, float* d_output,
+                              void* d_arena, uint64_t arena_bytes, void* s_copy, void* s_xform, void* s_exec,
+                              int32_t depth, nnv_timing_t* timings) {
+    NNV_REQUIRE(p && choices && h_weights && d_input && d_output && d_arena, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(depth >= 0 && depth <= p->opts.max_depth, NNV_ERR_INVALID_ARG, "depth %d outside 0..%d", depth, p->opts.max_depth);
+    NNV_REQUIRE(aligned256(d_arena) && aligned256(d_input) && aligned256(d_output), NNV_ERR_INVALID_ARG,
+                "device pointers must be 256-byte aligned");
+    NNV_REQUIRE(s_copy != s_xform && s_copy != s_exec && s_xform != s_exec, NNV_ERR_INVALID_ARG,
+                "the three streams must be distinct");
+    return run_model(p, choices, h_weights, w_bytes, h_cached, c_bytes, d_input, d_output, d_arena, arena_bytes,
+                     (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings, false, nullptr, nullptr,
+                     0, 0);
 }
 
 nnv_status_t nnv_cold_run_queues(nnv_plan_t* p, const nnv_choice_t* choices, const int32_t* queue_of, int32_t n_little,
@@ -644,6 +690,19 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
     int file_n;
     cache_geometry(cache, &raw_off, &cached_off, &w_bytes, &c_bytes, &file_choices, &file_n);
     NNV_REQUIRE(file_n == n, NNV_ERR_INVALID_ARG, "the file describes %d layers, the plan %d", file_n, n);
+    {
+        // the file must describe THIS model: same layers, same places in the raw blob
+        const nnv_layer_desc_t* fl = cache_layers(cache);
+        for (int i = 0; i < n; ++i) {
+            const nnv_layer_desc_t& a = p->layers[i];
+            const nnv_layer_desc_t& b = fl[i];
+            const bool same = a.op == b.op && a.C == b.C && a.K == b.K && a.R == b.R && a.S == b.S && a.stride == b.stride &&
+                              a.pad == b.pad && a.groups == b.groups && a.H == b.H && a.W == b.W && a.in0 == b.in0 && a.in1 == b.in1 &&
+                              a.act == b.act && a.has_bias == b.has_bias &&
+                              (a.op != NNV_OP_CONV || (a.w_off == b.w_off && (!a.has_bias || a.b_off == b.b_off)));
+            NNV_REQUIRE(same, NNV_ERR_INVALID_ARG, "layer %d of the file differs from the plan's (another model's file?)", i);
+        }
+    }
     NNV_REQUIRE(stage_w_bytes >= w_bytes, NNV_ERR_WORKSPACE_TOO_SMALL, "weight staging needs %llu bytes", (unsigned long long)w_bytes);
     std::vector<uint64_t> coff(n), fcoff(n);
     uint64_t ctotal = 0, fctotal = 0;
@@ -663,62 +722,84 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
         }
     }
 
-    // Reader thread: layer by layer, the bytes the layer's choice reads (cached blob entry, or raw
-    // weights; the bias) from the file into the pinned staging buffers, at the blobs' own offsets.
+    for (int i = 0; i < n; ++i)
+        if (p->layers[i].op == NNV_OP_CONV)
+            NNV_REQUIRE(p->layers[i].w_off + raw_weight_bytes(p->layers[i]) <= w_bytes &&
+                            (!p->layers[i].has_bias || p->layers[i].b_off + 4ull * p->layers[i].K <= w_bytes),
+                        NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the file's raw blob", i);
+
+    // Reader threads.  The bytes each layer's choice reads (its cached blob entry, or its raw weights;
+    // its bias) are cut into pieces of up to 2 MiB, listed in layer order; kReaders threads take the next
+    // piece off the list and pread it from the file into the pinned staging buffers, at the blobs' own
+    // offsets.  Several requests are then in flight at the storage device at once, which a single
+    // buffered reader never achieves.  A layer is ready once all its pieces have arrived.
+    struct Piece { uint64_t file_off; uint8_t* dst; uint64_t len; int layer; };
+    constexpr uint64_t kPiece = 2u << 20;
+    constexpr int kReaders = 4;
+    std::vector<Piece> pieces;
+    std::vector<int> left(n, 0);                              // pieces of layer i still to arrive
+    uint64_t bytes_total = 0;
+    auto add_range = [&](int i, uint64_t foff, uint8_t* dst, uint64_t len) {
+        for (uint64_t o = 0; o < len; o += kPiece) {
+            pieces.push_back(Piece{foff + o, dst + o, std::min(kPiece, len - o), i});
+            ++left[i];
+        }
+        bytes_total += len;
+    };
+    for (int i = 0; i < n; ++i) {
+        const nnv_layer_desc_t& L = p->layers[i];
+        if (L.op != NNV_OP_CONV) continue;
+        const nnv_choice_t ch = choices[i];
+        if (variant_has_transform(ch.variant) && ch.cached)
+            add_range(i, cached_off + coff[i], (uint8_t*)h_stage_cached + coff[i], transformed_bytes(*p, i, ch.variant, ch.math));
+        else
+            add_range(i, raw_off + L.w_off, (uint8_t*)h_stage_weights + L.w_off, raw_weight_bytes(L));
+        if (L.has_bias) add_range(i, raw_off + L.b_off, (uint8_t*)h_stage_weights + L.b_off, 4ull * L.K);
+    }
     std::vector<int> ready(n, 0);
+    for (int i = 0; i < n; ++i) ready[i] = left[i] == 0 ? 1 : 0;
     std::mutex mu;
     std::condition_variable cv;
     std::atomic<bool> stop{false};
+    std::atomic<size_t> next{0};
     nnv_status_t reader_rc = NNV_OK;
     std::string reader_err;
     uint64_t bytes_read = 0, ns_read = 0;
-    std::thread reader([&] {
-        const auto t0 = std::chrono::steady_clock::now();
-        for (int i = 0; i < n && !stop.load(); ++i) {
-            const nnv_layer_desc_t& L = p->layers[i];
-            nnv_status_t rc = NNV_OK;
-            if (L.op == NNV_OP_CONV) {
-                const nnv_choice_t ch = choices[i];
-                if (variant_has_transform(ch.variant) && ch.cached) {
-                    const uint64_t tb = transformed_bytes(*p, i, ch.variant, ch.math);
-                    rc = cache_read_range(cache, cached_off + coff[i], (uint8_t*)h_stage_cached + coff[i], tb);
-                    bytes_read += tb;
-                } else {
-                    rc = cache_read_range(cache, raw_off + L.w_off, (uint8_t*)h_stage_weights + L.w_off, raw_weight_bytes(L));
-                    bytes_read += raw_weight_bytes(L);
-                }
-                if (rc == NNV_OK && L.has_bias) {
-                    rc = cache_read_range(cache, raw_off + L.b_off, (uint8_t*)h_stage_weights + L.b_off, 4ull * L.K);
-                    bytes_read += 4ull * L.K;
-                }
-            }
+    const auto t_read0 = std::chrono::steady_clock::now();
+    auto reader_fn = [&] {
+        for (;;) {
+            const size_t k = next.fetch_add(1);
+            if (k >= pieces.size() || stop.load()) return;
+            const Piece& pc = pieces[k];
+            const nnv_status_t rc = cache_read_range(cache, pc.file_off, pc.dst, pc.len);
             std::lock_guard<std::mutex> lk(mu);
             if (rc != NNV_OK) {
-                reader_rc = rc;
-                reader_err = nnv_last_error();
-                ready[i] = -1;
+                if (reader_rc == NNV_OK) { reader_rc = rc; reader_err = nnv_last_error(); }
+                stop = true;
                 cv.notify_all();
                 return;
             }
-            ready[i] = 1;
-            cv.notify_all();
+            bytes_read += pc.len;
+            if (--left[pc.layer] == 0) { ready[pc.layer] = 1; cv.notify_all(); }
+            if (bytes_read == bytes_total)
+                ns_read = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t_read0).count();
         }
-        ns_read = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
-    });
+    };
+    std::vector<std::thread> readers;
+    for (int t = 0; t < kReaders; ++t) readers.emplace_back(reader_fn);
+    struct Joiner {
+        std::vector<std::thread>& ts; std::atomic<bool>& stop;
+        void join() { stop = true; for (std::thread& t : ts) if (t.joinable()) t.join(); }
+    } reader{readers, stop};
     const std::function<nnv_status_t(int)> gate = [&](int i) -> nnv_status_t {
         std::unique_lock<std::mutex> lk(mu);
         cv.wait(lk, [&] { return ready[i] != 0 || reader_rc != NNV_OK; });
         if (reader_rc != NNV_OK) return fail(reader_rc, "%s", reader_err.c_str());
         return NNV_OK;
     };
-    for (int i = 0; i < n; ++i)
-        if (p->layers[i].op == NNV_OP_CONV)
-            NNV_REQUIRE_OR(p->layers[i].w_off + raw_weight_bytes(p->layers[i]) <= w_bytes, { stop = true; reader.join(); },
-                           NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the file's raw blob", i);
     const nnv_status_t rc = run_model(p, choices, h_stage_weights, w_bytes, h_stage_cached, stage_c_bytes, h_input, h_output, d_arena,
                                       arena_bytes, (cudaStream_t)s_copy, (cudaStream_t)s_xform, (cudaStream_t)s_exec, depth, timings,
                                       false, nullptr, nullptr, 0, -1, nullptr, false, &gate);
-    stop = true;
     reader.join();
     if (rc != NNV_OK) {
         cudaStreamSynchronize((cudaStream_t)s_copy);            // nothing of the failed pass may still touch the staging buffers
@@ -728,6 +809,12 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
     }
     if (read_ns) *read_ns = ns_read;
     if (read_bytes) *read_bytes = bytes_read;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_last_enqueue_ns(const nnv_plan_t* p, uint64_t* ns) {
+    NNV_REQUIRE(p && ns, NNV_ERR_INVALID_ARG, "null argument");
+    *ns = p->last_enqueue_ns;
     return NNV_OK;
 }
 

@@ -4,6 +4,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "nnv_internal.h"
@@ -18,6 +19,62 @@ nnv_status_t fail(nnv_status_t code, const char* fmt, ...) {
     vsnprintf(g_err, sizeof(g_err), fmt, ap);
     va_end(ap);
     return code;
+}
+
+static std::mutex g_tuning_mu;
+static Tuning g_tuning;
+
+Tuning tuning() {
+    std::lock_guard<std::mutex> lk(g_tuning_mu);
+    return g_tuning;
+}
+
+// "key=value;key=value" -> *t.  Returns the offending item on a parse / range error, else nullptr.
+static const char* parse_tuning(const char* spec, Tuning* t, char* item, size_t item_cap) {
+    const char* s = spec;
+    while (*s) {
+        const char* e = std::strchr(s, ';');
+        const size_t len = e ? (size_t)(e - s) : std::strlen(s);
+        if (len >= item_cap) return "item too long";
+        std::memcpy(item, s, len);
+        item[len] = 0;
+        s += len + (e ? 1 : 0);
+        if (len == 0) continue;
+        char* eq = std::strchr(item, '=');
+        if (!eq) return item;
+        *eq = 0;
+        const char* key = item;
+        const char* val = eq + 1;
+        int a = 0, b = 0, c = 0, d = 0, f = 0;
+        auto flag = [&](int* dst) { return std::sscanf(val, "%d", &a) == 1 && (a == 0 || a == 1) ? (*dst = a, true) : false; };
+        bool ok = false;
+        if (!std::strcmp(key, "gemm_tile")) {
+            ok = std::sscanf(val, "%d,%d", &a, &b) == 2 && a >= 16 && a <= 128 && a % 16 == 0 && b >= 1 && b <= 8 && (b & (b - 1)) == 0;
+            if (ok) { t->gemm_bn = a; t->gemm_splits = b; }
+        } else if (!std::strcmp(key, "gemm_ring")) {
+            ok = std::sscanf(val, "%d", &a) == 1 && a >= 2 && a <= 8;
+            if (ok) t->gemm_ring = a;
+        } else if (!std::strcmp(key, "gemm_prefill")) {
+            ok = flag(&t->gemm_prefill);
+        } else if (!std::strcmp(key, "conv3x3")) {
+            if (!std::strcmp(val, "off")) { t->conv3x3 = 1; ok = true; }
+            else if (!std::strcmp(val, "auto")) { t->conv3x3 = 0; ok = true; }
+            else {
+                const int got = std::sscanf(val, "%d,%d,%d,%d,%d", &a, &b, &c, &d, &f);
+                ok = got >= 3 && (a == 1 || a == 2) && b >= 16 && b <= 128 && b % 16 == 0 && c >= 1 && c <= 8 && (c & (c - 1)) == 0 &&
+                     (got < 4 || (d >= 0 && d <= 4)) && (got < 5 || (f >= 0 && f <= 8));
+                if (ok) { t->conv3x3 = 2; t->conv_mt = a; t->conv_bn = b; t->conv_splits = c; t->conv_na = got >= 4 ? d : 0; t->conv_nb = got >= 5 ? f : 0; }
+            }
+        } else if (!std::strcmp(key, "side")) {
+            ok = flag(&t->side);
+        } else if (!std::strcmp(key, "merge")) {
+            ok = flag(&t->merge);
+        } else if (!std::strcmp(key, "group")) {
+            ok = flag(&t->group);
+        }
+        if (!ok) { *eq = '='; return item; }
+    }
+    return nullptr;
 }
 
 bool variant_has_transform(int v) { return v != NNV_VAR_DIRECT && v != NNV_VAR_DEPTHWISE; }
@@ -241,6 +298,19 @@ extern "C" {
 const char* nnv_last_error(void) { return g_err; }
 int32_t nnv_version(void) { return 100; }
 
+nnv_status_t nnv_tuning_set(const char* spec) {
+    Tuning t;                                                   // every call starts from the defaults
+    char item[128];
+    if (spec && *spec) {
+        const char* bad = parse_tuning(spec, &t, item, sizeof(item));
+        NNV_REQUIRE(!bad, NNV_ERR_INVALID_ARG, "tuning item not understood or out of range: %s", bad);
+    }
+    std::lock_guard<std::mutex> lk(g_tuning_mu);
+    t.generation = g_tuning.generation + 1;
+    g_tuning = t;
+    return NNV_OK;
+}
+
 nnv_status_t nnv_plan_create(const nnv_layer_desc_t* layers, int32_t n, const nnv_plan_opts_t* opts,
                              nnv_plan_t** out) {
     NNV_REQUIRE(layers && out, NNV_ERR_INVALID_ARG, "null argument");
@@ -309,6 +379,9 @@ nnv_status_t nnv_plan_create(const nnv_layer_desc_t* layers, int32_t n, const nn
 
 nnv_status_t nnv_plan_destroy(nnv_plan_t* p) {
     if (!p) return NNV_OK;
+    if (p->warm_pending)                                       // reads / transforms of K_warm - K_cold may still be queued
+        for (cudaEvent_t e : p->warm_ev)
+            if (e) cudaEventSynchronize(e);
     for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
     for (cudaEvent_t e : p->tev) cudaEventDestroy(e);
     for (cudaEvent_t e : p->warm_ev)

@@ -40,6 +40,73 @@ static uint64_t makespan(const nnv_plan& p, const uint64_t* pl, const uint64_t* 
     return exec_end[n - 1];
 }
 
+// The same latency on a machine where every queue's weights arrive over ONE host link.  A
+// preparation is two operations on its queue, read then transform; the link carries one read at a
+// time, and when it is free it takes, among the reads whose turn on their own queue has come, the
+// one of the lowest layer (reads are issued in layer order).  Event-driven: operations are started
+// as soon as they can be, time jumps to the next end.
+static uint64_t makespan_link(const nnv_plan& p, const uint64_t* rd, const uint64_t* xl, const uint64_t* xb, const uint64_t* ex,
+                              const int32_t* queue_of, int n_little) {
+    const int n = (int)p.layers.size();
+    enum { READ = 0, XFORM = 1, EXEC = 2 };
+    struct Op { int kind, layer; uint64_t dur; };
+    std::vector<std::vector<Op>> ops(n_little + 1);
+    for (int i = 0; i < n; ++i) {
+        const bool conv = p.layers[i].op == NNV_OP_CONV;
+        if (conv && queue_of[i] == 0) { ops[0].push_back({READ, i, rd[i]}); ops[0].push_back({XFORM, i, xb[i]}); }
+        ops[0].push_back({EXEC, i, ex[i]});
+        if (conv && queue_of[i] > 0) { ops[queue_of[i]].push_back({READ, i, rd[i]}); ops[queue_of[i]].push_back({XFORM, i, xl[i]}); }
+    }
+    constexpr uint64_t NOT_YET = ~0ull;
+    std::vector<uint64_t> end_of[3];
+    for (auto& v : end_of) v.assign(n, NOT_YET);
+    std::vector<size_t> head(n_little + 1, 0);
+    std::vector<uint64_t> busy(n_little + 1, 0);
+    uint64_t link_free = 0, t = 0;
+    auto ended = [&](int kind, int layer) { return end_of[kind][layer] != NOT_YET && end_of[kind][layer] <= t; };
+    while (end_of[EXEC][n - 1] == NOT_YET) {
+        bool progressed = true;
+        while (progressed) {
+            progressed = false;
+            int wq = -1;                                         // queue of the waiting read of the lowest layer
+            for (int q = 0; q <= n_little; ++q) {
+                if (head[q] >= ops[q].size() || busy[q] > t) continue;
+                const Op& o = ops[q][head[q]];
+                if (o.kind == READ) {
+                    if (wq < 0 || o.layer < ops[wq][head[wq]].layer) wq = q;
+                    continue;
+                }
+                bool ok;
+                if (o.kind == XFORM) {
+                    ok = ended(READ, o.layer);
+                } else {
+                    const nnv_layer_desc_t& L = p.layers[o.layer];
+                    ok = (L.op != NNV_OP_CONV || ended(XFORM, o.layer)) && (L.in0 < 0 || ended(EXEC, L.in0)) &&
+                         (L.in1 < 0 || ended(EXEC, L.in1));
+                }
+                if (!ok) continue;
+                end_of[o.kind][o.layer] = busy[q] = t + o.dur;
+                ++head[q];
+                progressed = true;
+            }
+            if (wq >= 0 && link_free <= t) {
+                const Op& o = ops[wq][head[wq]];
+                end_of[READ][o.layer] = busy[wq] = link_free = t + o.dur;
+                ++head[wq];
+                progressed = true;
+            }
+        }
+        if (end_of[EXEC][n - 1] != NOT_YET) break;
+        uint64_t next = NOT_YET;                                 // the earliest end after t
+        for (const auto& v : end_of)
+            for (uint64_t e : v)
+                if (e != NOT_YET && e > t) next = std::min(next, e);
+        if (next == NOT_YET) break;                              // cannot happen for a topologically ordered plan
+        t = next;
+    }
+    return end_of[EXEC][n - 1];
+}
+
 // Algorithm 1's little-core balancing step: round-robin start in layer order, then move operations
 // from the longest to the shortest little queue while one shorter than half the gap exists.
 struct Item { int layer; uint64_t t; };
@@ -119,9 +186,11 @@ static uint64_t schedule_queues(const nnv_plan& p, const uint64_t* pl, const uin
 // Outer loop of Algorithm 1 over the filtered candidates: exhaustive up to `limit` combinations,
 // else coordinate descent from the per-layer cold-cost minimum (first strict improvement in rank
 // order per layer, at most 8 sweeps).  Ties keep the earlier combination.
+// With `reads` (per layer and option, the part of the preparation that crosses the host link) the latency
+// compared and returned is makespan_link's; the queues still come from the heuristic on the bundled times.
 static uint64_t search(const nnv_plan& p, const std::vector<std::vector<Option>>& options, const uint64_t* pool_ns,
                        int n_little, uint64_t eps, int big_pct, uint64_t limit, std::vector<int>* pick_out,
-                       std::vector<int32_t>* queue_out) {
+                       std::vector<int32_t>* queue_out, const std::vector<std::vector<uint64_t>>* reads = nullptr) {
     const int n = (int)p.layers.size();
     std::vector<int> conv;
     for (int i = 0; i < n; ++i)
@@ -136,7 +205,16 @@ static uint64_t search(const nnv_plan& p, const std::vector<std::vector<Option>>
                 pl[i] = pb[i] = 0; ex[i] = pool_ns ? pool_ns[i] : 0;
             }
         }
-        return schedule_queues(p, pl.data(), pb.data(), ex.data(), n_little, eps, q);
+        const uint64_t t = schedule_queues(p, pl.data(), pb.data(), ex.data(), n_little, eps, q);
+        if (!reads) return t;
+        std::vector<uint64_t> rd(n, 0), xl(n, 0), xb(n, 0);
+        for (int i = 0; i < n; ++i)
+            if (p.layers[i].op == NNV_OP_CONV) {
+                rd[i] = (*reads)[i][pick[i]];
+                xl[i] = pl[i] - rd[i];
+                xb[i] = xl[i] * (uint64_t)big_pct / 100;
+            }
+        return makespan_link(p, rd.data(), xl.data(), xb.data(), ex.data(), q->data(), n_little);
     };
     uint64_t total = 1;
     for (int i : conv) {
@@ -217,9 +295,95 @@ nnv_status_t nnv_schedule_queues(const nnv_plan_t* p, const uint64_t* prep_littl
     return NNV_OK;
 }
 
+nnv_status_t nnv_simulate_link(const nnv_plan_t* p, const uint64_t* read_ns, const uint64_t* xform_little_ns,
+                               const uint64_t* xform_big_ns, const uint64_t* exec_ns, const int32_t* queue_of, int32_t n_little,
+                               uint64_t* t_cold_ns) {
+    NNV_REQUIRE(p && read_ns && xform_little_ns && xform_big_ns && exec_ns && queue_of && t_cold_ns, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(n_little >= 1 && n_little <= NNV_MAX_QUEUES, NNV_ERR_INVALID_ARG, "n_little %d outside 1..%d", n_little, NNV_MAX_QUEUES);
+    NNV_TRY(check_queues(*p, queue_of, n_little));
+    *t_cold_ns = makespan_link(*p, read_ns, xform_little_ns, xform_big_ns, exec_ns, queue_of, n_little);
+    return NNV_OK;
+}
+
+static nnv_status_t schedule_impl(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                                  const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
+                                  uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns, bool link);
+
 nnv_status_t nnv_schedule(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
                           const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
                           uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns) {
+    return schedule_impl(p, costs, n_costs, allow_cached, pool_ns, n_little, eps_ns, big_pct, combo_limit, out, queue_of, t_cold_ns, false);
+}
+
+nnv_status_t nnv_schedule_link(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                               const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
+                               uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns) {
+    return schedule_impl(p, costs, n_costs, allow_cached, pool_ns, n_little, eps_ns, big_pct, combo_limit, out, queue_of, t_cold_ns, true);
+}
+
+nnv_status_t nnv_schedule_eps(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                              int32_t eps_pct, uint64_t* eps_ns) {
+    NNV_REQUIRE(p && costs && eps_ns, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(eps_pct >= 0 && eps_pct <= 100, NNV_ERR_INVALID_ARG, "eps_pct %d outside 0..100", eps_pct);
+    const int n = (int)p->layers.size();
+    std::vector<nnv_choice_t> ch(n);
+    NNV_TRY(nnv_select_kernels(p, costs, n_costs, allow_cached, ch.data()));
+    uint64_t sum = 0;
+    for (int i = 0; i < n; ++i) {
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        for (int r = 0; r < n_costs; ++r)
+            if (costs[r].layer == i && costs[r].variant == ch[i].variant && costs[r].math == ch[i].math) { sum += costs[r].exec_ns; break; }
+    }
+    *eps_ns = sum * (uint64_t)eps_pct / 100;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_calibrate_costs(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, const nnv_choice_t* choices,
+                                 const nnv_timing_t* timings, nnv_cost_t* out, uint64_t* factors) {
+    NNV_REQUIRE(p && costs && choices && timings && out, NNV_ERR_INVALID_ARG, "null argument");
+    const int n = (int)p->layers.size();
+    uint64_t num[3] = {0, 0, 0}, den[3] = {0, 0, 0};             // read, transform, execution
+    for (int i = 0; i < n; ++i) {
+        if (p->layers[i].op != NNV_OP_CONV) continue;
+        NNV_TRY(check_choice(*p, i, choices[i].variant, choices[i].math));
+        const nnv_cost_t* row = nullptr;
+        for (int r = 0; r < n_costs && !row; ++r)
+            if (costs[r].layer == i && costs[r].variant == choices[i].variant && costs[r].math == choices[i].math) row = &costs[r];
+        NNV_REQUIRE(row, NNV_ERR_STATE, "no cost row for the kernel chosen for layer %d", i);
+        const nnv_timing_t& t = timings[i];
+        NNV_REQUIRE(t.h2d_end_ns >= t.h2d_start_ns && t.xform_end_ns >= t.xform_start_ns && t.exec_end_ns >= t.exec_start_ns,
+                    NNV_ERR_INVALID_ARG, "layer %d: a timing interval ends before it starts", i);
+        const bool has_xf = variant_has_transform(choices[i].variant);
+        const bool cached = has_xf && choices[i].cached;
+        num[0] += t.h2d_end_ns - t.h2d_start_ns;
+        den[0] += cached ? row->h2d_cached_ns : row->h2d_raw_ns;
+        if (has_xf && !cached) {
+            num[1] += t.xform_end_ns - t.xform_start_ns;
+            den[1] += row->xform_ns;
+        }
+        num[2] += t.exec_end_ns - t.exec_start_ns;
+        den[2] += row->exec_ns;
+    }
+    auto scale = [&](uint64_t v, int k) -> uint64_t {
+        if (num[k] == 0 || den[k] == 0) return v;
+        return (uint64_t)((unsigned __int128)v * num[k] / den[k]);
+    };
+    for (int r = 0; r < n_costs; ++r) {
+        nnv_cost_t c = costs[r];
+        c.h2d_raw_ns = scale(c.h2d_raw_ns, 0);
+        c.h2d_cached_ns = scale(c.h2d_cached_ns, 0);
+        c.xform_ns = scale(c.xform_ns, 1);
+        c.exec_ns = scale(c.exec_ns, 2);
+        out[r] = c;
+    }
+    if (factors)
+        for (int k = 0; k < 3; ++k) { factors[2 * k] = num[k]; factors[2 * k + 1] = den[k]; }
+    return NNV_OK;
+}
+
+static nnv_status_t schedule_impl(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, int32_t allow_cached,
+                                  const uint64_t* pool_ns, int32_t n_little, uint64_t eps_ns, int32_t big_pct,
+                                  uint64_t combo_limit, nnv_choice_t* out, int32_t* queue_of, uint64_t* t_cold_ns, bool link) {
     NNV_REQUIRE(p && costs && out && queue_of && t_cold_ns, NNV_ERR_INVALID_ARG, "null argument");
     NNV_REQUIRE(n_little >= 1 && n_little <= NNV_MAX_QUEUES, NNV_ERR_INVALID_ARG, "n_little %d outside 1..%d", n_little, NNV_MAX_QUEUES);
     NNV_REQUIRE(big_pct >= 0 && big_pct <= 1000, NNV_ERR_INVALID_ARG, "big_pct %d outside 0..1000", big_pct);
@@ -232,9 +396,22 @@ nnv_status_t nnv_schedule(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t 
         NNV_REQUIRE(!all.empty(), NNV_ERR_STATE, "no cost rows for conv layer %d", i);
         pareto(all, &options[i]);
     }
+    std::vector<std::vector<uint64_t>> reads(n);                 // per option, the part of prep that is the read
+    if (link) {
+        for (int i = 0; i < n; ++i)
+            for (const Option& o : options[i]) {
+                uint64_t rd = 0;
+                for (int r = 0; r < n_costs; ++r)
+                    if (costs[r].layer == i && costs[r].variant == o.variant && costs[r].math == o.math) {
+                        rd = o.cached ? costs[r].h2d_cached_ns : costs[r].h2d_raw_ns;
+                        break;
+                    }
+                reads[i].push_back(rd);
+            }
+    }
     std::vector<int> pick;
     std::vector<int32_t> q;
-    *t_cold_ns = search(*p, options, pool_ns, n_little, eps_ns, big_pct, combo_limit, &pick, &q);
+    *t_cold_ns = search(*p, options, pool_ns, n_little, eps_ns, big_pct, combo_limit, &pick, &q, link ? &reads : nullptr);
     for (int i = 0; i < n; ++i) {
         queue_of[i] = q[i];
         if (p->layers[i].op == NNV_OP_CONV) {

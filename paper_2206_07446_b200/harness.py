@@ -47,6 +47,11 @@ class Model:
         self.h_cached = None
         self.c_bytes = 0
 
+    def second_plan(self, use_graphs):
+        """Another plan over the same layers and weight blob (e.g. one that replays recorded graphs beside an eager one)."""
+        return nb.Plan(self.layers, self.w_off, self.b_off, opts=dict(default_math=nb.MATH_TF32, allow_cached=1, max_depth=4,
+                                                                      debug_checks=0, use_graphs=use_graphs))
+
     def out_hw(self, i):
         L = self.layers[i]
         if L["op"] == nb.OP_GAVGPOOL:
@@ -131,21 +136,18 @@ class Model:
                                     self.prep_streams(n_little), want_timings)
         return self.h_output.numpy().copy(), tm
 
-    def schedule(self, x_nchw, costs, n_little, allow_cached=1, rounds=2, eps_pct=1, big_pct=100, combo_limit=4096):
-        """Algorithm 1 with its calibration step: schedule from the cost table, run the schedule once with
-        per-operation timings, and rescale the table by how much slower each kind of operation (read,
-        transform, execution) ran while the other queues were busy than it did alone -- the queues share
-        one host link and one GPU, so co-running operations slow each other down; then schedule again
-        (`rounds` times).  Every option of a kind gets the same factor, so that options that were not
-        run are not favoured over the calibrated ones.  eps is eps_pct percent of the summed execution
-        time of the per-layer choice.  Returns (choices, queue_of, predicted ns, calibrated costs)."""
-        table = [dict(c) for c in costs]
-        base = nb.nnv_select_kernels(self.plan, table, allow_cached)
-        iso = {(c["layer"], c["variant"], c["math"]): c for c in costs}
-        eps = sum(iso[(i,) + ch[:2]]["exec_ns"] for i, ch in enumerate(base) if ch is not None) * eps_pct // 100
+    def schedule(self, x_nchw, costs, n_little, allow_cached=1, rounds=2, eps_pct=1, big_pct=100, combo_limit=4096, link=True):
+        """Algorithm 1 with its profiling step repeated under load: schedule from the cost table, run the
+        schedule once with per-operation timings, let the library rescale the table by how much slower each kind
+        of operation ran beside the others than alone (nnv_calibrate_costs), schedule again; `rounds` times.
+        This method only sequences library calls.  link=True evaluates schedules with the shared-link latency
+        (nnv_schedule_link).  Returns (choices, queue_of, predicted ns, calibrated costs)."""
+        table = costs
+        eps = nb.nnv_schedule_eps(self.plan, costs, allow_cached, eps_pct)
         out = None
+        self.calibration = None
         for r in range(rounds + 1):
-            out = nb.nnv_schedule(self.plan, table, allow_cached, n_little, eps, big_pct, combo_limit)
+            out = nb.nnv_schedule(self.plan, table, allow_cached, n_little, eps, big_pct, combo_limit, link=link)
             if r == rounds:
                 break
             choices, queue_of, _ = out
@@ -153,23 +155,9 @@ class Model:
                 self.build_cached_blob(choices)
             self.cold_run_queues(x_nchw, choices, queue_of, n_little, poison=False)          # warm
             _, tm = self.cold_run_queues(x_nchw, choices, queue_of, n_little, want_timings=True, poison=False)
-            got = dict(h2d=0, xform=0, exec=0)
-            alone = dict(h2d=0, xform=0, exec=0)
-            for i, ch in enumerate(choices):
-                if ch is None:
-                    continue
-                row, t = iso[(i,) + ch[:2]], tm[i]
-                got["exec"] += t["exec_end_ns"] - t["exec_start_ns"]
-                alone["exec"] += row["exec_ns"]
-                got["h2d"] += t["h2d_end_ns"] - t["h2d_start_ns"]
-                alone["h2d"] += row["h2d_cached_ns"] if ch[2] else row["h2d_raw_ns"]
-                if not ch[2]:
-                    got["xform"] += t["xform_end_ns"] - t["xform_start_ns"]
-                    alone["xform"] += row["xform_ns"]
-            f = {k: (got[k] / alone[k] if alone[k] else 1.0) for k in got}
-            self.calibration = f
-            table = [dict(c, h2d_raw_ns=int(c["h2d_raw_ns"] * f["h2d"]), h2d_cached_ns=int(c["h2d_cached_ns"] * f["h2d"]),
-                          xform_ns=int(c["xform_ns"] * f["xform"]), exec_ns=int(c["exec_ns"] * f["exec"])) for c in costs]
+            rows, fac = nb.nnv_calibrate_costs(self.plan, costs, choices, tm)
+            self.calibration = {k: (f[0] / f[1] if f[1] else None) for k, f in zip(("h2d", "xform", "exec"), fac)}
+            table = nb.CostTable(rows)
         return out[0], out[1], out[2], table
 
     def cold_run_continuous(self, x_nchw, cold, warm, want_timings=False):

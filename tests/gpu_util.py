@@ -35,6 +35,29 @@ def rel_l2(got, ref):
     return float(np.sqrt(np.sum((got - ref) ** 2)) / (den if den > 0 else 1.0))
 
 
+def max_abs_rel(got, ref):
+    """Largest element-wise error relative to the largest reference magnitude."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    den = float(np.max(np.abs(ref))) if ref.size else 0.0
+    return float(np.max(np.abs(got - ref))) / (den if den > 0 else 1.0) if ref.size else 0.0
+
+
+ELEMENTWISE_FACTOR = 8.0     # max |y - ref| <= 8 * tol * max |ref|: a norm alone would let single wrong outputs of a large layer through
+
+
+def assert_conv_close(got, ref, tol, what=None):
+    """The tolerance of a conv output: relative L2 error <= tol, and no single element off by more than
+    ELEMENTWISE_FACTOR * tol of the largest reference magnitude."""
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    assert np.all(np.isfinite(got)), what
+    err = rel_l2(got, ref)
+    assert err <= tol, (what, "rel L2", err)
+    worst = max_abs_rel(got, ref)
+    assert worst <= ELEMENTWISE_FACTOR * tol, (what, "element-wise", worst)
+    return err
+
+
 def run_conv(plan, i, L, variant, math, x_chw, w, bias=None, addend_chw=None):
     """Transform (if the variant has one) and execute layer i through the C ABI; returns CHW numpy."""
     d_raw = dev(w.astype(np.float32))

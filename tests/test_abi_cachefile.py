@@ -93,3 +93,24 @@ def test_damaged_files_are_refused(tmp_path):
     assert e.value.status == 3                                    # NNV_ERR_STATE
     with pytest.raises(nb.NnvError):                              # a choice the layer cannot run
         nb.nnv_cache_write(str(tmp_path / "bad.nnv"), plan, [(nb.VAR_DEPTHWISE, 0, 0)], None, 0, blob, blob.size, None, 0)
+
+
+def test_cold_run_refuses_a_file_written_for_another_model(tmp_path):
+    """Same layer count, fitting offsets, different shapes: nnv_cold_run_file must refuse before any device work
+    (the pointers below are never dereferenced: the comparison of the descriptors comes first)."""
+    layers = wl.tiny_net()
+    plan, descs, blob = _setup(layers, seed=1)
+    choices = _choices(plan, layers, 0)
+    path = str(tmp_path / "a.nnv")
+    nb.nnv_cache_write(path, plan, choices, None, 0, blob, blob.size, None, 0)
+    other = [dict(L) for L in layers]
+    conv = next(i for i, L in enumerate(other) if L["op"] == wl.OP_CONV)
+    other[conv]["act"] = (other[conv]["act"] + 1) % 3          # the same byte layout, another network
+    plan2, _, _ = _setup(other, seed=1)
+    cache = nb.CacheFile(path)
+    stage = np.zeros(blob.size, np.uint8)
+    io = np.zeros(1 << 16, np.float32)
+    with pytest.raises(nb.NnvError) as e:
+        nb.nnv_cold_run_file(plan2, choices, cache, stage, stage.size, None, 0, io, io, 256, 1 << 30, 1, 2, 3, 1)
+    assert e.value.status == 1 and "differs from the plan" in str(e.value)
+    cache.close()

@@ -202,3 +202,18 @@ def test_arena_and_workspace_sizes_are_consistent():
     offs, total = nb.nnv_cached_layout(plan, [None if c is None else (c[0], c[1], 1) for c in ch])
     assert total >= sum(nb.nnv_transformed_bytes(plan, i, c[0], c[1]) for i, c in enumerate(ch) if c)
     assert all(o % 256 == 0 for o in offs)
+
+
+def test_tuning_overrides_parse_and_reject():
+    """nnv_tuning_set: documented items are accepted, anything else is refused and changes nothing."""
+    try:
+        for ok in ("gemm_tile=64,4", "gemm_ring=6;gemm_prefill=0", "conv3x3=off", "conv3x3=auto", "conv3x3=2,64,4",
+                   "conv3x3=1,128,2,1,3", "side=0;merge=0;group=0", "", None, "gemm_tile=16,1;;side=1"):
+            nb.nnv_tuning_set(ok)
+        for bad in ("gemm_tile=48", "gemm_tile=24,2", "gemm_tile=64,3", "gemm_ring=9", "conv3x3=3,64,1", "conv3x3=1,64,16",
+                    "side=2", "unknown=1", "gemm_tile", "x" * 300):
+            with pytest.raises(nb.NnvError) as e:
+                nb.nnv_tuning_set(bad)
+            assert e.value.status == 1, bad
+    finally:
+        nb.nnv_tuning_set(None)

@@ -204,11 +204,11 @@ def test_residual_branch_layers_on_the_side_stream():
             if M["in1"] == i:
                 assert tm[j]["exec_start_ns"] >= tm[i]["exec_end_ns"], (i, j)
         assert tm[i]["exec_start_ns"] >= tm[layers[i]["in0"]]["exec_end_ns"]
-    os.environ["NNV_DEBUG_NO_SIDE"] = "1"
+    nb.nnv_tuning_set("side=0")
     try:
         y_main, _ = model.cold_run(x, ch, depth=0, want_timings=True)
     finally:
-        del os.environ["NNV_DEBUG_NO_SIDE"]
+        nb.nnv_tuning_set(None)
     assert np.array_equal(y_side, y_main)
     y_graph, _ = model.cold_run(x, ch, depth=0)
     assert np.array_equal(y_graph, y_side)
@@ -230,10 +230,10 @@ def test_merged_copies_at_depth_zero():
         L = layers[i]
         assert tm[i]["h2d_bytes"] == 4 * L["K"] * L["C"] * L["R"] * L["S"]
         assert tm[i]["exec_start_ns"] >= tm[i]["h2d_end_ns"]
-    os.environ["NNV_DEBUG_NO_MERGE"] = "1"
+    nb.nnv_tuning_set("merge=0")
     try:
         y_single, tm1 = model.cold_run(x, ch, depth=0, want_timings=True)
     finally:
-        del os.environ["NNV_DEBUG_NO_MERGE"]
+        nb.nnv_tuning_set(None)
     assert len({(tm1[i]["h2d_start_ns"], tm1[i]["h2d_end_ns"]) for i in convs}) == len(convs)
     assert np.array_equal(y_merged, y_single)

@@ -1,8 +1,6 @@
 """GPU parity of the halo-resident 3x3 tensor-core kernel: every tiling it can take (one or two MMA
 tiles per CTA, several channel-tile widths, K splits over a thread-block cluster) against the fp64
 direct-convolution oracle, and against the plain implicit GEMM that it replaces."""
-import os
-
 import numpy as np
 import pytest
 
@@ -12,23 +10,14 @@ from gpu_util import TOL, rel_l2, run_conv
 
 pytestmark = pytest.mark.gpu
 
-ENV = "NNV_DEBUG_CONV3X3"          # debug override read by the library at every launch
-
-
 def _run(L, x, w, b, add, setting):
-    old = os.environ.get(ENV)
-    if setting is None:
-        os.environ.pop(ENV, None)
-    else:
-        os.environ[ENV] = setting
+    """One layer with the 3x3 kernel's tiling forced through nnv_tuning_set (None = the library's own pick)."""
+    nb.nnv_tuning_set(None if setting is None else "conv3x3=" + setting)
     try:
         plan = nb.Plan([L], [0], [0])
         return run_conv(plan, 0, L, nb.VAR_IM2COL, nb.MATH_TF32, x, w, b, add)
     finally:
-        if old is None:
-            os.environ.pop(ENV, None)
-        else:
-            os.environ[ENV] = old
+        nb.nnv_tuning_set(None)
 
 
 @pytest.mark.parametrize("shape", [
