@@ -319,7 +319,7 @@ def run_ours(args):
     ws, bs = wl.make_weights(layers)
     x = wl.make_input(layers)
     # the headline is eager; a second plan over the same blob replays recorded graphs for the side arms
-    model = harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=0)
+    model = harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=0, kernel_stamps=1)
     plan_g = model.second_plan(use_graphs=1)
     math = nb.MATH_BF16 if args.math == "bf16" else nb.MATH_TF32
 
@@ -386,11 +386,11 @@ def run_ours(args):
     def step_value(k, timed):
         begin(k, timed, (s_copy, s_xform))
         ch = nb.nnv_select_kernels(model.plan, costs, 0)      # the selection call belongs to the cold inference
-        tm = nb.nnv_cold_run_dio(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
-                                 model.arena, need, s_copy, s_xform, s_exec, args.cold_depth, timed)
+        nb.nnv_cold_run_dio(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
+                            model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
         if timed:
             ev1[k].record(s_exec)
-        return tm
+            return nb.nnv_kernel_times(model.plan)            # the kernels' own device-clock stamps of this step
 
     sampler.start()
     torch.cuda.cudart().cudaProfilerStart()                  # a profiler attached with "profile from start off" sees the timed steps only
@@ -473,7 +473,12 @@ def run_ours(args):
                 ev1[k].record(s_exec)
 
         ms, _ = timed_region(step_sched, args.arm_steps, 3)
+        iso = {(c["layer"], c["variant"], c["math"]): c for c in costs}
+        chosen = [iso[(i,) + c[:2]] for i, c in enumerate(ch_s) if c is not None]
         alg1 = {"n_little": args.queues, "e2e_ms": ms, "predicted_ms": t_pred / 1e6,
+                "model": "shared host link (nnv_schedule_link); reads keep their isolated costs, transform and execution are rescaled by the calibration run",
+                "isolated_sums_ms": {"read": sum(c["h2d_raw_ns"] for c in chosen) / 1e6, "transform": sum(c["xform_ns"] for c in chosen) / 1e6,
+                                     "exec": sum(c["exec_ns"] for c in chosen) / 1e6},
                 "calibration_factors": getattr(model, "calibration", None),
                 "preps_on_queue0": sum(1 for q in q_s if q == 0),
                 "choices_differing_from_per_layer_argmin": sum(1 for a, b in zip(ch_s, choices_raw) if a != b),
@@ -591,66 +596,76 @@ def run_ours(args):
     clocks = sampler.stop()
     peaks = load_peaks()
 
-    # ---- rooflines from the per-layer events of the TIMED headline steps ----------------------------------
+    # ---- rooflines: kernel durations are the kernels' own device-clock stamps (first block in, last block
+    # out) taken INSIDE the timed headline steps; event pairs around 5 us kernels add microseconds of their own
+    # and serialise the streams (the same step with per-layer events takes 1.8x as long)
     xf, ex = {}, {}                                              # layer -> [ns] over the timed steps
-    for tm in step_timings:
-        for i, t in enumerate(tm):
-            if t["xform_bytes"]:
-                xf.setdefault(i, []).append(t["xform_end_ns"] - t["xform_start_ns"])
-            if layers[i]["op"] == wl.OP_CONV:
-                ex.setdefault(i, []).append(t["exec_end_ns"] - t["exec_start_ns"])
-    last_tm = step_timings[-1]
+    for xs, es in step_timings:
+        for i in range(len(layers)):
+            if xs[i]:
+                xf.setdefault(i, []).append(xs[i])
+            if es[i]:
+                ex.setdefault(i, []).append(es[i])
     avg = statistics.mean
+
+    def layer_flops(i):
+        L = layers[i]
+        oh, ow = wl.out_hw(L)
+        return 2 * oh * ow * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"]
+
     tf32_peak = peaks["bf16_tflops"] * 0.5
     tens_peak = peaks["bf16_tflops"] if math == nb.MATH_BF16 else tf32_peak
-    # the tensor-core GEMM launches that are a layer's whole execution (implicit-GEMM, 3x3 halo kernel, direct-operand 1x1)
+    # the tensor-core GEMM launches that are a layer's whole convolution (implicit GEMM, 3x3 halo kernel, direct-operand 1x1)
     single = [i for i in ex if choices_raw[i][0] in (nb.VAR_IM2COL, nb.VAR_GEMM1X1)
               and nb.nnv_exec_workspace_bytes(model.plan, i, choices_raw[i][0], choices_raw[i][1]) == 0]
     roof = None
     if single:
-        gfl = sum(last_tm[i]["exec_flops"] for i in single)
+        gfl = sum(layer_flops(i) for i in single)
         gby = sum(gemm_bytes(layers[i]) for i in single)
         gns = sum(avg(ex[i]) for i in single)
-        big = max(single, key=lambda i: last_tm[i]["exec_flops"])
+        big = max(single, key=layer_flops)
         t_tensor = gfl / (tens_peak * 1e3)                       # ns at the tensor peak
         t_hbm = gby / peaks["hbm_gbs"]                            # ns at the HBM peak (the weights arrive cold)
         tens = {"bound": "tensor", "achieved": gfl / gns / 1e3, "peak": tens_peak, "unit": "TFLOP/s", "frac": gfl / gns / 1e3 / tens_peak}
         hbm = {"bound": "hbm", "achieved": gby / gns, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gby / gns / peaks["hbm_gbs"]}
         roof = dict(hbm if t_hbm >= t_tensor else tens)           # the binding roofline of these launches
-        roof.update({"kernel": "gemm_tc_kernel / conv3x3_tc_kernel (tcgen05 GEMM; every launch that is a layer's whole execution)",
+        roof.update({"kernel": "gemm_tc_kernel / conv3x3_tc_kernel (tcgen05 GEMM; every launch that is a layer's whole convolution)",
                      "traffic": NCU_GEMM_TRAFFIC_BYTES.get((args.config, args.math)),
-                     "durations": "CUDA events around each layer on the execution stream, inside the timed headline steps",
+                     "durations": "device-clock stamps written by the kernels themselves inside the timed steps (CUDA events time the step)",
                      "peak_source": peaks["source"] + (" HBM copy" if t_hbm >= t_tensor else " bf16 burst" + ("" if math == nb.MATH_BF16 else " x 0.5 (tf32:bf16 nominal ratio)")),
                      "other_roofline": tens if t_hbm >= t_tensor else hbm,
                      "launches_per_step": len(single), "flops_per_step": gfl, "bytes_per_step": gby,
                      "sum_us_per_step": gns / 1e3, "avg_launch_us": gns / len(single) / 1e3,
-                     "largest_launch": {"layer": big, "flops": last_tm[big]["exec_flops"], "bytes": gemm_bytes(layers[big]),
-                                        "us": avg(ex[big]) / 1e3, "tflops": last_tm[big]["exec_flops"] / avg(ex[big]) / 1e3}})
-    # the weight-transform kernels: filter transform and repack, HBM-bound
+                     "largest_launch": {"layer": big, "flops": layer_flops(big), "bytes": gemm_bytes(layers[big]),
+                                        "us": avg(ex[big]) / 1e3, "tflops": layer_flops(big) / avg(ex[big]) / 1e3}})
+    # the weight-transform kernels: filter transform and repack, HBM-bound; a grouped launch is booked on its first layer
     xroof = None
     if xf:
-        launches = {}                                             # layers transformed by one launch share its interval
-        for i in xf:
-            key = (last_tm[i]["xform_start_ns"], last_tm[i]["xform_end_ns"])
-            ent = launches.setdefault(key, {"bytes": 0, "ns": avg(xf[i]), "layers": 0})
-            ent["bytes"] += last_tm[i]["xform_bytes"]
-            ent["layers"] += 1
-        tb = sum(e["bytes"] for e in launches.values())
-        tns = sum(e["ns"] for e in launches.values())
-        bigx = max(launches.values(), key=lambda e: e["bytes"])
-        xroof = {"kernel": "filter_transform / pack kernels of the timed headline steps", "bound": "hbm", "achieved": tb / tns,
-                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": tb / tns / peaks["hbm_gbs"], "traffic": None,
-                 "peak_source": peaks["source"], "launches_per_step": len(launches), "bytes_per_step": tb,
-                 "sum_us_per_step": tns / 1e3, "avg_launch_us": tns / len(launches) / 1e3,
-                 "largest_launch": {"layers": bigx["layers"], "bytes": bigx["bytes"], "us": bigx["ns"] / 1e3,
-                                    "gbs": bigx["bytes"] / bigx["ns"]}}
+        xbytes = sum(raw_bytes(layers[i]) + nb.nnv_transformed_bytes(model.plan, i, c[0], c[1]) for i, c in enumerate(choices_raw)
+                     if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
+        tns = sum(avg(v) for v in xf.values())
+        xroof = {"kernel": "multi_transform_kernel (filter transform + repack), the grouped launches of the timed headline steps",
+                 "bound": "hbm", "achieved": xbytes / tns, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": xbytes / tns / peaks["hbm_gbs"],
+                 "traffic": None, "peak_source": peaks["source"], "launches_per_step": len(xf), "bytes_per_step": xbytes,
+                 "sum_us_per_step": tns / 1e3, "avg_launch_us": tns / len(xf) / 1e3,
+                 "durations": "device-clock stamps written by the kernels themselves inside the timed steps"}
+    # per layer: the tensor-core kernel's duration inside the timed steps against the layer's own roofline
+    per_layer = []
+    for i in sorted(ex):
+        L = layers[i]
+        c = choices_raw[i]
+        fl, by, us = layer_flops(i), gemm_bytes(L), avg(ex[i]) / 1e3
+        t_min_us = max(fl / (tens_peak * 1e6), by / (peaks["hbm_gbs"] * 1e3))
+        per_layer.append({"layer": i, "shape": "%dx%d C=%d K=%d R=%d s=%d" % (L["H"], L["W"], L["C"], L["K"], L["R"], L["stride"]),
+                          "kernel": nb.VARIANT_NAMES[c[0]], "whole_conv": i in single, "us": round(us, 2),
+                          "roofline_us": round(t_min_us, 2), "bound": "tensor" if fl / (tens_peak * 1e6) >= by / (peaks["hbm_gbs"] * 1e3) else "hbm",
+                          "frac": round(t_min_us / us, 4)})
     # kernels that are not tensor-core GEMMs, each on the workload's layers that can run it (isolated launches, L2 flushed)
     krows = None if args.minimal else other_kernel_rooflines(layers, model, nb, torch, flush, peaks)
 
-    flops = sum(last_tm[i]["exec_flops"] for i in ex)
+    flops = sum(layer_flops(i) for i in ex)
     exec_ns = sum(avg(v) for v in ex.values())
     xform_ns = sum(avg(v) for v in xf.values())
-    h2d_ns = sum(last_tm[i]["h2d_end_ns"] - last_tm[i]["h2d_start_ns"] for i in ex)
     n_xf = sum(1 for c in choices_raw if c is not None and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
     per_step_launches = count_launches(layers, choices_raw, model.plan, nb)
 
@@ -677,12 +692,13 @@ def run_ours(args):
         "roofline_transform": xroof,
         "transform_all": xall,
         "kernel_rooflines": krows,
+        "per_layer": per_layer,
         "arms": arms,
         "algorithm1": alg1,
         "continuous": cont,
         "storage": storage,
-        "breakdown": {"sum_h2d_us": h2d_ns / 1e3, "sum_xform_us": xform_ns / 1e3, "sum_exec_us": exec_ns / 1e3,
-                      "exec_tflops": flops / exec_ns / 1e3 if exec_ns else None,
+        "breakdown": {"sum_xform_kernel_us": xform_ns / 1e3, "sum_tensor_core_kernel_us": exec_ns / 1e3,
+                      "tensor_core_tflops": flops / exec_ns / 1e3 if exec_ns else None,
                       "choices": names(choices_raw, nb), "choices_bypass_arm": names(choices_byp, nb),
                       "choices_resident_arm": names(choices_res, nb)},
     }
@@ -778,8 +794,28 @@ def time_conv(torch, nb, variant, math, C, K, R, stride, H, W, groups=1, reps=20
     med, best = _time(torch, lambda st: nb.nnv_conv_exec(plan, 0, variant, math, d_in, None, d_wt, None, d_out, d_ws, wsb, st),
                       reps, flush)
     flops = 2.0 * oh * ow * K * cg * R * R
-    return dict(op="conv", variant=nb.VARIANT_NAMES[variant], math=nb.MATH_NAMES[math], C=C, K=K, R=R, stride=stride,
-                H=H, W=W, groups=groups, direct_flops=flops, us=med, us_min=best, direct_tflops=flops / med / 1e6)
+    out = dict(op="conv", variant=nb.VARIANT_NAMES[variant], math=nb.MATH_NAMES[math], C=C, K=K, R=R, stride=stride,
+               H=H, W=W, groups=groups, direct_flops=flops, us=med, us_min=best, direct_tflops=flops / med / 1e6)
+    if variant not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE):
+        # the tensor-core kernel's own duration (device-clock stamps, no launch or event overhead): the layer as a
+        # one-layer model through nnv_resident_run with its transformed weights passed as the cached blob
+        from paper_2206_07446_b200 import harness
+        w = np.zeros((K, cg, R, R), np.float32)
+        m1 = harness.model_from_workload([L], [w], [None], wl.weight_blob, use_graphs=0, kernel_stamps=1)
+        ch = [(variant, math, 1)]
+        need = m1.ensure_arena(ch, 1)
+        d_w = _buf(torch, m1.w_bytes)
+        d_io_in, d_io_out = _rand(torch, C * H * W), _buf(torch, 4 * oh * ow * K)
+        ks = []
+        for r in range(reps + 2):
+            if flush is not None:
+                flush.fill_(r & 0xFF)
+            nb.nnv_resident_run(m1.plan, ch, d_w, m1.w_bytes, d_wt, d_wt.numel(), d_io_in, d_io_out, m1.arena, need,
+                                m1.streams[1], m1.streams[2], 1)
+            ks.append(nb.nnv_kernel_times(m1.plan)[1][0] / 1e3)
+        out["kernel_us"] = statistics.median(ks[2:])
+        out["kernel_tflops"] = flops / out["kernel_us"] / 1e6 if out["kernel_us"] else None
+    return out
 
 
 def _offsets(layers):

@@ -95,7 +95,9 @@ typedef struct {
     int32_t default_math;       /* nnv_math_t used where a caller passes -1; default TF32 */
     int32_t allow_cached;       /* default for selection; default 1                       */
     int32_t max_depth;          /* largest pipeline depth nnv_cold_run accepts; default 4 */
-    int32_t debug_checks;       /* reserved, 0                                            */
+    int32_t kernel_stamps;      /* 1: the tensor-core GEMM kernels and the weight-transform kernels of every run record
+                                   the device clock when their first block starts and their last block ends
+                                   (two atomics per block); nnv_kernel_times reads the durations.  Default 0. */
     int32_t use_graphs;         /* 1: nnv_cold_run / nnv_resident_run record their stream work into a
                                    CUDA graph on the first call with a given argument set (choices,
                                    buffer addresses, depth) and replay it afterwards; 0: always enqueue
@@ -144,6 +146,7 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* plan);
  *   gemm_tile=BN,splits   column tile (16..128, multiple of 16) and K splits (1,2,4,8) of the GEMM
  *   gemm_ring=N           shared-memory ring depth 2..8        gemm_prefill=0|1
  *   conv3x3=off|auto|MT,BN,splits[,boxes,weight_tiles]          the halo-resident 3x3 kernel
+ *   smallp=0|1|N          the weights-on-rows kernel for layers of at most 256 pixels: off, on, on with N K splits
  *   side=0|1  merge=0|1  group=0|1   side stream for residual branches, merged reads, grouped transforms
  * Every call replaces all settings (unnamed keys return to their defaults).  An item that does not
  * parse or is out of range -> NNV_ERR_INVALID_ARG and nothing changes; a setting that does not fit a
@@ -287,12 +290,15 @@ nnv_status_t nnv_schedule_eps(const nnv_plan_t* plan, const nnv_cost_t* costs, i
  * num_k = sum over the conv layers of the run's measured interval, den_k = sum of the chosen
  * kernels' isolated costs (read: h2d_cached_ns if the choice read cached weights, else
  * h2d_raw_ns; transform: only layers that transformed).  Every row's costs of kind k become
- * floor(cost * num_k / den_k), exactly; a kind with num_k = 0 or den_k = 0 is left alone.
+ * floor(cost * num_k / den_k), exactly; a kind with num_k = 0 or den_k = 0 is left alone, and
+ * so is a kind whose bit in `kinds` is clear (1 read, 2 transform, 4 execution): a table meant
+ * for nnv_schedule_link keeps its isolated read costs, because there the reads' waiting for one
+ * another -- which a measured read interval includes -- is what the link model itself adds.
  * Scaling by kind, not by kernel, keeps options that did not run from looking cheaper than
  * those that did.  out: n_costs rows (may alias costs).  factors: NULL or 6 values
  * {num, den} x {read, transform, execution}.  A chosen kernel without a row -> NNV_ERR_STATE. */
 nnv_status_t nnv_calibrate_costs(const nnv_plan_t* plan, const nnv_cost_t* costs, int32_t n_costs,
-                                 const nnv_choice_t* choices, const nnv_timing_t* timings,
+                                 const nnv_choice_t* choices, const nnv_timing_t* timings, int32_t kinds,
                                  nnv_cost_t* out, uint64_t* factors);
 
 /* ---- single operations (asynchronous on `stream`) ------------------------------------------ */
@@ -553,6 +559,15 @@ nnv_status_t nnv_layer_output(const nnv_plan_t* plan, int32_t layer, const void*
  * call of an eager run, or the one graph launch of a replayed one.  When this exceeds the
  * device time of the run, the host and not the GPU or the link bounds the cold latency. */
 nnv_status_t nnv_last_enqueue_ns(const nnv_plan_t* plan, uint64_t* ns);
+
+/* Device time of the kernels of the most recent run on a plan created with kernel_stamps = 1,
+ * per layer, in nanoseconds of the device clock: xform_ns[i] = from the first block's start to the
+ * last block's end of layer i's weight-transform launch (a grouped launch is booked on the first
+ * layer of its group, the others get 0), exec_ns[i] = the same for the layer's tensor-core GEMM
+ * kernel (0 for layers executed by other kernels).  Unlike event pairs around a kernel, which add
+ * microseconds of their own and serialise the streams, the stamps do not disturb the run they
+ * measure.  Both arrays hold one entry per layer; either may be NULL.  Synchronises the device. */
+nnv_status_t nnv_kernel_times(const nnv_plan_t* plan, uint64_t* xform_ns, uint64_t* exec_ns);
 
 /* Profile every eligible (variant, math) of every conv layer in isolation --
  * the per-operation profiling that feeds the paper's Algorithm 1 -- and write

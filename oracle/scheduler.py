@@ -262,7 +262,7 @@ def simulate_link(layers, read_t, xf_little, xf_big, exec_t, queue_of, n_little)
     return end[("e", n - 1)]
 
 
-def calibrate(rows, choices, timings):
+def calibrate(rows, choices, timings, kinds=(True, True, True)):
     """The re-profiling step of Algorithm 1 (its profiling of operations happens with the other queues
     busy; Section 3.3's remark on interference): scale the isolated cost table by how much slower each KIND
     of operation ran in a run of the schedule than it did alone.
@@ -272,7 +272,9 @@ def calibrate(rows, choices, timings):
     end stamps of that run.  For kind k in (read, transform, execution): num_k = sum over the chosen kernels
     of the measured interval, den_k = sum of their isolated costs (read: the cached or the raw read, whichever
     the choice made; transform: only where the choice transformed).  Every row's costs of kind k become
-    floor(cost * num_k / den_k); a kind with num_k = 0 or den_k = 0 stays as it is.
+    floor(cost * num_k / den_k); a kind with num_k = 0 or den_k = 0 stays as it is, and so does a kind whose
+    entry in `kinds` (read, transform, execution) is False -- under the shared-link model the reads' waiting for
+    one another is what simulate_link() itself accounts for, so their measured intervals must not be fed back.
     Returns (new rows, [(num, den) for read, transform, execution]).
     """
     iso = {(r["layer"], r["variant"], r["math"]): r for r in rows}
@@ -293,7 +295,7 @@ def calibrate(rows, choices, timings):
         den[2] += r["exec_ns"]
 
     def scale(v, k):
-        return v if num[k] == 0 or den[k] == 0 else v * num[k] // den[k]
+        return v if num[k] == 0 or den[k] == 0 or not kinds[k] else v * num[k] // den[k]
 
     out = [dict(r, h2d_raw_ns=scale(r["h2d_raw_ns"], 0), h2d_cached_ns=scale(r["h2d_cached_ns"], 0),
                 xform_ns=scale(r["xform_ns"], 1), exec_ns=scale(r["exec_ns"], 2)) for r in rows]

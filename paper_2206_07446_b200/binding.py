@@ -36,7 +36,7 @@ class LayerDesc(ctypes.Structure):
 
 
 class PlanOpts(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("default_math", "allow_cached", "max_depth", "debug_checks", "use_graphs")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("default_math", "allow_cached", "max_depth", "kernel_stamps", "use_graphs")]
 
 
 class Cost(ctypes.Structure):
@@ -81,7 +81,7 @@ _SIGS = {
     "nnv_simulate_link": [_vp, _P(_u64), _P(_u64), _P(_u64), _P(_u64), _P(_i32), _i32, _P(_u64)],
     "nnv_schedule_link": [_vp, _P(Cost), _i32, _i32, _P(_u64), _i32, _u64, _i32, _u64, _P(Choice), _P(_i32), _P(_u64)],
     "nnv_schedule_eps": [_vp, _P(Cost), _i32, _i32, _i32, _P(_u64)],
-    "nnv_calibrate_costs": [_vp, _P(Cost), _i32, _P(Choice), _P(Timing), _P(Cost), _P(_u64)],
+    "nnv_calibrate_costs": [_vp, _P(Cost), _i32, _P(Choice), _P(Timing), _i32, _P(Cost), _P(_u64)],
     "nnv_transform_weights": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
     "nnv_transformed_layout": [_vp, _P(Choice), _P(_u64), _P(_u64)],
     "nnv_transform_all": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp],
@@ -109,6 +109,7 @@ _SIGS = {
                           _P(_u64), _P(_u64)],
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
     "nnv_last_enqueue_ns": [_vp, _P(_u64)],
+    "nnv_kernel_times": [_vp, _P(_u64), _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
     "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
     "nnv_device_status": [_P(_i32)],
@@ -351,13 +352,14 @@ def _timings_array(plan, timings):
     return arr
 
 
-def nnv_calibrate_costs(plan, costs, choices, timings):
-    """Returns (rescaled cost rows as dicts, [(num, den) for read, transform, execution])."""
+def nnv_calibrate_costs(plan, costs, choices, timings, kinds=7):
+    """kinds: bit mask of the kinds to rescale (1 read, 2 transform, 4 execution).
+    Returns (rescaled cost rows as dicts, [(num, den) for read, transform, execution])."""
     n = len(costs)
     out = (Cost * max(1, n))()
     fac = (_u64 * 6)()
     _check(_lib.nnv_calibrate_costs(plan.handle, _costs_array(costs), n, _choices_array(plan, choices),
-                                    _timings_array(plan, timings), out, fac))
+                                    _timings_array(plan, timings), int(kinds), out, fac))
     rows = [{f: int(getattr(out[i], f)) for f, _ in Cost._fields_ if f != "reserved"} for i in range(n)]
     return rows, [(int(fac[2 * k]), int(fac[2 * k + 1])) for k in range(3)]
 
@@ -559,6 +561,13 @@ def nnv_layer_output(plan, layer):
     b = _u64(0)
     _check(_lib.nnv_layer_output(plan.handle, layer, ctypes.byref(p), ctypes.byref(b)))
     return int(p.value), int(b.value)
+
+
+def nnv_kernel_times(plan):
+    """(xform_ns, exec_ns) per layer from the kernels' own device-clock stamps of the last run (plan option kernel_stamps)."""
+    xf, ex = (_u64 * plan.n)(), (_u64 * plan.n)()
+    _check(_lib.nnv_kernel_times(plan.handle, xf, ex))
+    return [int(v) for v in xf], [int(v) for v in ex]
 
 
 def nnv_last_enqueue_ns(plan):

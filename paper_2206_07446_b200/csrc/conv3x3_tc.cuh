@@ -21,6 +21,7 @@
 #pragma once
 
 struct ConvDev {
+    unsigned long long* stamp;      // device-clock stamps of this launch, or null
     float* D;
     const float* bias;
     const float* addend;
@@ -72,6 +73,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *holder_ptr;
     pdl_wait();                                               // set-up above overlaps the previous kernel's tail
+    if (threadIdx.x == 32) stamp_start(g.stamp);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -277,6 +279,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) stamp_end(g.stamp);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");

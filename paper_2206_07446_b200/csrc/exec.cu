@@ -39,6 +39,9 @@ nnv_status_t do_exec(const nnv_plan& p, int layer, int v, int math, const void* 
         return launch_depthwise(x, (const float*)d_wt, bias, add, y, L.act, L.C, L.H, L.W, L.R, L.S, L.stride, L.pad,
                                 g.OH, g.OW, st);
 
+    const SmallPPlan spp = small_p_plan(L, g, v, math);
+    if (spp.use) return launch_gemm_sp(L, g, spp, x, (const float*)d_wt, bias, add, y, d_ws, st);
+
     GemmArgs a{};
     a.mode = bf16 ? GEMM_BF16 : GEMM_TF32;
     a.bias = bias; a.addend = add; a.act = L.act;

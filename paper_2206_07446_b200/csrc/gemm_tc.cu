@@ -41,6 +41,20 @@ nnv_status_t read_device_status(int32_t* code) {
     return NNV_OK;
 }
 
+__device__ unsigned long long g_stamps[2 * STAMP_SLOTS_PER_LAYER * STAMP_MAX_LAYERS];
+
+unsigned long long*& next_stamp() {
+    static thread_local unsigned long long* p = nullptr;
+    return p;
+}
+
+nnv_status_t stamps_device_base(unsigned long long** base) {
+    void* ptr = nullptr;
+    NNV_CUDA(cudaGetSymbolAddress(&ptr, g_stamps));
+    *base = static_cast<unsigned long long*>(ptr);
+    return NNV_OK;
+}
+
 nnv_status_t enqueue_status_read(int* h_pinned, cudaStream_t st) {
     NNV_CUDA(cudaMemcpyFromSymbolAsync(h_pinned, g_device_status, sizeof(int), 0, cudaMemcpyDeviceToHost, st));
     return NNV_OK;
@@ -98,6 +112,16 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
         : "memory");
 }
 
+// Tile store shared -> global through the tensor map (rows / columns outside the tensor are clipped).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// All of this thread's tile stores have finished READING shared memory (the global writes complete with the grid).
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
 // Barrier over every thread of every CTA in the cluster (release / acquire).
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -151,11 +175,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 struct GemmDev {
+    unsigned long long* stamp;        // device-clock stamps of this launch, or null
     float* D;
     const float* bias;
     const float* addend;
     long long ldd, strideD;
     int M, N, Kd, BN, act, tmem_cols, splits, stages, prefill;
+    int tma_out;                      // 0: plain stores; else the column width (16 or 32) of the staged tiles stored by TMA
+    uint32_t stage_off;               // byte offset (from the aligned base) of the dedicated staging tile; 0 = the idle ring
     // implicit im2col (A is the NHWC activation itself): 0 = off
     int ic_on, ic_C, ic_cblk, ic_S, ic_OW, ic_stride, ic_pad;
 };
@@ -230,7 +257,8 @@ __host__ __device__ constexpr uint32_t stage_bytes_of(int BN) {
 
 template <int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmDev g) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmAdd, const GemmDev g) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();
     const int STAGES = g.stages;                              // depth of the shared-memory ring (2..8)
@@ -247,6 +275,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     auto conv_bar = [&](int s) { return bars + 8u * (2 * MAXS + s); };
     const uint32_t tmem_full_bar = bars + 8u * (3 * MAXS);
     const uint32_t holder = bars + 8u * (3 * MAXS + 1);
+    const uint32_t addend_bar = bars + 8u * (3 * MAXS + 2);
+    // Write-out through shared memory (g.tma_out): the tile is staged as [column chunk][warp quarter] sub-tiles of
+    // 32 rows x CW columns in the swizzled layout of the output tensor map and stored by TMA.  With a residual
+    // addend the sub-tiles live in their own region and the addend is loaded INTO them while the K loop runs, so
+    // the epilogue adds in place; without one they reuse the ring, which is idle by then.
+    const int CW = g.tma_out;
+    const uint32_t chunk_bytes = 32u * (uint32_t)CW * 4u;
+    const uint32_t stg0 = sbase + g.stage_off;
     volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -268,6 +304,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(conv_bar(s), 128);
         }
         mbar_init(tmem_full_bar, 1);
+        mbar_init(addend_bar, 1);
+        if (CW) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmD)) : "memory");
+            if (g.addend) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmAdd)) : "memory");
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -314,12 +355,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0 && lane == 0) {
         pdl_wait();
         for (int it = 0; it < prefill; ++it) issue_stage(it, it);
+        if (CW && g.addend) {                                 // the residual tile, straight into the staging sub-tiles
+            const int nch = BN / CW;
+            mbar_expect_tx(addend_bar, (uint32_t)nch * 4u * chunk_bytes);
+            for (int j = 0; j < nch; ++j)
+                for (int q = 0; q < 4; ++q)
+                    tma_load_3d(stg0 + (uint32_t)(j * 4 + q) * chunk_bytes, &tmAdd, n0 + j * CW, m0 + q * 32, 0, addend_bar);
+        }
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *holder_ptr;
     pdl_wait();                                               // set-up above overlaps the previous kernel's tail
+    if (threadIdx.x == 32) stamp_start(g.stamp);
 
     bool epi_ok = false;
     if (warp == 0) {
@@ -401,6 +450,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         if (!ok) {
             if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        } else if (splits == 1 && CW) {
+            // lane = one accumulator row; per column chunk: TMEM -> registers -> (+ bias, + addend from the staging
+            // sub-tile, activation) -> staging sub-tile -> one TMA store per warp and chunk
+            const int quarter = warp & 3;
+            const int nch = BN / CW;
+            bool aok = true;
+            if (g.addend) aok = mbar_wait(addend_bar, 0);
+            if (!aok) {
+                if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+            } else {
+                const bool row_live = m0 + quarter * 32 < g.M;
+                for (int j = 0; j < nch; ++j) {
+                    const uint32_t buf = stg0 + (uint32_t)(j * 4 + quarter) * chunk_bytes;
+                    const uint32_t rowa = buf + (uint32_t)lane * (uint32_t)CW * 4u;
+                    const int nbase = n0 + j * CW;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (h * 16 >= CW) break;
+                        uint32_t r[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(j * CW + h * 16), r);
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            const int c = h * 4 + c4;                       // 16-byte chunk of the row
+                            const int n = nbase + c * 4;
+                            const uint32_t sw = (CW == 32) ? (uint32_t)(c ^ (lane & 7)) : (uint32_t)(c ^ ((lane >> 1) & 3));
+                            const uint32_t addr = rowa + sw * 16u;
+                            float4 v = make_float4(__uint_as_float(r[c4 * 4]), __uint_as_float(r[c4 * 4 + 1]),
+                                                   __uint_as_float(r[c4 * 4 + 2]), __uint_as_float(r[c4 * 4 + 3]));
+                            if (g.bias && n < g.N) {
+                                const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+                                v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                            }
+                            if (g.addend) {
+                                float4 aa;
+                                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(aa.x), "=f"(aa.y), "=f"(aa.z), "=f"(aa.w) : "r"(addr));
+                                v.x += aa.x; v.y += aa.y; v.z += aa.z; v.w += aa.w;
+                            }
+                            v.x = act_fn(v.x, g.act); v.y = act_fn(v.y, g.act); v.z = act_fn(v.z, g.act); v.w = act_fn(v.w, g.act);
+                            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA's reads
+                    __syncwarp();
+                    if (lane == 0 && row_live && nbase < g.N) {
+                        tma_store_3d(&tmD, buf, nbase, m0 + quarter * 32, b);
+                        tma_store_commit();
+                    }
+                }
+                if (lane == 0) tma_store_wait_read();
+            }
         } else if (splits == 1) {
             const int quarter = warp & 3;                     // TMEM lanes this warp may read
             const int m = m0 + quarter * 32 + lane;
@@ -470,7 +569,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (splits > 1) cluster_sync_all();
         if (splits > 1 && warp >= 2 && g_device_status == 0) {
             const int t = (int)threadIdx.x - 64;
-            const int rows_per = BM / splits, r0 = sp * rows_per;
+            // only the rows of the tile that exist are reduced, shared evenly by the cluster's CTAs
+            const int live = min(BM, g.M - m0);
+            const int rows_per = (live + splits - 1) / splits, r0 = sp * rows_per;
             const int c4n = BN / 4;
             const bool vec = ((g.ldd & 3) == 0) && ((g.N & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
                              (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
@@ -478,7 +579,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // Thread t walks the (row, 4-column group) grid in steps of 128 without divisions.  The loop
             // is kept small on purpose (no unrolling): each CTA runs it once, and instruction fetch of
             // cold code costs more here than the arithmetic.
-            const int total = rows_per * c4n;
+            const int total = max(0, min(rows_per, live - r0)) * c4n;
             const int qstep = 128 / c4n, rstep = 128 - qstep * c4n;
             int row = r0 + t / c4n, col4 = t % c4n;
             float* const dbase = g.D + (long long)b * g.strideD;
@@ -528,6 +629,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) stamp_end(g.stamp);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
@@ -535,6 +637,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 #include "conv3x3_tc.cuh"
+#include "gemm_sp.cuh"
 
 // ---- host side --------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
@@ -573,6 +676,20 @@ nnv_status_t encode_operand(CUtensorMap* map, const void* base, bool bf16, int K
                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return NNV_OK;
+}
+
+// 3-D map over the fp32 output (or the residual addend, same geometry): dims {N, M, batch}, boxes of
+// `cw` columns (32 with the 128-byte swizzle, 16 with the 64-byte one) x 32 rows.
+nnv_status_t encode_output(CUtensorMap* map, const void* base, int N, int M, int batch, int64_t ld, int64_t batch_stride, int cw) {
+    cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)(ld * 4), (cuuint64_t)(batch_stride * 4)};
+    cuuint32_t box[3] = {(cuuint32_t)cw, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, cw == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (output tiles) failed with code %d", (int)r);
     return NNV_OK;
 }
 
@@ -678,6 +795,7 @@ nnv_status_t gemm_tc_init() {
         cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(gemm_sp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     });
     return NNV_OK;
 }
@@ -687,6 +805,8 @@ static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, c
     NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 16 * ct.MT + 2));
     NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, ct.BN));
     ConvDev g;
+    g.stamp = next_stamp();
+    next_stamp() = nullptr;
     g.D = a.D; g.bias = a.bias; g.addend = a.addend;
     g.C = a.ic.C; g.H = a.ic.H; g.W = a.ic.W; g.K = a.N;
     g.BN = ct.BN; g.MT = ct.MT; g.act = a.act; g.tmem_cols = ct.tmem_cols; g.splits = ct.splits; g.na = ct.na; g.nb = ct.nb;
@@ -696,6 +816,51 @@ static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, c
     NNV_REQUIRE(grid.y <= 65535, NNV_ERR_UNSUPPORTED, "convolution grid too large");
     (void)launch_pdl_cluster(conv3x3_tc_kernel, grid, dim3(GEMM_THREADS), ct.smem, st, ct.splits, tmA, tmB, g);
     NNV_CUDA(cudaGetLastError());
+    return NNV_OK;
+}
+
+// 3-D tiled map over an NHWC fp32 activation {C, W, H} whose box is 32 channels of the WHOLE image.
+static nnv_status_t encode_image_operand(CUtensorMap* map, const void* base, int C, int H, int W) {
+    NNV_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0 && (C % 4) == 0 && W <= 256 && H <= 256, NNV_ERR_INVALID_ARG,
+                "activation must be 16-byte aligned with C a multiple of 4 and at most 256 pixels a side");
+    cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H};
+    cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)W * C * 4};
+    cuuint32_t box[3] = {32, (cuuint32_t)W, (cuuint32_t)H};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (whole-image boxes) failed with code %d", (int)r);
+    return NNV_OK;
+}
+
+nnv_status_t launch_gemm_sp(const nnv_layer_desc_t& L, const LayerGeom& geo, const SmallPPlan& sp, const float* x, const float* wt,
+                            const float* bias, const float* addend, float* y, void* ws, cudaStream_t st) {
+    NNV_TRY(gemm_tc_init());
+    NNV_REQUIRE(sp.splits == 1 || ws, NNV_ERR_INVALID_ARG, "the K split needs its scratch");
+    CUtensorMap tmW, tmX;
+    NNV_TRY(encode_operand(&tmW, wt, false, geo.Qp, L.K, 1, geo.Qp, (int64_t)L.K * geo.Qp, BM));
+    NNV_TRY(encode_image_operand(&tmX, x, L.C, L.H, L.W));
+    SpDev g;
+    g.stamp = next_stamp();
+    next_stamp() = nullptr;
+    g.D = y; g.part = (float*)ws; g.bias = bias; g.addend = addend;
+    g.P = geo.P; g.K = L.K; g.C = L.C; g.S = L.S; g.pad = L.pad; g.Npad = sp.Npad; g.act = L.act;
+    g.tmem_cols = 32;
+    while (g.tmem_cols < sp.Npad) g.tmem_cols *= 2;
+    g.splits = sp.splits; g.stages = sp.stages; g.cblk = L.C / 32; g.nkb_all = sp.nkb;
+    g.b_slot_bytes = sp.b_slot_bytes; g.b_tx_bytes = (uint32_t)(L.H * L.W) * 128u;
+    const size_t smem = (size_t)1024 + (size_t)sp.stages * (A_STAGE_BYTES + sp.b_slot_bytes) + 8 * (2 * SP_MAX_STAGES + 2);
+    dim3 grid(ceil_div(L.K, BM), sp.splits);
+    (void)launch_pdl(gemm_sp_kernel, grid, dim3(GEMM_THREADS), smem, st, tmW, tmX, g);
+    NNV_CUDA(cudaGetLastError());
+    if (sp.splits > 1) {
+        const long long n4 = (long long)geo.P * L.K / 4;
+        const unsigned blocks = (unsigned)((n4 + 31) / 32);
+        (void)launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, st, (const float*)ws, y, bias, addend, geo.P, L.K, sp.splits,
+                         L.act, g.stamp);
+        NNV_CUDA(cudaGetLastError());
+    }
     return NNV_OK;
 }
 
@@ -709,20 +874,29 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     const int bke = (a.mode == GEMM_BF16) ? 64 : 32;
     const int nkb_all = a.ic.on ? a.ic.R * a.ic.S * ceil_div(a.ic.C, 32) : ceil_div(a.Kd, bke);
     const int m_tiles = ceil_div(a.M, BM);
-    const int stages = (a.mode == GEMM_X3) ? 3 : 4;               // ring depth assumed by the cost model
+    // Ring depth: 8 stages when every CTA has an SM to itself (a lone CTA needs that many loads in flight to keep
+    // the SM's ~100 GB/s of shared-memory fill busy on weights that come cold from HBM), 4 when several share one.
+    auto ring_for = [&](int bn, long long ctas) {
+        const uint32_t stage = (a.mode == GEMM_X3) ? stage_bytes_of<2>(bn) : stage_bytes_of<0>(bn);
+        if (a.mode == GEMM_X3) return 3;
+        return (ctas <= 148 && (size_t)8 * stage <= 200u * 1024u) ? 8 : 4;
+    };
     int BN = 0, splits = 1;
     double best = 1e30;
     for (int nt = ceil_div(a.N, 128); nt <= ceil_div(a.N, 16); nt *= 2) {
         const int bn = ceil_div(ceil_div(a.N, nt), 16) * 16;
         const int n_tiles = ceil_div(a.N, bn);
         const double kb_bytes = (double)(A_STAGE_BYTES + bn * BK_BYTES);
-        const double smem = 1024.0 + stages * kb_bytes * (a.mode == GEMM_X3 ? 2 : 1);
-        const int occ = std::max(1, std::min(4, (int)(220.0 * 1024.0 / smem)));
         for (int sp = 1; sp <= 8 && sp <= nkb_all; sp *= 2) {
             const long long ctas = (long long)m_tiles * n_tiles * a.batch * sp;
-            const double waves = std::ceil((double)ctas / (148.0 * occ));
-            const double per_kb_us = std::max(kb_bytes * occ / 90e3, 0.12);   // bytes / (90 GB/s) in us, shared by co-resident CTAs
-            const double t = waves * (2.0 + (sp > 1 ? 4.5 : 0.0) + std::ceil((double)nkb_all / sp) * per_kb_us + bn * 0.004);
+            const int stages = ring_for(bn, ctas);
+            const double smem = 1024.0 + stages * kb_bytes * (a.mode == GEMM_X3 ? 2 : 1);
+            const int occ = std::max(1, std::min(4, (int)(220.0 * 1024.0 / smem)));
+            double waves = std::ceil((double)ctas / (148.0 * occ));
+            if (sp > 1 && occ == 1 && ctas > 96) waves = std::max(waves, 2.0);     // whole clusters must find free SMs in one GPC
+            const int resident = (int)std::min<long long>(occ, (ctas + 147) / 148);   // CTAs that really share an SM
+            const double per_kb_us = std::max(kb_bytes * resident / 100e3, 0.12) * (stages >= 8 ? 1.0 : 1.3);
+            const double t = waves * (2.0 + (sp > 1 ? 3.0 : 0.0) + std::ceil((double)nkb_all / sp) * per_kb_us + 0.3 + bn * 0.004);
             if (t < best - 1e-9) { best = t; BN = bn; splits = sp; }
         }
         if (bn <= 16) break;
@@ -749,16 +923,16 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     }
     int tmem_cols = 32;
     while (tmem_cols < BN) tmem_cols *= 2;
-    // Ring depth.  Measured: the K loop moves ~90 GB/s per SM whatever the depth beyond 4 (it is bound
-    // by the SM's L2 read rate, not by latency), so 4 stages (3 with the extra converted tiles).
     const uint32_t sb = (a.mode == GEMM_X3) ? stage_bytes_of<2>(BN) : stage_bytes_of<0>(BN);
-    int ring = (a.mode == GEMM_X3) ? 3 : 4;
+    int ring = ring_for(BN, (long long)m_tiles * ceil_div(a.N, BN) * a.batch * splits);
     if (tn.gemm_ring && (size_t)tn.gemm_ring * sb <= 210u * 1024u) ring = tn.gemm_ring;
-    while (splits > 1 && (uint32_t)ring * sb < (uint32_t)BM * (BN + 4) * 4u) ++ring;   // room to park the partial tile
+    while (splits > 1 && ring < 8 && (uint32_t)ring * sb < (uint32_t)BM * (BN + 4) * 4u) ++ring;   // room to park the partial tile
 
     const bool bf16 = a.mode == GEMM_BF16;
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmD, tmAdd;
     GemmDev g;
+    g.stamp = next_stamp();
+    next_stamp() = nullptr;
     g.D = a.D; g.bias = a.bias; g.addend = a.addend;
     g.ldd = a.ldd; g.strideD = a.strideD;
     g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits; g.stages = ring; g.prefill = tn.gemm_prefill;
@@ -774,15 +948,45 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     }
     NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
 
+    // Write-out by TMA through swizzled staging tiles when the output rows are 16-byte multiples (else plain stores).
+    // A residual addend needs a staging tile of its own beside the ring: the ring gives up stages for it.
+    if (a.addend && splits == 1)
+        while (ring > 4 && (size_t)2048 + (size_t)ring * sb + 8 * (3 * 8 + 3) + (size_t)BM * BN * 4 > 220u * 1024u) --ring;
+    g.stages = ring;
+    const size_t ring_and_bars = (size_t)ring * sb + 8 * (3 * 8 + 3);
+    size_t smem_bytes = (size_t)1024 + ring_and_bars;
+    g.tma_out = 0;
+    g.stage_off = 0;
+    const bool out_ok = splits == 1 && (a.N % 4) == 0 && (a.ldd % 4) == 0 && (a.strideD % 4) == 0 &&
+                        (reinterpret_cast<uintptr_t>(a.D) & 15) == 0 && (!a.addend || (reinterpret_cast<uintptr_t>(a.addend) & 15) == 0) &&
+                        (!a.bias || (reinterpret_cast<uintptr_t>(a.bias) & 15) == 0) && (!a.addend || a.batch == 1);
+    if (out_ok) {
+        const int cw = (BN % 32) == 0 ? 32 : 16;
+        size_t need = smem_bytes;
+        uint32_t off = 0;
+        if (a.addend) {                                          // the staging tile cannot share the ring: it is filled while the ring works
+            off = (uint32_t)align_up(ring_and_bars, 1024);
+            need = (size_t)1024 + off + (size_t)BM * BN * 4;
+        }
+        if (need <= 220u * 1024u) {
+            g.tma_out = cw;
+            g.stage_off = off;
+            smem_bytes = need;
+            NNV_TRY(encode_output(&tmD, a.D, a.N, a.M, a.batch, a.ldd, a.batch > 1 ? a.strideD : (int64_t)a.M * a.ldd, cw));
+            if (a.addend) NNV_TRY(encode_output(&tmAdd, a.addend, a.N, a.M, 1, a.ldd, (int64_t)a.M * a.ldd, cw));
+        }
+    }
+    if (!g.tma_out) tmD = tmA;                                   // unused by the kernel, but a kernel parameter must hold a valid object
+    if (!g.tma_out || !a.addend) tmAdd = tmA;
+
     dim3 grid(m_tiles, ceil_div(a.N, BN), a.batch * splits);
     NNV_REQUIRE(grid.y <= 65535 && grid.z <= 65535, NNV_ERR_UNSUPPORTED, "GEMM grid too large");
-    const size_t smem_bytes = (size_t)1024 + (size_t)ring * sb + 8 * (3 * 8 + 2);
     if (a.mode == GEMM_TF32)
-        (void)launch_pdl_cluster(gemm_tc_kernel<0>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<0>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
     else if (a.mode == GEMM_BF16)
-        (void)launch_pdl_cluster(gemm_tc_kernel<1>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<1>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
     else if (a.mode == GEMM_X3)
-        (void)launch_pdl_cluster(gemm_tc_kernel<2>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, g);
+        (void)launch_pdl_cluster(gemm_tc_kernel<2>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
     else
         return fail(NNV_ERR_INVALID_ARG, "unknown GEMM mode %d", a.mode);
     NNV_CUDA(cudaGetLastError());

@@ -87,6 +87,30 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(Params...), dim3 grid, dim3
     (void)::nnv::launch_pdl(kernel, dim3(grid), dim3(block), (size_t)(smem), st, __VA_ARGS__)
 #endif
 
+// ---- device-clock stamps of kernels ----------------------------------------------------------
+// A kernel given a non-null `stamp` pointer records the device-wide nanosecond clock when its first
+// block starts working (after the wait on the previous kernel) and when its last block has finished:
+// stamp[0] = max over blocks of ~start (i.e. ~ of the earliest start), stamp[1] = max over blocks of
+// end; both cleared to 0 before the run.  The launchers below take the pointer from
+// next_stamp() -- set by the caller right before the launch, cleared by the launch that uses it.
+#ifdef __CUDACC__
+__device__ __forceinline__ unsigned long long device_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void stamp_start(unsigned long long* stamp) {
+    if (stamp) atomicMax(stamp, ~device_ns());
+}
+__device__ __forceinline__ void stamp_end(unsigned long long* stamp) {
+    if (stamp) atomicMax(stamp + 1, device_ns());
+}
+#endif
+constexpr int STAMP_SLOTS_PER_LAYER = 2;                      // transform, execution
+constexpr int STAMP_MAX_LAYERS = 4096;
+unsigned long long*& next_stamp();                            // thread-local hand-over to the next stamped launch
+nnv_status_t stamps_device_base(unsigned long long** base);  // the stamp array on the current device (2 words per slot)
+
 static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -123,6 +147,8 @@ struct Tuning {
     int conv3x3 = 0;                          // 0 auto, 1 off, 2 forced tiling below
     int conv_mt = 0, conv_bn = 0, conv_splits = 0, conv_na = 0, conv_nb = 0;
     int side = 1, merge = 1, group = 1;       // pipeline features: side stream, merged reads, grouped transforms
+    int smallp = 1;                           // the weights-on-rows kernel for layers with few pixels
+    int smallp_splits = 0;                    // 0 = the cost model decides
     uint64_t generation = 0;
 };
 Tuning tuning();                              // a copy of the current overrides (thread safe)
@@ -166,6 +192,7 @@ struct nnv_plan {
     int* h_status = nullptr;              // pinned host word the device status is copied into
     cudaStream_t s_side = nullptr;        // the plan's own stream for residual-branch layers (created on first use)
     std::vector<cudaEvent_t> warm_ev;     // continuous mode: layer i's warm weights are prepared
+    int stamped_layers = 0;               // layers whose kernels stamped the device clock in the last run (opts.kernel_stamps)
     uint64_t last_enqueue_ns = 0;         // host time the last run spent putting its work on the streams
     bool warm_pending = false;            // warm preparations may still be running (first warm run waits)
 };
@@ -178,6 +205,10 @@ int wino_m(int variant);                                     // 2/4/6 or 0
 bool is_eligible(const nnv_layer_desc_t& L, int variant);
 uint64_t transformed_bytes(const nnv_plan& p, int layer, int variant, int math);
 uint64_t exec_ws_bytes(const nnv_plan& p, int layer, int variant, int math);
+// How the weights-on-rows kernel (gemm_sp.cuh) would run a layer: K splits, ring depth, padded pixel count and
+// the scratch for the partial tiles; use = false when the layer does not qualify.
+struct SmallPPlan { bool use; int splits, stages, Npad, nkb; uint32_t b_slot_bytes; uint64_t ws_bytes; };
+SmallPPlan small_p_plan(const nnv_layer_desc_t& L, const LayerGeom& g, int variant, int math);
 uint64_t raw_weight_bytes(const nnv_layer_desc_t& L);
 uint64_t exec_flops(const nnv_plan& p, int layer, int variant);
 nnv_status_t check_choice(const nnv_plan& p, int layer, int variant, int math);
@@ -207,7 +238,7 @@ struct XformDesc {
     int kind, bf16, block0;
 };
 constexpr int XF_BATCH_MAX = 56;
-struct XformBatch { int n; int total_blocks; XformDesc d[XF_BATCH_MAX]; };
+struct XformBatch { unsigned long long* stamp; int n; int total_blocks; XformDesc d[XF_BATCH_MAX]; };
 nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st);
 
 // Explicit im2col of an NHWC fp32 image: Xcol[P][Qp], q = (r*S+s)*C + c (fp32 or bf16).
@@ -252,6 +283,9 @@ struct GemmArgs {
 // as hi*hi + lo*hi + hi*lo on the bf16 tensor pipe (fp32-class accuracy, fp32 bytes in memory).
 enum { GEMM_TF32 = 0, GEMM_BF16 = 1, GEMM_X3 = 2 };
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
+// Convolution of a layer with few pixels by the weights-on-rows kernel: x NHWC [H*W][C], wt packed P[K][Qp].
+nnv_status_t launch_gemm_sp(const nnv_layer_desc_t& L, const LayerGeom& g, const SmallPPlan& sp, const float* x, const float* wt,
+                            const float* bias, const float* addend, float* y, void* ws, cudaStream_t st);
 // One-time host set-up of the GEMM (driver entry point, shared-memory attributes); call before
 // stream capture.
 nnv_status_t gemm_tc_init();

@@ -191,8 +191,17 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     const bool grouped = resident && depth == 0 && tn.group;
     std::vector<cudaEvent_t> group_event(n, nullptr);
 
+    // Kernel stamps: slot 2i for layer i's transform launch, 2i + 1 for its tensor-core kernel; two words each.
+    unsigned long long* stamp_base = nullptr;
+    if (p->opts.kernel_stamps && n <= STAMP_MAX_LAYERS) NNV_TRY(stamps_device_base(&stamp_base));
+    auto stamp_for = [&](int layer, int which) {
+        next_stamp() = stamp_base ? stamp_base + 2 * (STAMP_SLOTS_PER_LAYER * layer + which) : nullptr;
+    };
+    p->stamped_layers = stamp_base ? n : 0;
+
     // Everything the pass puts on the streams: fork from s_exec, the per-layer operations, join back.
     auto enqueue = [&]() -> nnv_status_t {
+    if (stamp_base) NNV_CUDA(cudaMemsetAsync(stamp_base, 0, sizeof(unsigned long long) * 2 * STAMP_SLOTS_PER_LAYER * n, s_exec));
     if (tm) NNV_CUDA(cudaEventRecord(p->tev[0], s_exec));
     NNV_CUDA(cudaEventRecord(p->ev[3 * n], s_exec));
     if (queued) {
@@ -217,6 +226,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // can start at once, the next ~8 MB, then all the rest) instead of one small launch per layer.
     if (grouped) {
         std::vector<XformDesc> descs[3];
+        int group_first[3] = {0, 0, 0};
         uint64_t first_bytes = 0;
         for (int i = 0; i < n; ++i) {
             const nnv_layer_desc_t& L = p->layers[i];
@@ -226,13 +236,16 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             const XformDesc d = make_xform_desc(*p, i, ch, (const uint8_t*)weights + L.w_off, base + A.xf_off[i]);
             const int g = first_bytes < (1u << 20) ? 0 : first_bytes < (9u << 20) ? 1 : 2;
             first_bytes += raw_weight_bytes(L);
+            if (descs[g].empty()) group_first[g] = i;
             descs[g].push_back(d);
             group_event[i] = p->ev[3 * n + 3 + g];
         }
         for (int g = 0; g < 3; ++g) {
             if (descs[g].empty()) continue;
             if (tm) NNV_CUDA(cudaEventRecord(p->tev[6 * n + 1 + 2 * g], s_xform));
+            stamp_for(group_first[g], 0);
             NNV_TRY(launch_transform_batch(descs[g].data(), (int)descs[g].size(), s_xform));
+            next_stamp() = nullptr;
             if (tm) NNV_CUDA(cudaEventRecord(p->tev[6 * n + 2 + 2 * g], s_xform));
             NNV_CUDA(cudaEventRecord(p->ev[3 * n + 3 + g], s_xform));
         }
@@ -294,7 +307,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), ps));
             if (has_xf && !cached) {
                 if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), ps));
+                stamp_for(i, 0);
                 NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, (void*)xf, ps));
+                next_stamp() = nullptr;
                 if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), ps));
             }
             if (ps != s_exec) {
@@ -333,7 +348,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                     if (!descs.empty()) {
                         NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(i, 0), 0));
                         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
+                        stamp_for(i, 0);
                         NNV_TRY(launch_transform_batch(descs.data(), (int)descs.size(), s_xform));
+                        next_stamp() = nullptr;
                         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
                         NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
                     }
@@ -371,7 +388,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (ready) NNV_CUDA(cudaStreamWaitEvent(s_xform, ready, 0));
             else if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
+            stamp_for(i, 0);
             NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, (void*)xf, s_xform));
+            next_stamp() = nullptr;
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
             NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
             ready = EV(i, 1);
@@ -382,8 +401,10 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         if (wait_warm && i < (int)p->warm_ev.size() && p->warm_ev[i]) NNV_CUDA(cudaStreamWaitEvent(se, p->warm_ev[i], 0));
         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 4), se));
         const void* add = L.in1 >= 0 ? base + A.act_off[L.in1] : nullptr;
+        stamp_for(i, 1);
         NNV_TRY(do_exec(*p, i, ch.variant, ch.math, in, add, has_xf ? xf : raw, L.has_bias ? bias : nullptr, out,
                         base + A.ws_off, A.ws_bytes, se));
+        next_stamp() = nullptr;
         if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 5), se));
         NNV_CUDA(cudaEventRecord(EV(i, 2), se));
         if (tm) {
@@ -809,6 +830,27 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
     }
     if (read_ns) *read_ns = ns_read;
     if (read_bytes) *read_bytes = bytes_read;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_kernel_times(const nnv_plan_t* p, uint64_t* xform_ns, uint64_t* exec_ns) {
+    NNV_REQUIRE(p, NNV_ERR_INVALID_ARG, "null argument");
+    const int n = (int)p->layers.size();
+    NNV_REQUIRE(p->opts.kernel_stamps && p->stamped_layers == n, NNV_ERR_STATE,
+                "no run with kernel stamps has used this plan (create it with kernel_stamps = 1)");
+    unsigned long long* base = nullptr;
+    NNV_TRY(stamps_device_base(&base));
+    std::vector<unsigned long long> h((size_t)2 * STAMP_SLOTS_PER_LAYER * n);
+    NNV_CUDA(cudaDeviceSynchronize());
+    NNV_CUDA(cudaMemcpy(h.data(), base, sizeof(unsigned long long) * h.size(), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < n; ++i)
+        for (int w = 0; w < STAMP_SLOTS_PER_LAYER; ++w) {
+            const unsigned long long ns = h[2 * (STAMP_SLOTS_PER_LAYER * i + w)], ne = h[2 * (STAMP_SLOTS_PER_LAYER * i + w) + 1];
+            const uint64_t start = ~ns;
+            const uint64_t d = (ns != 0 && ne >= start) ? ne - start : 0;
+            uint64_t* dst = w == 0 ? xform_ns : exec_ns;
+            if (dst) dst[i] = d;
+        }
     return NNV_OK;
 }
 

@@ -339,8 +339,9 @@ nnv_status_t nnv_schedule_eps(const nnv_plan_t* p, const nnv_cost_t* costs, int3
 }
 
 nnv_status_t nnv_calibrate_costs(const nnv_plan_t* p, const nnv_cost_t* costs, int32_t n_costs, const nnv_choice_t* choices,
-                                 const nnv_timing_t* timings, nnv_cost_t* out, uint64_t* factors) {
+                                 const nnv_timing_t* timings, int32_t kinds, nnv_cost_t* out, uint64_t* factors) {
     NNV_REQUIRE(p && costs && choices && timings && out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_REQUIRE(kinds >= 0 && kinds <= 7, NNV_ERR_INVALID_ARG, "kinds %d is not a mask of read (1), transform (2), execution (4)", kinds);
     const int n = (int)p->layers.size();
     uint64_t num[3] = {0, 0, 0}, den[3] = {0, 0, 0};             // read, transform, execution
     for (int i = 0; i < n; ++i) {
@@ -365,7 +366,7 @@ nnv_status_t nnv_calibrate_costs(const nnv_plan_t* p, const nnv_cost_t* costs, i
         den[2] += row->exec_ns;
     }
     auto scale = [&](uint64_t v, int k) -> uint64_t {
-        if (num[k] == 0 || den[k] == 0) return v;
+        if (num[k] == 0 || den[k] == 0 || !((kinds >> k) & 1)) return v;
         return (uint64_t)((unsigned __int128)v * num[k] / den[k]);
     };
     for (int r = 0; r < n_costs; ++r) {

@@ -72,18 +72,38 @@ template <> struct VecStore<__nv_bfloat16, 4> {
     }
 };
 
-constexpr int FT_THREADS = 256;
+template <> struct VecStore<__nv_bfloat16, 8> {
+    __device__ static void st(__nv_bfloat16* p, const float* v) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+        __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+        uint4 u;
+        u.x = *reinterpret_cast<uint32_t*>(&a);
+        u.y = *reinterpret_cast<uint32_t*>(&b);
+        u.z = *reinterpret_cast<uint32_t*>(&c);
+        u.w = *reinterpret_cast<uint32_t*>(&d);
+        *reinterpret_cast<uint4*>(p) = u;
+    }
+};
 
-// One thread transforms NF filters that are adjacent in the padded channel index, so that each
-// of the alpha^2 output planes receives one NF-wide vector store per thread and a warp writes
-// 32*NF consecutive elements of the plane.  With C == Cp the block's raw filters are one
-// contiguous range, staged through shared memory with 128-bit loads.
+constexpr int FT_THREADS = 256;
+constexpr int FT_FILTERS = 1024;                                // filters (padded (k, c) pairs) per block
+// Filters per thread: as many as make every store of a thread 16 bytes wide (4 fp32 or 8 bf16 values).
+template <typename OutT> struct FtNF { static constexpr int value = 4; };
+template <> struct FtNF<__nv_bfloat16> { static constexpr int value = 8; };
+
+// One thread transforms NF filters that are adjacent in the padded channel index, so that each of the alpha^2
+// output planes receives one NF-wide (16-byte) vector store per thread and a warp writes 32*NF consecutive
+// elements of the plane.  A block covers FT_FILTERS filters with FT_FILTERS / NF of its threads.  With C == Cp
+// the block's raw filters are one contiguous range, staged through shared memory with 128-bit loads by all
+// threads and read back with 128-bit loads (a thread's NF * 9 floats start on a 16-byte boundary; the eight
+// threads of a quarter warp then touch all 32 banks once).
 template <int M_, typename OutT, int NF>
 __device__ __forceinline__ void filter_transform_block(const float* __restrict__ g, OutT* __restrict__ U, int K, int C,
                                                        int Cp, unsigned block, float* sg) {
     constexpr int A = WinoG<M_>::A;
+    constexpr int ACTIVE = FT_FILTERS / NF;                       // threads that transform
     const long long F = (long long)K * Cp;                      // padded filter count = plane size
-    const long long f_block = (long long)block * (FT_THREADS * NF);
+    const long long f_block = (long long)block * FT_FILTERS;
     const long long f0 = f_block + (long long)threadIdx.x * NF;
     const bool contiguous = (C == Cp);
 
@@ -92,23 +112,33 @@ __device__ __forceinline__ void filter_transform_block(const float* __restrict__
         const long long base = f_block * 9;
         const float4* src = reinterpret_cast<const float4*>(g + base);
         float4* dst = reinterpret_cast<float4*>(sg);
-        constexpr int NV = FT_THREADS * NF * 9 / 4;
+        constexpr int NV = FT_FILTERS * 9 / 4;
         for (int i = threadIdx.x; i < NV; i += FT_THREADS) {
             if (base + 4ll * i < total) dst[i] = __ldg(src + i);
         }
         __syncthreads();
     }
-    if (f0 >= F) return;
+    if ((int)threadIdx.x >= ACTIVE || f0 >= F) return;
 
     float w[NF][9];
     bool pad[NF];
+    if (contiguous) {
+        const float4* s4 = reinterpret_cast<const float4*>(sg + (size_t)threadIdx.x * NF * 9);
+        float flat[NF * 9];
 #pragma unroll
-    for (int j = 0; j < NF; ++j) {
-        pad[j] = false;
-        if (contiguous) {
+        for (int i = 0; i < NF * 9 / 4; ++i) {
+            const float4 v = s4[i];
+            flat[4 * i] = v.x; flat[4 * i + 1] = v.y; flat[4 * i + 2] = v.z; flat[4 * i + 3] = v.w;
+        }
 #pragma unroll
-            for (int i = 0; i < 9; ++i) w[j][i] = sg[(threadIdx.x * NF + j) * 9 + i];
-        } else {
+        for (int j = 0; j < NF; ++j) {
+            pad[j] = false;
+#pragma unroll
+            for (int i = 0; i < 9; ++i) w[j][i] = flat[j * 9 + i];
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < NF; ++j) {
             const long long f = f0 + j;
             const int k = (int)(f / Cp), c = (int)(f % Cp);
             pad[j] = c >= C;
@@ -147,23 +177,27 @@ __device__ __forceinline__ void filter_transform_block(const float* __restrict__
     }
 }
 
-constexpr int XF_SMEM_FLOATS = 8192;                            // 32 KB staging buffer shared by all transform kernels
+constexpr int XF_SMEM_FLOATS = FT_FILTERS * 9;                   // 36 KB staging buffer shared by all transform kernels
 
 template <int M_, typename OutT, int NF>
 __global__ void __launch_bounds__(FT_THREADS)
-filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp) {
+filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp, unsigned long long* stamp) {
     pdl_enter();
+    if (threadIdx.x == 0) stamp_start(stamp);
     __shared__ __align__(16) float sg[XF_SMEM_FLOATS];
     filter_transform_block<M_, OutT, NF>(g, U, K, C, Cp, blockIdx.x, sg);
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_end(stamp);
 }
 
 template <int M_, typename OutT>
 static nnv_status_t launch_ft(const float* g, void* U, int K, int C, int Cp, cudaStream_t st) {
-    constexpr int NF = 2;
+    constexpr int NF = FtNF<OutT>::value;
     const long long F = (long long)K * Cp;
-    const long long per_block = (long long)FT_THREADS * NF;
-    const unsigned grid = (unsigned)((F + per_block - 1) / per_block);
-    NNV_LAUNCH((filter_transform_kernel<M_, OutT, NF>), grid, FT_THREADS, 0, st, g, reinterpret_cast<OutT*>(U), K, C, Cp);
+    const unsigned grid = (unsigned)((F + FT_FILTERS - 1) / FT_FILTERS);
+    unsigned long long* stamp = next_stamp();
+    next_stamp() = nullptr;
+    NNV_LAUNCH((filter_transform_kernel<M_, OutT, NF>), grid, FT_THREADS, 0, st, g, reinterpret_cast<OutT*>(U), K, C, Cp, stamp);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
@@ -172,8 +206,10 @@ nnv_status_t launch_filter_transform(int m, bool bf16, const float* g, void* U, 
                                      cudaStream_t st) {
     switch (m) {
         case 2: return bf16 ? launch_ft<2, __nv_bfloat16>(g, U, K, C, Cp, st) : launch_ft<2, float>(g, U, K, C, Cp, st);
-        case 4: return bf16 ? launch_ft<4, __nv_bfloat16>(g, U, K, C, Cp, st) : launch_ft<4, float>(g, U, K, C, Cp, st);
-        case 6: return bf16 ? launch_ft<6, __nv_bfloat16>(g, U, K, C, Cp, st) : launch_ft<6, float>(g, U, K, C, Cp, st);
+        // F(4,3) and F(6,3) exist with fp32 U only: their tile GEMM multiplies fp32 operands (one bf16 pass in
+        // those domains misses the output tolerance of the bf16 class)
+        case 4: NNV_REQUIRE(!bf16, NNV_ERR_UNSUPPORTED, "F(4x4,3x3) has no bf16 filter transform"); return launch_ft<4, float>(g, U, K, C, Cp, st);
+        case 6: NNV_REQUIRE(!bf16, NNV_ERR_UNSUPPORTED, "F(6x6,3x3) has no bf16 filter transform"); return launch_ft<6, float>(g, U, K, C, Cp, st);
         default: return fail(NNV_ERR_INVALID_ARG, "no Winograd tile size %d", m);
     }
 }
@@ -329,17 +365,23 @@ __device__ __forceinline__ void pack1x1_block(const float* __restrict__ w, OutT*
 
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
-pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp) {
+pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp, unsigned long long* stamp) {
     pdl_enter();
+    if (threadIdx.x == 0) stamp_start(stamp);
     __shared__ __align__(16) float sw[PACK_SMEM_FLOATS];
     pack_block<OutT>(w, P, K, C, RS, Qp, blockIdx.x, sw);
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_end(stamp);
 }
 
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
-pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp) {
+pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp, unsigned long long* stamp) {
     pdl_enter();
+    if (threadIdx.x == 0) stamp_start(stamp);
     pack1x1_block<OutT>(w, P, K, C, Qp, blockIdx.x);
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_end(stamp);
 }
 
 // ---- many layers in one launch ----------------------------------------------------------------
@@ -357,6 +399,7 @@ template <int GROUP>
 __global__ void __launch_bounds__(FT_THREADS)
 multi_transform_kernel(const __grid_constant__ XformBatch batch) {
     pdl_enter();
+    if (threadIdx.x == 0) stamp_start(batch.stamp);
     __shared__ __align__(16) float smem[XF_SMEM_FLOATS];
     const unsigned vb = blockIdx.x;
     int di = 0;
@@ -375,14 +418,16 @@ multi_transform_kernel(const __grid_constant__ XformBatch batch) {
         }
     } else if constexpr (GROUP == XG_WINO_SMALL) {
         switch (d.kind * 2 + d.bf16) {
-            case XF_WINO2 * 2: filter_transform_block<2, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
-            case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 2>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
-            case XF_WINO4 * 2: filter_transform_block<4, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO2 * 2: filter_transform_block<2, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 8>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO4 * 2: filter_transform_block<4, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
             default: break;
         }
     } else {
-        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem);
+        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem);
     }
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_end(batch.stamp);
 }
 
 static long long pack_blocks(int K, int C, int RS) {
@@ -394,13 +439,16 @@ int xform_blocks(const XformDesc& d) {
     switch (d.kind) {
         case XF_PACK: return (int)pack_blocks(d.K, d.C, d.RS);
         case XF_PACK1X1: return (int)(((long long)d.K * d.Qp + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
-        default: return (int)(((long long)d.K * d.Cp + FT_THREADS * 2 - 1) / (FT_THREADS * 2));
+        default: return (int)(((long long)d.K * d.Cp + FT_FILTERS - 1) / FT_FILTERS);
     }
 }
 
 nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st) {
+    unsigned long long* stamp = next_stamp();                  // every launch of the batch stamps the same slot
+    next_stamp() = nullptr;
     for (int grp = 0; grp < XG_COUNT; ++grp) {
         XformBatch b;
+        b.stamp = stamp;
         b.n = 0;
         int blocks = 0;
         auto flush = [&]() -> nnv_status_t {
@@ -430,16 +478,18 @@ nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st) {
 }
 
 nnv_status_t launch_pack(bool bf16, const float* w, void* P, int K, int C, int RS, int Qp, cudaStream_t st) {
+    unsigned long long* stamp = next_stamp();
+    next_stamp() = nullptr;
     if (RS == 1) {
         const long long n = (long long)K * Qp;
         const unsigned grid = (unsigned)((n + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
-        if (bf16) NNV_LAUNCH((pack1x1_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, Qp);
-        else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp);
+        if (bf16) NNV_LAUNCH((pack1x1_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, Qp, stamp);
+        else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp, stamp);
     } else {
         NNV_REQUIRE(8 * RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED, "filter window of %d taps is too large to repack", RS);
         const unsigned grid = (unsigned)pack_blocks(K, C, RS);
-        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, RS, Qp);
-        else NNV_LAUNCH((pack_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, RS, Qp);
+        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, RS, Qp, stamp);
+        else NNV_LAUNCH((pack_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, RS, Qp, stamp);
     }
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;

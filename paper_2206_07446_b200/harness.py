@@ -28,10 +28,10 @@ def dev_bytes(nbytes, fill=0xFF):
 class Model:
     """A plan plus its host-side weight blob, ready for cold runs."""
 
-    def __init__(self, layers, blob_u8, w_off, b_off, max_depth=4, use_graphs=1):
+    def __init__(self, layers, blob_u8, w_off, b_off, max_depth=4, use_graphs=1, kernel_stamps=0):
         self.layers = layers
         self.plan = nb.Plan(layers, w_off, b_off, opts=dict(default_math=nb.MATH_TF32, allow_cached=1,
-                                                            max_depth=max_depth, debug_checks=0,
+                                                            max_depth=max_depth, kernel_stamps=kernel_stamps,
                                                             use_graphs=use_graphs))
         self.h_weights = _pinned_bytes(np.ascontiguousarray(blob_u8))
         self.w_bytes = int(blob_u8.size)
@@ -50,7 +50,7 @@ class Model:
     def second_plan(self, use_graphs):
         """Another plan over the same layers and weight blob (e.g. one that replays recorded graphs beside an eager one)."""
         return nb.Plan(self.layers, self.w_off, self.b_off, opts=dict(default_math=nb.MATH_TF32, allow_cached=1, max_depth=4,
-                                                                      debug_checks=0, use_graphs=use_graphs))
+                                                                      kernel_stamps=0, use_graphs=use_graphs))
 
     def out_hw(self, i):
         L = self.layers[i]
@@ -141,7 +141,7 @@ class Model:
         schedule once with per-operation timings, let the library rescale the table by how much slower each kind
         of operation ran beside the others than alone (nnv_calibrate_costs), schedule again; `rounds` times.
         This method only sequences library calls.  link=True evaluates schedules with the shared-link latency
-        (nnv_schedule_link).  Returns (choices, queue_of, predicted ns, calibrated costs)."""
+        (nnv_schedule_link) and keeps the isolated read costs (the link model adds the reads' waiting itself).  Returns (choices, queue_of, predicted ns, calibrated costs)."""
         table = costs
         eps = nb.nnv_schedule_eps(self.plan, costs, allow_cached, eps_pct)
         out = None
@@ -155,7 +155,7 @@ class Model:
                 self.build_cached_blob(choices)
             self.cold_run_queues(x_nchw, choices, queue_of, n_little, poison=False)          # warm
             _, tm = self.cold_run_queues(x_nchw, choices, queue_of, n_little, want_timings=True, poison=False)
-            rows, fac = nb.nnv_calibrate_costs(self.plan, costs, choices, tm)
+            rows, fac = nb.nnv_calibrate_costs(self.plan, costs, choices, tm, kinds=6 if link else 7)
             self.calibration = {k: (f[0] / f[1] if f[1] else None) for k, f in zip(("h2d", "xform", "exec"), fac)}
             table = nb.CostTable(rows)
         return out[0], out[1], out[2], table
@@ -254,8 +254,8 @@ class Model:
         return costs
 
 
-def model_from_workload(layers, weights, biases, blob_fn, max_depth=4, use_graphs=1):
+def model_from_workload(layers, weights, biases, blob_fn, max_depth=4, use_graphs=1, kernel_stamps=0):
     """Build a Model from a layer list and per-layer numpy weights using `blob_fn`
     (workloads.weight_blob) to lay out the host blob."""
     blob, w_off, b_off = blob_fn(layers, weights, biases)
-    return Model(layers, blob, w_off, b_off, max_depth=max_depth, use_graphs=use_graphs)
+    return Model(layers, blob, w_off, b_off, max_depth=max_depth, use_graphs=use_graphs, kernel_stamps=kernel_stamps)

@@ -165,10 +165,11 @@ def test_calibrate_and_eps_match_oracle(seed):
             a, b, c = (int(rng.integers(0, hi)) for _ in range(3))
             tm.append(dict(h2d_start_ns=5, h2d_end_ns=5 + a, xform_start_ns=7, xform_end_ns=7 + (b if seed % 4 else 0),
                            exec_start_ns=9, exec_end_ns=9 + c))
-        want_rows, want_fac = osch.calibrate(costs, choices, tm)
-        got_rows, got_fac = nb.nnv_calibrate_costs(plan, costs, choices, tm)
-        assert got_fac == [tuple(f) for f in want_fac]
-        assert got_rows == [{k: r[k] for k in got_rows[0]} for r in want_rows]
+        for kinds in (7, 6, 5, 0):
+            want_rows, want_fac = osch.calibrate(costs, choices, tm, kinds=[bool(kinds & 1), bool(kinds & 2), bool(kinds & 4)])
+            got_rows, got_fac = nb.nnv_calibrate_costs(plan, costs, choices, tm, kinds)
+            assert got_fac == [tuple(f) for f in want_fac]
+            assert got_rows == [{k: r[k] for k in got_rows[0]} for r in want_rows]
         iso = {(c["layer"], c["variant"], c["math"]): c for c in costs}
         for pct in (0, 1, 7, 100):
             ex = [iso[(i,) + ch[:2]]["exec_ns"] for i, ch in enumerate(choices) if ch is not None]

@@ -237,3 +237,34 @@ def test_merged_copies_at_depth_zero():
         nb.nnv_tuning_set(None)
     assert len({(tm1[i]["h2d_start_ns"], tm1[i]["h2d_end_ns"]) for i in convs}) == len(convs)
     assert np.array_equal(y_merged, y_single)
+
+
+def test_kernel_stamps_measure_without_changing_the_result():
+    """A plan with kernel_stamps = 1: the tensor-core and transform kernels write device-clock stamps; the
+    result is bit for bit that of a plan without them, every stamped duration is positive and none is longer
+    than the whole run, and layers executed by the fp32 kernels report none."""
+    layers = wl.cfg2_resnet18()
+    ws, bs = wl.make_weights(layers)
+    x = wl.make_input(layers)
+    plain = harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=0)
+    stamped = harness.model_from_workload(layers, ws, bs, wl.weight_blob, use_graphs=0, kernel_stamps=1)
+    ch = _choices(plain, [nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    ch[0] = (nb.VAR_DIRECT, nb.MATH_FP32, 0)
+    y0, _ = plain.cold_run(x, ch, depth=0)
+    with pytest.raises(nb.NnvError):
+        nb.nnv_kernel_times(plain.plan)
+    for depth in (0, 2):
+        y1, tm = stamped.cold_run(x, ch, depth=depth, want_timings=True)
+        assert np.array_equal(y0.view(np.uint32), y1.view(np.uint32))
+        xf, ex = nb.nnv_kernel_times(stamped.plan)
+        total = max(t["exec_end_ns"] for t in tm)
+        convs = [i for i, L in enumerate(layers) if L["op"] == wl.OP_CONV]
+        assert ex[0] == 0                                      # the direct kernel is no tensor-core launch
+        assert depth == 0 or xf[0] == 0                        # (at depth 0 layer 0 books the grouped transform of its chunk)
+        for i in convs[1:]:
+            assert 0 < ex[i] < total, (i, ex[i], total)
+            # the stamps lie inside the event interval around the layer (1 us of slack for the two clocks)
+            assert ex[i] <= tm[i]["exec_end_ns"] - tm[i]["exec_start_ns"] + 1000, (i, ex[i], tm[i])
+        assert sum(1 for i in convs if xf[i] > 0) >= 1 and all(v < total for v in xf)
+        if depth:                                              # one transform launch per layer
+            assert all(xf[i] > 0 for i in convs[1:])

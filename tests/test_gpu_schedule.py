@@ -91,6 +91,12 @@ def test_profile_schedule_run():
     if any(c is not None and c[2] for c in choices):
         model.build_cached_blob(choices)
     y, _ = model.cold_run_queues(x, choices, queue_of, 2)
+    # the harness only sequences library calls: the calibrated table is nnv_calibrate_costs of a run's timings,
+    # which is the oracle's calibrate() of the same timings, exactly
+    _, tm = model.cold_run_queues(x, choices, queue_of, 2, want_timings=True, poison=False)
+    got_rows, got_fac = nb.nnv_calibrate_costs(model.plan, costs, choices, tm)
+    want_rows, want_fac = osch.calibrate(costs, choices, tm)
+    assert got_fac == [tuple(f) for f in want_fac] and got_rows == [{k: r[k] for k in got_rows[0]} for r in want_rows]
     y3, _ = model.cold_run(x, choices, depth=0)
     assert np.array_equal(y.view(np.uint32), y3.view(np.uint32))
     acts = omodel.run_model(layers, ws, bs, x)

@@ -250,6 +250,9 @@ def test_calibrate_hand_table():
     assert [r["h2d_cached_ns"] for r in out] == [300 * 1065 // 810, 500 * 1065 // 810, 10 * 1065 // 810, 700 * 1065 // 810]
     assert [r["xform_ns"] for r in out] == [60, 135, 0, 90]
     assert [r["exec_ns"] for r in out] == [65, 26, 91, 39]
+    # a kind switched off keeps its isolated costs, the others are scaled as before
+    out6, fac6 = sch.calibrate(rows, choices, tm, kinds=(False, True, True))
+    assert [r["h2d_raw_ns"] for r in out6] == [100, 100, 10, 200] and [r["exec_ns"] for r in out6] == [65, 26, 91, 39] and fac6 == fac
     # a run that measured nothing of a kind leaves that kind alone (no division by zero, no zeroed table)
     tm0 = [dict(t, xform_start_ns=0, xform_end_ns=0) for t in tm]
     out0, fac0 = sch.calibrate(rows, choices, tm0)
