@@ -433,6 +433,30 @@ def run_ours(args):
                                   "transform_launches": sum(1 for c in choices_byp if c is not None and not c[2] and c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE)),
                                   "h2d_bytes_per_step": h2d_bytes(layers, choices_byp, model.plan, nb, x.nbytes)}
 
+        # ---- zero-copy arm: the transform kernels read the raw weights in place in pinned host memory ----
+        choices_zc = nb.nnv_select_kernels(model.plan, costs, 2)
+        choices_zc_all = [None if c is None else (c[0], c[1], nb.ARM_ZERO_COPY if c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else 0)
+                          for c in choices_raw]
+        for name, chz in (("zero_copy_allowed", choices_zc), ("zero_copy_every_layer", choices_zc_all)):
+            def step_zc(k, timed, chz=chz):
+                begin(k, timed, (s_copy, s_xform))
+                nb.nnv_cold_run(model.plan, chz, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
+                                model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+                if timed:
+                    ev1[k].record(s_exec)
+
+            ms, _ = timed_region(step_zc, args.arm_steps, 3)
+            arms[name] = {"e2e_ms": ms, "zero_copy_layers": sum(1 for c in chz if c is not None and c[2] == nb.ARM_ZERO_COPY),
+                          "what": "nnv_cold_run, eager; " + ("selection with the zero-copy arm allowed (allow_cached = 2)" if name == "zero_copy_allowed"
+                                                             else "the headline's kernels, every transform reading host memory in place")}
+        # per layer, isolated: copy then transform against the fused zero-copy preparation (profiled costs)
+        by_size = {}
+        for c in costs:
+            if c["zc_ns"] and choices_raw[c["layer"]] is not None and (c["variant"], c["math"]) == tuple(choices_raw[c["layer"]][:2]):
+                by_size.setdefault(raw_bytes(layers[c["layer"]]), []).append((c["h2d_raw_ns"] + c["xform_ns"], c["zc_ns"]))
+        arms["zero_copy_by_layer_size"] = [{"raw_bytes": b, "layers": len(v), "copy_then_transform_us": statistics.mean(a for a, _ in v) / 1e3,
+                                            "zero_copy_us": statistics.mean(z for _, z in v) / 1e3} for b, v in sorted(by_size.items())]
+
         # ---- the headline step replayed from a recorded CUDA graph ----
         def step_graph(k, timed):
             begin(k, timed, (s_copy, s_xform))

@@ -110,9 +110,19 @@ typedef struct {
 typedef struct {
     int32_t layer, variant, math, reserved;
     uint64_t h2d_raw_ns, xform_ns, h2d_cached_ns, exec_ns;
+    uint64_t zc_ns;             /* the fused preparation: the transform kernel reads the raw weights straight from pinned
+                                   host memory, no copy before it (0 = not profiled / not offered) */
 } nnv_cost_t;
 
+/* One layer's kernel and how its weights are prepared.  cached: NNV_ARM_RAW = read raw weights, then
+ * transform; NNV_ARM_CACHED = read cached post-transform weights (Section 3.1.2); NNV_ARM_ZERO_COPY = the
+ * transform kernel reads the raw weights in place in pinned host memory and writes the transformed
+ * weights to device memory (the paper bundles read and transform into one preparation operation,
+ * Section 3.1.3; here they become one kernel, and the raw copy in device memory disappears). */
 typedef struct { int32_t variant, math, cached; } nnv_choice_t;
+#define NNV_ARM_RAW 0
+#define NNV_ARM_CACHED 1
+#define NNV_ARM_ZERO_COPY 2
 
 /* Per-layer record of one cold run.  Start/end stamps are nanoseconds since the
  * run's first enqueue; 0/0 where the operation does not exist for the layer. */
@@ -182,8 +192,10 @@ nnv_status_t nnv_cached_layout(const nnv_plan_t* plan, const nnv_choice_t* choic
 /* ---- selection (integer, exact) ------------------------------------------------------------ */
 
 /* Candidate filter that opens the paper's Algorithm 1: of one layer's options
- * (each cost row gives a raw arm, prep = h2d_raw + xform, and -- if the variant
- * has a transform and allow_cached -- a cached arm, prep = h2d_cached) drop every
+ * (each cost row gives a raw arm, prep = h2d_raw + xform; if the variant has a
+ * transform and bit 0 of allow_cached is set a cached arm, prep = h2d_cached; if it
+ * has a transform, bit 1 of allow_cached is set and zc_ns > 0 a zero-copy arm,
+ * prep = zc_ns) drop every
  * option for which another is no slower in both prep and exec and faster in one;
  * of exact duplicates keep the lowest (variant, math, cached).  Survivors are
  * written in ascending (variant, math, cached) order. */

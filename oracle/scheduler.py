@@ -285,12 +285,14 @@ def calibrate(rows, choices, timings, kinds=(True, True, True)):
             continue
         r, t = iso[(i, ch[0], ch[1])], timings[i]
         has_xf = ch[0] not in (0, 3)                           # DIRECT and DEPTHWISE read raw weights as they are
-        cached = bool(ch[2]) and has_xf
-        num[0] += t["h2d_end_ns"] - t["h2d_start_ns"]
-        den[0] += r["h2d_cached_ns"] if cached else r["h2d_raw_ns"]
+        cached = ch[2] == 1 and has_xf
+        fused = ch[2] == 2 and has_xf                          # read + transform as one operation (zc_ns): counts as a transform
+        if not fused:
+            num[0] += t["h2d_end_ns"] - t["h2d_start_ns"]
+            den[0] += r["h2d_cached_ns"] if cached else r["h2d_raw_ns"]
         if has_xf and not cached:
             num[1] += t["xform_end_ns"] - t["xform_start_ns"]
-            den[1] += r["xform_ns"]
+            den[1] += r.get("zc_ns", 0) if fused else r["xform_ns"]
         num[2] += t["exec_end_ns"] - t["exec_start_ns"]
         den[2] += r["exec_ns"]
 
@@ -298,7 +300,8 @@ def calibrate(rows, choices, timings, kinds=(True, True, True)):
         return v if num[k] == 0 or den[k] == 0 or not kinds[k] else v * num[k] // den[k]
 
     out = [dict(r, h2d_raw_ns=scale(r["h2d_raw_ns"], 0), h2d_cached_ns=scale(r["h2d_cached_ns"], 0),
-                xform_ns=scale(r["xform_ns"], 1), exec_ns=scale(r["exec_ns"], 2)) for r in rows]
+                xform_ns=scale(r["xform_ns"], 1), exec_ns=scale(r["exec_ns"], 2),
+                **({"zc_ns": scale(r["zc_ns"], 1)} if "zc_ns" in r else {})) for r in rows]
     return out, list(zip(num, den))
 
 

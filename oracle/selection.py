@@ -62,8 +62,11 @@ def options_from_costs(rows, allow_cached):
     for r in rows:
         v, mth = int(r["variant"]), int(r["math"])
         opts.append(((v, mth, 0), int(r["h2d_raw_ns"]) + int(r["xform_ns"]), int(r["exec_ns"])))
-        if allow_cached and has_transform(v):
+        if (int(allow_cached) & 1) and has_transform(v):
             opts.append(((v, mth, 1), int(r["h2d_cached_ns"]), int(r["exec_ns"])))
+        # third arm (bit 1 of allow_cached): read and transform fused into one operation whose time is zc_ns
+        if (int(allow_cached) & 2) and has_transform(v) and int(r.get("zc_ns", 0)) > 0:
+            opts.append(((v, mth, 2), int(r["zc_ns"]), int(r["exec_ns"])))
     return opts
 
 

@@ -18,6 +18,7 @@ OP_CONV, OP_MAXPOOL, OP_GAVGPOOL = 0, 1, 2
 VAR_DIRECT, VAR_IM2COL, VAR_GEMM1X1, VAR_DEPTHWISE, VAR_WINO_F2, VAR_WINO_F4, VAR_WINO_F6 = range(7)
 VARIANT_NAMES = ["direct", "im2col", "gemm1x1", "depthwise", "wino_f2", "wino_f4", "wino_f6"]
 MATH_FP32, MATH_TF32, MATH_BF16 = 0, 1, 2
+ARM_RAW, ARM_CACHED, ARM_ZERO_COPY = 0, 1, 2           # the `cached` field of a choice: how the weights are prepared
 MATH_NAMES = ["fp32", "tf32", "bf16"]
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "STATE", "WORKSPACE_TOO_SMALL", "CUDA", "TIMEOUT"]
 
@@ -41,7 +42,7 @@ class PlanOpts(ctypes.Structure):
 
 class Cost(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("layer", "variant", "math", "reserved")] + \
-               [(n, ctypes.c_uint64) for n in ("h2d_raw_ns", "xform_ns", "h2d_cached_ns", "exec_ns")]
+               [(n, ctypes.c_uint64) for n in ("h2d_raw_ns", "xform_ns", "h2d_cached_ns", "exec_ns", "zc_ns")]
 
 
 class Choice(ctypes.Structure):
@@ -268,7 +269,7 @@ def _costs_array(costs):
     arr = (Cost * max(1, len(costs)))()
     for i, c in enumerate(costs):
         arr[i] = Cost(int(c["layer"]), int(c["variant"]), int(c["math"]), 0, int(c["h2d_raw_ns"]),
-                      int(c["xform_ns"]), int(c["h2d_cached_ns"]), int(c["exec_ns"]))
+                      int(c["xform_ns"]), int(c["h2d_cached_ns"]), int(c["exec_ns"]), int(c.get("zc_ns", 0)))
     return arr
 
 

@@ -126,7 +126,7 @@ nnv_status_t nnv_cache_write(const char* path, const nnv_plan_t* p, const nnv_ch
                     NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the weight blob", i);
         NNV_REQUIRE(!queue_of || n_little == 0 || (queue_of[i] >= 0 && queue_of[i] <= n_little), NNV_ERR_INVALID_ARG,
                     "layer %d: queue %d outside 0..%d", i, queue_of ? queue_of[i] : 0, n_little);
-        rows[i] = PlanRow{choices[i].variant, choices[i].math, choices[i].cached ? 1 : 0, (queue_of && n_little) ? queue_of[i] : -1};
+        rows[i] = PlanRow{choices[i].variant, choices[i].math, choices[i].cached, (queue_of && n_little) ? queue_of[i] : -1};
     }
     FileHeader h{};
     memcpy(h.magic, MAGIC, 8);

@@ -5,14 +5,16 @@ using namespace nnv;
 
 namespace nnv {
 
+// host_src: d_raw is pinned host memory read in place (the zero-copy arm): the kernels then start loading
+// before they wait for the previous kernel of their stream, which they do not depend on.
 nnv_status_t do_transform(const nnv_plan& p, int layer, int v, int math, const void* d_raw, void* d_out,
-                          cudaStream_t st) {
+                          cudaStream_t st, bool host_src) {
     const nnv_layer_desc_t& L = p.layers[layer];
     const LayerGeom& g = p.geom[layer];
     const bool bf16 = math == NNV_MATH_BF16;
-    if (int m = wino_m(v)) return launch_filter_transform(m, bf16, (const float*)d_raw, d_out, L.K, L.C, g.Cp, st);
+    if (int m = wino_m(v)) return launch_filter_transform(m, bf16, (const float*)d_raw, d_out, L.K, L.C, g.Cp, st, host_src);
     if (v == NNV_VAR_IM2COL || v == NNV_VAR_GEMM1X1)
-        return launch_pack(bf16, (const float*)d_raw, d_out, L.K, L.C, L.R * L.S, g.Qp, st);
+        return launch_pack(bf16, (const float*)d_raw, d_out, L.K, L.C, L.R * L.S, g.Qp, st, host_src);
     return fail(NNV_ERR_UNSUPPORTED, "variant %d reads raw weights and has no transform", v);
 }
 
@@ -103,7 +105,7 @@ nnv_status_t nnv_transform_weights(const nnv_plan_t* p, int32_t layer, int32_t v
     NNV_REQUIRE(p && d_raw && d_out, NNV_ERR_INVALID_ARG, "null argument");
     NNV_TRY(check_choice(*p, layer, v, math));
     NNV_REQUIRE(aligned256(d_raw) && aligned256(d_out), NNV_ERR_INVALID_ARG, "device pointers must be 256-byte aligned");
-    return do_transform(*p, layer, v, math, d_raw, d_out, (cudaStream_t)stream);
+    return do_transform(*p, layer, v, math, d_raw, d_out, (cudaStream_t)stream, false);
 }
 
 nnv_status_t nnv_transformed_layout(const nnv_plan_t* p, const nnv_choice_t* choices, uint64_t* offsets, uint64_t* total) {

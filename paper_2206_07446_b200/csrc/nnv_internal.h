@@ -226,9 +226,10 @@ nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int de
 // ---- kernel launchers (device TUs) ----------------------------------------------------------
 // Winograd filter transform: g[K][C][3][3] fp32 -> U[alpha^2][K][Cp] (fp32 or bf16).
 nnv_status_t launch_filter_transform(int m, bool bf16, const float* d_g, void* d_U, int K, int C, int Cp,
-                                     cudaStream_t st);
+                                     cudaStream_t st, bool host_src = false);
 // GEMM-ready repack: W[K][C][R][S] -> P[K][Qp] (fp32 or bf16).
-nnv_status_t launch_pack(bool bf16, const float* d_w, void* d_P, int K, int C, int RS, int Qp, cudaStream_t st);
+nnv_status_t launch_pack(bool bf16, const float* d_w, void* d_P, int K, int C, int RS, int Qp, cudaStream_t st,
+                         bool host_src = false);
 
 // Several layers' weight transforms in one launch.
 enum { XF_PACK = 0, XF_PACK1X1 = 1, XF_WINO2 = 2, XF_WINO4 = 3, XF_WINO6 = 4 };
@@ -236,9 +237,10 @@ struct XformDesc {
     const void* src; void* dst;
     int K, C, Cp, RS, Qp;
     int kind, bf16, block0;
+    int host_src;                    // src is pinned host memory read in place
 };
 constexpr int XF_BATCH_MAX = 56;
-struct XformBatch { unsigned long long* stamp; int n; int total_blocks; XformDesc d[XF_BATCH_MAX]; };
+struct XformBatch { unsigned long long* stamp; int n; int total_blocks; int host_src; XformDesc d[XF_BATCH_MAX]; };
 nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st);
 
 // Explicit im2col of an NHWC fp32 image: Xcol[P][Qp], q = (r*S+s)*C + c (fp32 or bf16).

@@ -11,7 +11,7 @@
 #include "nnv_internal.h"
 
 namespace nnv {
-nnv_status_t do_transform(const nnv_plan& p, int layer, int v, int math, const void* d_raw, void* d_out, cudaStream_t st);
+nnv_status_t do_transform(const nnv_plan& p, int layer, int v, int math, const void* d_raw, void* d_out, cudaStream_t st, bool host_src = false);
 nnv_status_t do_exec(const nnv_plan& p, int layer, int v, int math, const void* d_in, const void* d_add,
                      const void* d_wt, const void* d_bias, void* d_out, void* d_ws, uint64_t ws_bytes, cudaStream_t st);
 nnv_status_t do_pool(const nnv_plan& p, int layer, const void* d_in, void* d_out, cudaStream_t st);
@@ -48,6 +48,13 @@ struct WarmCtx {
     uint64_t xf_region;
     std::vector<uint64_t> woff;
 };
+
+// True when kernels can read `h` in place: pinned (page-locked) host memory under unified addressing.
+static bool host_blob_is_mapped(const void* h) {
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, h) != cudaSuccess) { cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeHost && at.devicePointer == h;
+}
 
 static XformDesc make_xform_desc(const nnv_plan& p, int i, const nnv_choice_t& ch, const void* src, void* dst) {
     const nnv_layer_desc_t& L = p.layers[i];
@@ -89,6 +96,13 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         if (L.op != NNV_OP_CONV) continue;
         NNV_REQUIRE(L.w_off + raw_weight_bytes(L) <= w_bytes && (!L.has_bias || L.b_off + 4ull * L.K <= w_bytes),
                     NNV_ERR_INVALID_ARG, "layer %d: weights lie outside the weight blob", i);
+    }
+    if (!resident && !wc) {
+        bool any_zc = false;
+        for (int i = 0; i < n; ++i)
+            any_zc = any_zc || (p->layers[i].op == NNV_OP_CONV && variant_has_transform(choices[i].variant) && choices[i].cached == NNV_ARM_ZERO_COPY);
+        NNV_REQUIRE(!any_zc || host_blob_is_mapped(weights), NNV_ERR_INVALID_ARG,
+                    "the zero-copy arm needs the weight blob in pinned host memory that kernels can address");
     }
     NNV_TRY(ensure_events(*p, timings != nullptr));
     if (wc && p->warm_ev.size() != (size_t)n) {
@@ -138,7 +152,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // and destination ranges line up are read by ONE copy.  The chunks start at 256 KB, so that execution
     // begins early, and double up to 4 MB; all layers of a chunk become ready when it lands, and their
     // weight transforms are one grouped launch.
-    struct CopyChunk { const uint8_t* src; uint8_t* dst; uint64_t bytes; int first, last; };
+    struct CopyChunk { const uint8_t* src; uint8_t* dst; uint64_t bytes; int first, last; bool zero_copy; };
     std::vector<CopyChunk> chunks;
     std::vector<int> chunk_of(n, -1);
     bool merge = !resident && !queued && depth == 0 && !wc && tn.merge;
@@ -152,7 +166,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (p->layers[i].op != NNV_OP_CONV) continue;
             ++convs;
             const nnv_choice_t ch = choices[i];
-            bytes += (variant_has_transform(ch.variant) && ch.cached) ? transformed_bytes(*p, i, ch.variant, ch.math)
+            bytes += (variant_has_transform(ch.variant) && ch.cached == NNV_ARM_CACHED) ? transformed_bytes(*p, i, ch.variant, ch.math)
                                                                        : raw_weight_bytes(p->layers[i]);
         }
         merge = (double)bytes / 50e3 > 8.0 * convs;              // us
@@ -165,12 +179,14 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             const nnv_layer_desc_t& L = p->layers[i];
             if (L.op != NNV_OP_CONV) continue;
             const nnv_choice_t ch = choices[i];
-            const bool cached = variant_has_transform(ch.variant) && ch.cached;
+            const bool zc_l = variant_has_transform(ch.variant) && ch.cached == NNV_ARM_ZERO_COPY;   // read by its transform kernel, no copy
+            const bool cached = variant_has_transform(ch.variant) && ch.cached == NNV_ARM_CACHED;
+            const int kind = zc_l ? 2 : (int)cached;
             const uint8_t* src = cached ? (const uint8_t*)cached_blob + coff[i] : (const uint8_t*)weights + L.w_off;
             uint8_t* dst = (uint8_t*)d_arena + (cached ? A.xf_off[i] : A.raw_off[i]);
             const uint64_t len = cached ? transformed_bytes(*p, i, ch.variant, ch.math) : raw_weight_bytes(L);
             bool joined = false;
-            if (!chunks.empty() && cur_kind == (int)cached) {
+            if (!chunks.empty() && cur_kind == kind) {
                 CopyChunk& c = chunks.back();
                 if (src >= c.src + c.bytes && (uint64_t)(src - (c.src + c.bytes)) <= kMaxGap && src - c.src == dst - c.dst &&
                     c.bytes < target && i - c.first < XF_BATCH_MAX) {
@@ -181,8 +197,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             }
             if (!joined) {
                 if (!chunks.empty()) target = std::min(target * 2, kMaxTarget);
-                chunks.push_back(CopyChunk{src, dst, len, i, i});
-                cur_kind = (int)cached;
+                chunks.push_back(CopyChunk{src, dst, len, i, i, kind == 2});
+                cur_kind = kind;
             }
             chunk_of[i] = (int)chunks.size() - 1;
         }
@@ -232,7 +248,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             const nnv_layer_desc_t& L = p->layers[i];
             if (L.op != NNV_OP_CONV) continue;
             const nnv_choice_t ch = choices[i];
-            if (!variant_has_transform(ch.variant) || ch.cached) continue;
+            if (!variant_has_transform(ch.variant) || ch.cached == NNV_ARM_CACHED) continue;
             const XformDesc d = make_xform_desc(*p, i, ch, (const uint8_t*)weights + L.w_off, base + A.xf_off[i]);
             const int g = first_bytes < (1u << 20) ? 0 : first_bytes < (9u << 20) ? 1 : 2;
             first_bytes += raw_weight_bytes(L);
@@ -276,7 +292,10 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         const uint8_t* bias = depth ? raw + A.raw_bias_off : base + A.bias_off[i];
         const uint8_t* xf = depth ? base + A.xf_slot0 + (uint64_t)slot * A.xf_slot_bytes : base + A.xf_off[i];
         const bool has_xf = variant_has_transform(ch.variant);
-        const bool cached = has_xf && ch.cached;
+        const bool cached = has_xf && ch.cached == NNV_ARM_CACHED;
+        // zero-copy arm: no copy, the transform kernel reads the host blob itself (with the weights already on the
+        // device, or when the raw copy has to stay for warm runs, it is the raw arm)
+        const bool zc = has_xf && ch.cached == NNV_ARM_ZERO_COPY && !resident && !wc;
         const uint64_t rbytes = raw_weight_bytes(L), tbytes = transformed_bytes(*p, i, ch.variant, ch.math);
         if (wc) {
             // raw weights and biases are read straight into the copy that stays; a kernel that is also
@@ -293,7 +312,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             cudaStream_t ps = queue_of[i] == 0 ? s_exec : s_prep[queue_of[i] - 1];
             if (before_read) NNV_TRY((*before_read)(i));
             if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), ps));
-            if (cached) {
+            if (zc) {
+                // nothing to copy but the bias
+            } else if (cached) {
                 NNV_CUDA(cudaMemcpyAsync((void*)xf, (const uint8_t*)cached_blob + coff[i], tbytes, cudaMemcpyHostToDevice, ps));
                 copied += tbytes;
             } else {
@@ -308,7 +329,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             if (has_xf && !cached) {
                 if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), ps));
                 stamp_for(i, 0);
-                NNV_TRY(do_transform(*p, i, ch.variant, ch.math, raw, (void*)xf, ps));
+                NNV_TRY(do_transform(*p, i, ch.variant, ch.math, zc ? (const uint8_t*)weights + L.w_off : raw, (void*)xf, ps, zc));
                 next_stamp() = nullptr;
                 if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), ps));
             }
@@ -323,13 +344,28 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         } else {
             // read: the staging slot is free once the layer that used it last has executed
             if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_copy, EV(conv_ids[j - depth], 2), 0));
-            if (merge) {
+            if (zc && !merge) {
+                // fused preparation on the transform stream: (bias copy,) kernel reading the pinned host weights
+                if (before_read) NNV_TRY((*before_read)(i));
+                if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
+                if (L.has_bias) {
+                    NNV_CUDA(cudaMemcpyAsync((void*)bias, (const uint8_t*)weights + L.b_off, 4ull * L.K, cudaMemcpyHostToDevice, s_xform));
+                    copied += 4ull * L.K;
+                }
+                if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 2), s_xform));
+                stamp_for(i, 0);
+                NNV_TRY(do_transform(*p, i, ch.variant, ch.math, (const uint8_t*)weights + L.w_off, (void*)xf, s_xform, true));
+                next_stamp() = nullptr;
+                if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 3), s_xform));
+                NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
+                ready = EV(i, 1);
+            } else if (merge) {
                 const CopyChunk& c = chunks[chunk_of[i]];
                 if (c.first == i) {                             // the chunk's one copy, issued with its first layer
                     for (int k = c.first; k <= c.last; ++k)
                         if (before_read && p->layers[k].op == NNV_OP_CONV) NNV_TRY((*before_read)(k));
                     if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
-                    NNV_CUDA(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, s_copy));
+                    if (!c.zero_copy) NNV_CUDA(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, s_copy));
                     for (int k = c.first; k <= c.last; ++k) {
                         const nnv_layer_desc_t& Lk = p->layers[k];
                         if (Lk.op == NNV_OP_CONV && Lk.has_bias)
@@ -342,8 +378,12 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                     std::vector<XformDesc> descs;
                     for (int k = c.first; k <= c.last; ++k) {
                         const nnv_layer_desc_t& Lk = p->layers[k];
-                        if (Lk.op != NNV_OP_CONV || !variant_has_transform(choices[k].variant) || choices[k].cached) continue;
-                        descs.push_back(make_xform_desc(*p, k, choices[k], base + A.raw_off[k], base + A.xf_off[k]));
+                        if (Lk.op != NNV_OP_CONV || !variant_has_transform(choices[k].variant) || choices[k].cached == NNV_ARM_CACHED) continue;
+                        if ((choices[k].cached == NNV_ARM_ZERO_COPY) != c.zero_copy) continue;
+                        XformDesc d = make_xform_desc(*p, k, choices[k], c.zero_copy ? (const void*)((const uint8_t*)weights + Lk.w_off)
+                                                                                   : (const void*)(base + A.raw_off[k]), base + A.xf_off[k]);
+                        d.host_src = c.zero_copy ? 1 : 0;
+                        descs.push_back(d);
                     }
                     if (!descs.empty()) {
                         NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(i, 0), 0));
@@ -355,7 +395,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                         NNV_CUDA(cudaEventRecord(EV(i, 1), s_xform));
                     }
                 }
-                copied += (cached ? tbytes : rbytes) + (L.has_bias ? 4ull * L.K : 0);
+                copied += (zc ? 0 : cached ? tbytes : rbytes) + (L.has_bias ? 4ull * L.K : 0);
                 ready = (has_xf && !cached) ? EV(c.first, 1) : EV(c.first, 0);
             } else {
             if (before_read) NNV_TRY((*before_read)(i));         // the layer's bytes have arrived from storage
@@ -382,8 +422,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             // done above, inside the bundled preparation
         } else if (grouped) {
             if (has_xf && !cached) ready = group_event[i];
-        } else if (merge) {
-            // done with the chunk's copy
+        } else if (merge || zc) {
+            // done with the chunk's copy, or by the fused preparation above
         } else if (has_xf && !cached) {
             if (ready) NNV_CUDA(cudaStreamWaitEvent(s_xform, ready, 0));
             else if (depth && j >= depth) NNV_CUDA(cudaStreamWaitEvent(s_xform, EV(conv_ids[j - depth], 2), 0));
@@ -411,7 +451,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             timings[i].h2d_bytes = copied;
             timings[i].xform_bytes = (has_xf && !cached) ? rbytes + tbytes : 0;
             timings[i].exec_flops = exec_flops(*p, i, ch.variant);
-            timings[i].choice = nnv_choice_t{ch.variant, ch.math, cached ? 1 : 0};
+            timings[i].choice = nnv_choice_t{ch.variant, ch.math, cached ? NNV_ARM_CACHED : zc ? NNV_ARM_ZERO_COPY : NNV_ARM_RAW};
         }
     }
 
@@ -447,7 +487,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             const nnv_layer_desc_t& L = p->layers[i];
             if (L.op != NNV_OP_CONV) continue;
             const nnv_choice_t ch = choices[i], wm = wc->warm[i];
-            const bool cold_read_raw = !(variant_has_transform(ch.variant) && ch.cached);
+            const bool cold_read_raw = !(variant_has_transform(ch.variant) && ch.cached == NNV_ARM_CACHED);
             const bool warm_xf = variant_has_transform(wm.variant);
             if (same_kernel(ch, wm) || (cold_read_raw && !warm_xf)) continue;     // nothing left to prepare
             uint8_t* raw = wc->d_warm + L.w_off;
@@ -531,7 +571,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             NNV_TRY(stamp(TEV(i, 4), &timings[i].exec_start_ns));
             NNV_TRY(stamp(TEV(i, 5), &timings[i].exec_end_ns));
             if (L.op != NNV_OP_CONV) continue;
-            if (!resident || queued) {
+            const bool zc_i = !queued && !resident && !wc && !merge && variant_has_transform(choices[i].variant) &&
+                              choices[i].cached == NNV_ARM_ZERO_COPY;
+            if ((!resident || queued) && !zc_i) {
                 const int hi = (merge && chunk_of[i] >= 0) ? chunks[chunk_of[i]].first : i;   // a merged copy's interval
                 NNV_TRY(stamp(TEV(hi, 0), &timings[i].h2d_start_ns));
                 NNV_TRY(stamp(TEV(hi, 1), &timings[i].h2d_end_ns));
@@ -736,8 +778,8 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
                     "the cached blob (file %llu bytes, staging %llu) is smaller than the %llu bytes these choices read",
                     (unsigned long long)c_bytes, (unsigned long long)stage_c_bytes, (unsigned long long)ctotal);
         for (int i = 0; i < n; ++i) {
-            if (p->layers[i].op != NNV_OP_CONV || !(variant_has_transform(choices[i].variant) && choices[i].cached)) continue;
-            NNV_REQUIRE(file_choices[i].cached && file_choices[i].variant == choices[i].variant && file_choices[i].math == choices[i].math &&
+            if (p->layers[i].op != NNV_OP_CONV || !(variant_has_transform(choices[i].variant) && choices[i].cached == NNV_ARM_CACHED)) continue;
+            NNV_REQUIRE(file_choices[i].cached == NNV_ARM_CACHED && file_choices[i].variant == choices[i].variant && file_choices[i].math == choices[i].math &&
                             fcoff[i] == coff[i],
                         NNV_ERR_INVALID_ARG, "layer %d: the file holds no cached weights for this kernel at the expected place", i);
         }
@@ -771,7 +813,7 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
         const nnv_layer_desc_t& L = p->layers[i];
         if (L.op != NNV_OP_CONV) continue;
         const nnv_choice_t ch = choices[i];
-        if (variant_has_transform(ch.variant) && ch.cached)
+        if (variant_has_transform(ch.variant) && ch.cached == NNV_ARM_CACHED)
             add_range(i, cached_off + coff[i], (uint8_t*)h_stage_cached + coff[i], transformed_bytes(*p, i, ch.variant, ch.math));
         else
             add_range(i, raw_off + L.w_off, (uint8_t*)h_stage_weights + L.w_off, raw_weight_bytes(L));
@@ -936,6 +978,7 @@ nnv_status_t nnv_profile(nnv_plan_t* p, const void* h_weights, uint64_t w_bytes,
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t* base = (uint8_t*)d_arena;
     const int n = (int)p->layers.size();
+    const bool host_mapped = host_blob_is_mapped(h_weights);      // the zero-copy arm needs kernels to see the host blob
     cudaEvent_t e0, e1;
     NNV_CUDA(cudaEventCreate(&e0));
     NNV_CUDA(cudaEventCreate(&e1));
@@ -996,6 +1039,7 @@ nnv_status_t nnv_profile(nnv_plan_t* p, const void* h_weights, uint64_t w_bytes,
                     const uint64_t tbytes = transformed_bytes(*p, i, v, m);
                     if (has_xf) {
                         NNV_TRY(timed([&]() { return do_transform(*p, i, v, m, base + A.raw, base + A.xf, st); }, &c.xform_ns));
+                        if (host_mapped) NNV_TRY(timed([&]() { return do_transform(*p, i, v, m, hsrc, base + A.xf, st, true); }, &c.zc_ns));
                         // the cached blob is `tbytes` long; time a copy of that many bytes (scaled when the
                         // host blob is shorter than the layer's transformed weights)
                         const uint64_t cp = std::min<uint64_t>(tbytes, w_bytes);

@@ -267,7 +267,7 @@ nnv_status_t layout_arena(const nnv_plan& p, const nnv_choice_t* choices, int de
             if (L.op != NNV_OP_CONV) continue;
             a.raw_off[i] = raw_region + (L.w_off - lo);
             a.bias_off[i] = L.has_bias ? raw_region + (L.b_off - lo) : raw_region;
-            const bool cached = variant_has_transform(choices[i].variant) && choices[i].cached;
+            const bool cached = variant_has_transform(choices[i].variant) && choices[i].cached == NNV_ARM_CACHED;
             a.xf_off[i] = cached ? cached_region + coff[i] : take(transformed_bytes(p, i, choices[i].variant, choices[i].math));
         }
     } else {
@@ -300,8 +300,10 @@ nnv_status_t gather_options(const nnv_plan& p, int layer, const nnv_cost_t* cost
                         math_valid_for(c.variant, c.math),
                     NNV_ERR_INVALID_ARG, "cost row %d names a kernel layer %d cannot use", i, layer);
         opts->push_back({c.variant, c.math, 0, c.h2d_raw_ns + c.xform_ns, c.exec_ns});
-        if (allow_cached && variant_has_transform(c.variant))
-            opts->push_back({c.variant, c.math, 1, c.h2d_cached_ns, c.exec_ns});
+        if ((allow_cached & 1) && variant_has_transform(c.variant))
+            opts->push_back({c.variant, c.math, NNV_ARM_CACHED, c.h2d_cached_ns, c.exec_ns});
+        if ((allow_cached & 2) && variant_has_transform(c.variant) && c.zc_ns > 0)
+            opts->push_back({c.variant, c.math, NNV_ARM_ZERO_COPY, c.zc_ns, c.exec_ns});
     }
     return NNV_OK;
 }
@@ -471,7 +473,11 @@ nnv_status_t nnv_cached_layout(const nnv_plan_t* p, const nnv_choice_t* choices,
         offsets[i] = 0;
         if (p->layers[i].op != NNV_OP_CONV) continue;
         NNV_TRY(check_choice(*p, i, choices[i].variant, choices[i].math));
-        if (!choices[i].cached) continue;
+        NNV_REQUIRE(choices[i].cached >= NNV_ARM_RAW && choices[i].cached <= NNV_ARM_ZERO_COPY, NNV_ERR_INVALID_ARG,
+                    "layer %d: %d is not a preparation arm", i, choices[i].cached);
+        NNV_REQUIRE(choices[i].cached == NNV_ARM_RAW || variant_has_transform(choices[i].variant), NNV_ERR_INVALID_ARG,
+                    "layer %d: variant %d has no transform to cache or fuse", i, choices[i].variant);
+        if (choices[i].cached != NNV_ARM_CACHED) continue;
         NNV_REQUIRE(variant_has_transform(choices[i].variant), NNV_ERR_INVALID_ARG,
                     "layer %d: variant %d has no transform to cache", i, choices[i].variant);
         offsets[i] = pos;

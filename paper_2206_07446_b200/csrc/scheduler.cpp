@@ -355,12 +355,15 @@ nnv_status_t nnv_calibrate_costs(const nnv_plan_t* p, const nnv_cost_t* costs, i
         NNV_REQUIRE(t.h2d_end_ns >= t.h2d_start_ns && t.xform_end_ns >= t.xform_start_ns && t.exec_end_ns >= t.exec_start_ns,
                     NNV_ERR_INVALID_ARG, "layer %d: a timing interval ends before it starts", i);
         const bool has_xf = variant_has_transform(choices[i].variant);
-        const bool cached = has_xf && choices[i].cached;
-        num[0] += t.h2d_end_ns - t.h2d_start_ns;
-        den[0] += cached ? row->h2d_cached_ns : row->h2d_raw_ns;
+        const bool cached = has_xf && choices[i].cached == NNV_ARM_CACHED;
+        const bool zc = has_xf && choices[i].cached == NNV_ARM_ZERO_COPY;
+        if (!zc) {                                               // a zero-copy preparation has no read of its own:
+            num[0] += t.h2d_end_ns - t.h2d_start_ns;             // it is measured, and rescaled, as a transform
+            den[0] += cached ? row->h2d_cached_ns : row->h2d_raw_ns;
+        }
         if (has_xf && !cached) {
             num[1] += t.xform_end_ns - t.xform_start_ns;
-            den[1] += row->xform_ns;
+            den[1] += zc ? row->zc_ns : row->xform_ns;
         }
         num[2] += t.exec_end_ns - t.exec_start_ns;
         den[2] += row->exec_ns;
@@ -374,6 +377,7 @@ nnv_status_t nnv_calibrate_costs(const nnv_plan_t* p, const nnv_cost_t* costs, i
         c.h2d_raw_ns = scale(c.h2d_raw_ns, 0);
         c.h2d_cached_ns = scale(c.h2d_cached_ns, 0);
         c.xform_ns = scale(c.xform_ns, 1);
+        c.zc_ns = scale(c.zc_ns, 1);
         c.exec_ns = scale(c.exec_ns, 2);
         out[r] = c;
     }
@@ -404,7 +408,8 @@ static nnv_status_t schedule_impl(const nnv_plan_t* p, const nnv_cost_t* costs, 
                 uint64_t rd = 0;
                 for (int r = 0; r < n_costs; ++r)
                     if (costs[r].layer == i && costs[r].variant == o.variant && costs[r].math == o.math) {
-                        rd = o.cached ? costs[r].h2d_cached_ns : costs[r].h2d_raw_ns;
+                        // a zero-copy preparation holds the link for its whole length
+                        rd = o.cached == NNV_ARM_CACHED ? costs[r].h2d_cached_ns : o.cached == NNV_ARM_ZERO_COPY ? costs[r].zc_ns : costs[r].h2d_raw_ns;
                         break;
                     }
                 reads[i].push_back(rd);

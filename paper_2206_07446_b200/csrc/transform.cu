@@ -99,7 +99,7 @@ template <> struct FtNF<__nv_bfloat16> { static constexpr int value = 8; };
 // threads of a quarter warp then touch all 32 banks once).
 template <int M_, typename OutT, int NF>
 __device__ __forceinline__ void filter_transform_block(const float* __restrict__ g, OutT* __restrict__ U, int K, int C,
-                                                       int Cp, unsigned block, float* sg) {
+                                                       int Cp, unsigned block, float* sg, bool late_wait) {
     constexpr int A = WinoG<M_>::A;
     constexpr int ACTIVE = FT_FILTERS / NF;                       // threads that transform
     const long long F = (long long)K * Cp;                      // padded filter count = plane size
@@ -118,6 +118,9 @@ __device__ __forceinline__ void filter_transform_block(const float* __restrict__
         }
         __syncthreads();
     }
+    // Weights read in place from host memory do not depend on the previous kernel of the stream: those loads were
+    // issued above, before this wait (which then only orders the stores below).
+    if (late_wait) pdl_wait();
     if ((int)threadIdx.x >= ACTIVE || f0 >= F) return;
 
     float w[NF][9];
@@ -181,35 +184,38 @@ constexpr int XF_SMEM_FLOATS = FT_FILTERS * 9;                   // 36 KB stagin
 
 template <int M_, typename OutT, int NF>
 __global__ void __launch_bounds__(FT_THREADS)
-filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp, unsigned long long* stamp) {
-    pdl_enter();
+filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K, int C, int Cp, unsigned long long* stamp,
+                        int host_src) {
+    pdl_trigger();
+    if (!host_src) pdl_wait();
     if (threadIdx.x == 0) stamp_start(stamp);
     __shared__ __align__(16) float sg[XF_SMEM_FLOATS];
-    filter_transform_block<M_, OutT, NF>(g, U, K, C, Cp, blockIdx.x, sg);
+    filter_transform_block<M_, OutT, NF>(g, U, K, C, Cp, blockIdx.x, sg, host_src != 0);
     __syncthreads();
     if (threadIdx.x == 0) stamp_end(stamp);
 }
 
 template <int M_, typename OutT>
-static nnv_status_t launch_ft(const float* g, void* U, int K, int C, int Cp, cudaStream_t st) {
+static nnv_status_t launch_ft(const float* g, void* U, int K, int C, int Cp, cudaStream_t st, bool host_src) {
     constexpr int NF = FtNF<OutT>::value;
     const long long F = (long long)K * Cp;
     const unsigned grid = (unsigned)((F + FT_FILTERS - 1) / FT_FILTERS);
     unsigned long long* stamp = next_stamp();
     next_stamp() = nullptr;
-    NNV_LAUNCH((filter_transform_kernel<M_, OutT, NF>), grid, FT_THREADS, 0, st, g, reinterpret_cast<OutT*>(U), K, C, Cp, stamp);
+    NNV_LAUNCH((filter_transform_kernel<M_, OutT, NF>), grid, FT_THREADS, 0, st, g, reinterpret_cast<OutT*>(U), K, C, Cp, stamp,
+               host_src ? 1 : 0);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
 
 nnv_status_t launch_filter_transform(int m, bool bf16, const float* g, void* U, int K, int C, int Cp,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, bool host_src) {
     switch (m) {
-        case 2: return bf16 ? launch_ft<2, __nv_bfloat16>(g, U, K, C, Cp, st) : launch_ft<2, float>(g, U, K, C, Cp, st);
+        case 2: return bf16 ? launch_ft<2, __nv_bfloat16>(g, U, K, C, Cp, st, host_src) : launch_ft<2, float>(g, U, K, C, Cp, st, host_src);
         // F(4,3) and F(6,3) exist with fp32 U only: their tile GEMM multiplies fp32 operands (one bf16 pass in
         // those domains misses the output tolerance of the bf16 class)
-        case 4: NNV_REQUIRE(!bf16, NNV_ERR_UNSUPPORTED, "F(4x4,3x3) has no bf16 filter transform"); return launch_ft<4, float>(g, U, K, C, Cp, st);
-        case 6: NNV_REQUIRE(!bf16, NNV_ERR_UNSUPPORTED, "F(6x6,3x3) has no bf16 filter transform"); return launch_ft<6, float>(g, U, K, C, Cp, st);
+        case 4: NNV_REQUIRE(!bf16, NNV_ERR_UNSUPPORTED, "F(4x4,3x3) has no bf16 filter transform"); return launch_ft<4, float>(g, U, K, C, Cp, st, host_src);
+        case 6: NNV_REQUIRE(!bf16, NNV_ERR_UNSUPPORTED, "F(6x6,3x3) has no bf16 filter transform"); return launch_ft<6, float>(g, U, K, C, Cp, st, host_src);
         default: return fail(NNV_ERR_INVALID_ARG, "no Winograd tile size %d", m);
     }
 }
@@ -268,7 +274,7 @@ __host__ __device__ inline bool pack_fast(int C, int RS) {
 
 template <typename OutT>
 __device__ __forceinline__ void pack_fast_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS,
-                                                int Qp, unsigned block, float* sg) {
+                                                int Qp, unsigned block, float* sg, bool late_wait) {
     const long long F = (long long)K * C;
     const long long f_block = (long long)block * PACK_NF;
     const int nf = (int)min((long long)PACK_NF, F - f_block);    // multiple of 64
@@ -277,6 +283,7 @@ __device__ __forceinline__ void pack_fast_block(const float* __restrict__ w, Out
     const int nv = nf * RS / 4;
     for (int i = threadIdx.x; i < nv; i += PACK_THREADS) dst[i] = __ldg(src + i);
     __syncthreads();
+    if (late_wait) pdl_wait();                                    // host weights were loaded above; only the stores wait
     const int Cb = min(C, PACK_NF);                               // channels of one k row inside this block
     const int k0 = (int)(f_block / C), cbase = (int)(f_block - (long long)k0 * C);
     // Write-out.  A row is one (k, rs) pair: Cb consecutive output elements.  A warp takes four
@@ -303,11 +310,12 @@ __device__ __forceinline__ void pack_fast_block(const float* __restrict__ w, Out
 
 template <typename OutT>
 __device__ __forceinline__ void pack_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp,
-                                           unsigned block, float* smem) {
+                                           unsigned block, float* smem, bool late_wait) {
     if (pack_fast(C, RS)) {
-        pack_fast_block<OutT>(w, P, K, C, RS, Qp, block, smem);
+        pack_fast_block<OutT>(w, P, K, C, RS, Qp, block, smem, late_wait);
         return;
     }
+    if (late_wait) pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int CH = pack_ch(RS), upr = pack_units_per_row(C, RS);
     const long long unit = (long long)block * PACK_WARPS + warp;
@@ -336,7 +344,7 @@ __device__ __forceinline__ void pack_block(const float* __restrict__ w, OutT* __
 // PACK1X1_PER_BLOCK consecutive elements of P.
 template <typename OutT>
 __device__ __forceinline__ void pack1x1_block(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp,
-                                              unsigned block) {
+                                              unsigned block, bool late_wait) {
     const long long n = (long long)K * Qp;
     const long long base = (long long)block * PACK1X1_PER_BLOCK;
     if (C == Qp) {                                              // no padding: a straight conversion copy, 4 at a time
@@ -346,12 +354,14 @@ __device__ __forceinline__ void pack1x1_block(const float* __restrict__ w, OutT*
             const long long i = base + ((long long)u * PACK_THREADS + threadIdx.x) * 4;
             if (i < n) v[u] = __ldg(reinterpret_cast<const float4*>(w + i));
         }
+        if (late_wait) pdl_wait();
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const long long i = base + ((long long)u * PACK_THREADS + threadIdx.x) * 4;
             if (i < n) store4<OutT>(P + i, v[u].x, v[u].y, v[u].z, v[u].w);
         }
     } else {
+        if (late_wait) pdl_wait();
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
             const long long i = base + (long long)u * PACK_THREADS + threadIdx.x;
@@ -365,21 +375,23 @@ __device__ __forceinline__ void pack1x1_block(const float* __restrict__ w, OutT*
 
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
-pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp, unsigned long long* stamp) {
-    pdl_enter();
+pack_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int RS, int Qp, unsigned long long* stamp, int host_src) {
+    pdl_trigger();
+    if (!host_src) pdl_wait();
     if (threadIdx.x == 0) stamp_start(stamp);
     __shared__ __align__(16) float sw[PACK_SMEM_FLOATS];
-    pack_block<OutT>(w, P, K, C, RS, Qp, blockIdx.x, sw);
+    pack_block<OutT>(w, P, K, C, RS, Qp, blockIdx.x, sw, host_src != 0);
     __syncthreads();
     if (threadIdx.x == 0) stamp_end(stamp);
 }
 
 template <typename OutT>
 __global__ void __launch_bounds__(PACK_THREADS)
-pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp, unsigned long long* stamp) {
-    pdl_enter();
+pack1x1_kernel(const float* __restrict__ w, OutT* __restrict__ P, int K, int C, int Qp, unsigned long long* stamp, int host_src) {
+    pdl_trigger();
+    if (!host_src) pdl_wait();
     if (threadIdx.x == 0) stamp_start(stamp);
-    pack1x1_block<OutT>(w, P, K, C, Qp, blockIdx.x);
+    pack1x1_block<OutT>(w, P, K, C, Qp, blockIdx.x, host_src != 0);
     __syncthreads();
     if (threadIdx.x == 0) stamp_end(stamp);
 }
@@ -398,7 +410,9 @@ __host__ __device__ inline int xform_group(int kind) {
 template <int GROUP>
 __global__ void __launch_bounds__(FT_THREADS)
 multi_transform_kernel(const __grid_constant__ XformBatch batch) {
-    pdl_enter();
+    pdl_trigger();
+    const bool late = batch.host_src != 0;                      // sources in host memory: load first, wait before the stores
+    if (!late) pdl_wait();
     if (threadIdx.x == 0) stamp_start(batch.stamp);
     __shared__ __align__(16) float smem[XF_SMEM_FLOATS];
     const unsigned vb = blockIdx.x;
@@ -410,21 +424,21 @@ multi_transform_kernel(const __grid_constant__ XformBatch batch) {
     const float* src = static_cast<const float*>(d.src);
     if constexpr (GROUP == XG_PACK) {
         switch (d.kind * 2 + d.bf16) {
-            case XF_PACK * 2: pack_block<float>(src, (float*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem); break;
-            case XF_PACK * 2 + 1: pack_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem); break;
-            case XF_PACK1X1 * 2: pack1x1_block<float>(src, (float*)d.dst, d.K, d.C, d.Qp, lb); break;
-            case XF_PACK1X1 * 2 + 1: pack1x1_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Qp, lb); break;
+            case XF_PACK * 2: pack_block<float>(src, (float*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem, late); break;
+            case XF_PACK * 2 + 1: pack_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.RS, d.Qp, lb, smem, late); break;
+            case XF_PACK1X1 * 2: pack1x1_block<float>(src, (float*)d.dst, d.K, d.C, d.Qp, lb, late); break;
+            case XF_PACK1X1 * 2 + 1: pack1x1_block<__nv_bfloat16>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Qp, lb, late); break;
             default: break;
         }
     } else if constexpr (GROUP == XG_WINO_SMALL) {
         switch (d.kind * 2 + d.bf16) {
-            case XF_WINO2 * 2: filter_transform_block<2, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
-            case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 8>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
-            case XF_WINO4 * 2: filter_transform_block<4, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem); break;
+            case XF_WINO2 * 2: filter_transform_block<2, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
+            case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 8>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
+            case XF_WINO4 * 2: filter_transform_block<4, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
             default: break;
         }
     } else {
-        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem);
+        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late);
     }
     __syncthreads();
     if (threadIdx.x == 0) stamp_end(batch.stamp);
@@ -449,6 +463,7 @@ nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st) {
     for (int grp = 0; grp < XG_COUNT; ++grp) {
         XformBatch b;
         b.stamp = stamp;
+        b.host_src = (n > 0 && descs[0].host_src) ? 1 : 0;      // a batch is all device or all host sources
         b.n = 0;
         int blocks = 0;
         auto flush = [&]() -> nnv_status_t {
@@ -477,19 +492,20 @@ nnv_status_t launch_transform_batch(XformDesc* descs, int n, cudaStream_t st) {
     return NNV_OK;
 }
 
-nnv_status_t launch_pack(bool bf16, const float* w, void* P, int K, int C, int RS, int Qp, cudaStream_t st) {
+nnv_status_t launch_pack(bool bf16, const float* w, void* P, int K, int C, int RS, int Qp, cudaStream_t st, bool host_src) {
+    const int hs = host_src ? 1 : 0;
     unsigned long long* stamp = next_stamp();
     next_stamp() = nullptr;
     if (RS == 1) {
         const long long n = (long long)K * Qp;
         const unsigned grid = (unsigned)((n + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
-        if (bf16) NNV_LAUNCH((pack1x1_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, Qp, stamp);
-        else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp, stamp);
+        if (bf16) NNV_LAUNCH((pack1x1_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, Qp, stamp, hs);
+        else NNV_LAUNCH((pack1x1_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, Qp, stamp, hs);
     } else {
         NNV_REQUIRE(8 * RS <= PACK_SLICE, NNV_ERR_UNSUPPORTED, "filter window of %d taps is too large to repack", RS);
         const unsigned grid = (unsigned)pack_blocks(K, C, RS);
-        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, RS, Qp, stamp);
-        else NNV_LAUNCH((pack_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, RS, Qp, stamp);
+        if (bf16) NNV_LAUNCH((pack_kernel<__nv_bfloat16>), grid, PACK_THREADS, 0, st, w, (__nv_bfloat16*)P, K, C, RS, Qp, stamp, hs);
+        else NNV_LAUNCH((pack_kernel<float>), grid, PACK_THREADS, 0, st, w, (float*)P, K, C, RS, Qp, stamp, hs);
     }
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;

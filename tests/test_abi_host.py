@@ -75,7 +75,8 @@ def _random_costs(layers, rng, hi=50):
                     continue
                 costs.append(dict(layer=i, variant=v, math=m, h2d_raw_ns=int(rng.integers(0, hi)),
                                   xform_ns=int(rng.integers(0, hi)) if osel.has_transform(v) else 0,
-                                  h2d_cached_ns=int(rng.integers(0, hi)), exec_ns=int(rng.integers(0, hi))))
+                                  h2d_cached_ns=int(rng.integers(0, hi)), exec_ns=int(rng.integers(0, hi)),
+                                  zc_ns=int(rng.integers(0, 2 * hi)) if (osel.has_transform(v) and rng.random() < 0.7) else 0))
     return costs
 
 
@@ -85,7 +86,7 @@ def test_selection_matches_oracle_bit_exact(seed):
     layers = [wl.tiny_net, wl.cfg2_resnet18, wl.cfg3_mobilenetv2, wl.cfg5_vgg16][seed % 4]()
     plan = _plan(layers)
     costs = _random_costs(layers, rng, hi=8 if seed % 2 else 10 ** 9)
-    for allow in (0, 1):
+    for allow in (0, 1, 2, 3):                              # bit 0: cached arm, bit 1: zero-copy arm
         assert nb.nnv_select_kernels(plan, costs, allow) == osel.select_kernels(layers, costs, allow)
         for i, L in enumerate(layers):
             if L["op"] != wl.OP_CONV:

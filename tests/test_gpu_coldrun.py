@@ -268,3 +268,50 @@ def test_kernel_stamps_measure_without_changing_the_result():
         assert sum(1 for i in convs if xf[i] > 0) >= 1 and all(v < total for v in xf)
         if depth:                                              # one transform launch per layer
             assert all(xf[i] > 0 for i in convs[1:])
+
+
+def test_zero_copy_arm_is_bitwise_the_raw_arm():
+    """The third preparation arm: the transform kernels read the raw weights in place in pinned host memory.  Same
+    kernels, same arithmetic, same bytes out: the result equals the copy-then-transform run bit for bit at every
+    depth, on the scheduled queues and fed from a model file; only biases are still copied; layers without a
+    transform cannot take the arm."""
+    layers = wl.tiny_net()
+    model, ws, bs, x = _model(layers, seed=4)
+    raw = _choices(model, [nb.VAR_WINO_F4, nb.VAR_GEMM1X1, nb.VAR_IM2COL], nb.MATH_TF32)
+    zc = [None if c is None else (c[0], c[1], nb.ARM_ZERO_COPY if c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else 0) for c in raw]
+    assert any(c is not None and c[2] == nb.ARM_ZERO_COPY for c in zc)
+    y_raw, _ = model.cold_run(x, raw, depth=2)
+    for depth in (0, 1, 3):
+        y, tm = model.cold_run(x, zc, depth=depth, want_timings=True)
+        assert np.array_equal(y.view(np.uint32), y_raw.view(np.uint32)), depth
+        for i, L in enumerate(layers):
+            if zc[i] is None:
+                continue
+            if zc[i][2] == nb.ARM_ZERO_COPY:
+                assert tm[i]["choice"][2] == nb.ARM_ZERO_COPY
+                assert tm[i]["h2d_bytes"] == (4 * L["K"] if L["has_bias"] else 0)        # no weight copy
+                assert tm[i]["xform_bytes"] > 0 and tm[i]["exec_start_ns"] >= tm[i]["xform_end_ns"]
+            else:
+                assert tm[i]["h2d_bytes"] >= 4 * L["K"] * (L["C"] // L["groups"]) * L["R"] * L["S"]
+    q = [(-1 if c is None else (i % 3)) for i, c in enumerate(zc)]
+    q[next(i for i, c in enumerate(zc) if c is not None)] = 0
+    y_q, _ = model.cold_run_queues(x, zc, q, 2)
+    assert np.array_equal(y_q.view(np.uint32), y_raw.view(np.uint32))
+    bad = list(zc)
+    dw = next((i for i, c in enumerate(raw) if c is not None and c[0] in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE)), None)
+    if dw is not None:
+        bad[dw] = (raw[dw][0], raw[dw][1], nb.ARM_ZERO_COPY)
+        with pytest.raises(nb.NnvError):
+            model.cold_run(x, bad, depth=0)
+    # a larger model: ResNet-18-shaped, mixed arms picked by the selection on the profiled table
+    layers = wl.cfg2_resnet18()
+    model, ws, bs, x = _model(layers)
+    costs = model.profile(x, reps=3)
+    assert all(c["zc_ns"] > 0 for c in costs if c["variant"] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE))
+    mixed = nb.nnv_select_kernels(model.plan, costs, 2)
+    same_raw = [None if c is None else (c[0], c[1], 0) for c in mixed]
+    y_m, _ = model.cold_run(x, mixed, depth=0)
+    y_r, _ = model.cold_run(x, same_raw, depth=0)
+    assert np.array_equal(y_m.view(np.uint32), y_r.view(np.uint32))
+    print("zero-copy layers chosen:", sum(1 for c in mixed if c is not None and c[2] == nb.ARM_ZERO_COPY), "of",
+          sum(1 for c in mixed if c is not None))

@@ -141,3 +141,24 @@ def test_warm_selection_and_switch_set_properties():
             differs = (cold[i][0], cold[i][1]) != (warm[i][0], warm[i][1])
             assert (i in sw) == (differs and warm[i][0] != sel.DIRECT)
         assert sel.switch_set(warm, warm) == []
+
+
+def test_third_arm_fused_read_and_transform():
+    """The zero-copy arm (rank 2): offered only when allowed (bit 1) and profiled (zc_ns > 0), for kernels with a
+    transform; it competes on prep = zc_ns.  Hand table: one layer, two kernels."""
+    rows = [dict(variant=sel.IM2COL, math=sel.TF32, h2d_raw_ns=70, xform_ns=30, h2d_cached_ns=90, exec_ns=50, zc_ns=80),
+            dict(variant=sel.DIRECT, math=sel.FP32, h2d_raw_ns=70, xform_ns=0, h2d_cached_ns=70, exec_ns=200, zc_ns=40)]
+    ranks = lambda allow: [o[0] for o in sel.options_from_costs(rows, allow)]
+    assert ranks(0) == [(sel.IM2COL, sel.TF32, 0), (sel.DIRECT, sel.FP32, 0)]
+    assert ranks(1) == [(sel.IM2COL, sel.TF32, 0), (sel.IM2COL, sel.TF32, 1), (sel.DIRECT, sel.FP32, 0)]
+    assert ranks(2) == [(sel.IM2COL, sel.TF32, 0), (sel.IM2COL, sel.TF32, 2), (sel.DIRECT, sel.FP32, 0)]   # DIRECT: no transform, no arm
+    assert len(ranks(3)) == 4
+    # raw: 70 + 30 + 50 = 150; cached: 90 + 50 = 140; fused: 80 + 50 = 130
+    assert sel.choose(sel.options_from_costs(rows, 0))[0] == (sel.IM2COL, sel.TF32, 0)
+    assert sel.choose(sel.options_from_costs(rows, 1))[0] == (sel.IM2COL, sel.TF32, 1)
+    assert sel.choose(sel.options_from_costs(rows, 3))[0] == (sel.IM2COL, sel.TF32, 2)
+    # the fused arm dominates the raw arm of its kernel (80 <= 100, same execution): the filter drops the raw one
+    surv = [o[0] for o in sel.pareto_filter(sel.options_from_costs(rows, 2))]
+    assert (sel.IM2COL, sel.TF32, 2) in surv and (sel.IM2COL, sel.TF32, 0) not in surv
+    rows[0]["zc_ns"] = 0                                       # not profiled: not offered
+    assert ranks(3) == ranks(1)
