@@ -61,6 +61,7 @@ def parse():
     ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run (0 = skip)")
     ap.add_argument("--continuous-reps", type=int, default=10, help="cold + warm sequences for the kernel-switching report (0 = skip)")
     ap.add_argument("--file-reps", type=int, default=5, help="cold runs fed from a model file on local storage (0 = skip)")
+    ap.add_argument("--also", default="cfg2_resnet18,cfg5_vgg16", help="other workloads measured beside --config (headline, e2e and rooflines only)")
     ap.add_argument("--minimal", action="store_true", help="headline + e2e + rooflines only (no side arms or sections)")
     ap.add_argument("--save-costs", default=None, help="write the profiled cost table (JSON) to this file")
     ap.add_argument("--load-costs", default=None, help="use a cost table saved earlier instead of profiling (e.g. under a profiler)")
@@ -302,7 +303,6 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2206_07446_b200 import binding as nb
-    from paper_2206_07446_b200 import harness
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -314,6 +314,33 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     if args.tuning:
         nb.nnv_tuning_set(args.tuning)
+    line = measure(args, args.config, args.steps, args.warmup, args.minimal, rank, world, local)
+    # the other single-GPU configurations, headline numbers and rooflines only, beside the main workload
+    others = {}
+    for name in [c for c in args.also.split(",") if c and c != args.config]:
+        o = measure(args, name, args.arm_steps, 3, True, rank, world, local)
+        others[name] = {k: o[k] for k in ("value", "unit", "steps", "e2e", "roofline", "roofline_transform", "transform_all", "run", "per_layer")}
+        others[name]["e2e"] = {k: o["e2e"][k] for k in ("value", "h2d_bytes_per_step", "host_link")}
+    line["other_workloads"] = others
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure(args, config, steps, warmup, minimal, rank, world, local):
+    """All measurements of one workload; returns the JSON line as a dict."""
+    import torch
+    import torch.distributed as dist
+    from paper_2206_07446_b200 import binding as nb
+    from paper_2206_07446_b200 import harness
+
+    class _A:                                                  # the arguments with this call's workload and step counts
+        pass
+    a2 = _A()
+    a2.__dict__.update(vars(args))
+    a2.config, a2.steps, a2.warmup, a2.minimal = config, steps, warmup, minimal
+    args = a2
 
     layers = wl.CONFIGS[args.config]()
     ws, bs = wl.make_weights(layers)
@@ -387,7 +414,7 @@ def run_ours(args):
         begin(k, timed, (s_copy, s_xform))
         ch = nb.nnv_select_kernels(model.plan, costs, 0)      # the selection call belongs to the cold inference
         nb.nnv_cold_run_dio(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
-                            model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+                            model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
         if timed:
             ev1[k].record(s_exec)
             return nb.nnv_kernel_times(model.plan)            # the kernels' own device-clock stamps of this step
@@ -405,7 +432,7 @@ def run_ours(args):
         t0 = time.perf_counter()
         ch = nb.nnv_select_kernels(model.plan, costs, 0)
         nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
-                        model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+                        model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
         if timed:
             ev1[k].record(s_exec)
             wall.append(time.perf_counter() - t0)
@@ -423,7 +450,7 @@ def run_ours(args):
             begin(k, timed, (s_copy, s_xform))
             ch = nb.nnv_select_kernels(model.plan, costs, 1)
             nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes, model.h_input,
-                            model.h_output, model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+                            model.h_output, model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
             if timed:
                 ev1[k].record(s_exec)
 
@@ -438,10 +465,12 @@ def run_ours(args):
         choices_zc_all = [None if c is None else (c[0], c[1], nb.ARM_ZERO_COPY if c[0] not in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else 0)
                           for c in choices_raw]
         for name, chz in (("zero_copy_allowed", choices_zc), ("zero_copy_every_layer", choices_zc_all)):
+            need = max(need, model.ensure_arena(chz, args.cold_depth))
+
             def step_zc(k, timed, chz=chz):
                 begin(k, timed, (s_copy, s_xform))
                 nb.nnv_cold_run(model.plan, chz, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
-                                model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+                                model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
                 if timed:
                     ev1[k].record(s_exec)
 
@@ -462,7 +491,7 @@ def run_ours(args):
             begin(k, timed, (s_copy, s_xform))
             ch = nb.nnv_select_kernels(plan_g, costs, 0)
             nb.nnv_cold_run(plan_g, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
-                            model.arena, need, s_copy, s_xform, s_exec, args.cold_depth)
+                            model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
             if timed:
                 ev1[k].record(s_exec)
 
@@ -474,7 +503,7 @@ def run_ours(args):
             begin(k, timed, (s_xform,))
             ch = nb.nnv_select_kernels(plan_g, costs_res, 0)
             nb.nnv_resident_run(plan_g, ch, model.d_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
-                                model.arena, need, s_xform, s_exec, args.depth)
+                                model.arena, model.arena.numel(), s_xform, s_exec, args.depth)
             if timed:
                 ev1[k].record(s_exec)
 
@@ -492,7 +521,7 @@ def run_ours(args):
         def step_sched(k, timed):
             begin(k, timed, st_s[1:])
             nb.nnv_cold_run_queues(model.plan, ch_s, q_s, args.queues, model.h_weights, model.w_bytes, None, 0,
-                                   model.h_input, model.h_output, model.arena, need_s, st_s)
+                                   model.h_input, model.h_output, model.arena, model.arena.numel(), st_s)
             if timed:
                 ev1[k].record(s_exec)
 
@@ -529,7 +558,7 @@ def run_ours(args):
             s_copy.wait_event(evs[0])
             s_xform.wait_event(evs[0])
             nb.nnv_cold_run_continuous(model.plan, choices_raw, warm, model.h_weights, model.w_bytes, None, 0,
-                                       model.h_input, model.h_output, model.arena, need_c, d_warm, wbytes, s_copy, s_xform, s_exec)
+                                       model.h_input, model.h_output, model.arena, model.arena.numel(), d_warm, wbytes, s_copy, s_xform, s_exec)
             evs[1].record(s_exec)
             for j in range(3):
                 nb.nnv_warm_run(model.plan, warm, d_warm, wbytes, model.w_bytes, model.h_input, model.h_output, model.arena,
@@ -730,7 +759,7 @@ def run_ours(args):
         xall["peak"] = peaks["hbm_gbs"]
         xall["frac"] = xall["achieved"] / peaks["hbm_gbs"]
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.minimal:
         from oracle import conv as oconv
         from oracle import model as omodel
         oconv.build()
@@ -748,10 +777,7 @@ def run_ours(args):
             alg1["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_s[0] - ref) ** 2)) / den)
         if cont:
             cont["parity_rel_l2_end_to_end"] = float(np.sqrt(np.sum((y_w[0] - ref) ** 2)) / den)
-    if rank == 0:
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    return line
 
 
 # ------------------------------------------------------------------------------------------------
@@ -903,6 +929,23 @@ def other_kernel_rooflines(layers, model, nb, torch, flush, peaks):
         rows.append({"kernel": "depthwise_kernel", "bound": "hbm", "layer": "%dx%d C=%d stride %d" % (L["H"], L["W"], L["C"], L["stride"]),
                      "bytes": by, "us": r["us"], "achieved": by / r["us"] / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": by / r["us"] / 1e3 / peaks["hbm_gbs"]})
+    w3 = [L for L in layers if L["op"] == wl.OP_CONV and L["groups"] == 1 and L["R"] == 3 and L["S"] == 3 and L["stride"] == 1]
+    if w3:
+        # the Winograd data transforms on the largest 3x3 / stride-1 layer, F(4x4,3x3): V and M through HBM
+        L = dict(max(w3, key=lambda L: L["C"] * L["H"] * L["W"]), in0=-1, in1=-1, has_bias=0)
+        plan = nb.Plan([L], [0], [0])
+        v = nb.VAR_WINO_F4
+        T, vb, mb = nb.nnv_wino_sizes(plan, 0, v, nb.MATH_TF32)
+        oh, ow = wl.out_hw(L)
+        d_in, d_V, d_M = _rand(torch, L["C"] * L["H"] * L["W"]), _buf(torch, vb), _rand(torch, mb // 4)
+        d_out = _buf(torch, 4 * oh * ow * L["K"])
+        us_in, _ = _time(torch, lambda st: nb.nnv_wino_input_transform(plan, 0, v, nb.MATH_TF32, d_in, d_V, st), 10, flush)
+        us_out, _ = _time(torch, lambda st: nb.nnv_wino_output_transform(plan, 0, v, d_M, None, None, d_out, st), 10, flush)
+        shape = "%dx%d C=%d K=%d, F(4x4,3x3), %d tiles" % (L["H"], L["W"], L["C"], L["K"], T)
+        for name, by, us in (("wino_input_kernel", 4 * L["C"] * L["H"] * L["W"] + vb, us_in),
+                             ("wino_output_kernel", mb + 4 * oh * ow * L["K"], us_out)):
+            rows.append({"kernel": name, "bound": "hbm", "layer": shape, "bytes": by, "us": us, "achieved": by / us / 1e3,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": by / us / 1e3 / peaks["hbm_gbs"]})
     dense = [L for L in layers if L["op"] == wl.OP_CONV and L["groups"] == 1]
     if dense:
         L = max(dense, key=lambda L: wl.out_hw(L)[0] * wl.out_hw(L)[1] * L["K"] * L["C"] * L["R"] * L["S"])

@@ -156,6 +156,8 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* plan);
  *   gemm_tile=BN,splits   column tile (16..128, multiple of 16) and K splits (1,2,4,8) of the GEMM
  *   gemm_ring=N           shared-memory ring depth 2..8        gemm_prefill=0|1
  *   conv3x3=off|auto|MT,BN,splits[,boxes,weight_tiles]          the halo-resident 3x3 kernel
+ *   conv3x3p=off|BN,ctas_per_sm[,boxes,weight_tiles]           the persistent form of the 3x3 kernel (off unless asked for)
+ *   winofused=auto|0|1    F(2x2,3x3) with TF32 math as one kernel (input transform, tile GEMMs, output transform)
  *   smallp=0|1|N          the weights-on-rows kernel for layers of at most 256 pixels: off, on, on with N K splits
  *   side=0|1  merge=0|1  group=0|1   side stream for residual branches, merged reads, grouped transforms
  * Every call replaces all settings (unnamed keys return to their defaults).  An item that does not
@@ -343,6 +345,26 @@ nnv_status_t nnv_transform_all(const nnv_plan_t* plan, const nnv_choice_t* choic
 nnv_status_t nnv_conv_exec(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
                            const void* d_in, const void* d_addend, const void* d_wt, const void* d_bias,
                            void* d_out, void* d_ws, uint64_t ws_bytes, void* stream);
+
+/* The data transforms around the Winograd tile GEMM as single operations (nnv_conv_exec with a
+ * WINO variant runs input transform, batched tile GEMM and output transform back to back; the
+ * paper's engine does the same inside its winograd kernels, Section 2 / Figure 3 name only the
+ * weight side).  Tiles of alpha x alpha input pixels at stride m, starting at -pad, zero outside
+ * the image; tile t = th * TW + tw, TH = ceil(OH / m), TW = ceil(OW / m).
+ *   nnv_wino_sizes: tiles T and the bytes of V and M for (layer, variant, math).
+ *   nnv_wino_input_transform: d_in NHWC fp32 -> d_V[xi*alpha+nu][t][cp] = (B^T d B)[xi][nu], cp < Cp
+ *       (entries with cp >= C are +0); element type fp32, or bf16 with BF16 math; for F(2x2,3x3)
+ *       with TF32 math the fp32 words are rounded to TF32 precision (nearest even), since one TF32
+ *       pass multiplies them.
+ *   nnv_wino_output_transform: d_M[xi*alpha+nu][t][k] fp32 -> d_out NHWC fp32: each tile's
+ *       A^T M A, clipped to the output grid, + bias + addend, then the layer's activation.
+ * Asynchronous on `stream`; pointers 256-byte aligned. */
+nnv_status_t nnv_wino_sizes(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
+                            int32_t* tiles, uint64_t* v_bytes, uint64_t* m_bytes);
+nnv_status_t nnv_wino_input_transform(const nnv_plan_t* plan, int32_t layer, int32_t variant, int32_t math,
+                                      const void* d_in, void* d_V, void* stream);
+nnv_status_t nnv_wino_output_transform(const nnv_plan_t* plan, int32_t layer, int32_t variant,
+                                       const void* d_M, const void* d_addend, const void* d_bias, void* d_out, void* stream);
 
 /* nnv_conv_exec without a scratch argument.  (The paper has no counterpart to
  * this call; it is a convenience of this library.)  It is for callers that cannot

@@ -88,6 +88,9 @@ _SIGS = {
     "nnv_transform_all": [_vp, _P(Choice), _vp, _u64, _vp, _u64, _vp],
     "nnv_conv_exec": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _u64, _vp],
     "nnv_conv_exec_static": [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp],
+    "nnv_wino_sizes": [_vp, _i32, _i32, _i32, _P(_i32), _P(_u64), _P(_u64)],
+    "nnv_wino_input_transform": [_vp, _i32, _i32, _i32, _vp, _vp, _vp],
+    "nnv_wino_output_transform": [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp],
     "nnv_pool_exec": [_vp, _i32, _vp, _vp, _vp],
     "nnv_chw_to_hwc": [_vp, _vp, _i32, _i32, _i32, _vp],
     "nnv_hwc_to_chw": [_vp, _vp, _i32, _i32, _i32, _vp],
@@ -407,6 +410,22 @@ def nnv_conv_exec_static(plan, layer, variant, math, d_in, d_addend, d_wt, d_bia
     inside the library (STATIC_SCRATCH_BYTES); nothing is allocated by this call."""
     _check(_lib.nnv_conv_exec_static(plan.handle, layer, variant, math, _ptr(d_in), _ptr(d_addend), _ptr(d_wt),
                                      _ptr(d_bias), _ptr(d_out), _stream(stream)))
+
+
+def nnv_wino_sizes(plan, layer, variant, math):
+    """(tiles, bytes of V, bytes of M) of a Winograd variant of a layer."""
+    t, vb, mb = _i32(0), _u64(0), _u64(0)
+    _check(_lib.nnv_wino_sizes(plan.handle, layer, variant, math, ctypes.byref(t), ctypes.byref(vb), ctypes.byref(mb)))
+    return int(t.value), int(vb.value), int(mb.value)
+
+
+def nnv_wino_input_transform(plan, layer, variant, math, d_in, d_V, stream=None):
+    _check(_lib.nnv_wino_input_transform(plan.handle, layer, variant, math, _ptr(d_in), _ptr(d_V), _stream(stream)))
+
+
+def nnv_wino_output_transform(plan, layer, variant, d_M, d_addend, d_bias, d_out, stream=None):
+    _check(_lib.nnv_wino_output_transform(plan.handle, layer, variant, _ptr(d_M), _ptr(d_addend), _ptr(d_bias), _ptr(d_out),
+                                          _stream(stream)))
 
 
 def nnv_pool_exec(plan, layer, d_in, d_out, stream=None):

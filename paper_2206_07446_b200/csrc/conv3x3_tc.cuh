@@ -285,3 +285,212 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
     }
 }
+
+// ---- persistent form ----------------------------------------------------------------------------
+// One CTA per SM walks over the output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The rings keep
+// running from one tile into the next, so the producer is already filling tile t+1 while tile t drains; TMEM
+// holds TWO accumulators, so the MMAs of tile t+1 run while the epilogue warps read and write out tile t
+// (tmem_full / tmem_empty barriers per accumulator).  Set-up (barriers, TMEM allocation, descriptor fetch) is
+// paid once per CTA instead of once per tile.  No K split here: layers that need one take the kernel above.
+// The epilogue's per-warp staging tiles have their own shared memory, since the rings are never idle.
+struct ConvPDev {
+    unsigned long long* stamp;
+    float* D;
+    const float* bias;
+    const float* addend;
+    int C, H, W, K;
+    int BN, act, tmem_cols, na, nb, cblk, tiles_w, n_tiles, tiles_total;   // n_tiles: channel tiles; tiles_total = patches x n_tiles
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+conv3x3_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ConvPDev g) {
+    extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int BN = g.BN, NA = g.na, NB = g.nb;
+    constexpr uint32_t a_slot_bytes = 18u * 1024u;                 // (16 + 2) rows of 8 pixels x 128 bytes
+    const uint32_t b_slot_bytes = (uint32_t)BN * BK_BYTES;
+    const uint32_t a_ring = sbase, b_ring = sbase + NA * a_slot_bytes;
+    const uint32_t stage0 = b_ring + NB * b_slot_bytes;            // 4 warps x 32 rows x 36 words
+    const uint32_t bars = stage0 + 4u * 32u * 36u * 4u;
+    auto a_full = [&](int s) { return bars + 8u * s; };
+    auto a_empty = [&](int s) { return bars + 8u * (CONV_MAX_NA + s); };
+    auto b_full = [&](int s) { return bars + 8u * (2 * CONV_MAX_NA + s); };
+    auto b_empty = [&](int s) { return bars + 8u * (2 * CONV_MAX_NA + CONV_MAX_NB + s); };
+    auto t_full = [&](int a) { return bars + 8u * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + a); };
+    auto t_empty = [&](int a) { return bars + 8u * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 2 + a); };
+    const uint32_t holder = bars + 8u * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 4);
+    volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+        for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(t_full(a), 1); mbar_init(t_empty(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"((uint32_t)g.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *holder_ptr;
+    pdl_wait();                                               // set-up above overlaps the previous kernel's tail
+    if (threadIdx.x == 32) stamp_start(g.stamp);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int sa = 0, sb = 0;
+            uint32_t pa = 0, pb = 0;
+            for (int t = blockIdx.x; t < g.tiles_total && ok; t += gridDim.x) {
+                const int patch = t / g.n_tiles, nt = t - patch * g.n_tiles;
+                const int tile_h = patch / g.tiles_w, tile_w = patch - tile_h * g.tiles_w;
+                const int oh0 = tile_h * 16, ow0 = tile_w * 8, n0 = nt * BN;
+                for (int cbi = 0; cbi < g.cblk && ok; ++cbi) {
+                    const int c0 = cbi * 32;
+                    for (int s = 0; s < 3 && ok; ++s) {
+                        ok = mbar_wait(a_empty(sa), pa ^ 1u);
+                        if (!ok) break;
+                        mbar_expect_tx(a_full(sa), a_slot_bytes);
+                        tma_load_3d(a_ring + sa * a_slot_bytes, &tmA, c0, ow0 + s - 1, oh0 - 1, a_full(sa));
+                        if (++sa == NA) { sa = 0; pa ^= 1u; }
+                        for (int r = 0; r < 3; ++r) {
+                            ok = mbar_wait(b_empty(sb), pb ^ 1u);
+                            if (!ok) break;
+                            mbar_expect_tx(b_full(sb), b_slot_bytes);
+                            tma_load_3d(b_ring + sb * b_slot_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, b_full(sb));
+                            if (++sb == NB) { sb = 0; pb ^= 1u; }
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let loads already in flight land
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            int sa = 0, sb = 0;
+            uint32_t pa = 0, pb = 0;
+            int lt = 0;                                           // this CTA's tile count so far
+            for (int t = blockIdx.x; t < g.tiles_total && ok; t += gridDim.x, ++lt) {
+                const int acc = lt & 1;
+                ok = mbar_wait(t_empty(acc), (((uint32_t)lt >> 1) & 1u) ^ 1u);   // the epilogue has drained this accumulator
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
+                for (int cbi = 0; cbi < g.cblk && ok; ++cbi) {
+                    for (int s = 0; s < 3 && ok; ++s) {
+                        ok = mbar_wait(a_full(sa), pa);
+                        if (!ok) break;
+                        const uint32_t a_box = a_ring + sa * a_slot_bytes;
+                        for (int r = 0; r < 3; ++r) {
+                            ok = mbar_wait(b_full(sb), pb);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint64_t bdesc = make_smem_desc(b_ring + sb * b_slot_bytes);
+                            const uint64_t adesc = make_smem_desc(a_box + (uint32_t)r * 1024u);
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk)
+                                umma<false>(tmem_d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (cbi | s | r | kk) ? 1u : 0u);
+                            umma_commit(b_empty(sb));
+                            if (++sb == NB) { sb = 0; pb ^= 1u; }
+                        }
+                        if (ok) umma_commit(a_empty(sa));
+                        if (++sa == NA) { sa = 0; pa ^= 1u; }
+                    }
+                }
+                if (ok) umma_commit(t_full(acc));
+            }
+            if (!ok) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        }
+    } else {
+        const int quarter = warp & 3;                         // TMEM lanes this warp may read
+        const bool vec = ((g.K & 3) == 0) && ((reinterpret_cast<uintptr_t>(g.D) & 15) == 0) &&
+                         (!g.addend || (reinterpret_cast<uintptr_t>(g.addend) & 15) == 0) &&
+                         (!g.bias || (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0);
+        const uint32_t stage = stage0 + (uint32_t)quarter * (32u * 36u * 4u);
+        const int sub = lane >> 3, cc = (lane & 7) * 4;
+        int lt = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < g.tiles_total && ok; t += gridDim.x, ++lt) {
+            const int acc = lt & 1;
+            const int patch = t / g.n_tiles, nt = t - patch * g.n_tiles;
+            const int tile_h = patch / g.tiles_w, tile_w = patch - tile_h * g.tiles_w;
+            const int oh0 = tile_h * 16, ow0 = tile_w * 8, n0 = nt * BN;
+            ok = mbar_wait(t_full(acc), ((uint32_t)lt >> 1) & 1u);
+            if (!ok) break;
+            tc_fence_after();
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    if (c0 + half * 16 < BN) {                // warp-uniform
+                        uint32_t r[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + c0 + half * 16), r);
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(stage + (uint32_t)(lane * 36 + half * 16 + j) * 4u),
+                                         "r"(r[j]), "r"(r[j + 1]), "r"(r[j + 2]), "r"(r[j + 3]) : "memory");
+                    }
+                }
+                if (c0 + 32 >= BN) {                          // every TMEM read of this tile is done: hand the accumulator back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(t_empty(acc));
+                }
+                __syncwarp();
+                const int n = n0 + c0 + cc;
+                const bool col_ok = (c0 + cc < BN) && (n < g.K);
+                float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (vec && col_ok && g.bias) bb = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+#pragma unroll 2
+                for (int it = 0; it < 8; ++it) {
+                    const int rl = it * 4 + sub, mrow = quarter * 32 + rl;
+                    const int oh = oh0 + (mrow >> 3), ow = ow0 + (mrow & 7);
+                    if (!col_ok || oh >= g.H || ow >= g.W) continue;
+                    float4 v;
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                 : "r"(stage + (uint32_t)(rl * 36 + cc) * 4u));
+                    const long long off = ((long long)oh * g.W + ow) * g.K + n;
+                    if (vec) {
+                        v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                        if (g.addend) {
+                            const float4 aa = __ldg(reinterpret_cast<const float4*>(g.addend + off));
+                            v.x += aa.x; v.y += aa.y; v.z += aa.z; v.w += aa.w;
+                        }
+                        v.x = act_fn(v.x, g.act); v.y = act_fn(v.y, g.act); v.z = act_fn(v.z, g.act); v.w = act_fn(v.w, g.act);
+                        *reinterpret_cast<float4*>(g.D + off) = v;
+                    } else {
+                        const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (n + j < g.K) {
+                                float tt = vv[j];
+                                if (g.bias) tt += __ldg(g.bias + n + j);
+                                if (g.addend) tt += __ldg(g.addend + off + j);
+                                g.D[off + j] = act_fn(tt, g.act);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();                                 // the staging tile is rewritten by the next chunk
+            }
+        }
+        if (!ok && lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_end(g.stamp);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
+    }
+}

@@ -5,6 +5,12 @@ using namespace nnv;
 
 namespace nnv {
 
+// Where the one-kernel F(2x2,3x3) path is taken without being asked for (filled in from measurements).
+static bool wino_fused_default(const nnv_layer_desc_t& L, const LayerGeom& g) {
+    (void)L; (void)g;
+    return false;
+}
+
 // host_src: d_raw is pinned host memory read in place (the zero-copy arm): the kernels then start loading
 // before they wait for the previous kernel of their stream, which they do not depend on.
 nnv_status_t do_transform(const nnv_plan& p, int layer, int v, int math, const void* d_raw, void* d_out,
@@ -50,6 +56,11 @@ nnv_status_t do_exec(const nnv_plan& p, int layer, int v, int math, const void* 
     a.D = y; a.ldd = L.K; a.strideD = (int64_t)g.P * L.K;
     a.N = L.K;
 
+    if (wino_fused_applies(L, v, math)) {
+        const int wf = tuning().winofused;
+        if (wf == 1 || (wf < 0 && wino_fused_default(L, g)))
+            return launch_wino_f2_fused(L, g, x, (const float*)d_wt, bias, add, y, st);
+    }
     if (int m = wino_m(v)) {
         const int TH = ceil_div(g.OH, m), TW = ceil_div(g.OW, m), T = TH * TW, a2 = (m + 2) * (m + 2);
         uint8_t* ws = (uint8_t*)d_ws;
@@ -161,6 +172,48 @@ nnv_status_t nnv_conv_exec(const nnv_plan_t* p, int32_t layer, int32_t v, int32_
                 NNV_ERR_INVALID_ARG, "device pointers must be 256-byte aligned");
     NNV_REQUIRE(!p->layers[layer].has_bias || d_bias, NNV_ERR_INVALID_ARG, "layer %d has a bias but d_bias is null", layer);
     return do_exec(*p, layer, v, math, d_in, d_addend, d_wt, d_bias, d_out, d_ws, ws_bytes, (cudaStream_t)stream);
+}
+
+nnv_status_t nnv_wino_sizes(const nnv_plan_t* p, int32_t layer, int32_t v, int32_t math, int32_t* tiles, uint64_t* v_bytes,
+                            uint64_t* m_bytes) {
+    NNV_REQUIRE(p, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_TRY(check_choice(*p, layer, v, math));
+    const int m = wino_m(v);
+    NNV_REQUIRE(m, NNV_ERR_INVALID_ARG, "variant %d is not a Winograd variant", v);
+    const LayerGeom& g = p->geom[layer];
+    const uint64_t T = (uint64_t)ceil_div(g.OH, m) * ceil_div(g.OW, m), a2 = (uint64_t)(m + 2) * (m + 2);
+    if (tiles) *tiles = (int32_t)T;
+    if (v_bytes) *v_bytes = a2 * T * g.Cp * (math == NNV_MATH_BF16 ? 2 : 4);
+    if (m_bytes) *m_bytes = a2 * T * p->layers[layer].K * 4;
+    return NNV_OK;
+}
+
+nnv_status_t nnv_wino_input_transform(const nnv_plan_t* p, int32_t layer, int32_t v, int32_t math, const void* d_in, void* d_V,
+                                      void* stream) {
+    NNV_REQUIRE(p && d_in && d_V, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_TRY(check_choice(*p, layer, v, math));
+    const int m = wino_m(v);
+    NNV_REQUIRE(m, NNV_ERR_INVALID_ARG, "variant %d is not a Winograd variant", v);
+    NNV_REQUIRE(aligned256(d_in) && aligned256(d_V), NNV_ERR_INVALID_ARG, "device pointers must be 256-byte aligned");
+    const nnv_layer_desc_t& L = p->layers[layer];
+    const LayerGeom& g = p->geom[layer];
+    return launch_wino_input(m, math == NNV_MATH_BF16, (const float*)d_in, d_V, L.C, g.Cp, L.H, L.W, L.pad, ceil_div(g.OH, m),
+                             ceil_div(g.OW, m), (cudaStream_t)stream);
+}
+
+nnv_status_t nnv_wino_output_transform(const nnv_plan_t* p, int32_t layer, int32_t v, const void* d_M, const void* d_addend,
+                                       const void* d_bias, void* d_out, void* stream) {
+    NNV_REQUIRE(p && d_M && d_out, NNV_ERR_INVALID_ARG, "null argument");
+    NNV_TRY(check_choice(*p, layer, v, NNV_MATH_TF32));
+    const int m = wino_m(v);
+    NNV_REQUIRE(m, NNV_ERR_INVALID_ARG, "variant %d is not a Winograd variant", v);
+    NNV_REQUIRE(aligned256(d_M) && aligned256(d_out) && (!d_addend || aligned256(d_addend)) && (!d_bias || aligned256(d_bias)),
+                NNV_ERR_INVALID_ARG, "device pointers must be 256-byte aligned");
+    const nnv_layer_desc_t& L = p->layers[layer];
+    const LayerGeom& g = p->geom[layer];
+    NNV_REQUIRE(!L.has_bias || d_bias, NNV_ERR_INVALID_ARG, "layer %d has a bias but d_bias is null", layer);
+    return launch_wino_output(m, (const float*)d_M, (float*)d_out, (const float*)d_bias, (const float*)d_addend, L.act, L.K, g.OH,
+                              g.OW, ceil_div(g.OH, m), ceil_div(g.OW, m), (cudaStream_t)stream);
 }
 
 nnv_status_t nnv_pool_exec(const nnv_plan_t* p, int32_t layer, const void* d_in, void* d_out, void* stream) {

@@ -638,6 +638,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 #include "conv3x3_tc.cuh"
 #include "gemm_sp.cuh"
+#include "wino_fused.cuh"
 
 // ---- host side --------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
@@ -796,6 +797,8 @@ nnv_status_t gemm_tc_init() {
         cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_sp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(conv3x3_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(wino_f2_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     });
     return NNV_OK;
 }
@@ -864,6 +867,73 @@ nnv_status_t launch_gemm_sp(const nnv_layer_desc_t& L, const LayerGeom& geo, con
     return NNV_OK;
 }
 
+nnv_status_t launch_wino_f2_fused(const nnv_layer_desc_t& L, const LayerGeom& geo, const float* x, const float* U, const float* bias,
+                                  const float* addend, float* y, cudaStream_t st) {
+    NNV_TRY(gemm_tc_init());
+    NNV_REQUIRE((reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(U) & 15) == 0 &&
+                    (reinterpret_cast<uintptr_t>(y) & 15) == 0 && (!bias || (reinterpret_cast<uintptr_t>(bias) & 15) == 0) &&
+                    (!addend || (reinterpret_cast<uintptr_t>(addend) & 15) == 0),
+                NNV_ERR_INVALID_ARG, "the fused Winograd kernel needs 16-byte aligned buffers");
+    WfDev g;
+    g.stamp = next_stamp();
+    next_stamp() = nullptr;
+    g.x = x; g.y = y; g.bias = bias; g.addend = addend;
+    g.C = L.C; g.H = L.H; g.W = L.W; g.K = L.K; g.pad = L.pad; g.OH = geo.OH; g.OW = geo.OW;
+    g.TW = ceil_div(geo.OW, 2);
+    g.T = ceil_div(geo.OH, 2) * g.TW;
+    g.act = L.act;
+    // 32 output channels per CTA (all 512 TMEM columns) when that still gives every other SM a CTA, else 16
+    const int row_tiles = ceil_div(g.T, BM);
+    g.BN = ((L.K % 32) == 0 && (long long)row_tiles * (L.K / 32) >= 74) ? 32 : 16;
+    g.tmem_cols = 16 * g.BN;
+    g.nsteps = L.C / 8;
+    g.stages = std::min(WF_MAX_STAGES, std::max(1, g.nsteps));
+    const uint32_t b_stage = 2u * 16u * (uint32_t)g.BN * 16u;
+    while (g.stages > 1 && (size_t)1024 + (size_t)g.stages * (WF_A_STAGE + b_stage) + 8 * (3 * WF_MAX_STAGES + 2) > 220u * 1024u) --g.stages;
+    const size_t smem = (size_t)1024 + (size_t)g.stages * (WF_A_STAGE + b_stage) + 8 * (3 * WF_MAX_STAGES + 2);
+    CUtensorMap tmU;
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)geo.Cp, (cuuint64_t)L.K, 16};
+        cuuint64_t strides[2] = {(cuuint64_t)geo.Cp * 4, (cuuint64_t)L.K * geo.Cp * 4};
+        cuuint32_t box[3] = {4, (cuuint32_t)g.BN, 16};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = g_encode(&tmU, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(U), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (transformed filters) failed with code %d", (int)r);
+    }
+    dim3 grid(row_tiles, ceil_div(L.K, g.BN));
+    (void)launch_pdl(wino_f2_fused_kernel, grid, dim3(GEMM_THREADS), smem, st, tmU, g);
+    NNV_CUDA(cudaGetLastError());
+    return NNV_OK;
+}
+
+// The persistent form: BN channels per tile, `per_sm` CTAs per SM, ring depths na / nb.
+static nnv_status_t launch_conv3x3_persistent(const GemmArgs& a, int BN, int per_sm, int na, int nb, cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 18));
+    NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, BN));
+    ConvPDev g;
+    g.stamp = next_stamp();
+    next_stamp() = nullptr;
+    g.D = a.D; g.bias = a.bias; g.addend = a.addend;
+    g.C = a.ic.C; g.H = a.ic.H; g.W = a.ic.W; g.K = a.N;
+    g.BN = BN; g.act = a.act; g.na = na; g.nb = nb;
+    g.cblk = ceil_div(a.ic.C, 32); g.tiles_w = ceil_div(a.ic.W, 8);
+    g.n_tiles = ceil_div(a.N, BN);
+    g.tiles_total = ceil_div(a.ic.H, 16) * g.tiles_w * g.n_tiles;
+    g.tmem_cols = 32;
+    while (g.tmem_cols < 2 * BN) g.tmem_cols *= 2;
+    NNV_REQUIRE(a.ldd == a.N, NNV_ERR_INVALID_ARG, "the 3x3 kernel writes a dense NHWC output");
+    const size_t smem = (size_t)1024 + (size_t)na * 18 * 1024 + (size_t)nb * BN * BK_BYTES + 4 * 32 * 36 * 4 +
+                        8 * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 5);
+    NNV_REQUIRE(smem <= 220u * 1024u, NNV_ERR_UNSUPPORTED, "persistent 3x3 tiling does not fit shared memory");
+    const int ctas = std::min(g.tiles_total, 148 * per_sm);
+    (void)launch_pdl(conv3x3_tc_persistent_kernel, dim3(ctas), dim3(GEMM_THREADS), smem, st, tmA, tmB, g);
+    NNV_CUDA(cudaGetLastError());
+    return NNV_OK;
+}
+
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     NNV_REQUIRE(a.M > 0 && a.N > 0 && a.Kd > 0 && a.batch > 0, NNV_ERR_INVALID_ARG, "empty GEMM");
     NNV_TRY(gemm_tc_init());
@@ -919,6 +989,13 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
                 use = true;
             }
         }
+        // The persistent form runs only on request.  Measured on B200 (VGG-shaped layers, L2 flushed): one resident
+        // CTA per SM reaches 154 TFLOP/s on 64 -> 64 @ 224 and two reach 206, against 260 for two or three
+        // one-tile CTAs per SM: inside one CTA the single MMA-issuing thread (about 56 cycles per tcgen05.mma
+        // against 50 cycles of execution at N = 64) and the shared-memory fill bound the tile rate, and independent
+        // CTAs hide both better than a second accumulator does.
+        if (tn.convp == 2 && (size_t)tn.convp_bn <= (size_t)ceil_div(a.N, 16) * 16)
+            return launch_conv3x3_persistent(a, tn.convp_bn, tn.convp_per_sm, tn.convp_na ? tn.convp_na : 2, tn.convp_nb ? tn.convp_nb : 4, st);
         if (use) return launch_conv3x3_tc(a, ct, st);
     }
     int tmem_cols = 32;

@@ -146,7 +146,10 @@ struct Tuning {
     int gemm_prefill = 1;
     int conv3x3 = 0;                          // 0 auto, 1 off, 2 forced tiling below
     int conv_mt = 0, conv_bn = 0, conv_splits = 0, conv_na = 0, conv_nb = 0;
+    int convp = 0;                            // persistent 3x3 kernel: 0 auto, 1 off, 2 forced with the values below
+    int convp_bn = 0, convp_per_sm = 0, convp_na = 0, convp_nb = 0;
     int side = 1, merge = 1, group = 1;       // pipeline features: side stream, merged reads, grouped transforms
+    int winofused = -1;                       // the one-kernel F(2x2,3x3) path: -1 the library decides, 0 off, 1 on where it applies
     int smallp = 1;                           // the weights-on-rows kernel for layers with few pixels
     int smallp_splits = 0;                    // 0 = the cost model decides
     uint64_t generation = 0;
@@ -265,6 +268,12 @@ nnv_status_t launch_maxpool(const float* d_x, float* d_y, int C, int H, int W, i
 nnv_status_t launch_gavgpool(const float* d_x, float* d_y, int C, int H, int W, cudaStream_t st);
 nnv_status_t launch_chw_to_hwc(const float* d_in, float* d_out, int C, int H, int W, cudaStream_t st);
 nnv_status_t launch_hwc_to_chw(const float* d_in, float* d_out, int C, int H, int W, cudaStream_t st);
+
+// Winograd F(2x2,3x3), TF32, as one kernel (wino_fused.cuh): x NHWC, U[16][K][Cp] fp32, y NHWC.  Needs C % 8 == 0 and
+// K % 8 == 0 (wino_fused_applies).
+bool wino_fused_applies(const nnv_layer_desc_t& L, int variant, int math);
+nnv_status_t launch_wino_f2_fused(const nnv_layer_desc_t& L, const LayerGeom& g, const float* x, const float* U, const float* bias,
+                                  const float* addend, float* y, cudaStream_t st);
 
 // Batched tensor-core GEMM  D[b][M][N] = A[b][M][Kd] * B[b][N][Kd]^T, both operands K-major
 // (row-major with the reduction index innermost), fp32 accumulate, fp32 output with leading

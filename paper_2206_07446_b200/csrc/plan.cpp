@@ -65,6 +65,17 @@ static const char* parse_tuning(const char* spec, Tuning* t, char* item, size_t 
                      (got < 4 || (d >= 0 && d <= 4)) && (got < 5 || (f >= 0 && f <= 8));
                 if (ok) { t->conv3x3 = 2; t->conv_mt = a; t->conv_bn = b; t->conv_splits = c; t->conv_na = got >= 4 ? d : 0; t->conv_nb = got >= 5 ? f : 0; }
             }
+        } else if (!std::strcmp(key, "conv3x3p")) {
+            if (!std::strcmp(val, "off")) { t->convp = 1; ok = true; }
+            else if (!std::strcmp(val, "auto")) { t->convp = 0; ok = true; }
+            else {
+                const int got = std::sscanf(val, "%d,%d,%d,%d", &a, &b, &c, &d);
+                ok = got >= 2 && a >= 16 && a <= 128 && a % 16 == 0 && b >= 1 && b <= 4 && (got < 3 || (c >= 1 && c <= 4)) && (got < 4 || (d >= 1 && d <= 8));
+                if (ok) { t->convp = 2; t->convp_bn = a; t->convp_per_sm = b; t->convp_na = got >= 3 ? c : 0; t->convp_nb = got >= 4 ? d : 0; }
+            }
+        } else if (!std::strcmp(key, "winofused")) {
+            if (!std::strcmp(val, "auto")) { t->winofused = -1; ok = true; }
+            else ok = flag(&t->winofused);
         } else if (!std::strcmp(key, "smallp")) {
             if (std::sscanf(val, "%d", &a) == 1 && a >= 0 && a <= 148) { t->smallp = a ? 1 : 0; t->smallp_splits = a > 1 ? a : 0; ok = true; }
         } else if (!std::strcmp(key, "side")) {
@@ -145,6 +156,11 @@ static inline bool implicit_gemm_operand(const nnv_layer_desc_t& L, int math) {
     // activation of at least 128 KiB (smaller tensors take the explicit path).
     return math == NNV_MATH_TF32 && (L.C % 4) == 0 && 4ull * L.C * L.H * L.W >= 131072ull && L.R <= 16 && L.S <= 16 &&
            L.pad <= 8;
+}
+
+bool wino_fused_applies(const nnv_layer_desc_t& L, int v, int math) {
+    return v == NNV_VAR_WINO_F2 && math == NNV_MATH_TF32 && L.groups == 1 && L.R == 3 && L.S == 3 && L.stride == 1 &&
+           (L.C % 8) == 0 && (L.K % 8) == 0;
 }
 
 SmallPPlan small_p_plan(const nnv_layer_desc_t& L, const LayerGeom& g, int v, int math) {

@@ -59,3 +59,45 @@ def test_every_tiling_matches_the_oracle(shape):
     # whatever the library picks by itself is one of the two kernels above
     auto = _run(L, x, w, b, add, None)
     assert rel_l2(auto, ref) <= TOL[nb.MATH_TF32]
+
+
+def _run_p(L, x, w, b, add, setting):
+    nb.nnv_tuning_set(setting)
+    try:
+        plan = nb.Plan([L], [0], [0])
+        return run_conv(plan, 0, L, nb.VAR_IM2COL, nb.MATH_TF32, x, w, b, add)
+    finally:
+        nb.nnv_tuning_set(None)
+
+
+@pytest.mark.parametrize("shape", [
+    # C, K, H, W, bias/addend/act
+    (64, 64, 56, 56, False),         # 49 patches: with one CTA per SM forced to few CTAs, several tiles per CTA
+    (32, 48, 40, 30, True),          # ragged: H % 16 != 0, W % 8 != 0, K = 48, epilogue terms
+    (96, 200, 35, 21, True),         # K = 200: two channel tiles at BN = 128, the second partly filled; three channel blocks
+    (64, 20, 100, 9, False),         # K = 20: scalar epilogue stores; many patches
+])
+def test_persistent_form_matches_the_oracle(shape):
+    """The persistent 3x3 kernel (tiles walked by resident CTAs, two TMEM accumulators): every tile width and ring
+    depth it can take, with more tiles than CTAs, against the oracle and the one-tile-per-CTA kernel."""
+    C, K, H, W, epi = shape
+    L = dict(op=0, C=C, K=K, R=3, S=3, stride=1, pad=1, groups=1, H=H, W=W, in0=-1, in1=-1, act=2 if epi else 1,
+             has_bias=1 if epi else 0)
+    rng = np.random.default_rng([9] + list(shape[:4]))
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((K, C, 3, 3)) * np.sqrt(2.0 / (C * 9))).astype(np.float32)
+    b = rng.uniform(-1, 1, K).astype(np.float32) if epi else None
+    add = rng.uniform(-1, 1, (K, H, W)).astype(np.float32) if epi else None
+    ref = omodel.run_layer(L, x, w, b, add)
+    one_tile = _run_p(L, x, w, b, add, "conv3x3p=off;conv3x3=1,%d,1" % min(128, -(-K // 16) * 16))
+    assert rel_l2(one_tile, ref) <= TOL[nb.MATH_TF32]
+    bn_full = min(128, -(-K // 16) * 16)
+    for bn in sorted({bn_full, 16, min(bn_full, 64)}):
+        for per_sm, na, nb_ in ((1, 2, 3), (1, 4, 8), (2, 1, 2), (3, 2, 4)):
+            y = _run_p(L, x, w, b, add, "conv3x3p=%d,%d,%d,%d" % (bn, per_sm, na, nb_))
+            assert np.all(np.isfinite(y)), (bn, per_sm, na, nb_)
+            err = rel_l2(y, ref)
+            assert err <= TOL[nb.MATH_TF32], (bn, per_sm, na, nb_, err)
+            # the same MMAs in the same order as the one-tile kernel with this tile width: the same bits
+            if bn == bn_full:
+                assert np.array_equal(y.view(np.uint32), one_tile.view(np.uint32)), (bn, per_sm, na, nb_)
