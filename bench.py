@@ -37,7 +37,7 @@ import workloads as wl  # noqa: E402
 # DRAM bytes per tensor-core GEMM launch (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the
 # launches of one step) from an ncu capture of this command; the file under profiles/ gives the command.
 # An entry is dropped (traffic = null) whenever the kernel changes after the capture.
-NCU_GEMM_TRAFFIC_BYTES = {}
+NCU_GEMM_TRAFFIC_BYTES = {("cfg4_resnet50", "tf32"): 3269014}   # profiles/gemm_cfg4_dram_traffic.md
 
 METRIC = "cold_inference_ms_batch1"
 UNIT = "ms"
@@ -317,7 +317,7 @@ def run_ours(args):
     line = measure(args, args.config, args.steps, args.warmup, args.minimal, rank, world, local)
     # the other single-GPU configurations, headline numbers and rooflines only, beside the main workload
     others = {}
-    for name in [c for c in args.also.split(",") if c and c != args.config]:
+    for name in [c for c in args.also.split(",") if c and c != "none" and c != args.config]:
         o = measure(args, name, args.arm_steps, 3, True, rank, world, local)
         others[name] = {k: o[k] for k in ("value", "unit", "steps", "e2e", "roofline", "roofline_transform", "transform_all", "run", "per_layer")}
         others[name]["e2e"] = {k: o["e2e"][k] for k in ("value", "h2d_bytes_per_step", "host_link")}
@@ -668,9 +668,9 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
 
     tf32_peak = peaks["bf16_tflops"] * 0.5
     tens_peak = peaks["bf16_tflops"] if math == nb.MATH_BF16 else tf32_peak
-    # the tensor-core GEMM launches that are a layer's whole convolution (implicit GEMM, 3x3 halo kernel, direct-operand 1x1)
-    single = [i for i in ex if choices_raw[i][0] in (nb.VAR_IM2COL, nb.VAR_GEMM1X1)
-              and nb.nnv_exec_workspace_bytes(model.plan, i, choices_raw[i][0], choices_raw[i][1]) == 0]
+    # the tensor-core launches that carry a layer's convolution (implicit GEMM, 3x3 halo kernel, direct-operand 1x1, the
+    # weights-on-rows kernel together with its split reduction; the stem's GEMM after its explicit im2col)
+    single = [i for i in ex if choices_raw[i][0] in (nb.VAR_IM2COL, nb.VAR_GEMM1X1)]
     roof = None
     if single:
         gfl = sum(layer_flops(i) for i in single)
@@ -682,7 +682,7 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
         tens = {"bound": "tensor", "achieved": gfl / gns / 1e3, "peak": tens_peak, "unit": "TFLOP/s", "frac": gfl / gns / 1e3 / tens_peak}
         hbm = {"bound": "hbm", "achieved": gby / gns, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gby / gns / peaks["hbm_gbs"]}
         roof = dict(hbm if t_hbm >= t_tensor else tens)           # the binding roofline of these launches
-        roof.update({"kernel": "gemm_tc_kernel / conv3x3_tc_kernel (tcgen05 GEMM; every launch that is a layer's whole convolution)",
+        roof.update({"kernel": "gemm_tc_kernel / gemm_sp_kernel (+ splitk_reduce_kernel) / conv3x3_tc_kernel: the tcgen05 GEMM of every im2col / 1x1 layer",
                      "traffic": NCU_GEMM_TRAFFIC_BYTES.get((args.config, args.math)),
                      "durations": "device-clock stamps written by the kernels themselves inside the timed steps (CUDA events time the step)",
                      "peak_source": peaks["source"] + (" HBM copy" if t_hbm >= t_tensor else " bf16 burst" + ("" if math == nb.MATH_BF16 else " x 0.5 (tf32:bf16 nominal ratio)")),
@@ -822,8 +822,25 @@ def time_transform(torch, nb, variant, math, C, K, R=3, reps=20, flush=None):
     d_raw = _rand(torch, K * C * R * R, 0.05)
     d_out = _buf(torch, outb)
     med, best = _time(torch, lambda st: nb.nnv_transform_weights(plan, 0, variant, math, d_raw, d_out, st), reps, flush)
-    return dict(op="transform", variant=nb.VARIANT_NAMES[variant], math=nb.MATH_NAMES[math], C=C, K=K, R=R,
-                bytes=rawb + outb, us=med, us_min=best, gbs=(rawb + outb) / med / 1e3)
+    out = dict(op="transform", variant=nb.VARIANT_NAMES[variant], math=nb.MATH_NAMES[math], C=C, K=K, R=R,
+               bytes=rawb + outb, us=med, us_min=best, gbs=(rawb + outb) / med / 1e3)
+    # the kernel's own duration (device-clock stamps, no launch or event overhead): the layer as a one-layer model
+    # whose resident run transforms the weights before it executes
+    from paper_2206_07446_b200 import harness
+    w = np.zeros((K, C, R, R), np.float32)
+    m1 = harness.model_from_workload([L], [w], [None], wl.weight_blob, use_graphs=0, kernel_stamps=1)
+    ch = [(variant, math, 0)]
+    need = m1.ensure_arena(ch, 1)
+    d_io_in, d_io_out = _rand(torch, C * 64), _buf(torch, 4 * 64 * K)
+    ks = []
+    for r in range(reps + 2):
+        if flush is not None:
+            flush.fill_(r & 0xFF)
+        nb.nnv_resident_run(m1.plan, ch, d_raw, m1.w_bytes, None, 0, d_io_in, d_io_out, m1.arena, need, m1.streams[1], m1.streams[2], 1)
+        ks.append(nb.nnv_kernel_times(m1.plan)[0][0] / 1e3)
+    out["kernel_us"] = statistics.median(ks[2:])
+    out["kernel_gbs"] = (rawb + outb) / out["kernel_us"] / 1e3 if out["kernel_us"] else None
+    return out
 
 
 def time_conv(torch, nb, variant, math, C, K, R, stride, H, W, groups=1, reps=20, flush=None):

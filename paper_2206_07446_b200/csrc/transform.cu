@@ -86,10 +86,16 @@ template <> struct VecStore<__nv_bfloat16, 8> {
 };
 
 constexpr int FT_THREADS = 256;
-constexpr int FT_FILTERS = 1024;                                // filters (padded (k, c) pairs) per block
-// Filters per thread: as many as make every store of a thread 16 bytes wide (4 fp32 or 8 bf16 values).
-template <typename OutT> struct FtNF { static constexpr int value = 4; };
-template <> struct FtNF<__nv_bfloat16> { static constexpr int value = 8; };
+constexpr int FT_FILTERS = 1024;                                // most filters (padded (k, c) pairs) a block takes
+// Filters of one block: every thread busy, at most FT_FILTERS (which the shared staging buffer holds).
+__host__ __device__ constexpr int ft_filters(int nf) { return FT_THREADS * nf > FT_FILTERS ? FT_FILTERS : FT_THREADS * nf; }
+// Filters per thread.  F(2x2,3x3): as many as make every store of a thread 16 bytes wide (4 fp32 or 8 bf16
+// values).  F(4x4,3x3) and F(6x6,3x3) keep 2 -- four filters' intermediates need 128 registers and halve the
+// resident warps (measured: 1024^2 filters 47 us against 41) -- and reach 16-byte stores by exchanging halves
+// between neighbouring lanes: of every pair of planes the even lane stores one plane for both lanes' filters
+// and the odd lane the other.
+template <int M_, typename OutT> struct FtNF { static constexpr int value = (M_ == 2) ? 4 : 2; };
+template <int M_> struct FtNF<M_, __nv_bfloat16> { static constexpr int value = (M_ == 2) ? 8 : 2; };
 
 // One thread transforms NF filters that are adjacent in the padded channel index, so that each of the alpha^2
 // output planes receives one NF-wide (16-byte) vector store per thread and a warp writes 32*NF consecutive
@@ -101,9 +107,10 @@ template <int M_, typename OutT, int NF>
 __device__ __forceinline__ void filter_transform_block(const float* __restrict__ g, OutT* __restrict__ U, int K, int C,
                                                        int Cp, unsigned block, float* sg, bool late_wait) {
     constexpr int A = WinoG<M_>::A;
-    constexpr int ACTIVE = FT_FILTERS / NF;                       // threads that transform
+    constexpr int FPB = ft_filters(NF);                          // filters of this block
+    constexpr int ACTIVE = FPB / NF;                              // threads that transform
     const long long F = (long long)K * Cp;                      // padded filter count = plane size
-    const long long f_block = (long long)block * FT_FILTERS;
+    const long long f_block = (long long)block * FPB;
     const long long f0 = f_block + (long long)threadIdx.x * NF;
     const bool contiguous = (C == Cp);
 
@@ -112,7 +119,7 @@ __device__ __forceinline__ void filter_transform_block(const float* __restrict__
         const long long base = f_block * 9;
         const float4* src = reinterpret_cast<const float4*>(g + base);
         float4* dst = reinterpret_cast<float4*>(sg);
-        constexpr int NV = FT_FILTERS * 9 / 4;
+        constexpr int NV = FPB * 9 / 4;
         for (int i = threadIdx.x; i < NV; i += FT_THREADS) {
             if (base + 4ll * i < total) dst[i] = __ldg(src + i);
         }
@@ -126,12 +133,21 @@ __device__ __forceinline__ void filter_transform_block(const float* __restrict__
     float w[NF][9];
     bool pad[NF];
     if (contiguous) {
-        const float4* s4 = reinterpret_cast<const float4*>(sg + (size_t)threadIdx.x * NF * 9);
         float flat[NF * 9];
+        if constexpr ((NF * 9) % 4 == 0) {
+            const float4* s4 = reinterpret_cast<const float4*>(sg + (size_t)threadIdx.x * NF * 9);
 #pragma unroll
-        for (int i = 0; i < NF * 9 / 4; ++i) {
-            const float4 v = s4[i];
-            flat[4 * i] = v.x; flat[4 * i + 1] = v.y; flat[4 * i + 2] = v.z; flat[4 * i + 3] = v.w;
+            for (int i = 0; i < NF * 9 / 4; ++i) {
+                const float4 v = s4[i];
+                flat[4 * i] = v.x; flat[4 * i + 1] = v.y; flat[4 * i + 2] = v.z; flat[4 * i + 3] = v.w;
+            }
+        } else {                                                  // NF = 2: 18 floats on an 8-byte boundary, conflict-free as 64-bit loads
+            const float2* s2 = reinterpret_cast<const float2*>(sg + (size_t)threadIdx.x * NF * 9);
+#pragma unroll
+            for (int i = 0; i < NF * 9 / 2; ++i) {
+                const float2 v = s2[i];
+                flat[2 * i] = v.x; flat[2 * i + 1] = v.y;
+            }
         }
 #pragma unroll
         for (int j = 0; j < NF; ++j) {
@@ -163,19 +179,43 @@ __device__ __forceinline__ void filter_transform_block(const float* __restrict__
 
     // U[xi][nu] = sum_i G[xi][i] * t[i][nu]; plane xi*A+nu, element f0..f0+NF-1
     OutT* out = U + f0;
+    auto plane_values = [&](int xi, int nu, float* v) {
 #pragma unroll
-    for (int xi = 0; xi < A; ++xi) {
+        for (int j = 0; j < NF; ++j) {
+            v[j] = WinoG<M_>::g(xi, 0) * t[j][0][nu] + WinoG<M_>::g(xi, 1) * t[j][1][nu] + WinoG<M_>::g(xi, 2) * t[j][2][nu];
+            if (pad[j]) v[j] = 0.f;                              // padded channels hold +0, never -0
+        }
+    };
+    if constexpr (NF == 2 && sizeof(OutT) == 4) {
+        // pairs of planes (A is even): lanes 2i and 2i+1 hold four adjacent filters between them (the plane size is a
+        // multiple of 8, so both are live or neither); each sends the partner its two values of the plane the partner stores
+        const unsigned live = __activemask();
+        const bool odd = (threadIdx.x & 1) != 0;
 #pragma unroll
-        for (int nu = 0; nu < A; ++nu) {
-            float v[NF];
+        for (int xi = 0; xi < A; ++xi) {
 #pragma unroll
-            for (int j = 0; j < NF; ++j)
-                v[j] = WinoG<M_>::g(xi, 0) * t[j][0][nu] + WinoG<M_>::g(xi, 1) * t[j][1][nu] +
-                       WinoG<M_>::g(xi, 2) * t[j][2][nu];
+            for (int nu = 0; nu < A; nu += 2) {
+                float vp[2], vq[2];
+                plane_values(xi, nu, vp);
+                plane_values(xi, nu + 1, vq);
+                const float s0 = __shfl_xor_sync(live, odd ? vp[0] : vq[0], 1);
+                const float s1 = __shfl_xor_sync(live, odd ? vp[1] : vq[1], 1);
+                float v4[4];
+                if (!odd) { v4[0] = vp[0]; v4[1] = vp[1]; v4[2] = s0; v4[3] = s1; }
+                else { v4[0] = s0; v4[1] = s1; v4[2] = vq[0]; v4[3] = vq[1]; }
+                OutT* dst = out + (long long)(xi * A + nu + (odd ? 1 : 0)) * F - (odd ? 2 : 0);
+                VecStore<OutT, 4>::st(dst, v4);
+            }
+        }
+    } else {
 #pragma unroll
-            for (int j = 0; j < NF; ++j)
-                if (pad[j]) v[j] = 0.f;                          // padded channels hold +0, never -0
-            VecStore<OutT, NF>::st(out + (long long)(xi * A + nu) * F, v);
+        for (int xi = 0; xi < A; ++xi) {
+#pragma unroll
+            for (int nu = 0; nu < A; ++nu) {
+                float v[NF];
+                plane_values(xi, nu, v);
+                VecStore<OutT, NF>::st(out + (long long)(xi * A + nu) * F, v);
+            }
         }
     }
 }
@@ -197,9 +237,9 @@ filter_transform_kernel(const float* __restrict__ g, OutT* __restrict__ U, int K
 
 template <int M_, typename OutT>
 static nnv_status_t launch_ft(const float* g, void* U, int K, int C, int Cp, cudaStream_t st, bool host_src) {
-    constexpr int NF = FtNF<OutT>::value;
+    constexpr int NF = FtNF<M_, OutT>::value;
     const long long F = (long long)K * Cp;
-    const unsigned grid = (unsigned)((F + FT_FILTERS - 1) / FT_FILTERS);
+    const unsigned grid = (unsigned)((F + ft_filters(NF) - 1) / ft_filters(NF));
     unsigned long long* stamp = next_stamp();
     next_stamp() = nullptr;
     NNV_LAUNCH((filter_transform_kernel<M_, OutT, NF>), grid, FT_THREADS, 0, st, g, reinterpret_cast<OutT*>(U), K, C, Cp, stamp,
@@ -434,11 +474,11 @@ multi_transform_kernel(const __grid_constant__ XformBatch batch) {
         switch (d.kind * 2 + d.bf16) {
             case XF_WINO2 * 2: filter_transform_block<2, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
             case XF_WINO2 * 2 + 1: filter_transform_block<2, __nv_bfloat16, 8>(src, (__nv_bfloat16*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
-            case XF_WINO4 * 2: filter_transform_block<4, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
+            case XF_WINO4 * 2: filter_transform_block<4, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late); break;
             default: break;
         }
     } else {
-        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 4>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late);
+        if (d.kind == XF_WINO6 && !d.bf16) filter_transform_block<6, float, 2>(src, (float*)d.dst, d.K, d.C, d.Cp, lb, smem, late);
     }
     __syncthreads();
     if (threadIdx.x == 0) stamp_end(batch.stamp);
@@ -453,7 +493,10 @@ int xform_blocks(const XformDesc& d) {
     switch (d.kind) {
         case XF_PACK: return (int)pack_blocks(d.K, d.C, d.RS);
         case XF_PACK1X1: return (int)(((long long)d.K * d.Qp + PACK1X1_PER_BLOCK - 1) / PACK1X1_PER_BLOCK);
-        default: return (int)(((long long)d.K * d.Cp + FT_FILTERS - 1) / FT_FILTERS);
+        default: {                                              // the block size of the kind's instantiation in multi_transform_kernel
+            const int fpb = d.kind == XF_WINO2 ? ft_filters(d.bf16 ? 8 : 4) : ft_filters(2);
+            return (int)(((long long)d.K * d.Cp + fpb - 1) / fpb);
+        }
     }
 }
 
