@@ -83,6 +83,7 @@ nnv_status_t do_exec(const nnv_plan& p, int layer, int v, int math, const void* 
     a.M = g.P; a.Kd = g.Qp; a.batch = 1;
     a.B = d_wt; a.ldb = g.Qp; a.strideB = (int64_t)L.K * g.Qp;
     const bool direct_operand = (v == NNV_VAR_GEMM1X1) && need == 0 && L.stride == 1;
+    if ((direct_operand || need == 0) && bf16) a.mode = GEMM_BF16_CVT;   // fp32 activation rounded to bf16 inside the kernel
     if (direct_operand) {
         a.A = x; a.lda = L.C; a.Kd = L.C;                      // rows of X are the GEMM's rows
     } else if (need == 0) {

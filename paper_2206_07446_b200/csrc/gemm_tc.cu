@@ -243,6 +243,29 @@ __device__ __forceinline__ void convert_row(uint32_t src_tile, uint32_t hi_tile,
     }
 }
 
+// Converts one row (32 fp32, stored by TMA with the 128-byte swizzle) of a staged tile into ONE bf16 tile (round to
+// nearest even; un-swizzled core-matrix layout, `rows` rows tall).
+__device__ __forceinline__ void convert_row_bf16(uint32_t src_tile, uint32_t dst_tile, int r, int rows) {
+    const uint32_t src = src_tile + (uint32_t)r * 128u;
+    const uint32_t lbo = (uint32_t)rows * 16u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {                              // 4 chunks of 8 K-elements
+        float4 v0, v1;
+        const uint32_t a0 = src + ((uint32_t)((2 * c) ^ (r & 7)) << 4), a1 = src + ((uint32_t)((2 * c + 1) ^ (r & 7)) << 4);
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v0.x), "=f"(v0.y), "=f"(v0.z), "=f"(v0.w) : "r"(a0));
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v1.x), "=f"(v1.y), "=f"(v1.z), "=f"(v1.w) : "r"(a1));
+        const __nv_bfloat162 p0 = __floats2bfloat162_rn(v0.x, v0.y), p1 = __floats2bfloat162_rn(v0.z, v0.w);
+        const __nv_bfloat162 p2 = __floats2bfloat162_rn(v1.x, v1.y), p3 = __floats2bfloat162_rn(v1.z, v1.w);
+        const uint32_t off = (uint32_t)c * lbo + (uint32_t)r * 16u;
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(dst_tile + off), "r"(*reinterpret_cast<const uint32_t*>(&p0)),
+                     "r"(*reinterpret_cast<const uint32_t*>(&p1)), "r"(*reinterpret_cast<const uint32_t*>(&p2)),
+                     "r"(*reinterpret_cast<const uint32_t*>(&p3)) : "memory");
+    }
+}
+
+// MODE 3: A is fp32 (the activation itself, direct or through the TMA's im2col mode) and is rounded to bf16 by the
+// epilogue warps on its way through shared memory; B is the bf16 packed weight, fetched straight into the
+// un-swizzled core-matrix layout by four TMA boxes of 8 elements (16 bytes) x BN rows per stage.
 // MODE 0: TF32 operands (fp32 words), 1: BF16 operands, 2: fp32 operands multiplied as
 // hi*hi + lo*hi + hi*lo of their bf16 splits (error-compensated, fp32-class accuracy).
 template <int MODE> struct ModeTraits {
@@ -252,6 +275,7 @@ template <int MODE> struct ModeTraits {
 template <int MODE>
 __host__ __device__ constexpr uint32_t stage_bytes_of(int BN) {
     // staged TMA tiles (A: 128 rows x 128 B, B: BN rows x 128 B); mode 2 adds hi and lo bf16 tiles
+    if (MODE == 3) return (uint32_t)(A_STAGE_BYTES + A_STAGE_BYTES / 2 + BN * 64);   // fp32 A, bf16 A, bf16 B (32 elements per row)
     return (uint32_t)(A_STAGE_BYTES + BN * BK_BYTES) * (MODE == 2 ? 2u : 1u);
 }
 
@@ -267,7 +291,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int BN = g.BN;
     const uint32_t b_stage_bytes = (uint32_t)BN * BK_BYTES;
-    const uint32_t tma_bytes = A_STAGE_BYTES + b_stage_bytes;
+    const uint32_t tma_bytes = A_STAGE_BYTES + (MODE == 3 ? (uint32_t)BN * 64u : b_stage_bytes);
     const uint32_t stage_bytes = stage_bytes_of<MODE>(BN);
     const uint32_t bars = sbase + STAGES * stage_bytes;       // full[S], empty[S], conv[S], tmem_full, holder
     auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -338,14 +362,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (g.ic_on) {
             // A comes straight from the activation: block `kb` is channel block ic_cb of tap (ic_fr, ic_fs)
             tma_load_im2col_4d(a_dst, &tmA, ic_cb * BKE, ic_w0, ic_h0, 0, (uint16_t)ic_fs, (uint16_t)ic_fr, full_bar(s));
-            tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, ic_tap * g.ic_C + ic_cb * BKE, n0, b, full_bar(s));
+            if constexpr (MODE == 3) {   // B: four boxes of 8 elements x BN rows, staged after the fp32 and the bf16 A tile
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    tma_load_3d(a_dst + A_STAGE_BYTES + A_STAGE_BYTES / 2 + (uint32_t)c * (uint32_t)BN * 16u, &tmB,
+                                ic_tap * g.ic_C + ic_cb * BKE + 8 * c, n0, 0, full_bar(s));
+            } else {
+                tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, ic_tap * g.ic_C + ic_cb * BKE, n0, b, full_bar(s));
+            }
             if (++ic_cb == g.ic_cblk) {
                 ic_cb = 0; ++ic_tap;
                 if (++ic_fs == g.ic_S) { ic_fs = 0; ++ic_fr; }
             }
         } else {
             tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
-            tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
+            if constexpr (MODE == 3) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    tma_load_3d(a_dst + A_STAGE_BYTES + A_STAGE_BYTES / 2 + (uint32_t)c * (uint32_t)BN * 16u, &tmB, kb * BKE + 8 * c, n0, 0,
+                                full_bar(s));
+            } else {
+                tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
+            }
         }
     };
     // The producer fills the whole ring before the CTA-wide barrier: the first loads fly while
@@ -396,7 +434,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int s = 0;
             uint32_t ph = 0;
             for (int it = 0; it < nkb; ++it, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
-                ok = mbar_wait(MODE == 2 ? conv_bar(s) : full_bar(s), ph);
+                ok = mbar_wait((MODE == 2 || MODE == 3) ? conv_bar(s) : full_bar(s), ph);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_src = sbase + s * stage_bytes;
@@ -415,6 +453,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         umma<true>(tmem_base, ah, bl, idesc, 1u);
                         umma<true>(tmem_base, ah, bh, idesc, 1u);
                     }
+                } else if constexpr (MODE == 3) {
+                    const uint32_t a_bf = a_src + A_STAGE_BYTES, b_bf = a_bf + A_STAGE_BYTES / 2;
+                    const uint32_t lbo_a = BM * 16u, lbo_b = (uint32_t)BN * 16u;
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk)             // 2 K-steps of 16 bf16 = 2 core matrices each
+                        umma<true>(tmem_base, make_smem_desc_plain(a_bf + kk * 2 * lbo_a, lbo_a, 128),
+                                   make_smem_desc_plain(b_bf + kk * 2 * lbo_b, lbo_b, 128), idesc, (it | kk) ? 1u : 0u);
                 } else {
                     const uint64_t adesc = make_smem_desc(a_src);
                     const uint64_t bdesc = make_smem_desc(a_src + A_STAGE_BYTES);
@@ -429,6 +474,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         bool ok = true;
+        if constexpr (MODE == 3) {
+            // warps 2-5 first round every staged fp32 A tile to bf16 (the weights arrive as bf16)
+            const int idx = (int)threadIdx.x - 64;              // 0..127: one row of A each
+            int s = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < nkb; ++it, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0 ? 1u : 0u)) {
+                ok = mbar_wait(full_bar(s), ph);
+                if (!ok) break;
+                const uint32_t a_src = sbase + s * stage_bytes;
+                convert_row_bf16(a_src, a_src + A_STAGE_BYTES, idx, BM);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
+                mbar_arrive(conv_bar(s));
+            }
+        }
         if constexpr (MODE == 2) {
             // warps 2-5 first convert every staged fp32 tile into its bf16 hi / lo tiles
             const int idx = (int)threadIdx.x - 64;              // 0..127: one row of A (and of B) each
@@ -795,6 +854,7 @@ nnv_status_t gemm_tc_init() {
         cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(gemm_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(gemm_sp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(conv3x3_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
@@ -947,7 +1007,7 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     // Ring depth: 8 stages when every CTA has an SM to itself (a lone CTA needs that many loads in flight to keep
     // the SM's ~100 GB/s of shared-memory fill busy on weights that come cold from HBM), 4 when several share one.
     auto ring_for = [&](int bn, long long ctas) {
-        const uint32_t stage = (a.mode == GEMM_X3) ? stage_bytes_of<2>(bn) : stage_bytes_of<0>(bn);
+        const uint32_t stage = (a.mode == GEMM_X3) ? stage_bytes_of<2>(bn) : (a.mode == GEMM_BF16_CVT) ? stage_bytes_of<3>(bn) : stage_bytes_of<0>(bn);
         if (a.mode == GEMM_X3) return 3;
         return (ctas <= 148 && (size_t)8 * stage <= 200u * 1024u) ? 8 : 4;
     };
@@ -1000,7 +1060,7 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     }
     int tmem_cols = 32;
     while (tmem_cols < BN) tmem_cols *= 2;
-    const uint32_t sb = (a.mode == GEMM_X3) ? stage_bytes_of<2>(BN) : stage_bytes_of<0>(BN);
+    const uint32_t sb = (a.mode == GEMM_X3) ? stage_bytes_of<2>(BN) : (a.mode == GEMM_BF16_CVT) ? stage_bytes_of<3>(BN) : stage_bytes_of<0>(BN);
     int ring = ring_for(BN, (long long)m_tiles * ceil_div(a.N, BN) * a.batch * splits);
     if (tn.gemm_ring && (size_t)tn.gemm_ring * sb <= 210u * 1024u) ring = tn.gemm_ring;
     while (splits > 1 && ring < 8 && (uint32_t)ring * sb < (uint32_t)BM * (BN + 4) * 4u) ++ring;   // room to park the partial tile
@@ -1015,7 +1075,8 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     g.M = a.M; g.N = a.N; g.Kd = a.Kd; g.BN = BN; g.act = a.act; g.tmem_cols = tmem_cols; g.splits = splits; g.stages = ring; g.prefill = tn.gemm_prefill;
     g.ic_on = 0; g.ic_C = g.ic_cblk = g.ic_S = g.ic_OW = g.ic_stride = g.ic_pad = 0;
     if (a.ic.on) {
-        NNV_REQUIRE(a.mode == GEMM_TF32 && a.batch == 1, NNV_ERR_INVALID_ARG, "implicit im2col needs the TF32 mode and one batch");
+        NNV_REQUIRE((a.mode == GEMM_TF32 || a.mode == GEMM_BF16_CVT) && a.batch == 1, NNV_ERR_INVALID_ARG,
+                    "implicit im2col needs fp32 activations (TF32 or converting BF16 mode) and one batch");
         NNV_TRY(encode_im2col_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, a.ic.R, a.ic.S, a.ic.stride, a.ic.pad));
         g.ic_on = 1; g.ic_C = a.ic.C; g.ic_cblk = ceil_div(a.ic.C, 32); g.ic_S = a.ic.S; g.ic_OW = a.ic.OW;
         g.ic_stride = a.ic.stride; g.ic_pad = a.ic.pad;
@@ -1023,7 +1084,20 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     } else {
         NNV_TRY(encode_operand(&tmA, a.A, bf16, a.Kd, a.M, a.batch, a.lda, a.strideA, BM));
     }
-    NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
+    if (a.mode == GEMM_BF16_CVT) {
+        // bf16 weights, boxes of 8 elements x BN rows, no swizzle: four of them make the core-matrix layout of a stage
+        NNV_REQUIRE(a.batch == 1 && (a.ldb % 8) == 0, NNV_ERR_INVALID_ARG, "the converting BF16 mode needs one batch and 16-byte weight rows");
+        cuuint64_t dims[3] = {(cuuint64_t)a.ldb, (cuuint64_t)a.N, 1};
+        cuuint64_t strides[2] = {(cuuint64_t)a.ldb * 2, (cuuint64_t)a.ldb * 2 * (cuuint64_t)a.N};
+        cuuint32_t box[3] = {8, (cuuint32_t)BN, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = g_encode(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(a.B), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (bf16 weight chunks) failed with code %d", (int)r);
+    } else {
+        NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
+    }
 
     // Write-out by TMA through swizzled staging tiles when the output rows are 16-byte multiples (else plain stores).
     // A residual addend needs a staging tile of its own beside the ring: the ring gives up stages for it.
@@ -1062,6 +1136,8 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         (void)launch_pdl_cluster(gemm_tc_kernel<0>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
     else if (a.mode == GEMM_BF16)
         (void)launch_pdl_cluster(gemm_tc_kernel<1>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
+    else if (a.mode == GEMM_BF16_CVT)
+        (void)launch_pdl_cluster(gemm_tc_kernel<3>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
     else if (a.mode == GEMM_X3)
         (void)launch_pdl_cluster(gemm_tc_kernel<2>, grid, dim3(GEMM_THREADS), smem_bytes, st, splits, tmA, tmB, tmD, tmAdd, g);
     else

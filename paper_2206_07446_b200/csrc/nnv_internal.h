@@ -150,6 +150,7 @@ struct Tuning {
     int convp_bn = 0, convp_per_sm = 0, convp_na = 0, convp_nb = 0;
     int side = 1, merge = 1, group = 1;       // pipeline features: side stream, merged reads, grouped transforms
     int winofused = -1;                       // the one-kernel F(2x2,3x3) path: -1 the library decides, 0 off, 1 on where it applies
+    int bf16cvt = 1;                          // BF16 math straight from the fp32 activation (rounded inside the GEMM); 0: explicit bf16 im2col
     int smallp = 1;                           // the weights-on-rows kernel for layers with few pixels
     int smallp_splits = 0;                    // 0 = the cost model decides
     uint64_t generation = 0;
@@ -292,7 +293,9 @@ struct GemmArgs {
 };
 // GEMM_X3: fp32 operands; each is split on the fly into bf16 hi + lo and the product is formed
 // as hi*hi + lo*hi + hi*lo on the bf16 tensor pipe (fp32-class accuracy, fp32 bytes in memory).
-enum { GEMM_TF32 = 0, GEMM_BF16 = 1, GEMM_X3 = 2 };
+// GEMM_BF16_CVT: A is fp32 and is rounded to bf16 inside the kernel, B is bf16 (weights packed for BF16 math): the
+// BF16 accuracy class without a bf16 copy of the activation (direct operand or implicit im2col; batch 1).
+enum { GEMM_TF32 = 0, GEMM_BF16 = 1, GEMM_X3 = 2, GEMM_BF16_CVT = 3 };
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st);
 // Convolution of a layer with few pixels by the weights-on-rows kernel: x NHWC [H*W][C], wt packed P[K][Qp].
 nnv_status_t launch_gemm_sp(const nnv_layer_desc_t& L, const LayerGeom& g, const SmallPPlan& sp, const float* x, const float* wt,

@@ -76,6 +76,8 @@ static const char* parse_tuning(const char* spec, Tuning* t, char* item, size_t 
         } else if (!std::strcmp(key, "winofused")) {
             if (!std::strcmp(val, "auto")) { t->winofused = -1; ok = true; }
             else ok = flag(&t->winofused);
+        } else if (!std::strcmp(key, "bf16cvt")) {
+            ok = flag(&t->bf16cvt);
         } else if (!std::strcmp(key, "smallp")) {
             if (std::sscanf(val, "%d", &a) == 1 && a >= 0 && a <= 148) { t->smallp = a ? 1 : 0; t->smallp_splits = a > 1 ? a : 0; ok = true; }
         } else if (!std::strcmp(key, "side")) {
@@ -147,15 +149,16 @@ uint64_t transformed_bytes(const nnv_plan& p, int layer, int v, int math) {
 static inline bool gemm1x1_direct_operand(const nnv_layer_desc_t& L, int math) {
     // The activation itself can be the GEMM's A operand when no subsampling, padding or
     // conversion is needed: stride 1, fp32 words (TF32), rows a multiple of 16 bytes.
-    return math == NNV_MATH_TF32 && L.stride == 1 && (L.C % 4) == 0;
+    // BF16 math: the kernel rounds the fp32 rows to bf16 on their way through shared memory (C % 8: 16-byte weight chunks).
+    return L.stride == 1 && ((math == NNV_MATH_TF32 && (L.C % 4) == 0) || (math == NNV_MATH_BF16 && (L.C % 8) == 0 && tuning().bf16cvt));
 }
 
 static inline bool implicit_gemm_operand(const nnv_layer_desc_t& L, int math) {
     // The TMA's im2col mode gathers filter-window pixels straight from the NHWC activation, so no
     // Xcol matrix is materialised: fp32 words (TF32), pixel rows a multiple of 16 bytes, and an
     // activation of at least 128 KiB (smaller tensors take the explicit path).
-    return math == NNV_MATH_TF32 && (L.C % 4) == 0 && 4ull * L.C * L.H * L.W >= 131072ull && L.R <= 16 && L.S <= 16 &&
-           L.pad <= 8;
+    return ((math == NNV_MATH_TF32 && (L.C % 4) == 0) || (math == NNV_MATH_BF16 && (L.C % 8) == 0 && tuning().bf16cvt)) &&
+           4ull * L.C * L.H * L.W >= 131072ull && L.R <= 16 && L.S <= 16 && L.pad <= 8;
 }
 
 bool wino_fused_applies(const nnv_layer_desc_t& L, int v, int math) {

@@ -188,5 +188,40 @@ def test_workspace_too_small_is_reported():
     plan = nb.Plan(layers, [0], [0])
     buf = poisoned(1 << 20)
     with pytest.raises(nb.NnvError) as e:
-        nb.nnv_conv_exec(plan, 0, nb.VAR_IM2COL, nb.MATH_BF16, buf, None, buf, None, buf, buf, 1024, torch.cuda.current_stream())
+        nb.nnv_conv_exec(plan, 0, nb.VAR_WINO_F4, nb.MATH_TF32, buf, None, buf, None, buf, buf, 1024, torch.cuda.current_stream())
     assert e.value.status == 4
+
+
+@pytest.mark.parametrize("shape", [
+    # C, K, R, stride, H, W
+    (64, 64, 3, 1, 56, 56),           # implicit im2col, bf16 rounding inside the GEMM
+    (128, 128, 3, 1, 28, 28),         # K split over a cluster
+    (256, 512, 3, 2, 28, 28),         # stride 2
+    (256, 64, 1, 1, 56, 56),          # 1x1: the activation itself is the operand
+    (64, 24, 1, 1, 57, 43),           # ragged pixels, K = 24
+    (40, 72, 3, 1, 64, 64),           # C = 40: the last channel block is partly outside the tensor
+])
+def test_bf16_math_without_a_bf16_copy_of_the_activation(shape):
+    """BF16-class GEMM layers whose fp32 activation is rounded to bf16 inside the kernel (no Xcol matrix, no scratch)
+    against the oracle, and against the explicit bf16 im2col path: the same rounded operands, so fp32-rounding apart."""
+    C, K, R, stride, H, W = shape
+    L = dict(op=0, C=C, K=K, R=R, S=R, stride=stride, pad=R // 2, groups=1, H=H, W=W, in0=-1, in1=-1, act=1, has_bias=1)
+    rng = np.random.default_rng([51] + list(shape))
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((K, C, R, R)) * np.sqrt(2.0 / (C * R * R))).astype(np.float32)
+    b = rng.uniform(-1, 1, K).astype(np.float32)
+    ref = omodel.run_layer(L, x, w, b, None)
+    v = nb.VAR_GEMM1X1 if R == 1 else nb.VAR_IM2COL
+    plan = nb.Plan([L], [0], [0])
+    assert nb.nnv_exec_workspace_bytes(plan, 0, v, nb.MATH_BF16) == 0
+    y = run_conv(plan, 0, L, v, nb.MATH_BF16, x, w, b, None)
+    assert_conv_close(y, ref, TOL[nb.MATH_BF16], "rounded in the kernel")
+    nb.nnv_tuning_set("bf16cvt=0")
+    try:
+        plan2 = nb.Plan([L], [0], [0])
+        assert nb.nnv_exec_workspace_bytes(plan2, 0, v, nb.MATH_BF16) > 0
+        y2 = run_conv(plan2, 0, L, v, nb.MATH_BF16, x, w, b, None)
+    finally:
+        nb.nnv_tuning_set(None)
+    assert_conv_close(y2, ref, TOL[nb.MATH_BF16], "explicit bf16 im2col")
+    assert rel_l2(y, y2) <= 1e-5, rel_l2(y, y2)

@@ -34,7 +34,7 @@ def _run_static(plan, i, L, variant, math, x_chw, w, addend_chw=None):
 
 
 @pytest.mark.parametrize("variant,math", [(nb.VAR_WINO_F2, nb.MATH_TF32), (nb.VAR_WINO_F4, nb.MATH_TF32),
-                                          (nb.VAR_IM2COL, nb.MATH_BF16)])
+                                          (nb.VAR_WINO_F2, nb.MATH_BF16)])
 def test_static_scratch_matches_conv_exec_on_two_calls_in_a_row(variant, math):
     layers = wl.cfg1()
     L = layers[0]
@@ -55,8 +55,8 @@ def test_static_scratch_matches_conv_exec_on_two_calls_in_a_row(variant, math):
 def test_static_scratch_refuses_layers_that_do_not_fit():
     L = dict(op=0, C=64, K=64, R=3, S=3, stride=1, pad=1, groups=1, H=224, W=224, in0=-1, in1=-1, act=1, has_bias=0)
     plan = nb.Plan([L], [0], [0])
-    assert nb.nnv_exec_workspace_bytes(plan, 0, nb.VAR_IM2COL, nb.MATH_BF16) > nb.STATIC_SCRATCH_BYTES
+    assert nb.nnv_exec_workspace_bytes(plan, 0, nb.VAR_WINO_F4, nb.MATH_TF32) > nb.STATIC_SCRATCH_BYTES
     buf = poisoned(1 << 20)
     with pytest.raises(nb.NnvError) as e:
-        nb.nnv_conv_exec_static(plan, 0, nb.VAR_IM2COL, nb.MATH_BF16, buf, None, buf, None, buf, torch.cuda.current_stream())
+        nb.nnv_conv_exec_static(plan, 0, nb.VAR_WINO_F4, nb.MATH_TF32, buf, None, buf, None, buf, torch.cuda.current_stream())
     assert e.value.status == 4 and "scratch" in str(e.value)
