@@ -162,6 +162,8 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* plan);
  *   winofused=auto|0|1    F(2x2,3x3) with TF32 math as one kernel (input transform, tile GEMMs, output transform)
  *   smallp=0|1|N          the weights-on-rows kernel for layers of at most 256 pixels: off, on, on with N K splits
  *   side=0|1  merge=0|1  group=0|1   side stream for residual branches, merged reads, grouped transforms
+ *   copies_first=0|1      merged reads are all put on the copy stream before the first kernel (1, default) or layer by layer
+ *   chunk=first_kb,max_kb merged reads: size target of the first copy (>= 16) and the size the targets double up to
  * Every call replaces all settings (unnamed keys return to their defaults).  An item that does not
  * parse or is out of range -> NNV_ERR_INVALID_ARG and nothing changes; a setting that does not fit a
  * particular layer (more splits than K blocks, a tiling beyond shared memory) is ignored for it. */
@@ -604,6 +606,15 @@ nnv_status_t nnv_last_enqueue_ns(const nnv_plan_t* plan, uint64_t* ns);
  * microseconds of their own and serialise the streams, the stamps do not disturb the run they
  * measure.  Both arrays hold one entry per layer; either may be NULL.  Synchronises the device. */
 nnv_status_t nnv_kernel_times(const nnv_plan_t* plan, uint64_t* xform_ns, uint64_t* exec_ns);
+
+/* The same stamps as a timeline: xform_span[2i], xform_span[2i+1] = start and end of layer i's
+ * weight-transform launch, exec_span[2i], exec_span[2i+1] = the same for its tensor-core GEMM
+ * kernel, in nanoseconds of the device clock counted from the earliest stamped start of the run
+ * (0, 0 where no stamped kernel ran for the layer).  A transform starts when its copy has landed,
+ * so the spans show where a cold run (Section 3.1.3: read, transform and execution of different
+ * layers overlapping) waits for the link and where for the kernels.  Both arrays hold two entries
+ * per layer; either may be NULL.  Synchronises the device. */
+nnv_status_t nnv_kernel_spans(const nnv_plan_t* plan, uint64_t* xform_span, uint64_t* exec_span);
 
 /* Profile every eligible (variant, math) of every conv layer in isolation --
  * the per-operation profiling that feeds the paper's Algorithm 1 -- and write

@@ -114,6 +114,7 @@ _SIGS = {
     "nnv_layer_output": [_vp, _i32, _P(_vp), _P(_u64)],
     "nnv_last_enqueue_ns": [_vp, _P(_u64)],
     "nnv_kernel_times": [_vp, _P(_u64), _P(_u64)],
+    "nnv_kernel_spans": [_vp, _P(_u64), _P(_u64)],
     "nnv_profile_arena_bytes": [_vp, _P(_u64)],
     "nnv_profile": [_vp, _vp, _u64, _vp, _vp, _u64, _vp, _i32, _P(Cost), _i32, _P(_i32)],
     "nnv_device_status": [_P(_i32)],
@@ -229,6 +230,8 @@ def nnv_exec_workspace_bytes(plan, layer, variant, math):
 
 
 def _choices_array(plan, choices):
+    if isinstance(choices, ctypes.Array):                 # already marshalled (choices_array): latency-critical callers
+        return choices
     arr = (Choice * plan.n)()
     for i, c in enumerate(choices):
         if c is None:
@@ -236,6 +239,12 @@ def _choices_array(plan, choices):
         else:
             arr[i] = Choice(int(c[0]), int(c[1]), int(c[2]))
     return arr
+
+
+def choices_array(plan, choices):
+    """The per-layer choices as the C array the run calls take; building it once keeps ~1 us per layer of Python
+    out of every call that passes it."""
+    return _choices_array(plan, choices)
 
 
 def nnv_arena_bytes(plan, choices, depth):
@@ -588,6 +597,13 @@ def nnv_kernel_times(plan):
     xf, ex = (_u64 * plan.n)(), (_u64 * plan.n)()
     _check(_lib.nnv_kernel_times(plan.handle, xf, ex))
     return [int(v) for v in xf], [int(v) for v in ex]
+
+
+def nnv_kernel_spans(plan):
+    """Per layer ((xform_start, xform_end), (exec_start, exec_end)) in ns from the run's earliest stamped kernel start."""
+    xf, ex = (_u64 * (2 * plan.n))(), (_u64 * (2 * plan.n))()
+    _check(_lib.nnv_kernel_spans(plan.handle, xf, ex))
+    return [((int(xf[2 * i]), int(xf[2 * i + 1])), (int(ex[2 * i]), int(ex[2 * i + 1]))) for i in range(plan.n)]
 
 
 def nnv_last_enqueue_ns(plan):

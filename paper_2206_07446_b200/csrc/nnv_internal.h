@@ -149,6 +149,8 @@ struct Tuning {
     int convp = 0;                            // persistent 3x3 kernel: 0 auto, 1 off, 2 forced with the values below
     int convp_bn = 0, convp_per_sm = 0, convp_na = 0, convp_nb = 0;
     int side = 1, merge = 1, group = 1;       // pipeline features: side stream, merged reads, grouped transforms
+    int copies_first = 1;                     // merged reads all enqueued before the first kernel
+    int chunk_first_kb = 256, chunk_max_kb = 16384;   // merged reads: size target of the first chunk, doubling up to the maximum
     int winofused = -1;                       // the one-kernel F(2x2,3x3) path: -1 the library decides, 0 off, 1 on where it applies
     int bf16cvt = 1;                          // BF16 math straight from the fp32 activation (rounded inside the GEMM); 0: explicit bf16 im2col
     int smallp = 1;                           // the weights-on-rows kernel for layers with few pixels

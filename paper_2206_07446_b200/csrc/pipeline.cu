@@ -150,8 +150,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     // its stream (measured: 64 MB as 1 MB copies moves at 45 GB/s, as 4 MB copies at 52, as one copy at
     // 55), so at depth 0 (where the arena mirrors the host blobs' layouts) consecutive layers whose source
     // and destination ranges line up are read by ONE copy.  The chunks start at 256 KB, so that execution
-    // begins early, and double up to 4 MB; all layers of a chunk become ready when it lands, and their
-    // weight transforms are one grouped launch.
+    // begins early, and double up to 16 MB (measured on the ResNet-50-shaped model: 1.84 ms with 4 MB chunks,
+    // 1.80 ms with 16 MB ones, 1.71 ms for one bulk copy of the same bytes); all layers of a chunk become ready
+    // when it lands, and their weight transforms are one grouped launch.
     struct CopyChunk { const uint8_t* src; uint8_t* dst; uint64_t bytes; int first, last; bool zero_copy; };
     std::vector<CopyChunk> chunks;
     std::vector<int> chunk_of(n, -1);
@@ -172,9 +173,12 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         merge = (double)bytes / 50e3 > 8.0 * convs;              // us
     }
     if (merge) {
-        constexpr uint64_t kFirstTarget = 256u << 10, kMaxTarget = 4u << 20, kMaxGap = 4096;
+        const uint64_t kFirstTarget = (uint64_t)tn.chunk_first_kb << 10, kMaxTarget = (uint64_t)tn.chunk_max_kb << 10;
+        constexpr uint64_t kMaxGap = 4096;
         uint64_t target = kFirstTarget;
-        int cur_kind = -1;
+        int cur_kind = -1, last_conv = -1;
+        for (int i = 0; i < n; ++i)
+            if (p->layers[i].op == NNV_OP_CONV) last_conv = i;
         for (int i = 0; i < n; ++i) {
             const nnv_layer_desc_t& L = p->layers[i];
             if (L.op != NNV_OP_CONV) continue;
@@ -186,7 +190,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
             uint8_t* dst = (uint8_t*)d_arena + (cached ? A.xf_off[i] : A.raw_off[i]);
             const uint64_t len = cached ? transformed_bytes(*p, i, ch.variant, ch.math) : raw_weight_bytes(L);
             bool joined = false;
-            if (!chunks.empty() && cur_kind == kind) {
+            if (!chunks.empty() && cur_kind == kind && i != last_conv) {   // the last layer's copy is its own: nothing but its
+                                                                          // transform and execution then follows the last byte
                 CopyChunk& c = chunks.back();
                 if (src >= c.src + c.bytes && (uint64_t)(src - (c.src + c.bytes)) <= kMaxGap && src - c.src == dst - c.dst &&
                     c.bytes < target && i - c.first < XF_BATCH_MAX) {
@@ -227,13 +232,39 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
         NNV_CUDA(cudaStreamWaitEvent(s_xform, p->ev[3 * n], 0));
     }
 
-    // model input: NCHW -> device NHWC, on the execution stream
+    // The merged reads.  Nothing orders a chunk's copy behind any kernel (at depth 0 every layer has its own place in
+    // the arena), and the link is what the run waits for, so when the weights are already in host memory ALL copies go
+    // on the copy stream before anything else is enqueued: the link then never waits for the host to get through the
+    // launches of earlier layers (measured on the ResNet-50-shaped model: the second to fourth chunk used to land
+    // 15-35 us late each).  With a storage reader in front the copies stay in layer order, each behind its arrival.
+    std::vector<char> chunk_issued(chunks.size(), 0);
+    auto issue_chunk_copy = [&](int ci) -> nnv_status_t {
+        if (chunk_issued[ci]) return NNV_OK;
+        chunk_issued[ci] = 1;
+        const CopyChunk& c = chunks[ci];
+        for (int k = c.first; k <= c.last; ++k)
+            if (before_read && p->layers[k].op == NNV_OP_CONV) NNV_TRY((*before_read)(k));
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(c.first, 0), s_copy));
+        if (!c.zero_copy) NNV_CUDA(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, s_copy));
+        for (int k = c.first; k <= c.last; ++k) {
+            const nnv_layer_desc_t& Lk = p->layers[k];
+            if (Lk.op == NNV_OP_CONV && Lk.has_bias)
+                NNV_CUDA(cudaMemcpyAsync(base + A.bias_off[k], (const uint8_t*)weights + Lk.b_off, 4ull * Lk.K, cudaMemcpyHostToDevice, s_copy));
+        }
+        if (tm) NNV_CUDA(cudaEventRecord(TEV(c.first, 1), s_copy));
+        NNV_CUDA(cudaEventRecord(EV(c.first, 0), s_copy));
+        return NNV_OK;
+    };
+    // model input: NCHW -> device NHWC, on the execution stream (its copy ahead of the weights': copies of one
+    // direction are served in the order they were submitted, whatever their streams)
     const nnv_layer_desc_t& L0 = p->layers[0];
     const float* in_chw = input;
     if (host_io) {
         NNV_CUDA(cudaMemcpyAsync(base + A.in_chw, input, 4ull * L0.C * L0.H * L0.W, cudaMemcpyHostToDevice, s_exec));
         in_chw = (const float*)(base + A.in_chw);
     }
+    if (merge && !before_read && tn.copies_first)
+        for (size_t ci = 0; ci < chunks.size(); ++ci) NNV_TRY(issue_chunk_copy((int)ci));
     NNV_TRY(launch_chw_to_hwc(in_chw, (float*)(base + A.in_hwc), L0.C, L0.H, L0.W, s_exec));
     if (any_side) NNV_CUDA(cudaEventRecord(ev_input, s_exec));
 
@@ -361,19 +392,8 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
                 ready = EV(i, 1);
             } else if (merge) {
                 const CopyChunk& c = chunks[chunk_of[i]];
-                if (c.first == i) {                             // the chunk's one copy, issued with its first layer
-                    for (int k = c.first; k <= c.last; ++k)
-                        if (before_read && p->layers[k].op == NNV_OP_CONV) NNV_TRY((*before_read)(k));
-                    if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 0), s_copy));
-                    if (!c.zero_copy) NNV_CUDA(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, s_copy));
-                    for (int k = c.first; k <= c.last; ++k) {
-                        const nnv_layer_desc_t& Lk = p->layers[k];
-                        if (Lk.op == NNV_OP_CONV && Lk.has_bias)
-                            NNV_CUDA(cudaMemcpyAsync(base + A.bias_off[k], (const uint8_t*)weights + Lk.b_off, 4ull * Lk.K,
-                                                     cudaMemcpyHostToDevice, s_copy));
-                    }
-                    if (tm) NNV_CUDA(cudaEventRecord(TEV(i, 1), s_copy));
-                    NNV_CUDA(cudaEventRecord(EV(i, 0), s_copy));
+                if (c.first == i) {                             // the chunk's one copy (unless issued ahead) ...
+                    NNV_TRY(issue_chunk_copy(chunk_of[i]));
                     // the weight transforms of the chunk's layers: one grouped launch behind the copy
                     std::vector<XformDesc> descs;
                     for (int k = c.first; k <= c.last; ++k) {
@@ -875,7 +895,8 @@ nnv_status_t nnv_cold_run_file(nnv_plan_t* p, const nnv_choice_t* choices, const
     return NNV_OK;
 }
 
-nnv_status_t nnv_kernel_times(const nnv_plan_t* p, uint64_t* xform_ns, uint64_t* exec_ns) {
+// Reads the stamp array of the plan's most recent run: per layer and slot, {start, end} in device-clock ns (0, 0 = no launch).
+static nnv_status_t read_stamps(const nnv_plan_t* p, std::vector<uint64_t>* out) {
     NNV_REQUIRE(p, NNV_ERR_INVALID_ARG, "null argument");
     const int n = (int)p->layers.size();
     NNV_REQUIRE(p->opts.kernel_stamps && p->stamped_layers == n, NNV_ERR_STATE,
@@ -885,13 +906,41 @@ nnv_status_t nnv_kernel_times(const nnv_plan_t* p, uint64_t* xform_ns, uint64_t*
     std::vector<unsigned long long> h((size_t)2 * STAMP_SLOTS_PER_LAYER * n);
     NNV_CUDA(cudaDeviceSynchronize());
     NNV_CUDA(cudaMemcpy(h.data(), base, sizeof(unsigned long long) * h.size(), cudaMemcpyDeviceToHost));
+    out->assign(h.size(), 0);
+    for (size_t j = 0; j < h.size(); j += 2) {
+        const uint64_t start = ~h[j], end = h[j + 1];       // the start slot holds the maximum of ~clock over the blocks
+        if (h[j] != 0 && end >= start) { (*out)[j] = start; (*out)[j + 1] = end; }
+    }
+    return NNV_OK;
+}
+
+nnv_status_t nnv_kernel_times(const nnv_plan_t* p, uint64_t* xform_ns, uint64_t* exec_ns) {
+    std::vector<uint64_t> h;
+    NNV_TRY(read_stamps(p, &h));
+    const int n = (int)p->layers.size();
     for (int i = 0; i < n; ++i)
         for (int w = 0; w < STAMP_SLOTS_PER_LAYER; ++w) {
-            const unsigned long long ns = h[2 * (STAMP_SLOTS_PER_LAYER * i + w)], ne = h[2 * (STAMP_SLOTS_PER_LAYER * i + w) + 1];
-            const uint64_t start = ~ns;
-            const uint64_t d = (ns != 0 && ne >= start) ? ne - start : 0;
+            const size_t j = 2 * ((size_t)STAMP_SLOTS_PER_LAYER * i + w);
             uint64_t* dst = w == 0 ? xform_ns : exec_ns;
-            if (dst) dst[i] = d;
+            if (dst) dst[i] = h[j + 1] - h[j];
+        }
+    return NNV_OK;
+}
+
+nnv_status_t nnv_kernel_spans(const nnv_plan_t* p, uint64_t* xform_span, uint64_t* exec_span) {
+    std::vector<uint64_t> h;
+    NNV_TRY(read_stamps(p, &h));
+    const int n = (int)p->layers.size();
+    uint64_t t0 = ~0ull;
+    for (size_t j = 0; j < h.size(); j += 2)
+        if (h[j + 1]) t0 = std::min(t0, h[j]);
+    for (int i = 0; i < n; ++i)
+        for (int w = 0; w < STAMP_SLOTS_PER_LAYER; ++w) {
+            const size_t j = 2 * ((size_t)STAMP_SLOTS_PER_LAYER * i + w);
+            uint64_t* dst = w == 0 ? xform_span : exec_span;
+            if (!dst) continue;
+            dst[2 * i] = h[j + 1] ? h[j] - t0 : 0;
+            dst[2 * i + 1] = h[j + 1] ? h[j + 1] - t0 : 0;
         }
     return NNV_OK;
 }

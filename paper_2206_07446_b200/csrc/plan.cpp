@@ -86,6 +86,11 @@ static const char* parse_tuning(const char* spec, Tuning* t, char* item, size_t 
             ok = flag(&t->merge);
         } else if (!std::strcmp(key, "group")) {
             ok = flag(&t->group);
+        } else if (!std::strcmp(key, "copies_first")) {
+            ok = flag(&t->copies_first);
+        } else if (!std::strcmp(key, "chunk")) {
+            ok = std::sscanf(val, "%d,%d", &a, &b) == 2 && a >= 16 && b >= a && b <= (1 << 20);
+            if (ok) { t->chunk_first_kb = a; t->chunk_max_kb = b; }
         }
         if (!ok) { *eq = '='; return item; }
     }
