@@ -75,6 +75,7 @@ def parse():
     ap.add_argument("--R", type=int, default=3)
     ap.add_argument("--stride", type=int, default=1)
     ap.add_argument("--H", type=int, default=56)
+    ap.add_argument("--W", type=int, default=0, help="image width of --kernel conv (0 = H)")
     ap.add_argument("--groups", type=int, default=1)
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--no-flush", action="store_true")
@@ -1003,7 +1004,7 @@ def run_kernel(args):
     elif a.kernel == "conv":
         v = nb.VARIANT_NAMES.index(a.variant)
         m = nb.MATH_FP32 if v in (nb.VAR_DIRECT, nb.VAR_DEPTHWISE) else math
-        print(json.dumps(time_conv(torch, nb, v, m, a.C, a.K, a.R, a.stride, a.H, a.H, a.groups, a.reps, flush)))
+        print(json.dumps(time_conv(torch, nb, v, m, a.C, a.K, a.R, a.stride, a.H, a.W or a.H, a.groups, a.reps, flush)))
     else:
         shapes = [(64, 64, 3, 1, 56), (128, 128, 3, 1, 28), (256, 256, 3, 1, 14), (512, 512, 3, 1, 7),
                   (64, 64, 3, 1, 224), (128, 128, 3, 1, 112), (256, 256, 3, 1, 56), (512, 512, 3, 1, 28),

@@ -157,6 +157,8 @@ nnv_status_t nnv_plan_destroy(nnv_plan_t* plan);
  *   gemm_ring=N           shared-memory ring depth 2..8        gemm_prefill=0|1
  *   conv3x3=off|auto|MT,BN,splits[,boxes,weight_tiles]          the halo-resident 3x3 kernel
  *   conv3x3p=off|BN,ctas_per_sm[,boxes,weight_tiles]           the persistent form of the 3x3 kernel (off unless asked for)
+ *   conv3x3w=off|auto|on  the weights-stationary form of the 3x3 kernel (layers whose weight slice fits shared memory):
+ *                         on = wherever it fits; auto and off = never (it measured slower than the one-tile kernel)
  *   bf16cvt=0|1           BF16-math GEMMs read the fp32 activation and round it inside the kernel (1, default) or
  *                         from an explicit bf16 im2col matrix (0)
  *   winofused=auto|0|1    F(2x2,3x3) with TF32 math as one kernel (input transform, tile GEMMs, output transform)

@@ -27,12 +27,14 @@ struct ConvDev {
     const float* addend;
     int C, H, W, K;                 // input channels, image (input = output grid), output channels
     int BN, MT, act, tmem_cols, splits, na, nb, cblk, tiles_w;
+    int tma_out;                    // 0: plain stores; 16 / 32: columns per TMA-stored sub-tile (no K split, no addend)
 };
 
 constexpr int CONV_MAX_NA = 4, CONV_MAX_NB = 8;
 
 __global__ void __launch_bounds__(GEMM_THREADS)
-conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const ConvDev g) {
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmD, const ConvDev g) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -59,6 +61,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+        if (g.tma_out) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmD)) : "memory");
         for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
         for (int s = 0; s < NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
         mbar_init(tmem_full_bar, 1);
@@ -143,6 +146,48 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int row = quarter * 32 + lane;                  // MMA row = 8 * (patch row) + (patch column)
         if (!ok) {
             if (lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        } else if (splits == 1 && g.tma_out) {
+            // Write-out by TMA.  A warp's 32 accumulator rows are 4 image rows x 8 pixels of the patch: per chunk of CW
+            // output channels the lanes write their rows (+ bias, activation) into a sub-tile in the swizzled layout of
+            // the output tensor map {K, W, H}, box {CW, 8, 4}, and one lane stores it; pixels and channels outside the
+            // tensor are clipped by the TMA.  The sub-tiles reuse the rings, which are idle by now.
+            const int CW = g.tma_out, nch = BN / CW;
+            const uint32_t chunk_bytes = 32u * (uint32_t)CW * 4u;
+            for (int mt = 0; mt < MT; ++mt) {
+                const int oh = oh0 + mt * 16 + quarter * 4;
+                for (int j = 0; j < nch; ++j) {
+                    const uint32_t buf = sbase + (uint32_t)((mt * nch + j) * 4 + quarter) * chunk_bytes;
+                    const uint32_t rowa = buf + (uint32_t)lane * (uint32_t)CW * 4u;
+                    const int nbase = n0 + j * CW;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (h * 16 >= CW) break;
+                        uint32_t r[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mt * BN + j * CW + h * 16), r);
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            const int c = h * 4 + c4;                       // 16-byte chunk of the row
+                            const int n = nbase + c * 4;
+                            const uint32_t sw = (CW == 32) ? (uint32_t)(c ^ (lane & 7)) : (uint32_t)(c ^ ((lane >> 1) & 3));
+                            float4 v = make_float4(__uint_as_float(r[c4 * 4]), __uint_as_float(r[c4 * 4 + 1]),
+                                                   __uint_as_float(r[c4 * 4 + 2]), __uint_as_float(r[c4 * 4 + 3]));
+                            if (g.bias && n < g.K) {
+                                const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+                                v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                            }
+                            v.x = act_fn(v.x, g.act); v.y = act_fn(v.y, g.act); v.z = act_fn(v.z, g.act); v.w = act_fn(v.w, g.act);
+                            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(rowa + sw * 16u), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA's reads
+                    __syncwarp();
+                    if (lane == 0 && oh < g.H && ow0 < g.W && nbase < g.K) {
+                        tma_store_3d(&tmD, buf, nbase, ow0, oh);
+                        tma_store_commit();
+                    }
+                }
+            }
+            if (lane == 0) tma_store_wait_read();
         } else if (splits == 1) {
             // Each warp turns its 32 accumulator rows (one pixel per lane) into pixel-contiguous
             // stores through a private 32 x 32 staging tile (row pitch 36 words; both rings are idle
@@ -484,6 +529,200 @@ conv3x3_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __gr
                 __syncwarp();                                 // the staging tile is rewritten by the next chunk
             }
         }
+        if (!ok && lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0) stamp_end(g.stamp);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)g.tmem_cols) : "memory");
+    }
+}
+
+// ---- weights-stationary form ---------------------------------------------------------------------
+// For layers whose whole weight slice of one channel tile fits shared memory (C x BN <= 4096 words per tap, e.g.
+// 64 -> 64): every CTA of the one-tile kernel above re-reads that slice from L2 (147 KB for 46 KB of activation boxes
+// per channel block), and on an SM the fill of shared memory, not the tensor pipe, is what the tile rate waits for.
+// Here one CTA per SM loads its channel tile's 9 x C/32 weight tiles ONCE, each behind its own barrier so that the
+// first MMAs start as soon as the first tap has landed, and then walks over output patches p = blockIdx.x,
+// blockIdx.x + gridDim.x, ...: per patch only the halo boxes move.  TMEM holds two accumulators (the MMAs of patch
+// t+1 run while patch t is written out), and the write-out goes through swizzled sub-tiles and TMA stores as above
+// (one sub-tile per warp: a warp waits for its previous store to have read it before the next chunk overwrites it).
+struct ConvWDev {
+    unsigned long long* stamp;
+    const float* bias;
+    int C, H, W, K;
+    int BN, act, tmem_cols, cblk, tiles_w, patches, cw;       // cw: columns per stored sub-tile (16 or 32)
+};
+
+constexpr int CONVW_NA = 3;                                    // halo boxes in flight
+constexpr int CONVW_MAX_WT = 36;                               // weight tiles (9 taps x up to 4 channel blocks)
+
+__global__ void __launch_bounds__(GEMM_THREADS)
+conv3x3_tc_ws_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const __grid_constant__ CUtensorMap tmD, const ConvWDev g) {
+    extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int BN = g.BN, NWT = 9 * g.cblk;
+    constexpr uint32_t a_slot_bytes = 18u * 1024u;                 // (16 + 2) rows of 8 pixels x 128 bytes
+    const uint32_t w_tile_bytes = (uint32_t)BN * BK_BYTES;
+    const uint32_t w_base = sbase, a_ring = sbase + (uint32_t)NWT * w_tile_bytes;
+    const uint32_t stage0 = a_ring + CONVW_NA * a_slot_bytes;      // 4 warps x one sub-tile of 32 rows x 32 words
+    const uint32_t bars = stage0 + 4u * 4096u;
+    auto w_full = [&](int i) { return bars + 8u * i; };
+    auto a_full = [&](int s) { return bars + 8u * (CONVW_MAX_WT + s); };
+    auto a_empty = [&](int s) { return bars + 8u * (CONVW_MAX_WT + CONVW_NA + s); };
+    auto t_full = [&](int a) { return bars + 8u * (CONVW_MAX_WT + 2 * CONVW_NA + a); };
+    auto t_empty = [&](int a) { return bars + 8u * (CONVW_MAX_WT + 2 * CONVW_NA + 2 + a); };
+    const uint32_t holder = bars + 8u * (CONVW_MAX_WT + 2 * CONVW_NA + 4);
+    volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.y * BN;
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmD)) : "memory");
+        for (int i = 0; i < NWT; ++i) mbar_init(w_full(i), 1);
+        for (int s = 0; s < CONVW_NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(t_full(a), 1); mbar_init(t_empty(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder), "r"((uint32_t)g.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *holder_ptr;
+    pdl_wait();                                               // set-up above overlaps the previous kernel's tail
+    if (threadIdx.x == 32) stamp_start(g.stamp);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int sa = 0;
+            uint32_t pa = 0;
+            bool first = true;
+            for (int t = blockIdx.x; t < g.patches && ok; t += gridDim.x) {
+                const int tile_h = t / g.tiles_w, tile_w = t - tile_h * g.tiles_w;
+                const int oh0 = tile_h * 16, ow0 = tile_w * 8;
+                for (int cbi = 0; cbi < g.cblk && ok; ++cbi) {
+                    const int c0 = cbi * 32;
+                    for (int s = 0; s < 3; ++s) {
+                        ok = mbar_wait(a_empty(sa), pa ^ 1u);
+                        if (!ok) break;
+                        mbar_expect_tx(a_full(sa), a_slot_bytes);
+                        tma_load_3d(a_ring + sa * a_slot_bytes, &tmA, c0, ow0 + s - 1, oh0 - 1, a_full(sa));
+                        if (++sa == CONVW_NA) { sa = 0; pa ^= 1u; }
+                        if (first) {                              // the weight tiles, in the order the MMAs will want them
+                            for (int r = 0; r < 3; ++r) {
+                                const int wi = cbi * 9 + r * 3 + s;
+                                mbar_expect_tx(w_full(wi), w_tile_bytes);
+                                tma_load_3d(w_base + (uint32_t)wi * w_tile_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, w_full(wi));
+                            }
+                        }
+                    }
+                }
+                first = false;
+            }
+            if (!ok) {
+                atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let loads already in flight land
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            int sa = 0;
+            uint32_t pa = 0;
+            int lt = 0;                                           // this CTA's patch count so far
+            for (int t = blockIdx.x; t < g.patches && ok; t += gridDim.x, ++lt) {
+                const int acc = lt & 1;
+                ok = mbar_wait(t_empty(acc), (((uint32_t)lt >> 1) & 1u) ^ 1u);   // the epilogue has drained this accumulator
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
+                for (int cbi = 0; cbi < g.cblk && ok; ++cbi) {
+                    for (int s = 0; s < 3 && ok; ++s) {
+                        ok = mbar_wait(a_full(sa), pa);
+                        if (!ok) break;
+                        const uint32_t a_box = a_ring + sa * a_slot_bytes;
+                        for (int r = 0; r < 3; ++r) {
+                            const int wi = cbi * 9 + r * 3 + s;
+                            if (lt == 0) {                        // later patches find every weight tile in place
+                                ok = mbar_wait(w_full(wi), 0);
+                                if (!ok) break;
+                            }
+                            tc_fence_after();
+                            const uint64_t bdesc = make_smem_desc(w_base + (uint32_t)wi * w_tile_bytes);
+                            const uint64_t adesc = make_smem_desc(a_box + (uint32_t)r * 1024u);
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk)
+                                umma<false>(tmem_d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (cbi | s | r | kk) ? 1u : 0u);
+                        }
+                        if (ok) umma_commit(a_empty(sa));
+                        if (++sa == CONVW_NA) { sa = 0; pa ^= 1u; }
+                    }
+                }
+                if (ok) umma_commit(t_full(acc));
+            }
+            if (!ok) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+        }
+    } else {
+        const int quarter = warp & 3;                         // TMEM lanes this warp may read: 4 image rows x 8 pixels
+        const int CW = g.cw, nch = BN / CW;
+        const uint32_t buf = stage0 + (uint32_t)quarter * 4096u;
+        const uint32_t rowa = buf + (uint32_t)lane * (uint32_t)CW * 4u;
+        int lt = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < g.patches && ok; t += gridDim.x, ++lt) {
+            const int acc = lt & 1;
+            const int tile_h = t / g.tiles_w, tile_w = t - tile_h * g.tiles_w;
+            const int oh = tile_h * 16 + quarter * 4, ow0 = tile_w * 8;
+            ok = mbar_wait(t_full(acc), ((uint32_t)lt >> 1) & 1u);
+            if (!ok) break;
+            tc_fence_after();
+            for (int j = 0; j < nch; ++j) {
+                const int nbase = n0 + j * CW;
+                uint32_t ra[16], rb[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + j * CW), ra);
+                if (CW == 32) tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + j * CW + 16), rb);
+                if (j == nch - 1) {                           // every TMEM read of this patch is done: hand the accumulator back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(t_empty(acc));
+                }
+                if (lane == 0) tma_store_wait_read();         // the previous store has read the sub-tile
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {                 // 16-byte chunks of the row
+                    if (c * 4 >= CW) break;
+                    const int n = nbase + c * 4;
+                    const uint32_t sw = (CW == 32) ? (uint32_t)(c ^ (lane & 7)) : (uint32_t)(c ^ ((lane >> 1) & 3));
+                    const int q = (c & 3) * 4;
+                    float4 v = c < 4 ? make_float4(__uint_as_float(ra[q]), __uint_as_float(ra[q + 1]), __uint_as_float(ra[q + 2]), __uint_as_float(ra[q + 3]))
+                                     : make_float4(__uint_as_float(rb[q]), __uint_as_float(rb[q + 1]), __uint_as_float(rb[q + 2]), __uint_as_float(rb[q + 3]));
+                    if (g.bias && n < g.K) {
+                        const float4 bb = __ldg(reinterpret_cast<const float4*>(g.bias + n));
+                        v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                    }
+                    v.x = act_fn(v.x, g.act); v.y = act_fn(v.y, g.act); v.z = act_fn(v.z, g.act); v.w = act_fn(v.w, g.act);
+                    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(rowa + sw * 16u), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA's reads
+                __syncwarp();
+                if (lane == 0 && oh < g.H && ow0 < g.W && nbase < g.K) {
+                    tma_store_3d(&tmD, buf, nbase, ow0, oh);
+                    tma_store_commit();
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_read();
         if (!ok && lane == 0) atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
     }
     tc_fence_before();

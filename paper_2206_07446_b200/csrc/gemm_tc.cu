@@ -859,12 +859,27 @@ nnv_status_t gemm_tc_init() {
         cudaFuncSetAttribute(gemm_sp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(conv3x3_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(wino_f2_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(conv3x3_tc_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
     });
     return NNV_OK;
 }
 
+// 3-D tiled map over the NHWC fp32 output {K, W, H}: boxes of `cw` channels x 8 pixels x 4 rows (what one warp of the
+// 3x3 kernel holds), in the swizzled layout the epilogue writes.
+static nnv_status_t encode_conv_output(CUtensorMap* map, const void* base, int K, int H, int W, int cw) {
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)W, (cuuint64_t)H};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 4, (cuuint64_t)W * K * 4};
+    cuuint32_t box[3] = {(cuuint32_t)cw, 8, 4};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, cw == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (3x3 output boxes) failed with code %d", (int)r);
+    return NNV_OK;
+}
+
 static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, cudaStream_t st) {
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmD;
     NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 16 * ct.MT + 2));
     NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, ct.BN));
     ConvDev g;
@@ -875,9 +890,20 @@ static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, c
     g.BN = ct.BN; g.MT = ct.MT; g.act = a.act; g.tmem_cols = ct.tmem_cols; g.splits = ct.splits; g.na = ct.na; g.nb = ct.nb;
     g.cblk = ceil_div(a.ic.C, 32); g.tiles_w = ceil_div(a.ic.W, 8);
     NNV_REQUIRE(a.ldd == a.N, NNV_ERR_INVALID_ARG, "the 3x3 kernel writes a dense NHWC output");
+    // Write-out by TMA when nothing is added after the K loop but the bias, the output rows are 16-byte multiples and
+    // the staged tile fits into the (then idle) rings; else plain stores.
+    g.tma_out = 0;
+    const size_t rings = (size_t)ct.na * (16 * ct.MT + 2) * 1024 + (size_t)ct.nb * ct.BN * BK_BYTES;
+    if (ct.splits == 1 && !a.addend && (a.N % 4) == 0 && (reinterpret_cast<uintptr_t>(a.D) & 15) == 0 &&
+        (!a.bias || (reinterpret_cast<uintptr_t>(a.bias) & 15) == 0) && (size_t)ct.MT * BM * ct.BN * 4 <= rings) {
+        g.tma_out = (ct.BN % 32) == 0 ? 32 : 16;
+        NNV_TRY(encode_conv_output(&tmD, a.D, a.N, a.ic.H, a.ic.W, g.tma_out));
+    } else {
+        tmD = tmA;                                               // unused by the kernel, but a kernel parameter must hold a valid object
+    }
     dim3 grid(ceil_div(a.ic.H, 16 * ct.MT) * g.tiles_w, ceil_div(a.N, ct.BN), ct.splits);
     NNV_REQUIRE(grid.y <= 65535, NNV_ERR_UNSUPPORTED, "convolution grid too large");
-    (void)launch_pdl_cluster(conv3x3_tc_kernel, grid, dim3(GEMM_THREADS), ct.smem, st, ct.splits, tmA, tmB, g);
+    (void)launch_pdl_cluster(conv3x3_tc_kernel, grid, dim3(GEMM_THREADS), ct.smem, st, ct.splits, tmA, tmB, tmD, g);
     NNV_CUDA(cudaGetLastError());
     return NNV_OK;
 }
@@ -968,6 +994,45 @@ nnv_status_t launch_wino_f2_fused(const nnv_layer_desc_t& L, const LayerGeom& ge
     return NNV_OK;
 }
 
+// The weights-stationary form; `fits` tells whether the layer's weight slice and the kernel's other buffers fit.
+static size_t convw_smem_bytes(int cblk, int BN) {
+    return (size_t)1024 + (size_t)9 * cblk * BN * BK_BYTES + (size_t)CONVW_NA * 18 * 1024 + 4 * 4096 + 8 * (CONVW_MAX_WT + 2 * CONVW_NA + 5);
+}
+static bool convw_fits(const GemmArgs& a, int* BN_out) {
+    const int cblk = ceil_div(a.ic.C, 32);
+    const int BN = std::min(128, ceil_div(a.N, 16) * 16);
+    if (9 * cblk > CONVW_MAX_WT || (BN % 16) != 0 || a.addend || (a.N % 4) != 0 || a.ldd != a.N) return false;
+    if ((reinterpret_cast<uintptr_t>(a.D) & 15) != 0 || (a.bias && (reinterpret_cast<uintptr_t>(a.bias) & 15) != 0)) return false;
+    // the widest channel tile (a multiple of 16, at most 128) whose weight slice fits
+    for (int bn = BN; bn >= 16; bn -= 16) {
+        if (convw_smem_bytes(cblk, bn) <= 226u * 1024u) { *BN_out = bn; return true; }
+    }
+    return false;
+}
+static nnv_status_t launch_conv3x3_ws(const GemmArgs& a, int BN, cudaStream_t st) {
+    CUtensorMap tmA, tmB, tmD;
+    NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 18));
+    NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, BN));
+    ConvWDev g;
+    g.stamp = next_stamp();
+    next_stamp() = nullptr;
+    g.bias = a.bias;
+    g.C = a.ic.C; g.H = a.ic.H; g.W = a.ic.W; g.K = a.N;
+    g.BN = BN; g.act = a.act;
+    g.cblk = ceil_div(a.ic.C, 32); g.tiles_w = ceil_div(a.ic.W, 8);
+    g.patches = ceil_div(a.ic.H, 16) * g.tiles_w;
+    g.cw = (BN % 32) == 0 ? 32 : 16;
+    g.tmem_cols = 32;
+    while (g.tmem_cols < 2 * BN) g.tmem_cols *= 2;
+    NNV_TRY(encode_conv_output(&tmD, a.D, a.N, a.ic.H, a.ic.W, g.cw));
+    const int n_tiles = ceil_div(a.N, BN);
+    const int ctas_x = std::max(1, std::min(g.patches, 148 / n_tiles));
+    const size_t smem = convw_smem_bytes(g.cblk, BN);
+    (void)launch_pdl(conv3x3_tc_ws_kernel, dim3(ctas_x, n_tiles), dim3(GEMM_THREADS), smem, st, tmA, tmB, tmD, g);
+    NNV_CUDA(cudaGetLastError());
+    return NNV_OK;
+}
+
 // The persistent form: BN channels per tile, `per_sm` CTAs per SM, ring depths na / nb.
 static nnv_status_t launch_conv3x3_persistent(const GemmArgs& a, int BN, int per_sm, int na, int nb, cudaStream_t st) {
     CUtensorMap tmA, tmB;
@@ -1054,6 +1119,12 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         // one-tile CTAs per SM: inside one CTA the single MMA-issuing thread (about 56 cycles per tcgen05.mma
         // against 50 cycles of execution at N = 64) and the shared-memory fill bound the tile rate, and independent
         // CTAs hide both better than a second accumulator does.
+        // The weights-stationary form runs only on request.  Measured on B200 (64 -> 64, L2 flushed or not): 20.4 us on
+        // a 224 x 224 image against 13.1 for the one-tile kernel, and 5.4 us for every further patch of a CTA.  A tile load
+        // takes 1.5-2 us from request to arrival, so an SM's fill rate is its bytes in flight divided by that; the
+        // resident weights leave room for three halo boxes (55 KB) in flight where three one-tile CTAs keep 180 KB.
+        int wbn = 0;
+        if (tn.convw == 2 && convw_fits(a, &wbn)) return launch_conv3x3_ws(a, wbn, st);
         if (tn.convp == 2 && (size_t)tn.convp_bn <= (size_t)ceil_div(a.N, 16) * 16)
             return launch_conv3x3_persistent(a, tn.convp_bn, tn.convp_per_sm, tn.convp_na ? tn.convp_na : 2, tn.convp_nb ? tn.convp_nb : 4, st);
         if (use) return launch_conv3x3_tc(a, ct, st);

@@ -268,6 +268,21 @@ def test_kernel_stamps_measure_without_changing_the_result():
         assert sum(1 for i in convs if xf[i] > 0) >= 1 and all(v < total for v in xf)
         if depth:                                              # one transform launch per layer
             assert all(xf[i] > 0 for i in convs[1:])
+        # the same stamps as a timeline: same durations, the earliest start is 0, a layer's GEMM starts after the
+        # transform that produced its weights has ended, and the main branch executes in layer order
+        spans = nb.nnv_kernel_spans(stamped.plan)
+        assert [b - a for (a, b), _ in spans] == xf and [d - c for _, (c, d) in spans] == ex
+        starts = [a for (a, b), _ in spans if b] + [c for _, (c, d) in spans if d]
+        assert min(starts) == 0
+        last_xf_end = 0
+        for i in convs:
+            (a, b), (c, d) = spans[i]
+            last_xf_end = b if b else last_xf_end              # a grouped launch is booked on its first layer
+            if i == convs[0]:
+                continue                                       # (executed by the fp32 kernel: no stamp)
+            assert c >= last_xf_end > 0, (i, spans[i], last_xf_end)
+            if depth:
+                assert c >= b > a, (i, spans[i])
 
 
 def test_zero_copy_arm_is_bitwise_the_raw_arm():

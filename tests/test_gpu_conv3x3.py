@@ -101,3 +101,41 @@ def test_persistent_form_matches_the_oracle(shape):
             # the same MMAs in the same order as the one-tile kernel with this tile width: the same bits
             if bn == bn_full:
                 assert np.array_equal(y.view(np.uint32), one_tile.view(np.uint32)), (bn, per_sm, na, nb_)
+
+
+@pytest.mark.parametrize("shape", [
+    # C, K, H, W, bias + ReLU6, addend
+    (64, 64, 200, 100, True, False),    # 169 patches for 148 CTAs: some CTAs walk two patches (both accumulators, ring wrap)
+    (32, 128, 150, 90, False, False),   # one channel block, channel tile 128
+    (64, 96, 57, 59, True, False),      # ragged patches; the slice fits at a channel tile of 64 only: two tiles, the second half full
+    (128, 40, 40, 30, True, False),     # four channel blocks (36 weight tiles), channel tile 32, K = 40 clipped by the store
+    (64, 20, 100, 9, False, False),     # K = 20
+    (64, 64, 40, 24, True, True),       # a residual addend: the layer stays on the one-tile kernel
+])
+def test_weights_stationary_form_matches_the_oracle(shape):
+    """The weights-stationary 3x3 kernel (the channel tile's whole weight slice resident in shared memory, patches
+    walked by one CTA per SM, write-out by TMA): against the oracle, and bit for bit against the one-tile kernel with
+    the same channel tile, which issues the same MMAs in the same order."""
+    C, K, H, W, epi, with_add = shape
+    L = dict(op=0, C=C, K=K, R=3, S=3, stride=1, pad=1, groups=1, H=H, W=W, in0=-1, in1=-1, act=2 if epi else 1,
+             has_bias=1 if epi else 0)
+    rng = np.random.default_rng([11] + list(shape[:4]))
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((K, C, 3, 3)) * np.sqrt(2.0 / (C * 9))).astype(np.float32)
+    b = rng.uniform(-1, 1, K).astype(np.float32) if epi else None
+    add = rng.uniform(-1, 1, (K, H, W)).astype(np.float32) if with_add else None
+    ref = omodel.run_layer(L, x, w, b, add)
+    y = _run_p(L, x, w, b, add, "conv3x3w=on")
+    assert np.all(np.isfinite(y))
+    assert rel_l2(y, ref) <= TOL[nb.MATH_TF32], rel_l2(y, ref)
+    assert np.max(np.abs(y - ref)) <= 8 * TOL[nb.MATH_TF32] * np.max(np.abs(ref))
+    bn = min(128, -(-K // 16) * 16)
+    while 9 * (C // 32) * bn * 128 > 150 * 1024:
+        bn -= 16
+    one_tile = _run_p(L, x, w, b, add, "conv3x3w=off;conv3x3=1,%d,1" % bn)
+    if with_add:                                           # another kernel took the layer: fp32 summation order apart
+        assert rel_l2(y, one_tile) <= 1e-5
+    else:
+        assert np.array_equal(y.view(np.uint32), one_tile.view(np.uint32))
+    again = _run_p(L, x, w, b, add, "conv3x3w=on")
+    assert np.array_equal(y.view(np.uint32), again.view(np.uint32))
