@@ -78,11 +78,14 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     pdl_wait();                                               // set-up above overlaps the previous kernel's tail
     if (threadIdx.x == 32) stamp_start(g.stamp);
 
+    // Two producers: a shared-memory fill costs its issuing thread ~150 cycles whatever its size, so the halo boxes
+    // and the (smaller, three times as many) weight tiles are issued by different warps -- warp 2's first lane serves
+    // the weight ring before it joins the epilogue.
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
-            int sa = 0, sb = 0;                               // ring slots and their phases, carried along (no divisions:
-            uint32_t pa = 0, pb = 0;                          // every instruction of this single-thread loop is latency)
+            int sa = 0;                                       // ring slot and its phase, carried along (no divisions:
+            uint32_t pa = 0;                                  // every instruction of this single-thread loop is latency)
             for (int cbi = 0; cbi < ncb && ok; ++cbi) {
                 const int c0 = (cb0 + cbi) * 32;
                 for (int s = 0; s < 3 && ok; ++s) {
@@ -91,13 +94,6 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     mbar_expect_tx(a_full(sa), a_slot_bytes);
                     tma_load_3d(a_ring + sa * a_slot_bytes, &tmA, c0, ow0 + s - 1, oh0 - 1, a_full(sa));
                     if (++sa == NA) { sa = 0; pa ^= 1u; }
-                    for (int r = 0; r < 3; ++r) {
-                        ok = mbar_wait(b_empty(sb), pb ^ 1u);
-                        if (!ok) break;
-                        mbar_expect_tx(b_full(sb), b_slot_bytes);
-                        tma_load_3d(b_ring + sb * b_slot_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, b_full(sb));
-                        if (++sb == NB) { sb = 0; pb ^= 1u; }
-                    }
                 }
             }
             if (!ok) {
@@ -140,7 +136,30 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             else atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
         }
     } else {
-        const bool ok = mbar_wait(tmem_full_bar, 0);
+        bool ok = true;
+        if (warp == 2 && lane == 0) {                         // the weight-tile producer
+            int sb = 0;
+            uint32_t pb = 0;
+            for (int cbi = 0; cbi < ncb && ok; ++cbi) {
+                const int c0 = (cb0 + cbi) * 32;
+                for (int s = 0; s < 3 && ok; ++s) {
+                    for (int r = 0; r < 3; ++r) {
+                        ok = mbar_wait(b_empty(sb), pb ^ 1u);
+                        if (!ok) break;
+                        mbar_expect_tx(b_full(sb), b_slot_bytes);
+                        tma_load_3d(b_ring + sb * b_slot_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, b_full(sb));
+                        if (++sb == NB) { sb = 0; pb ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                atomicExch(&g_device_status, (int)NNV_ERR_TIMEOUT);
+                for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let loads already in flight land
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;       // the whole warp takes the producer's verdict
+        ok = mbar_wait(tmem_full_bar, 0) && ok;
+        ok = __all_sync(0xffffffffu, (int)ok) != 0;           // (the epilogue's TMEM reads are warp-wide instructions)
         tc_fence_after();
         const int quarter = warp & 3;                         // TMEM lanes this warp may read
         const int row = quarter * 32 + lane;                  // MMA row = 8 * (patch row) + (patch column)
