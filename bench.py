@@ -817,6 +817,24 @@ def _time(torch, fn, reps, flush):
     return statistics.median(ts), min(ts)
 
 
+def _time_rotating(torch, fns, launches, reps):
+    """Per-launch time of `launches` back-to-back launches between ONE pair of events, cycling through `fns` (the same
+    kernel on different buffer sets whose total exceeds the L2): the events' own few microseconds are shared by all
+    launches and every launch finds its data in DRAM."""
+    st = torch.cuda.current_stream()
+    ts = []
+    for r in range(reps + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for i in range(launches):
+            fns[i % len(fns)](st)
+        e1.record(st)
+        e1.synchronize()
+        if r >= 2:
+            ts.append(e0.elapsed_time(e1) * 1e3 / launches)  # us
+    return statistics.median(ts)
+
+
 def time_transform(torch, nb, variant, math, C, K, R=3, reps=20, flush=None):
     L = _layer(C, K, R, 1, 8, 8)
     plan = nb.Plan([L], [0], [0])
@@ -966,6 +984,26 @@ def other_kernel_rooflines(layers, model, nb, torch, flush, peaks):
                              ("wino_output_kernel", mb + 4 * oh * ow * L["K"], us_out)):
             rows.append({"kernel": name, "bound": "hbm", "layer": shape, "bytes": by, "us": us, "achieved": by / us / 1e3,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": by / us / 1e3 / peaks["hbm_gbs"]})
+    # The same kernels on an instance large enough for a bandwidth figure (the layers of the workloads above are 1-13 MB:
+    # a few microseconds of launch ramp and tail around 0.2-2 us of data): 64 channels on 224 x 224, F(4x4,3x3) data
+    # transforms and a 3x3 depthwise layer, eight launches per event pair over four buffer sets (> L2 in total).
+    Lb = dict(op=0, C=64, K=64, R=3, S=3, stride=1, pad=1, groups=1, H=224, W=224, in0=-1, in1=-1, act=1, has_bias=0)
+    planb = nb.Plan([Lb], [0], [0])
+    T, vb, mb = nb.nnv_wino_sizes(planb, 0, nb.VAR_WINO_F4, nb.MATH_TF32)
+    sets = [(_rand(torch, 64 * 224 * 224), _buf(torch, vb), _rand(torch, mb // 4), _buf(torch, 4 * 224 * 224 * 64)) for _ in range(4)]
+    us_in = _time_rotating(torch, [lambda st, b=b: nb.nnv_wino_input_transform(planb, 0, nb.VAR_WINO_F4, nb.MATH_TF32, b[0], b[1], st) for b in sets], 8, 5)
+    us_out = _time_rotating(torch, [lambda st, b=b: nb.nnv_wino_output_transform(planb, 0, nb.VAR_WINO_F4, b[2], None, None, b[3], st) for b in sets], 8, 5)
+    for name, by, us in (("wino_input_kernel", 4 * 64 * 224 * 224 + vb, us_in), ("wino_output_kernel", mb + 4 * 224 * 224 * 64, us_out)):
+        rows.append({"kernel": name, "bound": "hbm", "layer": "large instance: 224x224 C=64 K=64, F(4x4,3x3), %d tiles; 8 launches per event pair over 4 buffer sets" % T,
+                     "bytes": by, "us": us, "achieved": by / us / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": by / us / 1e3 / peaks["hbm_gbs"]})
+    Ld = dict(op=0, C=64, K=64, R=3, S=3, stride=1, pad=1, groups=64, H=224, W=224, in0=-1, in1=-1, act=1, has_bias=0)
+    pland = nb.Plan([Ld], [0], [0])
+    wd = _rand(torch, 64 * 9, 0.3)
+    dsets = [(_rand(torch, 64 * 224 * 224), _buf(torch, 4 * 224 * 224 * 64)) for _ in range(6)]
+    us_dw = _time_rotating(torch, [lambda st, b=b: nb.nnv_conv_exec(pland, 0, nb.VAR_DEPTHWISE, nb.MATH_FP32, b[0], None, wd, None, b[1], None, 0, st) for b in dsets], 12, 5)
+    by = 4 * (2 * 64 * 224 * 224 + 64 * 9)
+    rows.append({"kernel": "depthwise3x3_v4_kernel", "bound": "hbm", "layer": "large instance: 224x224 C=64 3x3 stride 1; 12 launches per event pair over 6 buffer sets",
+                 "bytes": by, "us": us_dw, "achieved": by / us_dw / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": by / us_dw / 1e3 / peaks["hbm_gbs"]})
     dense = [L for L in layers if L["op"] == wl.OP_CONV and L["groups"] == 1]
     if dense:
         L = max(dense, key=lambda L: wl.out_hw(L)[0] * wl.out_hw(L)[1] * L["K"] * L["C"] * L["R"] * L["S"])

@@ -1116,13 +1116,14 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         }
         // The persistent form runs only on request.  Measured on B200 (VGG-shaped layers, L2 flushed): one resident
         // CTA per SM reaches 154 TFLOP/s on 64 -> 64 @ 224 and two reach 206, against 260 for two or three
-        // one-tile CTAs per SM: inside one CTA the single MMA-issuing thread (about 56 cycles per tcgen05.mma
-        // against 50 cycles of execution at N = 64) and the shared-memory fill bound the tile rate, and independent
-        // CTAs hide both better than a second accumulator does.
+        // one-tile CTAs per SM: inside one CTA the single MMA-issuing thread (about 82 cycles per tcgen05.mma
+        // against 32 cycles of execution at N = 64) bounds the tile rate, and independent CTAs, each with its own
+        // issuing thread, lift that bound where a second accumulator does not.
         // The weights-stationary form runs only on request.  Measured on B200 (64 -> 64, L2 flushed or not): 20.4 us on
-        // a 224 x 224 image against 13.1 for the one-tile kernel, and 5.4 us for every further patch of a CTA.  A tile load
-        // takes 1.5-2 us from request to arrival, so an SM's fill rate is its bytes in flight divided by that; the
-        // resident weights leave room for three halo boxes (55 KB) in flight where three one-tile CTAs keep 180 KB.
+        // a 224 x 224 image against 12.8 for the one-tile kernel, and 5.4 us for every further patch of a CTA.  One thread
+        // issues one tcgen05.mma per ~82 cycles whatever N is, so the 72 MMAs (N = 64) of a patch take 3 us of issue time
+        // alone where the tensor pipe needs 1.2; three one-tile CTAs per SM issue from three threads, and the resident
+        // weights leave room for only three halo boxes in flight.
         int wbn = 0;
         if (tn.convw == 2 && convw_fits(a, &wbn)) return launch_conv3x3_ws(a, wbn, st);
         if (tn.convp == 2 && (size_t)tn.convp_bn <= (size_t)ceil_div(a.N, 16) * 16)

@@ -225,3 +225,30 @@ def test_bf16_math_without_a_bf16_copy_of_the_activation(shape):
         nb.nnv_tuning_set(None)
     assert_conv_close(y2, ref, TOL[nb.MATH_BF16], "explicit bf16 im2col")
     assert rel_l2(y, y2) <= 1e-5, rel_l2(y, y2)
+
+
+@pytest.mark.parametrize("shape", [
+    # C, H, W, stride, pad, bias + addend + ReLU6
+    (8, 9, 7, 1, 1, True),             # ragged grid: output width 7 = one group of four pixels and a tail of three
+    (8, 9, 7, 2, 1, True),             # stride 2, output 5 x 4
+    (32, 17, 21, 1, 0, False),         # pad 0
+    (32, 18, 22, 2, 0, True),          # stride 2, pad 0
+    (96, 112, 112, 1, 1, False),       # MobileNetV2-shaped, stride 1
+    (96, 112, 112, 2, 1, True),        # MobileNetV2-shaped, stride 2
+    (4, 1, 1, 1, 1, True),             # one pixel
+    (6, 9, 7, 1, 1, True),             # C % 4 != 0: the one-channel-per-thread kernel
+])
+def test_depthwise_kernels(shape):
+    """3x3 depthwise layers on the vectorised kernel (four channels x four output pixels per thread) and its scalar
+    fallback: fp32 arithmetic, so the fp32 tolerance, element by element."""
+    C, H, W, stride, pad, epi = shape
+    L = dict(op=0, C=C, K=C, R=3, S=3, stride=stride, pad=pad, groups=C, H=H, W=W, in0=-1, in1=-1, act=2 if epi else 1,
+             has_bias=1 if epi else 0)
+    rng = np.random.default_rng([13] + [int(v) for v in shape])
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((C, 1, 3, 3)) * np.sqrt(2.0 / 9)).astype(np.float32)
+    oh, ow = wl.out_hw(L)
+    b = rng.uniform(-1, 1, C).astype(np.float32) if epi else None
+    add = rng.uniform(-1, 1, (C, oh, ow)).astype(np.float32) if epi else None
+    seen = _check_layer([L], 0, x, w, b, add, variants=[nb.VAR_DEPTHWISE])
+    assert [s[:2] for s in seen] == [("depthwise", "fp32")]
