@@ -300,9 +300,42 @@ def gemm_bytes(L):
     return 4 * (L["C"] * L["H"] * L["W"] + L["K"] * qp + oh * ow * L["K"])
 
 
+class Ranks:
+    """The only cross-rank traffic of the benchmark: a barrier around the timed steps and the maximum of a timing over
+    the ranks.  The path itself does not shard (every rank runs its own replica), so nothing else is exchanged.
+    backend "nccl" reduces on the rank's GPU, "gloo" on the host (CPU tests)."""
+
+    def __init__(self, backend=None, device=None):
+        import torch.distributed as dist
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.device = device
+        self.dist = dist
+        if self.world > 1:
+            if backend == "nccl":
+                dist.init_process_group("nccl", device_id=device)
+            else:
+                dist.init_process_group(backend)
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+
+    def reduce_max(self, v):
+        if self.world == 1:
+            return v
+        import torch
+        t = torch.tensor([v], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_2206_07446_b200 import binding as nb
 
     rank = int(os.environ.get("RANK", "0"))
@@ -311,28 +344,25 @@ def run_ours(args):
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ranks = Ranks("nccl", torch.device("cuda", local))
     if args.tuning:
         nb.nnv_tuning_set(args.tuning)
-    line = measure(args, args.config, args.steps, args.warmup, args.minimal, rank, world, local)
+    line = measure(args, args.config, args.steps, args.warmup, args.minimal, rank, world, local, ranks)
     # the other single-GPU configurations, headline numbers and rooflines only, beside the main workload
     others = {}
     for name in [c for c in args.also.split(",") if c and c != "none" and c != args.config]:
-        o = measure(args, name, args.arm_steps, 3, True, rank, world, local)
+        o = measure(args, name, args.arm_steps, 3, True, rank, world, local, ranks)
         others[name] = {k: o[k] for k in ("value", "unit", "steps", "e2e", "roofline", "roofline_transform", "transform_all", "run", "per_layer")}
         others[name]["e2e"] = {k: o["e2e"][k] for k in ("value", "h2d_bytes_per_step", "host_link")}
     line["other_workloads"] = others
     if rank == 0:
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.close()
 
 
-def measure(args, config, steps, warmup, minimal, rank, world, local):
+def measure(args, config, steps, warmup, minimal, rank, world, local, ranks):
     """All measurements of one workload; returns the JSON line as a dict."""
     import torch
-    import torch.distributed as dist
     from paper_2206_07446_b200 import binding as nb
     from paper_2206_07446_b200 import harness
 
@@ -373,16 +403,10 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
     ev1 = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
-    def reduce_max(v):
-        if world > 1:
-            t = torch.tensor([v], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return v
+    reduce_max = ranks.reduce_max
 
     def timed_region(step_fn, steps, warmup):
         """W untimed + K timed steps between barriers; mean ms per step (max over ranks)."""
@@ -410,7 +434,9 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
     if any(c is not None and c[2] for c in choices_byp):
         model.build_cached_blob(choices_byp)
 
-    ch_raw_c = nb.choices_array(model.plan, choices_raw)
+    ch_raw_c = nb.choices_array(model.plan, choices_raw)      # marshalled once: ~1 us of Python per layer stays out of the steps
+    ch_byp_c = nb.choices_array(model.plan, choices_byp)
+    ch_res_c = nb.choices_array(model.plan, choices_res)
 
     # ---- headline: raw weights from pinned host memory, transform, execute; input / output on the device ----
     def step_value(k, timed):
@@ -451,7 +477,7 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
         # ---- bypass arm (the paper's Section 3.1.2): selection may read cached post-transform weights ----
         def step_bypass(k, timed):
             begin(k, timed, (s_copy, s_xform))
-            ch = choices_byp
+            ch = ch_byp_c
             nb.nnv_cold_run(model.plan, ch, model.h_weights, model.w_bytes, model.h_cached, model.c_bytes, model.h_input,
                             model.h_output, model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
             if timed:
@@ -470,7 +496,7 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
         for name, chz in (("zero_copy_allowed", choices_zc), ("zero_copy_every_layer", choices_zc_all)):
             need = max(need, model.ensure_arena(chz, args.cold_depth))
 
-            def step_zc(k, timed, chz=chz):
+            def step_zc(k, timed, chz=nb.choices_array(model.plan, chz)):
                 begin(k, timed, (s_copy, s_xform))
                 nb.nnv_cold_run(model.plan, chz, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
                                 model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
@@ -492,7 +518,7 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
         # ---- the headline step replayed from a recorded CUDA graph ----
         def step_graph(k, timed):
             begin(k, timed, (s_copy, s_xform))
-            ch = choices_raw
+            ch = ch_raw_c
             nb.nnv_cold_run(plan_g, ch, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
                             model.arena, model.arena.numel(), s_copy, s_xform, s_exec, args.cold_depth)
             if timed:
@@ -504,7 +530,7 @@ def measure(args, config, steps, warmup, minimal, rank, world, local):
         # ---- weights already resident in HBM: transform + execution only ----
         def step_resident(k, timed):
             begin(k, timed, (s_xform,))
-            ch = choices_res
+            ch = ch_res_c
             nb.nnv_resident_run(plan_g, ch, model.d_weights, model.w_bytes, None, 0, model.d_input, model.d_output,
                                 model.arena, model.arena.numel(), s_xform, s_exec, args.depth)
             if timed:

@@ -209,10 +209,13 @@ def test_tuning_overrides_parse_and_reject():
     """nnv_tuning_set: documented items are accepted, anything else is refused and changes nothing."""
     try:
         for ok in ("gemm_tile=64,4", "gemm_ring=6;gemm_prefill=0", "conv3x3=off", "conv3x3=auto", "conv3x3=2,64,4",
-                   "conv3x3=1,128,2,1,3", "side=0;merge=0;group=0", "", None, "gemm_tile=16,1;;side=1"):
+                   "conv3x3=1,128,2,1,3", "side=0;merge=0;group=0", "", None, "gemm_tile=16,1;;side=1",
+                   "conv3x3p=64,2,2,6", "conv3x3p=off", "conv3x3w=on", "conv3x3w=auto;conv3x3w=off", "bf16cvt=0", "winofused=auto",
+                   "smallp=0", "smallp=24", "copies_first=0", "chunk=64,8192", "chunk=256,256"):
             nb.nnv_tuning_set(ok)
         for bad in ("gemm_tile=48", "gemm_tile=24,2", "gemm_tile=64,3", "gemm_ring=9", "conv3x3=3,64,1", "conv3x3=1,64,16",
-                    "side=2", "unknown=1", "gemm_tile", "x" * 300):
+                    "side=2", "unknown=1", "gemm_tile", "x" * 300, "conv3x3w=2", "conv3x3p=24,1", "copies_first=2", "chunk=8,64",
+                    "chunk=512,256", "chunk=256", "bf16cvt=yes", "smallp=149"):
             with pytest.raises(nb.NnvError) as e:
                 nb.nnv_tuning_set(bad)
             assert e.value.status == 1, bad
