@@ -426,7 +426,11 @@ nnv_status_t nnv_hwc_to_chw(const float* d_in, float* d_out, int32_t C, int32_t 
  *   timings:   NULL, or n entries filled from CUDA events (adds event records).
  * At depth 0, when the weights' copy time is estimated to exceed the execution
  * time, consecutive layers whose host and arena ranges line up are read by one
- * copy of up to ~1 MB (the per-layer timings then share that copy's interval).
+ * copy (256 KB at first, doubling up to 16 MB, the last layer by itself; the
+ * per-layer timings then share that copy's interval, and the layers' weight
+ * transforms are one grouped launch), and all these copies are put on s_copy,
+ * in layer order, before the first kernel is enqueued, so that the host link
+ * never waits for the host (nnv_tuning_set: chunk, copies_first, merge).
  * A conv layer whose output is only ever the residual addend of a later layer
  * and which needs no execution scratch runs on a fourth stream that the plan
  * creates and owns, beside the main branch; the result is the same bit for bit.

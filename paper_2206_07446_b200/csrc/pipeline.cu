@@ -147,7 +147,7 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     const cudaEvent_t ev_input = p->ev[3 * n + 6 + NNV_MAX_QUEUES], ev_side_join = p->ev[3 * n + 7 + NNV_MAX_QUEUES];
 
     // A host-to-device copy costs ~4 us on top of its bytes even when it directly follows another one on
-    // its stream (measured: 64 MB as 1 MB copies moves at 45 GB/s, as 4 MB copies at 52, as one copy at
+    // its stream (measured: 96 MB as 1 MB copies moves at 45 GB/s, as 4 MB copies at 51, as 16 MB copies at 53, as one copy at
     // 55), so at depth 0 (where the arena mirrors the host blobs' layouts) consecutive layers whose source
     // and destination ranges line up are read by ONE copy.  The chunks start at 256 KB, so that execution
     // begins early, and double up to 16 MB (measured on the ResNet-50-shaped model: 1.84 ms with 4 MB chunks,
