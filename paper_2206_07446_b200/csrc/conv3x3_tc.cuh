@@ -157,7 +157,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let loads already in flight land
             }
         }
-        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;       // the whole warp takes the producer's verdict
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;       // the whole warp takes the producer's result
         ok = mbar_wait(tmem_full_bar, 0) && ok;
         ok = __all_sync(0xffffffffu, (int)ok) != 0;           // (the epilogue's TMEM reads are warp-wide instructions)
         tc_fence_after();
