@@ -58,6 +58,7 @@ def parse():
     ap.add_argument("--cpu-passes", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--arm-steps", type=int, default=20, help="timed steps of each side arm (bypass, graph replay, resident)")
+    ap.add_argument("--depth-steps", type=int, default=10, help="timed steps per pipeline depth of the depth sweep (0 = skip)")
     ap.add_argument("--queues", type=int, default=2, help="preparation queues for the Algorithm 1 run (0 = skip)")
     ap.add_argument("--continuous-reps", type=int, default=10, help="cold + warm sequences for the kernel-switching report (0 = skip)")
     ap.add_argument("--file-reps", type=int, default=5, help="cold runs fed from a model file on local storage (0 = skip)")
@@ -352,7 +353,7 @@ def run_ours(args):
     others = {}
     for name in [c for c in args.also.split(",") if c and c != "none" and c != args.config]:
         o = measure(args, name, args.arm_steps, 3, True, rank, world, local, ranks)
-        others[name] = {k: o[k] for k in ("value", "unit", "steps", "e2e", "roofline", "roofline_transform", "transform_all", "run", "per_layer")}
+        others[name] = {k: o[k] for k in ("value", "unit", "steps", "e2e", "roofline", "roofline_transform", "transform_all", "run", "per_layer", "pipeline_depth_ms")}
         others[name]["e2e"] = {k: o["e2e"][k] for k in ("value", "h2d_bytes_per_step", "host_link")}
     line["other_workloads"] = others
     if rank == 0:
@@ -471,6 +472,22 @@ def measure(args, config, steps, warmup, minimal, rank, world, local, ranks):
     torch.cuda.cudart().cudaProfilerStop()
     y_e2e = model.h_output.numpy().copy()
     e2e_wall = reduce_max(1e3 * sum(wall) / len(wall))
+
+    # ---- the same step at every pipeline depth (staging slots; 1 = read, transform, execute one layer after the other) ----
+    depth_ms = {}
+    if args.depth_steps > 0:
+        for d in (1, 2, 3, 4, 0):
+            need_d = model.ensure_arena(choices_raw, d)
+
+            def step_depth(k, timed, d=d, need_d=need_d):
+                begin(k, timed, (s_copy, s_xform))
+                nb.nnv_cold_run(model.plan, ch_raw_c, model.h_weights, model.w_bytes, None, 0, model.h_input, model.h_output,
+                                model.arena, need_d, s_copy, s_xform, s_exec, d)
+                if timed:
+                    ev1[k].record(s_exec)
+
+            depth_ms["unbounded" if d == 0 else str(d)] = timed_region(step_depth, min(args.depth_steps, nev), 3)[0]
+        model.ensure_arena(choices_raw, args.cold_depth)
 
     arms = {}
     if not args.minimal:
@@ -775,6 +792,7 @@ def measure(args, config, steps, warmup, minimal, rank, world, local, ranks):
         "transform_all": xall,
         "kernel_rooflines": krows,
         "per_layer": per_layer,
+        "pipeline_depth_ms": {"what": "e2e of the headline's kernels at each pipeline depth (staging slots); the headline runs unbounded", **depth_ms} if depth_ms else None,
         "arms": arms,
         "algorithm1": alg1,
         "continuous": cont,
