@@ -154,7 +154,15 @@ class Model:
             if any(c is not None and c[2] for c in choices):
                 self.build_cached_blob(choices)
             self.cold_run_queues(x_nchw, choices, queue_of, n_little, poison=False)          # warm
-            _, tm = self.cold_run_queues(x_nchw, choices, queue_of, n_little, want_timings=True, poison=False)
+            # three timed runs, per operation the median duration: one stalled run on a shared GPU must not set the factors
+            runs = [self.cold_run_queues(x_nchw, choices, queue_of, n_little, want_timings=True, poison=False)[1] for _ in range(3)]
+            tm = []
+            for per_layer in zip(*runs):
+                t = dict(per_layer[0])
+                for op in ("h2d", "xform", "exec"):
+                    t[op + "_start_ns"] = 0
+                    t[op + "_end_ns"] = sorted(r[op + "_end_ns"] - r[op + "_start_ns"] for r in per_layer)[1]
+                tm.append(t)
             rows, fac = nb.nnv_calibrate_costs(self.plan, costs, choices, tm, kinds=6 if link else 7)
             self.calibration = {k: (f[0] / f[1] if f[1] else None) for k, f in zip(("h2d", "xform", "exec"), fac)}
             table = nb.CostTable(rows)
