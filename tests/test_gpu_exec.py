@@ -252,3 +252,80 @@ def test_depthwise_kernels(shape):
     add = rng.uniform(-1, 1, (C, oh, ow)).astype(np.float32) if epi else None
     seen = _check_layer([L], 0, x, w, b, add, variants=[nb.VAR_DEPTHWISE])
     assert [s[:2] for s in seen] == [("depthwise", "fp32")]
+
+
+def _random_shapes(count, seed):
+    """Seeded layer shapes that no hand-written list would think of: ragged channels, grids, strides and pads.
+    Kept to >= 2048 outputs (the tolerance is a statement about many rounding errors, see the degenerate-shape test)
+    and to a reduction of >= 32 products per output."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        R = int(rng.choice([1, 3, 3, 5]))
+        stride = int(rng.choice([1, 1, 2]))
+        pad = int(rng.choice([0, R // 2]))
+        C = int(rng.choice([int(rng.integers(1, 48)), int(rng.integers(48, 200)), int(8 * rng.integers(1, 40))]))
+        K = int(rng.choice([int(rng.integers(1, 48)), int(rng.integers(48, 200)), int(16 * rng.integers(1, 20))]))
+        H, W = int(rng.integers(R, 48)), int(rng.integers(R, 48))
+        oh, ow = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - R) // stride + 1
+        if oh < 1 or ow < 1 or K * oh * ow < 2048 or C * R * R < 32:
+            continue
+        out.append((C, K, R, stride, pad, H, W, int(rng.integers(0, 2)), int(rng.integers(0, 2)), int(rng.integers(0, 3))))
+    return out
+
+
+@pytest.mark.parametrize("shape", _random_shapes(36, 20240607))
+def test_random_shapes_on_every_variant(shape):
+    """Every eligible variant and math mode of a randomly drawn layer against the fp64 oracle."""
+    C, K, R, stride, pad, H, W, has_bias, has_add, act = shape
+    L = dict(op=0, C=C, K=K, R=R, S=R, stride=stride, pad=pad, groups=1, H=H, W=W, in0=-1, in1=-1, act=act, has_bias=has_bias)
+    rng = np.random.default_rng([5] + [int(v) for v in shape])
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((K, C, R, R)) * np.sqrt(2.0 / (C * R * R))).astype(np.float32)
+    oh, ow = wl.out_hw(L)
+    b = rng.uniform(-1, 1, K).astype(np.float32) if has_bias else None
+    add = rng.uniform(-1, 1, (K, oh, ow)).astype(np.float32) if has_add else None
+    seen = _check_layer([L], 0, x, w, b, add)
+    assert len(seen) >= 2
+
+
+def _random_kernel_shapes(seed):
+    """Random shapes inside the domains of the two specialised tensor-core kernels: the halo 3x3 kernel (3x3, stride
+    1, pad 1, C % 32 == 0, enough patches to fill the GPU) and the weights-on-rows kernel (grids of at most 64 pixels,
+    C % 32 == 0, K % 4 == 0)."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(6):
+        out.append((int(32 * rng.integers(1, 4)), int(rng.integers(8, 140)), 3, int(rng.integers(130, 200)), int(rng.integers(100, 150)), 1))
+    for _ in range(8):
+        R = int(rng.choice([1, 3]))
+        out.append((int(32 * rng.integers(1, 17)), int(4 * rng.integers(1, 130)), R, int(rng.integers(1, 9)), int(rng.integers(1, 9)), R // 2))
+    return out
+
+
+@pytest.mark.parametrize("shape", _random_kernel_shapes(77))
+def test_random_shapes_in_the_domains_of_the_specialised_kernels(shape):
+    C, K, R, H, W, pad = shape
+    L = dict(op=0, C=C, K=K, R=R, S=R, stride=1, pad=pad, groups=1, H=H, W=W, in0=-1, in1=-1, act=1, has_bias=1)
+    rng = np.random.default_rng([6] + [int(v) for v in shape])
+    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
+    w = (rng.standard_normal((K, C, R, R)) * np.sqrt(2.0 / (C * R * R))).astype(np.float32)
+    b = rng.uniform(-1, 1, K).astype(np.float32)
+    variants = [nb.VAR_IM2COL] + ([nb.VAR_GEMM1X1] if R == 1 else [])
+    if K * H * W < 2048:                                   # few outputs: pool the error over instances (see the degenerate-shape test)
+        errs = {}
+        for inst in range(8):
+            xi = np.random.default_rng([7, inst] + [int(v) for v in shape]).uniform(-1, 1, (C, H, W)).astype(np.float32)
+            ref = omodel.run_layer(L, xi, w, b, None)
+            plan = nb.Plan([L], [0], [0])
+            for v in variants:
+                for m in _maths(v):
+                    y = run_conv(plan, 0, L, v, m, xi, w, b, None)
+                    assert np.all(np.isfinite(y))
+                    num, den = errs.get((v, m), (0.0, 0.0))
+                    errs[(v, m)] = (num + float(np.sum((y - ref) ** 2)), den + float(np.sum(ref * ref)))
+        for (v, m), (num, den) in errs.items():
+            assert np.sqrt(num / max(den, 1e-30)) <= TOL[m], (v, m, np.sqrt(num / den))
+    else:
+        seen = _check_layer([L], 0, x, w, b, None, variants=variants)
+        assert seen
