@@ -102,3 +102,45 @@ def test_transform_rejects_variants_without_transform():
     with pytest.raises(nb.NnvError) as e:
         nb.nnv_transform_weights(plan, 0, nb.VAR_DIRECT, nb.MATH_FP32, buf, buf, torch.cuda.current_stream())
     assert e.value.status == 2
+
+
+def _random_banks(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        K = int(rng.choice([int(rng.integers(1, 40)), int(rng.integers(40, 700)), int(64 * rng.integers(1, 9))]))
+        C = int(rng.choice([int(rng.integers(1, 40)), int(rng.integers(40, 700)), int(64 * rng.integers(1, 9))]))
+        out.append((K, C))
+    return out
+
+
+@pytest.mark.parametrize("K,C", _random_banks(16, 31))
+def test_random_filter_banks(K, C):
+    """Seeded random filter-bank sizes (ragged and multiples of the kernels' block sizes alike): all three Winograd
+    filter transforms to 1e-5 of the largest element, the 3x3 and 1x1 repacks byte for byte in both precisions."""
+    w = _weights(K, C, 3, 77)
+    plan = nb.Plan([_layer(C, K)], [0], [0])
+    Cp = -(-C // 8) * 8
+    for m in (2, 4, 6):
+        ref = owin.pad_channels(owin.filter_transform(w, m), Cp)
+        nbytes = nb.nnv_transformed_bytes(plan, 0, WINO[m], nb.MATH_TF32)
+        d_out = poisoned(nbytes)
+        nb.nnv_transform_weights(plan, 0, WINO[m], nb.MATH_TF32, dev(w), d_out, torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        got = d_out[:nbytes].view(torch.float32).cpu().numpy().reshape(ref.shape)
+        assert np.max(np.abs(got.astype(np.float64) - ref)) <= 1e-5 * np.max(np.abs(ref)), m
+    for R in (3, 1):
+        wr = _weights(K, C, R, 78)
+        L = _layer(C, K, R)
+        L["pad"] = R // 2
+        planr = nb.Plan([L], [0], [0])
+        variant = nb.VAR_GEMM1X1 if R == 1 else nb.VAR_IM2COL
+        for bf16 in (False, True):
+            math = nb.MATH_BF16 if bf16 else nb.MATH_TF32
+            ref = opack.pack_weights(wr, bf16=bf16)
+            nbytes = nb.nnv_transformed_bytes(planr, 0, variant, math)
+            assert nbytes == ref.nbytes
+            d_out = poisoned(nbytes)
+            nb.nnv_transform_weights(planr, 0, variant, math, dev(wr), d_out, torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            assert np.array_equal(d_out[:nbytes].cpu().numpy(), ref.view(np.uint8).reshape(-1)), (R, bf16)
