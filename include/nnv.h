@@ -424,8 +424,7 @@ nnv_status_t nnv_hwc_to_chw(const float* d_in, float* d_out, int32_t C, int32_t 
  *              receives the LAST layer's output.
  *   d_arena:   nnv_arena_bytes() bytes of device memory.
  *   timings:   NULL, or n entries filled from CUDA events (adds event records).
- * At depth 0, when the weights' copy time is estimated to exceed the execution
- * time, consecutive layers whose host and arena ranges line up are read by one
+ * At depth 0 consecutive layers whose host and arena ranges line up are read by one
  * copy (256 KB at first, doubling up to 16 MB, the last layer by itself; the
  * per-layer timings then share that copy's interval, and the layers' weight
  * transforms are one grouped launch), and all these copies are put on s_copy,

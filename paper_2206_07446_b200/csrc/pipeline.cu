@@ -157,21 +157,9 @@ static nnv_status_t run_model(nnv_plan* p, const nnv_choice_t* choices, const vo
     std::vector<CopyChunk> chunks;
     std::vector<int> chunk_of(n, -1);
     bool merge = !resident && !queued && depth == 0 && !wc && tn.merge;
-    if (merge) {
-        // Coarser copies make layers ready later (a layer waits for its whole chunk), which only pays when
-        // the link, not execution, is what the run waits for: rough estimate, bytes at 50 GB/s against
-        // 8 us per layer (measured: ResNet / VGG shapes gain 2-4 %, a MobileNetV2 shape loses 14 %).
-        uint64_t bytes = 0;
-        int convs = 0;
-        for (int i = 0; i < n; ++i) {
-            if (p->layers[i].op != NNV_OP_CONV) continue;
-            ++convs;
-            const nnv_choice_t ch = choices[i];
-            bytes += (variant_has_transform(ch.variant) && ch.cached == NNV_ARM_CACHED) ? transformed_bytes(*p, i, ch.variant, ch.math)
-                                                                       : raw_weight_bytes(p->layers[i]);
-        }
-        merge = (double)bytes / 50e3 > 8.0 * convs;              // us
-    }
+    // (Merging pays on every model shape measured once the copies go first: a MobileNetV2 shape, whose 52 layers hold only
+    // 8.8 MB, went from 0.62 to 0.41 ms -- its run is bound by the host's API calls, and merged copies and grouped
+    // transforms save two thirds of them.)
     if (merge) {
         const uint64_t kFirstTarget = (uint64_t)tn.chunk_first_kb << 10, kMaxTarget = (uint64_t)tn.chunk_max_kb << 10;
         constexpr uint64_t kMaxGap = 4096;
