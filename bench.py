@@ -389,7 +389,9 @@ def measure(args, config, steps, warmup, minimal, rank, world, local, ranks):
         costs = model.profile(x, reps=5)
     if args.save_costs and rank == 0:
         json.dump(costs, open(args.save_costs, "w"))
-    costs = nb.CostTable([c for c in costs if c["math"] in (nb.MATH_FP32, math) or c["variant"] in (nb.VAR_WINO_F4, nb.VAR_WINO_F6)])
+    # math modes are accuracy classes: the BF16 class (output rel-L2 <= 1e-2) admits every kernel of the TF32 class (<= 1e-3) too
+    admitted = (nb.MATH_FP32, nb.MATH_TF32) if math == nb.MATH_TF32 else (nb.MATH_FP32, nb.MATH_TF32, nb.MATH_BF16)
+    costs = nb.CostTable([c for c in costs if c["math"] in admitted])
     choices_raw = nb.nnv_select_kernels(model.plan, costs, 0)        # headline: every layer reads RAW weights and transforms them
     choices_byp = nb.nnv_select_kernels(model.plan, costs, 1)        # bypass arm: cached post-transform weights allowed
     costs_res = nb.CostTable([dict(c, h2d_raw_ns=0, h2d_cached_ns=0) for c in costs])
