@@ -28,6 +28,7 @@ struct ConvDev {
     int C, H, W, K;                 // input channels, image (input = output grid), output channels
     int BN, MT, act, tmem_cols, splits, na, nb, cblk, tiles_w;
     int tma_out;                    // 0: plain stores; 16 / 32: columns per TMA-stored sub-tile (no K split, no addend)
+    int bf16;                       // 1: BF16 math -- the fp32 halo boxes are rounded to bf16 in shared memory, the weights arrive as bf16
 };
 
 constexpr int CONV_MAX_NA = 4, CONV_MAX_NB = 8;
@@ -39,8 +40,15 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     pdl_trigger();
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int BN = g.BN, MT = g.MT, NA = g.na, NB = g.nb;
-    const uint32_t a_slot_bytes = (uint32_t)(16 * MT + 2) * 1024u;
-    const uint32_t b_slot_bytes = (uint32_t)BN * BK_BYTES;
+    // BF16 math: a box slot holds the fp32 box as the TMA delivers it (128-byte rows, swizzled) and, behind it, the same
+    // pixels rounded to bf16 in the un-swizzled core-matrix layout [8-channel chunk][pixel row][16 bytes]; there an
+    // image row of the patch (8 pixels) is 128 bytes, so a vertical tap offset is again a shift of the descriptor's
+    // start address.  The weights arrive as bf16 in the same layout (one box of four 8-element chunks x BN rows per tile).
+    const bool bf16 = g.bf16 != 0;
+    const uint32_t box_rows = (uint32_t)(16 * MT + 2) * 8u;        // pixel rows of a halo box
+    const uint32_t a_box_bytes = box_rows * 128u;
+    const uint32_t a_slot_bytes = a_box_bytes + (bf16 ? box_rows * 64u : 0u);
+    const uint32_t b_slot_bytes = (uint32_t)BN * (bf16 ? 64u : (uint32_t)BK_BYTES);
     const uint32_t a_ring = sbase, b_ring = sbase + NA * a_slot_bytes;
     const uint32_t bars = b_ring + NB * b_slot_bytes;
     auto a_full = [&](int s) { return bars + 8u * s; };
@@ -49,6 +57,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     auto b_empty = [&](int s) { return bars + 8u * (2 * CONV_MAX_NA + CONV_MAX_NB + s); };
     const uint32_t tmem_full_bar = bars + 8u * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB);
     const uint32_t holder = tmem_full_bar + 8u;
+    auto a_conv = [&](int s) { return bars + 8u * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 2 + s); };   // box s is converted
     volatile uint32_t* holder_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (holder - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -62,7 +71,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
         if (g.tma_out) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmD)) : "memory");
-        for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < NA; ++s) { mbar_init(a_full(s), 1); mbar_init(a_empty(s), 1); mbar_init(a_conv(s), 128); }
         for (int s = 0; s < NB; ++s) { mbar_init(b_full(s), 1); mbar_init(b_empty(s), 1); }
         mbar_init(tmem_full_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -78,22 +87,41 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     pdl_wait();                                               // set-up above overlaps the previous kernel's tail
     if (threadIdx.x == 32) stamp_start(g.stamp);
 
-    // Two producers: a shared-memory fill costs its issuing thread ~150 cycles whatever its size, so the halo boxes
+    // One weight tile into ring slot `sb`: a 128-byte-swizzled fp32 tile, or a box of four 8-element bf16 chunks x BN rows
+    auto issue_b = [&](int sb, int tap, int c0) {
+        const uint32_t dst = b_ring + sb * b_slot_bytes;
+        mbar_expect_tx(b_full(sb), b_slot_bytes);
+        if (bf16) {
+            tma_load_3d(dst, &tmB, 0, n0, (tap * g.C + c0) >> 3, b_full(sb));   // {8 elements, BN rows, 4 chunks} in one load
+        } else {
+            tma_load_3d(dst, &tmB, tap * g.C + c0, n0, 0, b_full(sb));
+        }
+    };
+
+    // Two producers (TF32 math; with BF16 math warps 2-5 convert the boxes, so warp 0 issues the weight tiles too): a shared-memory fill costs its issuing thread ~150 cycles whatever its size, so the halo boxes
     // and the (smaller, three times as many) weight tiles are issued by different warps -- warp 2's first lane serves
     // the weight ring before it joins the epilogue.
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
-            int sa = 0;                                       // ring slot and its phase, carried along (no divisions:
-            uint32_t pa = 0;                                  // every instruction of this single-thread loop is latency)
+            int sa = 0, sb0 = 0;                              // ring slots and their phases, carried along (no divisions:
+            uint32_t pa = 0, pb0 = 0;                         // every instruction of this single-thread loop is latency)
             for (int cbi = 0; cbi < ncb && ok; ++cbi) {
                 const int c0 = (cb0 + cbi) * 32;
                 for (int s = 0; s < 3 && ok; ++s) {
                     ok = mbar_wait(a_empty(sa), pa ^ 1u);
                     if (!ok) break;
-                    mbar_expect_tx(a_full(sa), a_slot_bytes);
+                    mbar_expect_tx(a_full(sa), a_box_bytes);
                     tma_load_3d(a_ring + sa * a_slot_bytes, &tmA, c0, ow0 + s - 1, oh0 - 1, a_full(sa));
                     if (++sa == NA) { sa = 0; pa ^= 1u; }
+                    if (bf16) {
+                        for (int r = 0; r < 3; ++r) {
+                            ok = mbar_wait(b_empty(sb0), pb0 ^ 1u);
+                            if (!ok) break;
+                            issue_b(sb0, r * 3 + s, c0);
+                            if (++sb0 == NB) { sb0 = 0; pb0 ^= 1u; }
+                        }
+                    }
                 }
             }
             if (!ok) {
@@ -103,20 +131,32 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            // instruction descriptor: fp32 accumulate, TF32 operands, both K-major, N = BN, M = 128
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            // instruction descriptor: fp32 accumulate, TF32 (or bf16) operands, both K-major, N = BN, M = 128
+            const uint32_t fmt = bf16 ? 1u : 2u;
+            const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            const uint32_t lbo_a = box_rows * 16u, lbo_b = (uint32_t)BN * 16u;
             bool ok = true;
             int sa = 0, sb = 0;
             uint32_t pa = 0, pb = 0;
             for (int cbi = 0; cbi < ncb && ok; ++cbi) {
                 for (int s = 0; s < 3 && ok; ++s) {
-                    ok = mbar_wait(a_full(sa), pa);
+                    ok = mbar_wait(bf16 ? a_conv(sa) : a_full(sa), pa);
                     if (!ok) break;
                     const uint32_t a_box = a_ring + sa * a_slot_bytes;
                     for (int r = 0; r < 3; ++r) {
                         ok = mbar_wait(b_full(sb), pb);
                         if (!ok) break;
                         tc_fence_after();
+                        if (bf16) {
+                            const uint32_t a_bf = a_box + a_box_bytes, b_bf = b_ring + sb * b_slot_bytes;
+                            for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+                                for (int kk = 0; kk < 2; ++kk)     // 2 MMAs of 16 bf16 of K = two core matrices each
+                                    umma<true>(tmem_base + (uint32_t)(mt * BN),
+                                               make_smem_desc_plain(a_bf + (uint32_t)(mt * 16 + r) * 128u + (uint32_t)kk * 2u * lbo_a, lbo_a, 128),
+                                               make_smem_desc_plain(b_bf + (uint32_t)kk * 2u * lbo_b, lbo_b, 128), idesc, (cbi | s | r | kk) ? 1u : 0u);
+                            }
+                        } else {
                         const uint64_t bdesc = make_smem_desc(b_ring + sb * b_slot_bytes);
                         for (int mt = 0; mt < MT; ++mt) {
                             const uint64_t adesc = make_smem_desc(a_box + (uint32_t)(mt * 16 + r) * 1024u);
@@ -124,6 +164,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                             for (int kk = 0; kk < 4; ++kk)     // 4 MMAs of 32 bytes of K each
                                 umma<false>(tmem_base + (uint32_t)(mt * BN), adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2),
                                             idesc, (cbi | s | r | kk) ? 1u : 0u);
+                        }
                         }
                         umma_commit(b_empty(sb));
                         if (++sb == NB) { sb = 0; pb ^= 1u; }
@@ -137,7 +178,21 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
     } else {
         bool ok = true;
-        if (warp == 2 && lane == 0) {                         // the weight-tile producer
+        if (bf16) {
+            // warps 2-5 round every halo box to bf16 as it lands (one pixel row of 32 channels per thread and pass)
+            int sa = 0;
+            uint32_t pa = 0;
+            for (int it = 0; it < 3 * ncb && ok; ++it) {
+                ok = mbar_wait(a_full(sa), pa);
+                if (!ok) break;
+                const uint32_t a_box = a_ring + sa * a_slot_bytes;
+                for (uint32_t row = threadIdx.x - 64; row < box_rows; row += 128) convert_row_bf16(a_box, a_box + a_box_bytes, (int)row, (int)box_rows);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
+                mbar_arrive(a_conv(sa));
+                if (++sa == NA) { sa = 0; pa ^= 1u; }
+            }
+            ok = __all_sync(0xffffffffu, (int)ok) != 0;
+        } else if (warp == 2 && lane == 0) {                  // the weight-tile producer
             int sb = 0;
             uint32_t pb = 0;
             for (int cbi = 0; cbi < ncb && ok; ++cbi) {
@@ -146,8 +201,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     for (int r = 0; r < 3; ++r) {
                         ok = mbar_wait(b_empty(sb), pb ^ 1u);
                         if (!ok) break;
-                        mbar_expect_tx(b_full(sb), b_slot_bytes);
-                        tma_load_3d(b_ring + sb * b_slot_bytes, &tmB, (r * 3 + s) * g.C + c0, n0, 0, b_full(sb));
+                        issue_b(sb, r * 3 + s, c0);
                         if (++sb == NB) { sb = 0; pb ^= 1u; }
                     }
                 }

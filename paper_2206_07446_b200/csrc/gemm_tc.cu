@@ -265,7 +265,7 @@ __device__ __forceinline__ void convert_row_bf16(uint32_t src_tile, uint32_t dst
 
 // MODE 3: A is fp32 (the activation itself, direct or through the TMA's im2col mode) and is rounded to bf16 by the
 // epilogue warps on its way through shared memory; B is the bf16 packed weight, fetched straight into the
-// un-swizzled core-matrix layout by four TMA boxes of 8 elements (16 bytes) x BN rows per stage.
+// un-swizzled core-matrix layout by ONE TMA box per stage over the rows seen as {8 elements, N rows, chunks}.
 // MODE 0: TF32 operands (fp32 words), 1: BF16 operands, 2: fp32 operands multiplied as
 // hi*hi + lo*hi + hi*lo of their bf16 splits (error-compensated, fp32-class accuracy).
 template <int MODE> struct ModeTraits {
@@ -362,11 +362,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (g.ic_on) {
             // A comes straight from the activation: block `kb` is channel block ic_cb of tap (ic_fr, ic_fs)
             tma_load_im2col_4d(a_dst, &tmA, ic_cb * BKE, ic_w0, ic_h0, 0, (uint16_t)ic_fs, (uint16_t)ic_fr, full_bar(s));
-            if constexpr (MODE == 3) {   // B: four boxes of 8 elements x BN rows, staged after the fp32 and the bf16 A tile
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    tma_load_3d(a_dst + A_STAGE_BYTES + A_STAGE_BYTES / 2 + (uint32_t)c * (uint32_t)BN * 16u, &tmB,
-                                ic_tap * g.ic_C + ic_cb * BKE + 8 * c, n0, 0, full_bar(s));
+            if constexpr (MODE == 3) {   // B: one box of four 8-element chunks x BN rows, staged after the fp32 and the bf16 A tile
+                tma_load_3d(a_dst + A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmB, 0, n0, (ic_tap * g.ic_C + ic_cb * BKE) >> 3, full_bar(s));
             } else {
                 tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, ic_tap * g.ic_C + ic_cb * BKE, n0, b, full_bar(s));
             }
@@ -377,10 +374,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         } else {
             tma_load_3d(a_dst, &tmA, kb * BKE, m0, b, full_bar(s));
             if constexpr (MODE == 3) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    tma_load_3d(a_dst + A_STAGE_BYTES + A_STAGE_BYTES / 2 + (uint32_t)c * (uint32_t)BN * 16u, &tmB, kb * BKE + 8 * c, n0, 0,
-                                full_bar(s));
+                tma_load_3d(a_dst + A_STAGE_BYTES + A_STAGE_BYTES / 2, &tmB, 0, n0, (kb * BKE) >> 3, full_bar(s));
             } else {
                 tma_load_3d(a_dst + A_STAGE_BYTES, &tmB, kb * BKE, n0, b, full_bar(s));
             }
@@ -788,23 +782,28 @@ nnv_status_t encode_halo_operand(CUtensorMap* map, const void* base, int C, int 
 }
 
 // Tiling of conv3x3_tc_kernel for one layer.
-struct ConvTiling { int MT, BN, splits, na, nb, tmem_cols; size_t smem; };
+struct ConvTiling { int MT, BN, splits, na, nb, tmem_cols, bf16; size_t smem; };
 
-size_t conv_smem_bytes(int MT, int BN, int na, int nb) {
-    return (size_t)1024 + (size_t)na * (16 * MT + 2) * 1024 + (size_t)nb * BN * BK_BYTES + 8 * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 2);
+// Bytes of one halo-box slot and one weight-tile slot: with BF16 math a box slot also holds the box rounded to bf16
+// (half its size) and a weight tile is bf16.
+size_t conv_a_slot(int MT, int bf16) { return (size_t)(16 * MT + 2) * 1024 * (bf16 ? 3 : 2) / 2; }
+size_t conv_b_slot(int BN, int bf16) { return (size_t)BN * (bf16 ? 64 : BK_BYTES); }
+
+size_t conv_smem_bytes(int MT, int BN, int na, int nb, int bf16) {
+    return (size_t)1024 + (size_t)na * conv_a_slot(MT, bf16) + (size_t)nb * conv_b_slot(BN, bf16) + 8 * (3 * CONV_MAX_NA + 2 * CONV_MAX_NB + 2);
 }
 
 // Fills in ring depths (unless given), shared-memory size and TMEM columns; false if the tiling does
 // not fit (shared memory, or room to park the partial tiles of a K split).
 bool finish_conv_tiling(ConvTiling* t) {
     const size_t park = t->splits > 1 ? (size_t)t->MT * BM * (t->BN + 4) * 4 : 0;
-    auto rings = [&] { return (size_t)t->na * (16 * t->MT + 2) * 1024 + (size_t)t->nb * t->BN * BK_BYTES; };
+    auto rings = [&] { return (size_t)t->na * conv_a_slot(t->MT, t->bf16) + (size_t)t->nb * conv_b_slot(t->BN, t->bf16); };
     if (t->na <= 0 || t->nb <= 0) {
         t->na = 2; t->nb = 3;
         while (rings() < park && t->nb < CONV_MAX_NB) ++t->nb;      // deeper rings only to make room for the parked tiles
         while (rings() < park && t->na < CONV_MAX_NA) ++t->na;
     }
-    t->smem = conv_smem_bytes(t->MT, t->BN, t->na, t->nb);
+    t->smem = conv_smem_bytes(t->MT, t->BN, t->na, t->nb, t->bf16);
     t->tmem_cols = 32;
     while (t->tmem_cols < t->MT * t->BN) t->tmem_cols *= 2;
     return t->smem <= 200u * 1024u && rings() >= park;
@@ -818,10 +817,11 @@ bool finish_conv_tiling(ConvTiling* t) {
 // to one slot when that makes them fit.  Layers with fewer than four channel blocks and fewer than
 // two patches per SM, and layers too small to give every SM a CTA even with 8 splits, stay on the
 // plain implicit GEMM, which is faster there.
-bool pick_conv_tiling(int C, int H, int W, int N, ConvTiling* out) {
+bool pick_conv_tiling(int C, int H, int W, int N, int bf16, ConvTiling* out) {
     const int cblk = ceil_div(C, 32);
     ConvTiling t{};
     t.MT = 1;
+    t.bf16 = bf16;
     t.BN = std::min(128, ceil_div(N, 16) * 16);
     const long long tiles = (long long)ceil_div(H, 16) * ceil_div(W, 8) * ceil_div(N, t.BN);
     int max_sp = 1;
@@ -864,6 +864,23 @@ nnv_status_t gemm_tc_init() {
     return NNV_OK;
 }
 
+// bf16 packed weights [N][ld]: boxes of 8 elements (16 bytes) x BN rows, no swizzle -- four of them make the
+// un-swizzled core-matrix layout of a 32-element K block.
+static nnv_status_t encode_bf16_weight_chunks(CUtensorMap* map, const void* base, int64_t ld, int N, int BN) {
+    NNV_REQUIRE((ld % 8) == 0 && (reinterpret_cast<uintptr_t>(base) & 15) == 0, NNV_ERR_INVALID_ARG, "bf16 weight rows must be 16-byte multiples");
+    // the rows seen as {8 elements, N rows, ld / 8 chunks}: one box of {8, BN, 4} lands as [chunk][row][16 bytes], i.e. a whole
+    // 32-element K block of BN rows in the core-matrix layout with ONE load (a fill costs ~150 cycles whatever its size)
+    cuuint64_t dims[3] = {8, (cuuint64_t)N, (cuuint64_t)(ld / 8)};
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 2, 16};
+    cuuint32_t box[3] = {8, (cuuint32_t)BN, 4};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (bf16 weight chunks) failed with code %d", (int)r);
+    return NNV_OK;
+}
+
 // 3-D tiled map over the NHWC fp32 output {K, W, H}: boxes of `cw` channels x 8 pixels x 4 rows (what one warp of the
 // 3x3 kernel holds), in the swizzled layout the epilogue writes.
 static nnv_status_t encode_conv_output(CUtensorMap* map, const void* base, int K, int H, int W, int cw) {
@@ -881,7 +898,8 @@ static nnv_status_t encode_conv_output(CUtensorMap* map, const void* base, int K
 static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, cudaStream_t st) {
     CUtensorMap tmA, tmB, tmD;
     NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 16 * ct.MT + 2));
-    NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, ct.BN));
+    if (ct.bf16) NNV_TRY(encode_bf16_weight_chunks(&tmB, a.B, a.ldb, a.N, ct.BN));
+    else NNV_TRY(encode_operand(&tmB, a.B, false, a.Kd, a.N, 1, a.ldb, a.strideB, ct.BN));
     ConvDev g;
     g.stamp = next_stamp();
     next_stamp() = nullptr;
@@ -889,11 +907,12 @@ static nnv_status_t launch_conv3x3_tc(const GemmArgs& a, const ConvTiling& ct, c
     g.C = a.ic.C; g.H = a.ic.H; g.W = a.ic.W; g.K = a.N;
     g.BN = ct.BN; g.MT = ct.MT; g.act = a.act; g.tmem_cols = ct.tmem_cols; g.splits = ct.splits; g.na = ct.na; g.nb = ct.nb;
     g.cblk = ceil_div(a.ic.C, 32); g.tiles_w = ceil_div(a.ic.W, 8);
+    g.bf16 = ct.bf16;
     NNV_REQUIRE(a.ldd == a.N, NNV_ERR_INVALID_ARG, "the 3x3 kernel writes a dense NHWC output");
     // Write-out by TMA when nothing is added after the K loop but the bias, the output rows are 16-byte multiples and
     // the staged tile fits into the (then idle) rings; else plain stores.
     g.tma_out = 0;
-    const size_t rings = (size_t)ct.na * (16 * ct.MT + 2) * 1024 + (size_t)ct.nb * ct.BN * BK_BYTES;
+    const size_t rings = (size_t)ct.na * conv_a_slot(ct.MT, ct.bf16) + (size_t)ct.nb * conv_b_slot(ct.BN, ct.bf16);
     if (ct.splits == 1 && !a.addend && (a.N % 4) == 0 && (reinterpret_cast<uintptr_t>(a.D) & 15) == 0 &&
         (!a.bias || (reinterpret_cast<uintptr_t>(a.bias) & 15) == 0) && (size_t)ct.MT * BM * ct.BN * 4 <= rings) {
         g.tma_out = (ct.BN % 32) == 0 ? 32 : 16;
@@ -1100,15 +1119,22 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     if (tn.gemm_bn && tn.gemm_splits <= nkb_all) { BN = tn.gemm_bn; splits = tn.gemm_splits; }   // override (nnv_tuning_set)
     // A 3x3 / stride 1 / pad 1 layer large enough to fill the GPU runs on the halo-resident kernel,
     // which moves fewer operand bytes through L2 and shared memory.
-    if (a.ic.on && a.mode == GEMM_TF32 && a.batch == 1 && a.ic.R == 3 && a.ic.S == 3 && a.ic.stride == 1 && a.ic.pad == 1 &&
-        (a.ic.C % 32) == 0) {
+    if (a.ic.on && (a.mode == GEMM_TF32 || a.mode == GEMM_BF16_CVT) && a.batch == 1 && a.ic.R == 3 && a.ic.S == 3 && a.ic.stride == 1 &&
+        a.ic.pad == 1 && (a.ic.C % 32) == 0) {
+        const int cbf = a.mode == GEMM_BF16_CVT ? 1 : 0;
         ConvTiling ct;
-        bool use = pick_conv_tiling(a.ic.C, a.ic.H, a.ic.W, a.N, &ct);
+        bool use = pick_conv_tiling(a.ic.C, a.ic.H, a.ic.W, a.N, cbf, &ct);
+        // BF16 math: every box passes through the conversion warps before its MMAs, which a CTA with a single channel
+        // block (three boxes) cannot hide -- measured on 128 -> 128 @112: 29.7 us against 18.2 for the converting implicit
+        // GEMM; with two or more blocks per CTA the halo kernel is ahead (64 -> 64 @224: 19.6 against 29.3 us,
+        // 256 -> 256 @56: 20.4 against 26.2, 512 -> 512 @28: 20.7 against 26.9).
+        if (use && cbf && ceil_div(a.ic.C, 32) / ct.splits < 2) use = false;
         if (tn.conv3x3 == 1) {
             use = false;
         } else if (tn.conv3x3 == 2) {
             ConvTiling f{};
             f.MT = tn.conv_mt; f.BN = tn.conv_bn; f.splits = tn.conv_splits; f.na = tn.conv_na; f.nb = tn.conv_nb;
+            f.bf16 = cbf;
             if (f.splits <= ceil_div(a.ic.C, 32) && finish_conv_tiling(&f)) {
                 ct = f;
                 use = true;
@@ -1125,8 +1151,8 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         // alone where the tensor pipe needs 1.2; three one-tile CTAs per SM issue from three threads, and the resident
         // weights leave room for only three halo boxes in flight.
         int wbn = 0;
-        if (tn.convw == 2 && convw_fits(a, &wbn)) return launch_conv3x3_ws(a, wbn, st);
-        if (tn.convp == 2 && (size_t)tn.convp_bn <= (size_t)ceil_div(a.N, 16) * 16)
+        if (!cbf && tn.convw == 2 && convw_fits(a, &wbn)) return launch_conv3x3_ws(a, wbn, st);
+        if (!cbf && tn.convp == 2 && (size_t)tn.convp_bn <= (size_t)ceil_div(a.N, 16) * 16)
             return launch_conv3x3_persistent(a, tn.convp_bn, tn.convp_per_sm, tn.convp_na ? tn.convp_na : 2, tn.convp_nb ? tn.convp_nb : 4, st);
         if (use) return launch_conv3x3_tc(a, ct, st);
     }
@@ -1157,16 +1183,8 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         NNV_TRY(encode_operand(&tmA, a.A, bf16, a.Kd, a.M, a.batch, a.lda, a.strideA, BM));
     }
     if (a.mode == GEMM_BF16_CVT) {
-        // bf16 weights, boxes of 8 elements x BN rows, no swizzle: four of them make the core-matrix layout of a stage
-        NNV_REQUIRE(a.batch == 1 && (a.ldb % 8) == 0, NNV_ERR_INVALID_ARG, "the converting BF16 mode needs one batch and 16-byte weight rows");
-        cuuint64_t dims[3] = {(cuuint64_t)a.ldb, (cuuint64_t)a.N, 1};
-        cuuint64_t strides[2] = {(cuuint64_t)a.ldb * 2, (cuuint64_t)a.ldb * 2 * (cuuint64_t)a.N};
-        cuuint32_t box[3] = {8, (cuuint32_t)BN, 1};
-        cuuint32_t estr[3] = {1, 1, 1};
-        CUresult r = g_encode(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(a.B), dims, strides, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (bf16 weight chunks) failed with code %d", (int)r);
+        NNV_REQUIRE(a.batch == 1, NNV_ERR_INVALID_ARG, "the converting BF16 mode needs one batch");
+        NNV_TRY(encode_bf16_weight_chunks(&tmB, a.B, a.ldb, a.N, BN));
     } else {
         NNV_TRY(encode_operand(&tmB, a.B, bf16, a.Kd, a.N, a.batch, a.ldb, a.strideB, BN));
     }

@@ -10,12 +10,12 @@ from gpu_util import TOL, rel_l2, run_conv
 
 pytestmark = pytest.mark.gpu
 
-def _run(L, x, w, b, add, setting):
+def _run(L, x, w, b, add, setting, math=nb.MATH_TF32):
     """One layer with the 3x3 kernel's tiling forced through nnv_tuning_set (None = the library's own pick)."""
     nb.nnv_tuning_set(None if setting is None else "conv3x3=" + setting)
     try:
         plan = nb.Plan([L], [0], [0])
-        return run_conv(plan, 0, L, nb.VAR_IM2COL, nb.MATH_TF32, x, w, b, add)
+        return run_conv(plan, 0, L, nb.VAR_IM2COL, math, x, w, b, add)
     finally:
         nb.nnv_tuning_set(None)
 
@@ -59,6 +59,22 @@ def test_every_tiling_matches_the_oracle(shape):
     # whatever the library picks by itself is one of the two kernels above
     auto = _run(L, x, w, b, add, None)
     assert rel_l2(auto, ref) <= TOL[nb.MATH_TF32]
+    # BF16 math on the same tilings: the halo boxes are rounded to bf16 in shared memory, the weights arrive as bf16;
+    # the same products as the converting implicit GEMM (conv3x3=off), summed in another order
+    plain16 = _run(L, x, w, b, add, "off", nb.MATH_BF16)
+    assert rel_l2(plain16, ref) <= TOL[nb.MATH_BF16]
+    ran16 = 0
+    for mt in (1, 2):
+        for bn in sorted({bn_full, 16, min(bn_full, 64)}):
+            for sp in (1, 2, 4, 8):
+                if sp > cblk:
+                    continue
+                y = _run(L, x, w, b, add, "%d,%d,%d" % (mt, bn, sp), nb.MATH_BF16)
+                assert np.all(np.isfinite(y)), (mt, bn, sp)
+                assert rel_l2(y, ref) <= TOL[nb.MATH_BF16], (mt, bn, sp, rel_l2(y, ref))
+                assert rel_l2(y, plain16) <= 1e-5, (mt, bn, sp, rel_l2(y, plain16))
+                ran16 += 1
+    assert ran16 >= 4
 
 
 def _run_p(L, x, w, b, add, setting):
