@@ -690,7 +690,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 #include "conv3x3_tc.cuh"
-#include "conv3x3_tc2.cuh"
 #include "gemm_sp.cuh"
 #include "wino_fused.cuh"
 
@@ -861,7 +860,6 @@ nnv_status_t gemm_tc_init() {
         cudaFuncSetAttribute(conv3x3_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(wino_f2_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         cudaFuncSetAttribute(conv3x3_tc_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);
-        cudaFuncSetAttribute(conv3x3_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     });
     return NNV_OK;
 }
@@ -1080,92 +1078,6 @@ static nnv_status_t launch_conv3x3_persistent(const GemmArgs& a, int BN, int per
     return NNV_OK;
 }
 
-// ---- the 3x3 kernel on CTA pairs -----------------------------------------------------------------
-struct ConvPairTiling { int BN, splits, na, nb, tmem_cols; size_t smem; };
-
-static size_t conv_pair_rings(const ConvPairTiling& t) { return (size_t)t.na * 18 * 1024 + (size_t)t.nb * 3 * (t.BN / 2) * BK_BYTES; }
-
-// Fills in ring depths (unless given), shared-memory size and TMEM columns; false if the tiling does not fit.
-static bool finish_conv_pair_tiling(ConvPairTiling* t) {
-    if (t->BN < 16 || t->BN > 256 || (t->BN % 16) || (t->splits != 1 && t->splits != 2 && t->splits != 4)) return false;
-    const size_t park = t->splits > 1 ? (size_t)BM * (t->BN + 4) * 4 : 0;
-    if (t->na <= 0 || t->nb <= 0) {
-        t->na = 2; t->nb = 2;
-        while (conv_pair_rings(*t) < park && t->nb < CONV_MAX_NB) ++t->nb;
-        while (conv_pair_rings(*t) < park && t->na < CONV_MAX_NA) ++t->na;
-    }
-    if (t->na > CONV_MAX_NA || t->nb > CONV_MAX_NB) return false;
-    t->smem = (size_t)1024 + conv_pair_rings(*t) + 8 * (2 * CONV_MAX_NA + 2 * CONV_MAX_NB + 2);
-    t->tmem_cols = 32;
-    while (t->tmem_cols < t->BN) t->tmem_cols *= 2;
-    return t->smem <= 200u * 1024u && conv_pair_rings(*t) >= park && conv_pair_rings(*t) >= 4u * 32u * 36u * 4u;
-}
-
-// The packed 3x3 weights P[k][(r * 3 + s) * C + c] seen as {c, k, s, r}: one box of {32 channels, rows filters, 1, 3} is the
-// weight tiles of the taps (0, s), (1, s), (2, s) for one block of channels, one tile after the other in shared memory.
-static nnv_status_t encode_weight_taps(CUtensorMap* map, const void* base, int C, int N, int64_t ld, int rows) {
-    NNV_REQUIRE((reinterpret_cast<uintptr_t>(base) & 15) == 0 && (C % 4) == 0 && (ld % 4) == 0, NNV_ERR_INVALID_ARG,
-                "packed weights must be 16-byte aligned with rows of 16-byte multiples");
-    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)N, 3, 3};
-    cuuint64_t strides[3] = {(cuuint64_t)ld * 4, (cuuint64_t)C * 4, (cuuint64_t)C * 12};
-    cuuint32_t box[4] = {32, (cuuint32_t)rows, 1, 3};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    NNV_REQUIRE(r == CUDA_SUCCESS, NNV_ERR_CUDA, "cuTensorMapEncodeTiled (weight taps) failed with code %d", (int)r);
-    return NNV_OK;
-}
-
-static nnv_status_t launch_conv3x3_pair(const GemmArgs& a, const ConvPairTiling& ct, cudaStream_t st) {
-    CUtensorMap tmA, tmB, tmD;
-    NNV_TRY(encode_halo_operand(&tmA, a.A, a.ic.C, a.ic.H, a.ic.W, 18));
-    NNV_TRY(encode_weight_taps(&tmB, a.B, a.ic.C, a.N, a.ldb, ct.BN / 2));
-    ConvPairDev g;
-    g.stamp = next_stamp();
-    next_stamp() = nullptr;
-    g.D = a.D; g.bias = a.bias; g.addend = a.addend;
-    g.C = a.ic.C; g.H = a.ic.H; g.W = a.ic.W; g.K = a.N;
-    g.BN = ct.BN; g.act = a.act; g.tmem_cols = ct.tmem_cols; g.splits = ct.splits; g.na = ct.na; g.nb = ct.nb;
-    g.cblk = ceil_div(a.ic.C, 32); g.tiles_w = ceil_div(a.ic.W, 8);
-    NNV_REQUIRE(a.ldd == a.N, NNV_ERR_INVALID_ARG, "the 3x3 kernel writes a dense NHWC output");
-    NNV_REQUIRE(ct.splits <= g.cblk, NNV_ERR_INVALID_ARG, "more K splits than channel blocks");
-    g.tma_out = 0;
-    if (ct.splits == 1 && !a.addend && (a.N % 4) == 0 && (reinterpret_cast<uintptr_t>(a.D) & 15) == 0 &&
-        (!a.bias || (reinterpret_cast<uintptr_t>(a.bias) & 15) == 0) && (size_t)BM * ct.BN * 4 <= conv_pair_rings(ct)) {
-        g.tma_out = (ct.BN % 32) == 0 ? 32 : 16;
-        NNV_TRY(encode_conv_output(&tmD, a.D, a.N, a.ic.H, a.ic.W, g.tma_out));
-    } else {
-        tmD = tmA;                                               // unused by the kernel, but a kernel parameter must hold a valid object
-    }
-    const int patches = ceil_div(a.ic.H, 16) * g.tiles_w;
-    dim3 grid((unsigned)((patches + 1) & ~1), ceil_div(a.N, ct.BN), ct.splits);
-    NNV_REQUIRE(grid.y <= 65535, NNV_ERR_UNSUPPORTED, "convolution grid too large");
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(GEMM_THREADS);
-    cfg.dynamicSmemBytes = ct.smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = 2;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = (unsigned)ct.splits;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    (void)cudaLaunchKernelEx(&cfg, conv3x3_tc_pair_kernel, tmA, tmB, tmD, g);
-    NNV_CUDA(cudaGetLastError());
-    return NNV_OK;
-}
-
-// Where the pair kernel is taken without being asked for (filled in from measurements).
-static bool pick_conv_pair_tiling(int C, int H, int W, int N, ConvPairTiling* out) {
-    (void)C; (void)H; (void)W; (void)N; (void)out;
-    return false;
-}
-
 nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
     NNV_REQUIRE(a.M > 0 && a.N > 0 && a.Kd > 0 && a.batch > 0, NNV_ERR_INVALID_ARG, "empty GEMM");
     NNV_TRY(gemm_tc_init());
@@ -1238,17 +1150,6 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
         // issues one tcgen05.mma per ~82 cycles whatever N is, so the 72 MMAs (N = 64) of a patch take 3 us of issue time
         // alone where the tensor pipe needs 1.2; three one-tile CTAs per SM issue from three threads, and the resident
         // weights leave room for only three halo boxes in flight.
-        if (!cbf && tn.conv2 != 1) {
-            ConvPairTiling pt{};
-            bool pair = false;
-            if (tn.conv2 == 2) {
-                pt.BN = tn.conv2_bn; pt.splits = tn.conv2_splits; pt.na = tn.conv2_na; pt.nb = tn.conv2_nb;
-                pair = pt.BN <= ceil_div(a.N, 16) * 16 && pt.splits <= ceil_div(a.ic.C, 32) && finish_conv_pair_tiling(&pt);
-            } else {
-                pair = pick_conv_pair_tiling(a.ic.C, a.ic.H, a.ic.W, a.N, &pt);
-            }
-            if (pair) return launch_conv3x3_pair(a, pt, st);
-        }
         int wbn = 0;
         if (!cbf && tn.convw == 2 && convw_fits(a, &wbn)) return launch_conv3x3_ws(a, wbn, st);
         if (!cbf && tn.convp == 2 && (size_t)tn.convp_bn <= (size_t)ceil_div(a.N, 16) * 16)

@@ -149,8 +149,6 @@ struct Tuning {
     int convp = 0;                            // persistent 3x3 kernel: 0 auto, 1 off, 2 forced with the values below
     int convp_bn = 0, convp_per_sm = 0, convp_na = 0, convp_nb = 0;
     int convw = 0;                            // weights-stationary 3x3 kernel: 0 the library decides, 1 off, 2 wherever it fits
-    int conv2 = 0;                            // 3x3 kernel on CTA pairs (cta_group::2): 0 the library decides, 1 off, 2 forced with the values below
-    int conv2_bn = 0, conv2_splits = 0, conv2_na = 0, conv2_nb = 0;
     int side = 1, merge = 1, group = 1;       // pipeline features: side stream, merged reads, grouped transforms
     int copies_first = 1;                     // merged reads all enqueued before the first kernel
     int chunk_first_kb = 256, chunk_max_kb = 16384;   // merged reads: size target of the first chunk, doubling up to the maximum

@@ -73,15 +73,6 @@ static const char* parse_tuning(const char* spec, Tuning* t, char* item, size_t 
                 ok = got >= 2 && a >= 16 && a <= 128 && a % 16 == 0 && b >= 1 && b <= 4 && (got < 3 || (c >= 1 && c <= 4)) && (got < 4 || (d >= 1 && d <= 8));
                 if (ok) { t->convp = 2; t->convp_bn = a; t->convp_per_sm = b; t->convp_na = got >= 3 ? c : 0; t->convp_nb = got >= 4 ? d : 0; }
             }
-        } else if (!std::strcmp(key, "conv3x3x2")) {
-            if (!std::strcmp(val, "off")) { t->conv2 = 1; ok = true; }
-            else if (!std::strcmp(val, "auto")) { t->conv2 = 0; ok = true; }
-            else {
-                const int got = std::sscanf(val, "%d,%d,%d,%d", &a, &b, &c, &d);
-                ok = got >= 2 && a >= 16 && a <= 256 && a % 16 == 0 && (b == 1 || b == 2 || b == 4) && (got < 3 || (c >= 0 && c <= 4)) &&
-                     (got < 4 || (d >= 0 && d <= 8));
-                if (ok) { t->conv2 = 2; t->conv2_bn = a; t->conv2_splits = b; t->conv2_na = got >= 3 ? c : 0; t->conv2_nb = got >= 4 ? d : 0; }
-            }
         } else if (!std::strcmp(key, "conv3x3w")) {
             if (!std::strcmp(val, "off")) { t->convw = 1; ok = true; }
             else if (!std::strcmp(val, "auto")) { t->convw = 0; ok = true; }

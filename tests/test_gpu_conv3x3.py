@@ -155,47 +155,3 @@ def test_weights_stationary_form_matches_the_oracle(shape):
         assert np.array_equal(y.view(np.uint32), one_tile.view(np.uint32))
     again = _run_p(L, x, w, b, add, "conv3x3w=on")
     assert np.array_equal(y.view(np.uint32), again.view(np.uint32))
-
-
-@pytest.mark.parametrize("shape", [
-    # C, K, H, W, bias + addend + ReLU6
-    (64, 64, 56, 56, False),         # 49 patches: the last pair's second CTA has no patch at all
-    (32, 48, 40, 30, True),          # ragged: H % 16 != 0, W % 8 != 0, K = 48 (weight halves of 24 rows), epilogue terms
-    (128, 256, 28, 28, False),       # a channel tile of 256 (both CTAs fetch 128 filters); four channel blocks: K splits 2 and 4
-    (96, 200, 35, 21, True),         # K = 200: the second half tile partly beyond the filters; three channel blocks
-    (256, 20, 17, 9, True),          # K = 20: scalar epilogue stores; one pair
-])
-def test_pair_kernel_matches_the_oracle(shape):
-    """The 3x3 kernel on CTA pairs (one MMA stream of M = 256 over two patches, every CTA fetching half of each weight
-    tile): every channel-tile width and K split it can take against the oracle and the plain implicit GEMM."""
-    C, K, H, W, epi = shape
-    L = dict(op=0, C=C, K=K, R=3, S=3, stride=1, pad=1, groups=1, H=H, W=W, in0=-1, in1=-1, act=2 if epi else 1,
-             has_bias=1 if epi else 0)
-    rng = np.random.default_rng([11] + list(shape[:4]))
-    x = rng.uniform(-1, 1, (C, H, W)).astype(np.float32)
-    w = (rng.standard_normal((K, C, 3, 3)) * np.sqrt(2.0 / (C * 9))).astype(np.float32)
-    b = rng.uniform(-1, 1, K).astype(np.float32) if epi else None
-    add = rng.uniform(-1, 1, (K, H, W)).astype(np.float32) if epi else None
-    ref = omodel.run_layer(L, x, w, b, add)
-    plain = _run_p(L, x, w, b, add, "conv3x3x2=off;conv3x3=off")
-    assert rel_l2(plain, ref) <= TOL[nb.MATH_TF32]
-    bn_full = min(256, -(-K // 16) * 16)
-    cblk = C // 32
-    ran = 0
-    for bn in sorted({bn_full, min(bn_full, 128), min(bn_full, 64), 16}):
-        for sp in (1, 2, 4):
-            if sp > cblk:
-                continue
-            for rings in ("", ",1,1", ",4,3"):
-                y = _run_p(L, x, w, b, add, "conv3x3x2=%d,%d%s" % (bn, sp, rings))
-                assert np.all(np.isfinite(y)), (bn, sp, rings)
-                err = rel_l2(y, ref)
-                assert err <= TOL[nb.MATH_TF32], (bn, sp, rings, err)
-                # same products, other summation order than the plain kernel: fp32 rounding apart only
-                assert rel_l2(y, plain) <= 1e-5, (bn, sp, rings, rel_l2(y, plain))
-                ran += 1
-    assert ran >= 6
-    # run to run the same bits (the K split adds in a fixed order)
-    again = _run_p(L, x, w, b, add, "conv3x3x2=%d,%d" % (min(bn_full, 64), min(2, cblk)))
-    once = _run_p(L, x, w, b, add, "conv3x3x2=%d,%d" % (min(bn_full, 64), min(2, cblk)))
-    assert np.array_equal(again.view(np.uint32), once.view(np.uint32))
