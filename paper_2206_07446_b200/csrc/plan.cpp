@@ -191,11 +191,13 @@ SmallPPlan small_p_plan(const nnv_layer_desc_t& L, const LayerGeom& g, int v, in
     sp.nkb = L.R * L.S * (L.C / 32);
     const int m_tiles = ceil_div(L.K, 128);
     const int s_max = std::min(sp.nkb, std::max(1, 148 / m_tiles));
-    // microseconds: fixed cost + K blocks per CTA at ~100 GB/s of shared-memory fill per SM + (split) the second
-    // kernel and the partial tiles' trip through L2
+    // microseconds: fixed cost + K blocks per CTA at ~70 GB/s of shared-memory fill per SM + (split) the second
+    // kernel and the partial tiles' trip through L2.  Refit on sweeps of the split count (L2 flushed): 512 -> 2048 1x1 @7
+    // takes 7.8 / 6.7 / 6.3 / 6.1 / 6.5 us with 1 / 2 / 3 / 6 / 9 splits, 2048 -> 512 1x1 @7 14.5 / 10.6 / 8.2 / 7.9 / 8.3 us
+    // with 2 / 4 / 8 / 16 / 37, 512 -> 512 3x3 @7 11.7 / 9.6 / 9.7 us with 8 / 18 / 37.
     double best = 1e30;
     for (int s = 1; s <= s_max; ++s) {
-        const double t = 2.0 + ceil_div(sp.nkb, s) * stage / 100e3 + (s > 1 ? 3.0 + 3.0 * s * g.P * L.K * 4.0 / 4e6 : 0.0);
+        const double t = 2.0 + ceil_div(sp.nkb, s) * stage / 69e3 + (s > 1 ? 1.6 + 2.5 * s * g.P * L.K * 4.0 / 4e6 : 0.0);
         if (t < best - 1e-9) { best = t; sp.splits = s; }
     }
     if (tn.smallp_splits && tn.smallp_splits <= sp.nkb) sp.splits = tn.smallp_splits;
