@@ -1107,10 +1107,15 @@ nnv_status_t launch_gemm_tc(const GemmArgs& a, cudaStream_t st) {
             const double smem = 1024.0 + stages * kb_bytes * (a.mode == GEMM_X3 ? 2 : 1);
             const int occ = std::max(1, std::min(4, (int)(220.0 * 1024.0 / smem)));
             double waves = std::ceil((double)ctas / (148.0 * occ));
-            if (sp > 1 && occ == 1 && ctas > 96) waves = std::max(waves, 2.0);     // whole clusters must find free SMs in one GPC
+            // whole clusters must find free SMs in one GPC (16 - 20 SMs): measured in one wave are 14 clusters of 8
+            // (128 -> 128 3x3 @28 at BN = 64: 6.3 us against 8.3) and 32 clusters of 4 (1024 -> 2048 1x1 / 2 @14 at BN = 64: 6.8 against 9.0)
+            if (sp > 1 && occ == 1 && ctas > (sp == 8 ? 112 : sp == 4 ? 128 : 144)) waves = std::max(waves, 2.0);
             const int resident = (int)std::min<long long>(occ, (ctas + 147) / 148);   // CTAs that really share an SM
-            const double per_kb_us = std::max(kb_bytes * resident / 100e3, 0.12) * (stages >= 8 ? 1.0 : 1.3);
-            const double t = waves * (2.0 + (sp > 1 ? 3.0 : 0.0) + std::ceil((double)nkb_all / sp) * per_kb_us + 0.3 + bn * 0.004);
+            // refit on a sweep of every (BN, splits) over the GEMM layer shapes of the ResNet-shaped configurations (kernel
+            // stamps, L2 flushed): a K block costs a CTA at least 0.25 us however narrow its tile (an unsplit BN = 16 launch of
+            // 512 -> 128 @28 took 6.5 us where 5.3 was predicted, 64 x 8 splits 6.0), a split 2.5 us
+            const double per_kb_us = std::max(kb_bytes * resident / 100e3, 0.25) * (stages >= 8 ? 1.0 : 1.3);
+            const double t = waves * (2.0 + (sp > 1 ? 2.5 : 0.0) + std::ceil((double)nkb_all / sp) * per_kb_us + 0.3 + bn * 0.004);
             if (t < best - 1e-9) { best = t; BN = bn; splits = sp; }
         }
         if (bn <= 16) break;
