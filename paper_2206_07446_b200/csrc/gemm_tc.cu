@@ -827,6 +827,11 @@ bool pick_conv_tiling(int C, int H, int W, int N, int bf16, ConvTiling* out) {
     int max_sp = 1;
     while (max_sp * 2 <= std::min(8, cblk)) max_sp *= 2;
     if (tiles * max_sp < 148 || (cblk < 4 && tiles < 296)) return false;
+    // Against the implicit GEMM with its refit tiling model (kernel stamps, L2 flushed; halo kernel / implicit GEMM, us):
+    // 64 -> 64 @224 13.4 / 18.0 and 256 -> 256 @56 18.8 / 24.0, but 128 -> 128 @112 17.7 / 14.9, 128 -> 256 @56 14.7 / 12.8,
+    // 256 -> 512 @28 14.7 / 12.9, 512 -> 512 @28 19.0 / 18.6: the halo kernel keeps the layers with two or more patches per SM
+    // and the deep ones (eight or more channel blocks) that still have ~50 tiles.
+    if (tiles < 296 && !(cblk >= 8 && tiles >= 48)) return false;
     t.splits = 1;
     while (t.splits < max_sp && tiles * t.splits < 224) t.splits *= 2;
     const long long ctas = tiles * t.splits;

@@ -136,8 +136,8 @@ def test_degenerate_shapes_on_every_variant(shape):
 
 
 def test_halo_kernel_on_a_ragged_full_size_grid():
-    """128 -> 128, 3x3 on 57 x 59 (H % 16 != 0, W % 8 != 0): large enough that the library's own choice is the
-    halo-resident 3x3 kernel; compared with the plain implicit GEMM as well."""
+    """128 -> 128, 3x3 on 57 x 59 (H % 16 != 0, W % 8 != 0) with bias, residual addend and ReLU: the library's own choice,
+    the plain implicit GEMM and the halo-resident 3x3 kernel (tiling forced, with and without a K split) agree."""
     L = dict(op=0, C=128, K=128, R=3, S=3, stride=1, pad=1, groups=1, H=57, W=59, in0=-1, in1=-1, act=1, has_bias=1)
     rng = np.random.default_rng(57)
     x = rng.uniform(-1, 1, (128, 57, 59)).astype(np.float32)
@@ -155,6 +155,14 @@ def test_halo_kernel_on_a_ragged_full_size_grid():
         nb.nnv_tuning_set(None)
     assert_conv_close(y_plain, ref, TOL[nb.MATH_TF32], "plain implicit GEMM")
     assert rel_l2(y, y_plain) <= 1e-5
+    for tiling in ("1,128,4", "1,128,1", "2,64,2"):
+        nb.nnv_tuning_set("conv3x3=" + tiling)
+        try:
+            y_halo = run_conv(plan, 0, L, nb.VAR_IM2COL, nb.MATH_TF32, x, w, b, add)
+        finally:
+            nb.nnv_tuning_set(None)
+        assert_conv_close(y_halo, ref, TOL[nb.MATH_TF32], "halo kernel " + tiling)
+        assert rel_l2(y_halo, y_plain) <= 1e-5
 
 
 def test_residual_and_bias_epilogues_on_every_variant():
